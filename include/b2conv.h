@@ -1,0 +1,171 @@
+/*
+ * b2conv — int8 2-D convolution embedded into the Blackwell dense MMA intrinsic.
+ *
+ * C ABI of the library.  Every entry point is `extern "C"`, takes plain integers, structs of
+ * integers and raw pointers, and never throws, aborts or prints.  Unless a parameter says
+ * otherwise, pointers named *_dev are DEVICE pointers (global memory of the current CUDA
+ * device) and must be 16-byte aligned; all other pointers are HOST pointers.  `cuda_stream`
+ * is a `cudaStream_t` passed as `void*` (NULL = the legacy default stream).
+ *
+ * The operation follows Rieber, Acosta, Froening, "Joint Program and Layout Transformations to
+ * enable Convolutional Operators on Specialized Hardware based on Constraint Programming"
+ * (2021): a convolution is executed on a fixed matrix-multiply intrinsic (Section 5.1: 8-bit
+ * operands, 32-bit accumulation, C_xy += A_xz * B_zy^T, followed by a quantisation step) by
+ * choosing which convolution axes feed the intrinsic's x/y/z dimensions and rewriting the data
+ * layout to match (Table 2: stencil unroll, image pack, pad, split, reorder, fuse).  Here the
+ * intrinsic is `tcgen05.mma.kind::i8` (M = 128 rows, N = 16..256 columns, K = 32 per
+ * instruction, int32 accumulators in tensor memory).
+ *
+ * All calls return 0 (B2C_OK) or a negative B2C_E_* code.
+ */
+#ifndef B2CONV_H_
+#define B2CONV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes --------------------------------------------------------------------------- */
+#define B2C_OK 0
+#define B2C_E_INVALID_ARG (-1)         /* null pointer, misaligned pointer, value out of range   */
+#define B2C_E_UNSUPPORTED (-2)         /* valid request this library does not execute            */
+#define B2C_E_WORKSPACE_TOO_SMALL (-3) /* fixed-size scratch cannot hold this problem            */
+#define B2C_E_CUDA (-4)                /* a CUDA runtime/driver call failed; see b2c_last_cuda_error */
+#define B2C_E_TIMEOUT (-5)             /* a bounded device-side wait expired (device status word) */
+#define B2C_E_NOT_READY (-6)           /* plan has no weights yet                                */
+
+/* ---- problem description -------------------------------------------------------------------- */
+/* Convolution y[n][k][p][q] = sum_{c,r,s} x[n][c][p*stride_h - pad_h + r*dil_h][q*stride_w - pad_w + s*dil_w] * w[k][c][r][s]
+ * (Figure 5 step 1 and the access function [n, i + k] of Table 2: cross-correlation, zero
+ * padding per Section 4.2.4), int8 operands, exact int32 sums (Section 5.1).
+ * P = floor((H + 2*pad_h - dil_h*(R-1) - 1)/stride_h) + 1, Q likewise. */
+typedef struct {
+  int32_t N, C, H, W; /* input: batch, channels, height, width (all >= 1)                        */
+  int32_t K, R, S;    /* weights: output channels, kernel height, kernel width (all >= 1)        */
+  int32_t stride_h, stride_w; /* >= 1                                                            */
+  int32_t pad_h, pad_w;       /* >= 0, zeros on both sides                                       */
+  int32_t dil_h, dil_w;       /* >= 1                                                            */
+  int32_t shift;      /* 0..31: int8 output = clip(floor(acc / 2^shift), -128, 127)              */
+  int32_t in_layout;  /* B2C_LAYOUT_NCHW or B2C_LAYOUT_NHWC; tensors are dense, no strides       */
+  int32_t out_layout; /* B2C_LAYOUT_NCHW (= NKPQ) or B2C_LAYOUT_NHWC (= NPQK)                    */
+  int32_t out_mode;   /* bit 0: write int32 accumulators; bit 1: write requantised int8          */
+} b2c_conv_desc;
+
+#define B2C_LAYOUT_NCHW 0
+#define B2C_LAYOUT_NHWC 1
+#define B2C_OUT_I32 1
+#define B2C_OUT_I8 2
+
+/* ---- embeddings ------------------------------------------------------------------------------ */
+/* An embedding says which convolution axes feed the intrinsic's M / N / K dimensions and which
+ * layout rewrite makes that possible (Section 5.1 for the reference map n->x, oc->y, ic->z;
+ * Table 2 for the rewrites; Section 6 for the relaxed family). */
+#define B2C_AXIS_NPQ 1 /* fused batch and output pixels (Fuse rule)                              */
+#define B2C_AXIS_K 2   /* output channels                                                        */
+#define B2C_AXIS_C 3   /* input channels, padded to the intrinsic block (Pad + Split); r, s sequential */
+#define B2C_AXIS_CRS 4 /* fused (c, r, s) (Stencil Unroll + Fuse), padded to the K block         */
+
+#define B2C_VARIANT_CP_TMA 0         /* channel pack: NHWC C-padded activations, im2col-mode TMA */
+#define B2C_VARIANT_IM2COL_EXPLICIT 1 /* stencil unroll materialised as a matrix in scratch memory */
+#define B2C_VARIANT_IM2COL_GATHER 2  /* stencil unroll formed in shared memory inside the conv kernel */
+
+typedef struct {
+  int32_t id;       /* index in the enumeration for this descriptor; pass to b2c_plan_create      */
+  int32_t map_m, map_n, map_k; /* B2C_AXIS_*                                                      */
+  int32_t variant;  /* B2C_VARIANT_*                                                              */
+  int32_t tile_m, tile_n; /* accumulator tile of one thread block                                */
+  int32_t split_k;  /* number of thread blocks sharing one output tile's reduction                */
+  int64_t o_mac;    /* MACs issued to the intrinsic minus N*K*P*Q*C*R*S (Section 4.4)             */
+  int64_t o_data;   /* tensor elements moved minus (|x| + |w| + |y|) (Section 4.4)                */
+  int64_t workspace_bytes; /* scratch the caller passes to run                                    */
+  float device_us;  /* measured device time per run, or -1 if this candidate was not timed        */
+} b2c_embedding;
+
+#define B2C_POLICY_AUTO_TIMED (-1)   /* time the 5 lowest-overhead candidates, keep the fastest (Section 6.1) */
+#define B2C_POLICY_MIN_OVERHEAD (-2) /* lowest |[o_mac, o_data] . [1, 1]| without timing (Section 4.4)        */
+#define B2C_POLICY_MIN_WORKSPACE (-3) /* smallest scratch footprint (Table 4)                                 */
+
+typedef struct b2c_plan b2c_plan; /* opaque, library-owned */
+
+/* Output extent (host only).  *P or *Q is 0 when the dilated kernel does not fit; that is
+ * reported as B2C_E_UNSUPPORTED by the calls below.  INVALID_ARG on null or bad fields. */
+int b2c_out_shape(const b2c_conv_desc* desc, int32_t* P, int32_t* Q);
+
+/* Lists every legal embedding of `desc` (host only, no CUDA call), sorted by increasing
+ * o_mac + o_data.  Writes at most `cap` records to `out` (may be NULL when cap == 0) and the
+ * total number to *count.  UNSUPPORTED when C*R*S > 131071 (an int32 accumulator could
+ * overflow) or the output is empty. */
+int b2c_enumerate(const b2c_conv_desc* desc, b2c_embedding* out, int32_t cap, int32_t* count);
+
+/* Creates a plan for `desc` on the current device.  `policy_or_id` is a B2C_POLICY_* value or
+ * an embedding id from b2c_enumerate.  AUTO_TIMED allocates temporary device buffers, runs
+ * each candidate on `cuda_stream` and synchronises that stream.  The plan owns its packed
+ * weights, lookup tables and a device status word; free it with b2c_plan_destroy. */
+int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_stream, b2c_plan** out);
+
+/* Copies the chosen embedding (with device_us if it was timed) to *chosen. */
+int b2c_plan_info(const b2c_plan* plan, b2c_embedding* chosen);
+
+/* Bytes of scratch `run` needs (0 for embeddings that need none). */
+int b2c_plan_workspace_bytes(const b2c_plan* plan, size_t* bytes);
+
+/* Weight pack (Section 5.1: the B operand is held transposed, reduction index contiguous):
+ * reads w_kcrs_dev (int8 [K][C][R][S], device) and writes the plan's own packed copy,
+ * asynchronously on `cuda_stream`.  Call once per weight tensor, before run. */
+int b2c_plan_set_weights(b2c_plan* plan, const int8_t* w_kcrs_dev, void* cuda_stream);
+
+/* Enqueues the whole path on `cuda_stream` and returns without waiting: activation layout
+ * rewrite (if the embedding has one), the MMA kernel with fused shift/clip epilogue, stores in
+ * desc.out_layout.  x_dev: int8 input in desc.in_layout.  y_i32_dev / y_i8_dev: outputs
+ * selected by desc.out_mode (a selected output must be non-null; an unselected one is ignored).
+ * workspace_dev: at least b2c_plan_workspace_bytes bytes (may be NULL when that is 0); its
+ * contents are scratch.  The caller owns all four buffers and must keep them alive until the
+ * stream has run the work.  A plan must not be used from two threads at once. */
+int b2c_conv2d_int8_run(b2c_plan* plan, const int8_t* x_dev, int32_t* y_i32_dev, int8_t* y_i8_dev,
+                        void* workspace_dev, void* cuda_stream);
+
+/* One-shot form of the paper's problem statement: NCHW int8 input, KCRS int8 weights, NKPQ
+ * outputs (either may be NULL, not both), symmetric stride / pad / dilation.  All four tensor
+ * pointers are DEVICE pointers.  Picks the minimum-overhead embedding, keeps plans and scratch
+ * in a library-owned cache keyed by shape (so it may allocate on first use of a shape),
+ * re-packs the weights on every call, and enqueues on `cuda_stream`. */
+int b2c_conv2d_int8(int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int dilation,
+                    int shift, const int8_t* x_dev, const int8_t* w_dev, int32_t* y_i32_dev,
+                    int8_t* y_i8_dev, void* cuda_stream);
+
+/* Same operation with HOST tensors: copies x and w to the device, runs, copies the requested
+ * outputs back and synchronises.  Convenience for callers without device memory of their own. */
+int b2c_conv2d_int8_host(int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int dilation,
+                         int shift, const int8_t* x_host, const int8_t* w_host, int32_t* y_i32_host,
+                         int8_t* y_i8_host);
+
+/* Reads the plan's device status word (synchronises with the device).  *status is B2C_OK or
+ * B2C_E_TIMEOUT if a kernel of this plan gave up on a bounded wait; the word is then cleared. */
+int b2c_plan_device_status(b2c_plan* plan, int32_t* status);
+
+void b2c_plan_destroy(b2c_plan* plan);
+
+/* Layout rewrites on their own (the Pad / Reorder / Stencil Unroll rules of Table 2), exposed so
+ * they can be checked and timed separately.  b2c_pack_activations is asynchronous on
+ * `cuda_stream`; b2c_im2col builds a temporary lookup table and synchronises the stream.
+ * b2c_pack_activations: int8 NCHW [N][C][H][W] -> NHWC [N][H][W][C_pad], channels >= C zero;
+ *   C_pad must be a multiple of 16 and >= C.
+ * b2c_im2col: int8 input in desc.in_layout -> A[N*P*Q][K_pad], row m = (n, p, q), column
+ *   (c*R + r)*S + s, zeros for taps outside the image and for columns >= C*R*S; K_pad must be a
+ *   multiple of 16 and >= C*R*S. */
+int b2c_pack_activations(const int8_t* x_nchw_dev, int8_t* out_dev, int N, int C, int H, int W, int C_pad,
+                         void* cuda_stream);
+int b2c_im2col(const b2c_conv_desc* desc, const int8_t* x_dev, int8_t* a_dev, int K_pad, void* cuda_stream);
+
+const char* b2c_status_string(int status);
+
+/* The last CUDA error code (cudaError_t or CUresult as int) seen by this thread's failing call. */
+int b2c_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* B2CONV_H_ */

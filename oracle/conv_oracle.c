@@ -13,7 +13,7 @@
  *     the quantisation; tensors are NCHW.
  *   - Figure 5, step 1: the baseline conv2d is the seven-loop nest over n, oc, oh, ow, ic, kh, kw.
  *   - Table 2: the stencil access function is [n, i + k], i.e. cross-correlation (no kernel flip).
- *   - Section 4.4 (Padding): padded positions hold zeros.
+ *   - Section 4.2.4 (Padding): padded positions hold zeros.
  *   - Section 5 (Validation Experiments): all values are integers, so every association order
  *     of the sum gives the same result; there is exactly one correct output tensor.
  *

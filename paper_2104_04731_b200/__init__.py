@@ -1,0 +1,222 @@
+"""Python binding of libb2conv (argument marshalling only; every step runs in the CUDA library).
+
+The functions mirror the C ABI in ``include/b2conv.h`` one to one.  Tensors are ``torch`` CUDA
+tensors (used for device memory and streams only) or, for the ``*_host`` call, numpy arrays.
+There is no fallback: if the shared library is missing, ``load()`` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libb2conv.so")
+
+OK = 0
+E_INVALID_ARG, E_UNSUPPORTED, E_WORKSPACE_TOO_SMALL, E_CUDA, E_TIMEOUT, E_NOT_READY = -1, -2, -3, -4, -5, -6
+LAYOUT_NCHW, LAYOUT_NHWC = 0, 1
+OUT_I32, OUT_I8 = 1, 2
+AXIS_NPQ, AXIS_K, AXIS_C, AXIS_CRS = 1, 2, 3, 4
+VARIANT_CP_TMA, VARIANT_IM2COL_EXPLICIT, VARIANT_IM2COL_GATHER = 0, 1, 2
+POLICY_AUTO_TIMED, POLICY_MIN_OVERHEAD, POLICY_MIN_WORKSPACE = -1, -2, -3
+VARIANT_NAMES = {0: "channel_pack_tma_im2col", 1: "im2col_explicit", 2: "im2col_gather"}
+
+EXPORTS = [
+    "b2c_out_shape", "b2c_enumerate", "b2c_plan_create", "b2c_plan_info", "b2c_plan_workspace_bytes",
+    "b2c_plan_set_weights", "b2c_conv2d_int8_run", "b2c_conv2d_int8", "b2c_conv2d_int8_host",
+    "b2c_plan_device_status", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_status_string",
+    "b2c_last_cuda_error",
+]
+
+
+class ConvDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "N", "C", "H", "W", "K", "R", "S", "stride_h", "stride_w", "pad_h", "pad_w", "dil_h", "dil_w",
+        "shift", "in_layout", "out_layout", "out_mode")]
+
+
+class Embedding(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("id", "map_m", "map_n", "map_k", "variant", "tile_m", "tile_n", "split_k")] + [
+        ("o_mac", ctypes.c_int64), ("o_data", ctypes.c_int64), ("workspace_bytes", ctypes.c_int64),
+        ("device_us", ctypes.c_float)]
+
+    def as_dict(self):
+        d = {n: getattr(self, n) for n, _ in self._fields_}
+        d["variant_name"] = VARIANT_NAMES.get(self.variant, "?")
+        return d
+
+
+class B2CError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = _lib.b2c_status_string(code).decode() if _lib is not None else str(code)
+        extra = ""
+        if code == E_CUDA and _lib is not None:
+            extra = " (cuda error %d)" % _lib.b2c_last_cuda_error()
+        super().__init__("%s: %s%s" % (where, msg, extra))
+
+
+_lib = None
+
+
+def load():
+    """Loads libb2conv.so; raises if it has not been built (no fallback path exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            "libb2conv.so is missing: build it with `python -m paper_2104_04731_b200.build` "
+            "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    i32, vp = ctypes.c_int, ctypes.c_void_p
+    pd, pe = ctypes.POINTER(ConvDesc), ctypes.POINTER(Embedding)
+    pi32 = ctypes.POINTER(ctypes.c_int32)
+    lib.b2c_out_shape.argtypes = [pd, pi32, pi32]
+    lib.b2c_enumerate.argtypes = [pd, pe, ctypes.c_int32, pi32]
+    lib.b2c_plan_create.argtypes = [pd, ctypes.c_int32, vp, ctypes.POINTER(vp)]
+    lib.b2c_plan_info.argtypes = [vp, pe]
+    lib.b2c_plan_workspace_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
+    lib.b2c_plan_set_weights.argtypes = [vp, vp, vp]
+    lib.b2c_conv2d_int8_run.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.b2c_conv2d_int8.argtypes = [i32] * 11 + [vp] * 5
+    lib.b2c_conv2d_int8_host.argtypes = [i32] * 11 + [vp] * 4
+    lib.b2c_plan_device_status.argtypes = [vp, pi32]
+    lib.b2c_plan_destroy.argtypes = [vp]
+    lib.b2c_plan_destroy.restype = None
+    lib.b2c_pack_activations.argtypes = [vp, vp] + [i32] * 5 + [vp]
+    lib.b2c_im2col.argtypes = [pd, vp, vp, i32, vp]
+    lib.b2c_status_string.argtypes = [i32]
+    lib.b2c_status_string.restype = ctypes.c_char_p
+    lib.b2c_last_cuda_error.argtypes = []
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if name not in ("b2c_plan_destroy", "b2c_status_string"):
+            fn.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise B2CError(code, where)
+
+
+def _pair(v) -> Tuple[int, int]:
+    if isinstance(v, (tuple, list)):
+        return int(v[0]), int(v[1])
+    return int(v), int(v)
+
+
+def make_desc(N, C, H, W, K, R, S, stride=1, pad=0, dilation=1, shift=0, in_layout=LAYOUT_NCHW,
+              out_layout=LAYOUT_NCHW, out_mode=OUT_I32) -> ConvDesc:
+    sh, sw = _pair(stride)
+    ph, pw = _pair(pad)
+    dh, dw = _pair(dilation)
+    return ConvDesc(N, C, H, W, K, R, S, sh, sw, ph, pw, dh, dw, shift, in_layout, out_layout, out_mode)
+
+
+def status_string(code: int) -> str:
+    return load().b2c_status_string(code).decode()
+
+
+def out_shape(desc: ConvDesc) -> Tuple[int, int]:
+    P, Q = ctypes.c_int32(), ctypes.c_int32()
+    _check(load().b2c_out_shape(ctypes.byref(desc), ctypes.byref(P), ctypes.byref(Q)), "b2c_out_shape")
+    return P.value, Q.value
+
+
+def enumerate_embeddings(desc: ConvDesc) -> List[Embedding]:
+    lib = load()
+    n = ctypes.c_int32()
+    _check(lib.b2c_enumerate(ctypes.byref(desc), None, 0, ctypes.byref(n)), "b2c_enumerate")
+    arr = (Embedding * n.value)()
+    _check(lib.b2c_enumerate(ctypes.byref(desc), arr, n.value, ctypes.byref(n)), "b2c_enumerate")
+    return list(arr)
+
+
+def _stream_ptr(stream=None):
+    import torch
+
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+class Plan:
+    """Owns a ``b2c_plan``.  ``run`` enqueues the whole path on the current torch stream."""
+
+    def __init__(self, desc: ConvDesc, policy_or_id: int = POLICY_MIN_OVERHEAD, stream=None):
+        self._lib = load()
+        self.desc = desc
+        h = ctypes.c_void_p()
+        _check(self._lib.b2c_plan_create(ctypes.byref(desc), policy_or_id, _stream_ptr(stream), ctypes.byref(h)),
+               "b2c_plan_create")
+        self._h = h
+
+    def info(self) -> Embedding:
+        e = Embedding()
+        _check(self._lib.b2c_plan_info(self._h, ctypes.byref(e)), "b2c_plan_info")
+        return e
+
+    def workspace_bytes(self) -> int:
+        n = ctypes.c_size_t()
+        _check(self._lib.b2c_plan_workspace_bytes(self._h, ctypes.byref(n)), "b2c_plan_workspace_bytes")
+        return n.value
+
+    def set_weights(self, w, stream=None):
+        _check(self._lib.b2c_plan_set_weights(self._h, _dptr(w), _stream_ptr(stream)), "b2c_plan_set_weights")
+
+    def run(self, x, y32=None, y8=None, workspace=None, stream=None):
+        _check(self._lib.b2c_conv2d_int8_run(self._h, _dptr(x), _dptr(y32), _dptr(y8), _dptr(workspace),
+                                              _stream_ptr(stream)), "b2c_conv2d_int8_run")
+
+    def device_status(self) -> int:
+        s = ctypes.c_int32()
+        _check(self._lib.b2c_plan_device_status(self._h, ctypes.byref(s)), "b2c_plan_device_status")
+        return s.value
+
+    def destroy(self):
+        if getattr(self, "_h", None):
+            self._lib.b2c_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def conv2d_int8(x, w, stride=1, pad=0, dilation=1, shift=0, y32=None, y8=None, stream=None):
+    """One-shot call on CUDA tensors: x int8 [N,C,H,W], w int8 [K,C,R,S]; writes y32 / y8 ([N,K,P,Q])."""
+    N, C, H, W = x.shape
+    K, _, R, S = w.shape
+    _check(load().b2c_conv2d_int8(N, C, H, W, K, R, S, stride, pad, dilation, shift, _dptr(x), _dptr(w), _dptr(y32),
+                                  _dptr(y8), _stream_ptr(stream)), "b2c_conv2d_int8")
+
+
+def conv2d_int8_host(x, w, stride=1, pad=0, dilation=1, shift=0, y32=None, y8=None):
+    """One-shot call on numpy host arrays (copies in, runs, copies out, synchronises)."""
+    N, C, H, W = x.shape
+    K, _, R, S = w.shape
+
+    def hp(a):
+        return a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
+
+    _check(load().b2c_conv2d_int8_host(N, C, H, W, K, R, S, stride, pad, dilation, shift, hp(x), hp(w), hp(y32),
+                                       hp(y8)), "b2c_conv2d_int8_host")
+
+
+def pack_activations(x, out, C_pad: int, stream=None):
+    N, C, H, W = x.shape
+    _check(load().b2c_pack_activations(_dptr(x), _dptr(out), N, C, H, W, C_pad, _stream_ptr(stream)),
+           "b2c_pack_activations")
+
+
+def im2col(desc: ConvDesc, x, a, K_pad: int, stream=None):
+    _check(load().b2c_im2col(ctypes.byref(desc), _dptr(x), _dptr(a), K_pad, _stream_ptr(stream)), "b2c_im2col")

@@ -1,0 +1,571 @@
+// C ABI of libb2conv: descriptor validation, plan objects, the run path (layout rewrite ->
+// MMA kernel with fused epilogue -> optional split-reduction finish), the one-shot calls and
+// the timed candidate selection.  See include/b2conv.h for the contract of each entry point.
+#include <algorithm>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "b2c_internal.h"
+
+using namespace b2c;
+
+struct b2c_plan {
+  Geom g;
+  b2c_embedding emb;
+  int device = 0;
+  int8_t* w_packed = nullptr;   // device, plan-owned
+  size_t w_packed_bytes = 0;
+  GatherEntry* table = nullptr;  // device, plan-owned (stencil lookup table)
+  int table_len = 0;
+  int* status = nullptr;         // device status word
+  bool weights_set = false;
+  // derived launch parameters
+  int amode = 0;
+  int C_pad = 0, K_pad = 0, bk = 128;
+  size_t ws_layout_bytes = 0;    // bytes of the layout rewrite's output at the start of the workspace
+  size_t ws_total = 0;
+  ConvArgs args;
+  CUtensorMap tmap_b;
+  // one-shot cache extras
+  void* own_ws = nullptr;
+};
+
+namespace {
+
+#define CUDA_TRY(expr)                  \
+  do {                                  \
+    cudaError_t e__ = (expr);           \
+    if (e__ != cudaSuccess) {           \
+      set_last_cuda_error((int)e__);    \
+      return B2C_E_CUDA;                \
+    }                                   \
+  } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int tmem_cols_for(int n) {
+  int c = 32;
+  while (c < n) c <<= 1;
+  return c;
+}
+
+// Stencil lookup table: reduction index (c, r, s) -> input offset and displacement, in the
+// element strides of the activation layout.
+void build_table(const Geom& g, int K_pad, std::vector<GatherEntry>* t) {
+  const b2c_conv_desc& d = g.d;
+  long long sc, sh, sw;
+  if (d.in_layout == B2C_LAYOUT_NCHW) {
+    sc = (long long)d.H * d.W;
+    sh = d.W;
+    sw = 1;
+  } else {
+    sc = 1;
+    sh = (long long)d.W * d.C;
+    sw = d.C;
+  }
+  t->assign(K_pad, GatherEntry{-1, 0, 0});
+  int kg = 0;
+  for (int c = 0; c < d.C; ++c)
+    for (int r = 0; r < d.R; ++r)
+      for (int s = 0; s < d.S; ++s, ++kg) {
+        GatherEntry e;
+        e.off = (int32_t)(c * sc + (long long)r * d.dil_h * sh + (long long)s * d.dil_w * sw);
+        e.dh = (int16_t)(r * d.dil_h);
+        e.dw = (int16_t)(s * d.dil_w);
+        (*t)[kg] = e;
+      }
+}
+
+bool table_variant_legal(const Geom& g) {
+  const b2c_conv_desc& d = g.d;
+  return (long long)(d.R - 1) * d.dil_h < 32768 && (long long)(d.S - 1) * d.dil_w < 32768 &&
+         (long long)d.C * d.H * d.W < 0x7FFFFFFFLL;
+}
+
+void fill_common_args(b2c_plan* p) {
+  const b2c_conv_desc& d = p->g.d;
+  ConvArgs& a = p->args;
+  std::memset(&a, 0, sizeof(a));
+  a.status = p->status;
+  a.table = p->table;
+  if (d.in_layout == B2C_LAYOUT_NCHW) {
+    a.x_stride_n = (long long)d.C * d.H * d.W;
+    a.x_stride_h = d.W;
+    a.x_stride_w = 1;
+  } else {
+    a.x_stride_n = (long long)d.C * d.H * d.W;
+    a.x_stride_h = d.W * d.C;
+    a.x_stride_w = d.C;
+  }
+  a.Mg = (int)p->g.Mg;
+  a.K = d.K;
+  a.PQ = p->g.PQ;
+  a.Q = p->g.Q;
+  a.H = d.H;
+  a.W = d.W;
+  a.stride_h = d.stride_h;
+  a.stride_w = d.stride_w;
+  a.pad_h = d.pad_h;
+  a.pad_w = d.pad_w;
+  a.dil_h = d.dil_h;
+  a.dil_w = d.dil_w;
+  a.S = d.S;
+  a.tile_n = p->emb.tile_n;
+  a.tmem_cols = tmem_cols_for(p->emb.tile_n);
+  a.split_k = p->emb.split_k;
+  a.shift = d.shift;
+  a.out_mode = d.out_mode;
+  a.out_layout = d.out_layout;
+  a.table_len = p->table_len;
+  if (p->emb.variant == B2C_VARIANT_CP_TMA) {
+    p->amode = A_IM2COL_TMA;
+    p->C_pad = cp_channel_pad(d.C);
+    p->bk = cp_block_bytes(p->C_pad);
+    a.bk = p->bk;
+    a.kb_per_tap = p->C_pad / p->bk;
+    a.tap_cols = p->C_pad;
+    a.num_kb = d.R * d.S * a.kb_per_tap;
+    a.ksteps_full = p->bk / kMmaK;
+    a.ksteps_last = a.ksteps_full;
+  } else {
+    p->amode = p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT ? A_TILED : A_GATHER;
+    p->K_pad = im2col_k_pad(p->g.Kg);
+    p->bk = 128;
+    a.bk = 128;
+    a.num_kb = (p->K_pad + 127) / 128;
+    a.ksteps_full = 4;
+    a.ksteps_last = (p->K_pad - (a.num_kb - 1) * 128) / kMmaK;
+    a.kb_per_tap = 1;
+  }
+  // Pipeline depth: as many stages as the reduction slice has blocks, at most 6, within 160 KB.
+  int per_cta_kb = (a.num_kb + a.split_k - 1) / a.split_k;
+  int stages = std::min(6, std::max(1, per_cta_kb));
+  while (stages > 1 && (size_t)stages * (kTileM + a.tile_n) * a.bk > 160 * 1024) --stages;
+  a.stages = stages;
+}
+
+int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
+  b2c_plan* p = new (std::nothrow) b2c_plan();
+  if (!p) return B2C_E_INVALID_ARG;
+  p->g = g;
+  p->emb = emb;
+  cudaGetDevice(&p->device);
+  const b2c_conv_desc& d = g.d;
+  auto fail = [&](int code) {
+    b2c_plan_destroy(p);
+    return code;
+  };
+  if (cudaMalloc(&p->status, sizeof(int)) != cudaSuccess) return fail(B2C_E_CUDA);
+  if (cudaMemset(p->status, 0, sizeof(int)) != cudaSuccess) return fail(B2C_E_CUDA);
+  if (emb.variant == B2C_VARIANT_CP_TMA) {
+    int C_pad = cp_channel_pad(d.C);
+    p->w_packed_bytes = (size_t)d.K * d.R * d.S * C_pad;
+  } else {
+    int K_pad = im2col_k_pad(g.Kg);
+    p->w_packed_bytes = (size_t)d.K * K_pad;
+    std::vector<GatherEntry> t;
+    build_table(g, K_pad, &t);
+    p->table_len = K_pad;
+    if (cudaMalloc(&p->table, t.size() * sizeof(GatherEntry)) != cudaSuccess) return fail(B2C_E_CUDA);
+    if (cudaMemcpy(p->table, t.data(), t.size() * sizeof(GatherEntry), cudaMemcpyHostToDevice) != cudaSuccess)
+      return fail(B2C_E_CUDA);
+  }
+  // Room for one extra box row block so that a TMA box never starts past the allocation.
+  if (cudaMalloc(&p->w_packed, p->w_packed_bytes + 256) != cudaSuccess) return fail(B2C_E_CUDA);
+  fill_common_args(p);
+  p->ws_total = workspace_bytes_for(g, emb.variant, emb.split_k);
+  if (emb.variant == B2C_VARIANT_CP_TMA) {
+    bool direct = d.in_layout == B2C_LAYOUT_NHWC && p->C_pad == d.C;
+    p->ws_layout_bytes = direct ? 0 : ((size_t)d.N * d.H * d.W * p->C_pad + 255) / 256 * 256;
+  } else if (emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
+    p->ws_layout_bytes = ((size_t)g.Mg * p->K_pad + 255) / 256 * 256;
+  }
+  // Tensor map of the packed weights (plan-owned memory, so it is encoded once).
+  int rc;
+  if (emb.variant == B2C_VARIANT_CP_TMA) {
+    uint64_t cols = (uint64_t)d.R * d.S * p->C_pad;
+    rc = encode_tiled_2d(&p->tmap_b, p->w_packed, cols, d.K, cols, p->bk, emb.tile_n, p->bk);
+  } else {
+    rc = encode_tiled_2d(&p->tmap_b, p->w_packed, p->K_pad, d.K, p->K_pad, 128, emb.tile_n, 128);
+  }
+  if (rc != B2C_OK) return fail(rc);
+  *out = p;
+  return B2C_OK;
+}
+
+int time_plan(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, cudaStream_t st, float* us) {
+  cudaEvent_t e0, e1;
+  CUDA_TRY(cudaEventCreate(&e0));
+  CUDA_TRY(cudaEventCreate(&e1));
+  const int warm = 3, iters = 20;
+  int rc = B2C_OK;
+  for (int i = 0; i < warm && rc == B2C_OK; ++i) rc = b2c_conv2d_int8_run(p, x, y32, y8, ws, st);
+  if (rc == B2C_OK) {
+    cudaEventRecord(e0, st);
+    for (int i = 0; i < iters && rc == B2C_OK; ++i) rc = b2c_conv2d_int8_run(p, x, y32, y8, ws, st);
+    cudaEventRecord(e1, st);
+    cudaError_t e = cudaEventSynchronize(e1);
+    if (e != cudaSuccess) {
+      set_last_cuda_error((int)e);
+      rc = B2C_E_CUDA;
+    } else {
+      float ms = 0;
+      cudaEventElapsedTime(&ms, e0, e1);
+      *us = ms * 1000.0f / iters;
+    }
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (rc == B2C_OK) {
+    int32_t s = 0;
+    rc = b2c_plan_device_status(p, &s);
+    if (rc == B2C_OK && s != B2C_OK) rc = s;
+  }
+  return rc;
+}
+
+struct ShapeKey {
+  int v[12];
+  bool operator<(const ShapeKey& o) const { return std::memcmp(v, o.v, sizeof(v)) < 0; }
+};
+std::mutex g_cache_mu;
+std::map<ShapeKey, b2c_plan*> g_cache;
+
+}  // namespace
+
+extern "C" {
+
+const char* b2c_status_string(int s) {
+  switch (s) {
+    case B2C_OK: return "ok";
+    case B2C_E_INVALID_ARG: return "invalid argument";
+    case B2C_E_UNSUPPORTED: return "unsupported problem";
+    case B2C_E_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case B2C_E_CUDA: return "CUDA call failed";
+    case B2C_E_TIMEOUT: return "bounded device wait expired";
+    case B2C_E_NOT_READY: return "plan has no weights";
+    default: return "unknown status";
+  }
+}
+
+int b2c_out_shape(const b2c_conv_desc* desc, int32_t* P, int32_t* Q) {
+  if (!desc || !P || !Q) return B2C_E_INVALID_ARG;
+  Geom g;
+  int rc = resolve_geom(desc, &g);
+  if (rc == B2C_E_INVALID_ARG) return rc;
+  *P = g.P;
+  *Q = g.Q;
+  return B2C_OK;
+}
+
+int b2c_enumerate(const b2c_conv_desc* desc, b2c_embedding* out, int32_t cap, int32_t* count) {
+  if (!desc || !count || cap < 0 || (cap > 0 && !out)) return B2C_E_INVALID_ARG;
+  Geom g;
+  int rc = resolve_geom(desc, &g);
+  if (rc != B2C_OK) return rc;
+  std::vector<b2c_embedding> all;
+  enumerate_embeddings(g, &all);
+  if (!table_variant_legal(g))
+    all.erase(std::remove_if(all.begin(), all.end(), [](const b2c_embedding& e) { return e.variant != B2C_VARIANT_CP_TMA; }),
+              all.end());
+  for (size_t i = 0; i < all.size(); ++i) all[i].id = (int)i;
+  *count = (int32_t)all.size();
+  for (int i = 0; i < cap && i < (int)all.size(); ++i) out[i] = all[i];
+  return all.empty() ? B2C_E_UNSUPPORTED : B2C_OK;
+}
+
+int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_stream, b2c_plan** out) {
+  if (!desc || !out) return B2C_E_INVALID_ARG;
+  *out = nullptr;
+  Geom g;
+  int rc = resolve_geom(desc, &g);
+  if (rc != B2C_OK) return rc;
+  int32_t count = 0;
+  rc = b2c_enumerate(desc, nullptr, 0, &count);
+  if (rc != B2C_OK) return rc;
+  std::vector<b2c_embedding> all(count);
+  rc = b2c_enumerate(desc, all.data(), count, &count);
+  if (rc != B2C_OK) return rc;
+  if (policy_or_id < B2C_POLICY_MIN_WORKSPACE) return B2C_E_INVALID_ARG;
+  if (policy_or_id != B2C_POLICY_AUTO_TIMED) {
+    int idx = pick_by_policy(all, policy_or_id);
+    if (idx < 0) return B2C_E_INVALID_ARG;
+    return create_plan_for(g, all[idx], out);
+  }
+  // Timed selection (Section 6.1: the best candidates by the overhead metric are tuned and the
+  // fastest is kept).  All schedules of the five lowest-overhead (axis map, layout variant)
+  // groups are run on scratch tensors.
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  std::vector<int> groups;
+  for (const b2c_embedding& e : all)
+    if (std::find(groups.begin(), groups.end(), e.variant) == groups.end() && groups.size() < 5)
+      groups.push_back(e.variant);
+  size_t ws_max = 0;
+  for (const b2c_embedding& e : all) ws_max = std::max(ws_max, (size_t)e.workspace_bytes);
+  int8_t *x = nullptr, *w = nullptr, *y8 = nullptr;
+  int32_t* y32 = nullptr;
+  void* ws = nullptr;
+  auto cleanup = [&]() {
+    cudaFree(x);
+    cudaFree(w);
+    cudaFree(y8);
+    cudaFree(y32);
+    cudaFree(ws);
+  };
+  if (cudaMalloc(&x, g.x_elems + 256) != cudaSuccess || cudaMalloc(&w, g.w_elems + 256) != cudaSuccess ||
+      cudaMalloc(&y8, g.y_elems + 256) != cudaSuccess || cudaMalloc(&y32, g.y_elems * 4 + 256) != cudaSuccess ||
+      cudaMalloc(&ws, ws_max + 256) != cudaSuccess) {
+    set_last_cuda_error((int)cudaGetLastError());
+    cleanup();
+    return B2C_E_CUDA;
+  }
+  cudaMemsetAsync(x, 1, g.x_elems, st);
+  cudaMemsetAsync(w, 1, g.w_elems, st);
+  int best = -1;
+  float best_us = 0;
+  for (size_t i = 0; i < all.size(); ++i) {
+    if (std::find(groups.begin(), groups.end(), all[i].variant) == groups.end()) continue;
+    b2c_plan* p = nullptr;
+    rc = create_plan_for(g, all[i], &p);
+    if (rc != B2C_OK) break;
+    rc = b2c_plan_set_weights(p, w, st);
+    float us = -1;
+    if (rc == B2C_OK) rc = time_plan(p, x, y32, y8, ws, st, &us);
+    b2c_plan_destroy(p);
+    if (rc != B2C_OK) break;
+    all[i].device_us = us;
+    if (best < 0 || us < best_us) {
+      best = (int)i;
+      best_us = us;
+    }
+  }
+  cleanup();
+  if (rc != B2C_OK) return rc;
+  if (best < 0) return B2C_E_UNSUPPORTED;
+  return create_plan_for(g, all[best], out);
+}
+
+int b2c_plan_info(const b2c_plan* plan, b2c_embedding* chosen) {
+  if (!plan || !chosen) return B2C_E_INVALID_ARG;
+  *chosen = plan->emb;
+  return B2C_OK;
+}
+
+int b2c_plan_workspace_bytes(const b2c_plan* plan, size_t* bytes) {
+  if (!plan || !bytes) return B2C_E_INVALID_ARG;
+  *bytes = plan->ws_total;
+  return B2C_OK;
+}
+
+int b2c_plan_set_weights(b2c_plan* p, const int8_t* w, void* cuda_stream) {
+  if (!p || !w) return B2C_E_INVALID_ARG;
+  if (!aligned16(w)) return B2C_E_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const b2c_conv_desc& d = p->g.d;
+  if (p->emb.variant == B2C_VARIANT_CP_TMA)
+    CUDA_TRY(launch_pack_weights_cp(w, p->w_packed, d.K, d.C, d.R, d.S, p->C_pad, st));
+  else
+    CUDA_TRY(launch_pack_weights_rows(w, p->w_packed, d.K, p->g.Kg, p->K_pad, st));
+  p->weights_set = true;
+  return B2C_OK;
+}
+
+int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, void* cuda_stream) {
+  if (!p || !x) return B2C_E_INVALID_ARG;
+  if (!p->weights_set) return B2C_E_NOT_READY;
+  const b2c_conv_desc& d = p->g.d;
+  if ((d.out_mode & B2C_OUT_I32) && !y32) return B2C_E_INVALID_ARG;
+  if ((d.out_mode & B2C_OUT_I8) && !y8) return B2C_E_INVALID_ARG;
+  if (p->ws_total > 0 && !ws) return B2C_E_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(y32) || !aligned16(y8) || !aligned16(ws)) return B2C_E_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const Geom& g = p->g;
+  ConvArgs a = p->args;
+  a.x = x;
+  a.y32 = y32;
+  a.y8 = y8;
+  CUtensorMap tmap_a;
+  std::memset(&tmap_a, 0, sizeof(tmap_a));
+  uint8_t* wsb = static_cast<uint8_t*>(ws);
+  int rc = B2C_OK;
+
+  // ---- layout rewrite of the activations ----
+  if (p->emb.variant == B2C_VARIANT_CP_TMA) {
+    const int8_t* act = x;
+    if (p->ws_layout_bytes) {
+      CUDA_TRY(launch_pack_activations(x, reinterpret_cast<int8_t*>(wsb), d.N, d.C, d.H, d.W, p->C_pad, st));
+      act = reinterpret_cast<int8_t*>(wsb);
+    }
+    rc = encode_im2col_nhwc(&tmap_a, act, p->C_pad, d.W, d.H, d.N, d.pad_w, d.pad_h, d.S, d.R, d.dil_w, d.dil_h,
+                            d.stride_w, d.stride_h, p->bk, kTileM, p->bk);
+    if (rc != B2C_OK) return rc;
+  } else if (p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
+    int8_t* A = reinterpret_cast<int8_t*>(wsb);
+    CUDA_TRY(launch_im2col(x, A, p->table, g.Mg, g.PQ, g.Q, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
+                           a.x_stride_n, a.x_stride_h, a.x_stride_w, p->K_pad, st));
+    rc = encode_tiled_2d(&tmap_a, A, p->K_pad, (uint64_t)g.Mg, p->K_pad, 128, kTileM, 128);
+    if (rc != B2C_OK) return rc;
+  } else {
+    tmap_a = p->tmap_b;  // unused by the gather kernel; any valid map
+  }
+
+  // ---- split reduction: partial sums meet in a zeroed int32 buffer ----
+  bool need_finish = false;
+  if (a.split_k > 1) {
+    if (d.out_mode == B2C_OUT_I32) {
+      a.acc = y32;
+    } else {
+      a.acc = reinterpret_cast<int32_t*>(wsb + p->ws_layout_bytes);
+      need_finish = true;
+    }
+    CUDA_TRY(cudaMemsetAsync(a.acc, 0, (size_t)g.y_elems * 4, st));
+  }
+
+  CUDA_TRY(launch_conv_mma(p->amode, &tmap_a, &p->tmap_b, a, st));
+  if (need_finish) CUDA_TRY(launch_splitk_finish(a.acc, y32, y8, g.y_elems, d.shift, d.out_mode, st));
+  return B2C_OK;
+}
+
+int b2c_plan_device_status(b2c_plan* p, int32_t* status) {
+  if (!p || !status) return B2C_E_INVALID_ARG;
+  int s = 0;
+  CUDA_TRY(cudaMemcpy(&s, p->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (s != 0) CUDA_TRY(cudaMemset(p->status, 0, sizeof(int)));
+  *status = s;
+  return B2C_OK;
+}
+
+void b2c_plan_destroy(b2c_plan* p) {
+  if (!p) return;
+  cudaFree(p->w_packed);
+  cudaFree(p->table);
+  cudaFree(p->status);
+  cudaFree(p->own_ws);
+  delete p;
+}
+
+int b2c_conv2d_int8(int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int dilation, int shift,
+                    const int8_t* x, const int8_t* w, int32_t* y32, int8_t* y8, void* cuda_stream) {
+  if (!x || !w || (!y32 && !y8)) return B2C_E_INVALID_ARG;
+  b2c_conv_desc d;
+  std::memset(&d, 0, sizeof(d));
+  d.N = N; d.C = C; d.H = H; d.W = W; d.K = K; d.R = R; d.S = S;
+  d.stride_h = d.stride_w = stride;
+  d.pad_h = d.pad_w = pad;
+  d.dil_h = d.dil_w = dilation;
+  d.shift = shift;
+  d.in_layout = B2C_LAYOUT_NCHW;
+  d.out_layout = B2C_LAYOUT_NCHW;
+  d.out_mode = (y32 ? B2C_OUT_I32 : 0) | (y8 ? B2C_OUT_I8 : 0);
+  int dev = 0;
+  cudaGetDevice(&dev);
+  ShapeKey key = {{N, C, H, W, K, R, S, stride, pad, dilation, shift, d.out_mode * 64 + dev}};
+  std::lock_guard<std::mutex> lock(g_cache_mu);
+  b2c_plan* p = nullptr;
+  auto it = g_cache.find(key);
+  if (it == g_cache.end()) {
+    int rc = b2c_plan_create(&d, B2C_POLICY_MIN_OVERHEAD, cuda_stream, &p);
+    if (rc != B2C_OK) return rc;
+    if (p->ws_total) {
+      if (cudaMalloc(&p->own_ws, p->ws_total) != cudaSuccess) {
+        set_last_cuda_error((int)cudaGetLastError());
+        b2c_plan_destroy(p);
+        return B2C_E_CUDA;
+      }
+    }
+    g_cache[key] = p;
+  } else {
+    p = it->second;
+  }
+  int rc = b2c_plan_set_weights(p, w, cuda_stream);
+  if (rc != B2C_OK) return rc;
+  return b2c_conv2d_int8_run(p, x, y32, y8, p->own_ws, cuda_stream);
+}
+
+int b2c_conv2d_int8_host(int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int dilation, int shift,
+                         const int8_t* xh, const int8_t* wh, int32_t* y32h, int8_t* y8h) {
+  if (!xh || !wh || (!y32h && !y8h)) return B2C_E_INVALID_ARG;
+  b2c_conv_desc d;
+  std::memset(&d, 0, sizeof(d));
+  d.N = N; d.C = C; d.H = H; d.W = W; d.K = K; d.R = R; d.S = S;
+  d.stride_h = d.stride_w = stride;
+  d.pad_h = d.pad_w = pad;
+  d.dil_h = d.dil_w = dilation;
+  d.shift = shift;
+  d.out_mode = (y32h ? B2C_OUT_I32 : 0) | (y8h ? B2C_OUT_I8 : 0);
+  Geom g;
+  int rc = resolve_geom(&d, &g);
+  if (rc != B2C_OK) return rc;
+  // Device staging buffers, grown on demand and kept for the next call (per process).
+  static std::mutex mu;
+  static int8_t *dx = nullptr, *dw = nullptr, *dy8 = nullptr;
+  static int32_t* dy32 = nullptr;
+  static size_t cx = 0, cw = 0, cy8 = 0, cy32 = 0;
+  std::lock_guard<std::mutex> lock(mu);
+  auto grow = [](void** p, size_t* cap, size_t need) -> bool {
+    if (need <= *cap) return true;
+    cudaFree(*p);
+    *p = nullptr;
+    *cap = 0;
+    if (cudaMalloc(p, need + 256) != cudaSuccess) return false;
+    *cap = need;
+    return true;
+  };
+  bool ok = grow((void**)&dx, &cx, (size_t)g.x_elems) && grow((void**)&dw, &cw, (size_t)g.w_elems);
+  if (ok && y8h) ok = grow((void**)&dy8, &cy8, (size_t)g.y_elems);
+  if (ok && y32h) ok = grow((void**)&dy32, &cy32, (size_t)g.y_elems * 4);
+  if (!ok) {
+    set_last_cuda_error((int)cudaGetLastError());
+    return B2C_E_CUDA;
+  }
+  cudaStream_t st = 0;
+  CUDA_TRY(cudaMemcpyAsync(dx, xh, g.x_elems, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(dw, wh, g.w_elems, cudaMemcpyHostToDevice, st));
+  rc = b2c_conv2d_int8(N, C, H, W, K, R, S, stride, pad, dilation, shift, dx, dw, y32h ? dy32 : nullptr,
+                       y8h ? dy8 : nullptr, st);
+  if (rc != B2C_OK) return rc;
+  if (y32h) CUDA_TRY(cudaMemcpyAsync(y32h, dy32, g.y_elems * 4, cudaMemcpyDeviceToHost, st));
+  if (y8h) CUDA_TRY(cudaMemcpyAsync(y8h, dy8, g.y_elems, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  return B2C_OK;
+}
+
+int b2c_pack_activations(const int8_t* x, int8_t* out, int N, int C, int H, int W, int C_pad, void* cuda_stream) {
+  if (!x || !out || N < 1 || C < 1 || H < 1 || W < 1 || C_pad < C || (C_pad % 16) != 0) return B2C_E_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(out)) return B2C_E_INVALID_ARG;
+  CUDA_TRY(launch_pack_activations(x, out, N, C, H, W, C_pad, (cudaStream_t)cuda_stream));
+  return B2C_OK;
+}
+
+int b2c_im2col(const b2c_conv_desc* desc, const int8_t* x, int8_t* a, int K_pad, void* cuda_stream) {
+  if (!desc || !x || !a || !aligned16(x) || !aligned16(a)) return B2C_E_INVALID_ARG;
+  b2c_conv_desc d = *desc;
+  if ((d.out_mode & 3) == 0) d.out_mode = B2C_OUT_I32;
+  Geom g;
+  int rc = resolve_geom(&d, &g);
+  if (rc != B2C_OK) return rc;
+  if (K_pad < g.Kg || (K_pad % 16) != 0) return B2C_E_INVALID_ARG;
+  if (!table_variant_legal(g)) return B2C_E_UNSUPPORTED;
+  std::vector<GatherEntry> t;
+  build_table(g, K_pad, &t);
+  GatherEntry* dt = nullptr;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CUDA_TRY(cudaMalloc(&dt, t.size() * sizeof(GatherEntry)));
+  cudaError_t e = cudaMemcpyAsync(dt, t.data(), t.size() * sizeof(GatherEntry), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);  // the host table goes out of scope below
+  long long sn = (long long)d.C * d.H * d.W;
+  int sh = d.in_layout == B2C_LAYOUT_NCHW ? d.W : d.W * d.C;
+  int sw = d.in_layout == B2C_LAYOUT_NCHW ? 1 : d.C;
+  if (e == cudaSuccess)
+    e = launch_im2col(x, a, dt, g.Mg, g.PQ, g.Q, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w, sn, sh, sw, K_pad,
+                      st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  cudaFree(dt);
+  CUDA_TRY(e);
+  return B2C_OK;
+}
+
+}  // extern "C"

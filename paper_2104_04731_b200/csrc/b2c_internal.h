@@ -1,0 +1,110 @@
+// Internal declarations shared by the host code and the kernel launchers of libb2conv.
+// Nothing here is part of the public ABI (see include/b2conv.h).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "b2conv.h"
+
+namespace b2c {
+
+constexpr int kTileM = 128;       // rows of one tcgen05.mma accumulator tile (cta_group::1)
+constexpr int kMmaK = 32;         // reduction depth of one kind::i8 instruction (bytes per row)
+constexpr int kMaxKg = 131071;    // C*R*S bound that keeps |acc| <= Kg * 2^14 inside int32
+constexpr int kNumSMs = 148;
+
+// Resolved geometry of one convolution.
+struct Geom {
+  b2c_conv_desc d;
+  int P, Q;
+  int PQ;
+  long long Mg;  // N*P*Q
+  int Kg;        // C*R*S
+  long long x_elems, w_elems, y_elems;
+};
+
+// One entry of the stencil lookup table used by the in-kernel gather and the explicit unroll:
+// reduction index kg = (c*R + r)*S + s  ->  element offset from the window's top-left input
+// element and the (dh, dw) displacement used for the bounds test.  Entries past C*R*S (the
+// zero padding of the reduction axis) have off = -1.
+struct GatherEntry {
+  int32_t off;
+  int16_t dh;
+  int16_t dw;
+};
+
+enum AMode { A_TILED = 0, A_IM2COL_TMA = 1, A_GATHER = 2 };
+
+// Everything the MMA kernel needs besides its two tensor maps.
+struct ConvArgs {
+  int32_t* y32;
+  int8_t* y8;
+  int32_t* acc;  // split-K accumulation buffer (int32, output index order), or nullptr
+  int* status;
+  const int8_t* x;
+  const GatherEntry* table;
+  long long x_stride_n;
+  int x_stride_h, x_stride_w;
+  int Mg, K, PQ, Q, H, W;
+  int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
+  int S;
+  int num_kb;       // 128-byte (or bk-byte) reduction blocks in total
+  int ksteps_full;  // MMA instructions per full block (bk / 32)
+  int ksteps_last;  // MMA instructions in the last block
+  int kb_per_tap;   // channel-pack map: blocks per filter tap
+  int tap_cols;     // channel-pack map: columns of the packed weight matrix per tap (C_pad)
+  int table_len;    // gather: entries of the lookup table (padded reduction length)
+  int bk;           // bytes of reduction per block: 32, 64 or 128
+  int tile_n;
+  int tmem_cols;
+  int stages;
+  int split_k;
+  int shift, out_mode, out_layout;
+};
+
+struct Schedule {
+  int variant;
+  int tile_n;
+  int split_k;
+};
+
+// --- planner.cpp -------------------------------------------------------------------------------
+int resolve_geom(const b2c_conv_desc* d, Geom* g);  // validation + derived sizes; B2C_* code
+int round_up(int v, int m);
+int cp_channel_pad(int C);           // channels after Pad for the channel-pack map
+int cp_block_bytes(int C_pad);       // reduction bytes per block for the channel-pack map
+int im2col_k_pad(int Kg);            // padded reduction length for the stencil-unroll maps
+void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out);
+int pick_by_policy(const std::vector<b2c_embedding>& all, int policy);  // index or -1
+size_t workspace_bytes_for(const Geom& g, int variant, int split_k);
+
+// --- tma.cpp -----------------------------------------------------------------------------------
+// Tensor-map encoders obtained through cudaGetDriverEntryPoint (no link-time libcuda dependency).
+int encode_tiled_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
+                    uint32_t box_inner, uint32_t box_outer, int swizzle_bytes);
+int encode_im2col_nhwc(CUtensorMap* map, const void* base, int C_pad, int W, int H, int N, int pad_w, int pad_h,
+                       int S, int R, int dil_w, int dil_h, int stride_w, int stride_h, int channels_per_pixel,
+                       int pixels_per_column, int swizzle_bytes);
+void set_last_cuda_error(int e);
+int get_last_cuda_error();
+
+// --- kernel launchers (layout.cu, conv_mma.cu) -------------------------------------------------
+cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, int H, int W, int C_pad,
+                                    cudaStream_t st);
+cudaError_t launch_pack_weights_cp(const int8_t* w, int8_t* out, int K, int C, int R, int S, int C_pad,
+                                   cudaStream_t st);
+cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg, int K_pad, cudaStream_t st);
+cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, long long Mg, int PQ, int Q, int H,
+                          int W, int stride_h, int stride_w, int pad_h, int pad_w, long long x_stride_n,
+                          int x_stride_h, int x_stride_w, int K_pad, cudaStream_t st);
+cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, long long elems, int shift,
+                                 int out_mode, cudaStream_t st);
+cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,
+                            cudaStream_t st);
+size_t conv_mma_smem_bytes(int amode, const ConvArgs& args);
+
+}  // namespace b2c

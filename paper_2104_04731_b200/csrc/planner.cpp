@@ -1,0 +1,197 @@
+// Host-side embedding planner: which convolution axes feed the MMA's M / N / K dimensions, with
+// which layout rewrite, tile width and reduction split.
+//
+// The paper finds embeddings by constraint solving over the scalar data-flow graph (Section 4)
+// and derives the layout rewrites of Table 2 from the solution.  For a 2-D convolution on a
+// matrix-multiply intrinsic the legal, axis-aligned, dense solutions form a small closed family
+// (the hyper-rectangle and linear-access constraints of Section 4.2 leave only: feed K from the
+// padded channel axis, or from the unrolled stencil), so this planner writes that family out
+// directly, ranks it with the overhead terms of Section 4.4 and leaves the final choice to
+// measured device time, as Section 6.1 does with its five best candidates.
+#include <algorithm>
+#include <cstring>
+
+#include "b2c_internal.h"
+
+namespace b2c {
+
+int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+static int out_extent(int in, int k, int stride, int pad, int dil) {
+  long long span = (long long)in + 2LL * pad - (long long)dil * (k - 1) - 1;
+  if (span < 0) return 0;
+  return (int)(span / stride) + 1;
+}
+
+int resolve_geom(const b2c_conv_desc* d, Geom* g) {
+  if (!d || !g) return B2C_E_INVALID_ARG;
+  if (d->N < 1 || d->C < 1 || d->H < 1 || d->W < 1 || d->K < 1 || d->R < 1 || d->S < 1) return B2C_E_INVALID_ARG;
+  if (d->stride_h < 1 || d->stride_w < 1 || d->pad_h < 0 || d->pad_w < 0 || d->dil_h < 1 || d->dil_w < 1)
+    return B2C_E_INVALID_ARG;
+  if (d->shift < 0 || d->shift > 31) return B2C_E_INVALID_ARG;
+  if (d->in_layout != B2C_LAYOUT_NCHW && d->in_layout != B2C_LAYOUT_NHWC) return B2C_E_INVALID_ARG;
+  if (d->out_layout != B2C_LAYOUT_NCHW && d->out_layout != B2C_LAYOUT_NHWC) return B2C_E_INVALID_ARG;
+  if ((d->out_mode & ~3) != 0 || (d->out_mode & 3) == 0) return B2C_E_INVALID_ARG;
+  g->d = *d;
+  g->P = out_extent(d->H, d->R, d->stride_h, d->pad_h, d->dil_h);
+  g->Q = out_extent(d->W, d->S, d->stride_w, d->pad_w, d->dil_w);
+  long long kg = (long long)d->C * d->R * d->S;
+  if (g->P == 0 || g->Q == 0) return B2C_E_UNSUPPORTED;
+  if (kg > kMaxKg) return B2C_E_UNSUPPORTED;
+  g->PQ = g->P * g->Q;
+  g->Mg = (long long)d->N * g->PQ;
+  g->Kg = (int)kg;
+  g->x_elems = (long long)d->N * d->C * d->H * d->W;
+  g->w_elems = (long long)d->K * kg;
+  g->y_elems = g->Mg * d->K;
+  // Index arithmetic in the kernels is 32-bit for rows/columns and 64-bit for byte offsets.
+  if (g->Mg > 0x7FFFFF00LL || g->x_elems > (1LL << 40) || g->y_elems > (1LL << 40)) return B2C_E_UNSUPPORTED;
+  if ((long long)d->H * d->W * d->C > 0x7FFFFFFFLL) return B2C_E_UNSUPPORTED;
+  return B2C_OK;
+}
+
+// Pad rule (Table 2, rule 2) for the channel axis: the intrinsic consumes 32 channels per
+// instruction, so C is padded to a multiple of 32.
+int cp_channel_pad(int C) { return round_up(C, kMmaK); }
+
+// Split rule (Table 2, rule 3): the padded channel axis is cut into blocks of the largest of
+// 128 / 64 / 32 bytes that divides it (one shared-memory swizzle row per block).
+int cp_block_bytes(int C_pad) {
+  if (C_pad % 128 == 0) return 128;
+  if (C_pad % 64 == 0) return 64;
+  return 32;
+}
+
+int im2col_k_pad(int Kg) { return round_up(Kg, kMmaK); }
+
+static int tmem_pow2(int n) {
+  int c = 32;
+  while (c < n) c <<= 1;
+  return c;
+}
+
+size_t workspace_bytes_for(const Geom& g, int variant, int split_k) {
+  size_t ws = 0;
+  const b2c_conv_desc& d = g.d;
+  if (variant == B2C_VARIANT_CP_TMA) {
+    int C_pad = cp_channel_pad(d.C);
+    bool direct = d.in_layout == B2C_LAYOUT_NHWC && C_pad == d.C;
+    if (!direct) ws += (size_t)d.N * d.H * d.W * C_pad;
+  } else if (variant == B2C_VARIANT_IM2COL_EXPLICIT) {
+    ws += (size_t)g.Mg * im2col_k_pad(g.Kg);
+  }
+  ws = (ws + 255) / 256 * 256;
+  // A split reduction accumulates int32 partial sums in scratch unless the int32 output itself
+  // can serve (int32-only output in any layout).
+  if (split_k > 1 && (d.out_mode & B2C_OUT_I8)) ws += (size_t)g.y_elems * 4;
+  return ws;
+}
+
+static bool cp_legal(const Geom& g) {
+  const b2c_conv_desc& d = g.d;
+  // Limits of the 4-D im2col-mode tensor map: corners in [-128, 127], tap offsets in [0, 255],
+  // traversal strides in [1, 8], dimensions < 2^32, row pitch a multiple of 16 bytes.
+  int up_w = d.pad_w - (d.S - 1) * d.dil_w, up_h = d.pad_h - (d.R - 1) * d.dil_h;
+  if (d.pad_w > 128 || d.pad_h > 128 || up_w < -128 || up_h < -128 || up_w > 127 || up_h > 127) return false;
+  if ((d.S - 1) * d.dil_w > 255 || (d.R - 1) * d.dil_h > 255) return false;
+  if (d.stride_w > 8 || d.stride_h > 8) return false;
+  // NHWC source that is not already a multiple of 32 channels would need a re-pad kernel that
+  // this build does not have.
+  if (d.in_layout == B2C_LAYOUT_NHWC && cp_channel_pad(d.C) != d.C) return false;
+  return true;
+}
+
+static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int tile_n, int split_k) {
+  const b2c_conv_desc& d = g.d;
+  b2c_embedding e;
+  std::memset(&e, 0, sizeof(e));
+  e.map_m = B2C_AXIS_NPQ;
+  e.map_n = B2C_AXIS_K;
+  e.variant = variant;
+  e.tile_m = kTileM;
+  e.tile_n = tile_n;
+  e.split_k = split_k;
+  e.device_us = -1.0f;
+  long long M_pad = (g.Mg + kTileM - 1) / kTileM * kTileM;
+  long long N_pad = (long long)round_up(d.K, tile_n);
+  long long k_issued, moved;
+  long long mac_min = g.Mg * d.K * g.Kg;
+  long long data_min = g.x_elems + g.w_elems + g.y_elems;
+  if (variant == B2C_VARIANT_CP_TMA) {
+    e.map_k = B2C_AXIS_C;
+    int C_pad = cp_channel_pad(d.C);
+    k_issued = (long long)d.R * d.S * C_pad;
+    long long packed = (long long)d.N * d.H * d.W * C_pad;
+    bool direct = d.in_layout == B2C_LAYOUT_NHWC && C_pad == d.C;
+    moved = (direct ? 0 : g.x_elems + packed) + packed + (long long)d.K * k_issued + g.y_elems;
+  } else {
+    e.map_k = B2C_AXIS_CRS;
+    int K_pad = im2col_k_pad(g.Kg);
+    k_issued = K_pad;
+    if (variant == B2C_VARIANT_IM2COL_EXPLICIT)
+      moved = g.x_elems + 2 * g.Mg * K_pad + (long long)d.K * K_pad + g.y_elems;
+    else
+      moved = g.x_elems + (long long)d.K * K_pad + g.y_elems;
+  }
+  if (split_k > 1) moved += 2 * g.y_elems;  // partial sums written and read once more
+  e.o_mac = M_pad * N_pad * k_issued - mac_min;
+  e.o_data = moved - data_min;
+  e.workspace_bytes = (int64_t)workspace_bytes_for(g, variant, split_k);
+  out->push_back(e);
+}
+
+void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
+  out->clear();
+  const b2c_conv_desc& d = g.d;
+  // Tile widths: every MMA N extent up to the first one that covers K.
+  std::vector<int> tiles;
+  for (int t = 16; t <= 256; t <<= 1) {
+    tiles.push_back(t);
+    if (t >= d.K) break;
+  }
+  long long tiles_m = (g.Mg + kTileM - 1) / kTileM;
+  for (int variant = 0; variant < 3; ++variant) {
+    if (variant == B2C_VARIANT_CP_TMA && !cp_legal(g)) continue;
+    int num_kb;
+    if (variant == B2C_VARIANT_CP_TMA) {
+      int C_pad = cp_channel_pad(d.C);
+      num_kb = d.R * d.S * (C_pad / cp_block_bytes(C_pad));
+    } else {
+      num_kb = (im2col_k_pad(g.Kg) + 127) / 128;
+    }
+    // The in-kernel gather keeps its lookup table in shared memory.
+    if (variant == B2C_VARIANT_IM2COL_GATHER && im2col_k_pad(g.Kg) > 4096) continue;
+    for (int t : tiles) {
+      // Skip widths that only add padding: keep t if it is the covering width or K % t == 0
+      // or it wastes less than a quarter of the columns.
+      int n_pad = round_up(d.K, t);
+      if (t < tiles.back() && (n_pad - d.K) * 4 > n_pad) continue;
+      long long ctas = tiles_m * (n_pad / t);
+      for (int split = 1; split <= 32; split <<= 1) {
+        if (split > num_kb) break;
+        // A split reduction only helps while the grid is smaller than the machine.
+        if (split > 1 && ctas * (split / 2) >= kNumSMs) break;
+        add(out, g, variant, t, split);
+      }
+    }
+  }
+  std::stable_sort(out->begin(), out->end(), [](const b2c_embedding& a, const b2c_embedding& b) {
+    return a.o_mac + a.o_data < b.o_mac + b.o_data;
+  });
+  for (size_t i = 0; i < out->size(); ++i) (*out)[i].id = (int)i;
+  (void)tmem_pow2;
+}
+
+int pick_by_policy(const std::vector<b2c_embedding>& all, int policy) {
+  if (all.empty()) return -1;
+  if (policy >= 0) return policy < (int)all.size() ? policy : -1;
+  if (policy == B2C_POLICY_MIN_WORKSPACE) {
+    int best = 0;
+    for (size_t i = 1; i < all.size(); ++i)
+      if (all[i].workspace_bytes < all[best].workspace_bytes) best = (int)i;
+    return best;
+  }
+  return 0;  // MIN_OVERHEAD (AUTO_TIMED is resolved by the caller)
+}
+
+}  // namespace b2c

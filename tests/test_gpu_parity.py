@@ -1,0 +1,187 @@
+"""Parity of the CUDA path against the CPU oracle, bit for bit, through the C ABI."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2104_04731_b200 as b2c
+from paper_2104_04731_b200.synth import CONFIGS, int8_uniform
+
+from gpu_util import check_against_oracle, run_embedding, to_dev
+
+pytestmark = pytest.mark.gpu
+
+_ref_cache = {}
+
+
+def cfg_reference(cfg):
+    if cfg.name not in _ref_cache:
+        x, w = cfg.tensors()
+        _ref_cache[cfg.name] = (x, w, oracle.conv2d_int8(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift))
+    return _ref_cache[cfg.name]
+
+
+# ---- layout kernels on their own ---------------------------------------------------------------------
+@pytest.mark.parametrize("shape,C_pad", [((1, 16, 14, 14), 32), ((2, 3, 30, 23), 16), ((3, 70, 9, 13), 96),
+                                         ((2, 256, 14, 14), 256), ((1, 1, 96, 480), 32), ((2, 64, 56, 56), 64)])
+def test_pack_activations(lib, shape, C_pad):
+    x = int8_uniform(shape, 301)
+    want = oracle.pack_nhwc_cpad(x, C_pad)
+    out = torch.full(want.shape, 55, dtype=torch.int8, device="cuda")
+    lib.pack_activations(to_dev(x), out, C_pad)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("geom", [(2, 3, 20, 21, 7, 7, 2, 3, 1), (1, 1, 30, 60, 9, 21, 2, 0, 1), (2, 16, 9, 9, 3, 3, 1, 1, 1),
+                                  (1, 5, 17, 13, 3, 2, (2, 1), (0, 2), (2, 3))])
+@pytest.mark.parametrize("in_layout", [0, 1])
+def test_im2col_matrix(lib, geom, in_layout):
+    N, C, H, W, R, S, stride, pad, dil = geom
+    x = int8_uniform((N, C, H, W), 302)
+    A = oracle.im2col(x, R, S, stride, pad, dil)
+    K_pad = -(-A.shape[1] // 32) * 32
+    d = lib.make_desc(N, C, H, W, 1, R, S, stride, pad, dil, in_layout=in_layout)
+    xin = x if in_layout == 0 else x.transpose(0, 2, 3, 1)
+    out = torch.full((A.shape[0], K_pad), 55, dtype=torch.int8, device="cuda")
+    lib.im2col(d, to_dev(xin), out, K_pad)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    assert np.array_equal(got[:, :A.shape[1]], A)
+    assert not got[:, A.shape[1]:].any()
+
+
+# ---- the five benchmark shapes, every enumerated embedding ------------------------------------------
+@pytest.mark.parametrize("cfg", CONFIGS, ids=lambda c: c.name)
+def test_config_every_embedding(lib, cfg):
+    x, w, ref = cfg_reference(cfg)
+    d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
+                      out_mode=cfg.out_mode)
+    embs = lib.enumerate_embeddings(d)
+    assert {e.variant for e in embs} == {0, 1, 2}
+    for e in embs:
+        check_against_oracle(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, cfg.out_mode, e.id, ref=ref)
+
+
+@pytest.mark.parametrize("cfg", CONFIGS[:2] + CONFIGS[4:], ids=lambda c: c.name)
+@pytest.mark.parametrize("in_layout,out_layout", [(1, 1), (0, 1), (1, 0)])
+def test_config_layouts(lib, cfg, in_layout, out_layout):
+    x, w, ref = cfg_reference(cfg)
+    for variant in (0, 1, 2):
+        d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
+                          in_layout, out_layout, 3)
+        ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant]
+        for i in ids[:2] + ids[-1:]:
+            check_against_oracle(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, 3, i, ref=ref,
+                                 in_layout=in_layout, out_layout=out_layout)
+
+
+# ---- randomised small shapes: ragged tiles, odd channels, strides, dilation, big pads, shifts -------
+def _random_cases():
+    rng = np.random.default_rng(2104)
+    cases = []
+    for i in range(36):
+        C = int(rng.choice([1, 2, 3, 5, 17, 32, 33, 64, 72, 130]))
+        K = int(rng.choice([1, 8, 15, 16, 17, 40, 64, 129]))
+        R, S = int(rng.integers(1, 5)), int(rng.integers(1, 6))
+        sh, sw = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        dh, dw = int(rng.integers(1, 4)), int(rng.integers(1, 3))
+        ph, pw = int(rng.integers(0, 4)), int(rng.integers(0, 5))
+        H = int(rng.integers(dh * (R - 1) + 1, dh * (R - 1) + 20))
+        W = int(rng.integers(dw * (S - 1) + 1, dw * (S - 1) + 24))
+        N = int(rng.integers(1, 4))
+        shift = int(rng.choice([0, 1, 8, 12, 31]))
+        cases.append((N, C, H, W, K, R, S, (sh, sw), (ph, pw), (dh, dw), shift, 400 + i))
+    return cases
+
+
+@pytest.mark.parametrize("case", _random_cases(), ids=lambda c: "n%dc%dh%dw%dk%dr%ds%d" % c[:7])
+def test_random_shapes(lib, case):
+    N, C, H, W, K, R, S, stride, pad, dil, shift, seed = case
+    x = int8_uniform((N, C, H, W), seed)
+    w = int8_uniform((K, C, R, S), seed + 1000)
+    ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode=3)
+    embs = lib.enumerate_embeddings(d)
+    for variant in (0, 1, 2):
+        ids = [e.id for e in embs if e.variant == variant]
+        for i in ids[:1] + ids[-1:]:
+            check_against_oracle(x, w, stride, pad, dil, shift, 3, i, ref=ref)
+    # NHWC in and out through the lowest-overhead embedding that accepts it
+    d2 = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, 1, 1, 3)
+    e2 = lib.enumerate_embeddings(d2)[0]
+    check_against_oracle(x, w, stride, pad, dil, shift, 3, e2.id, ref=ref, in_layout=1, out_layout=1)
+
+
+def test_extreme_values_and_shift_clip(lib):
+    # -128 * -128 is the largest product; all-(-128) tensors with 9*64 taps reach 9437184.
+    x = np.full((1, 64, 6, 6), -128, dtype=np.int8)
+    w = np.full((16, 64, 3, 3), -128, dtype=np.int8)
+    ref = oracle.conv2d_int8(x, w, 1, 1, 1, 16)
+    for variant in (0, 1, 2):
+        d = lib.make_desc(1, 64, 6, 6, 16, 3, 3, 1, 1, 1, 16, out_mode=3)
+        i = next(e.id for e in lib.enumerate_embeddings(d) if e.variant == variant)
+        check_against_oracle(x, w, 1, 1, 1, 16, 3, i, ref=ref)
+    x = int8_uniform((1, 32, 5, 5), 501)
+    w = int8_uniform((8, 32, 3, 3), 502)
+    for shift in (0, 1, 8, 31):
+        ref = oracle.conv2d_int8(x, w, 1, 1, 1, shift)
+        check_against_oracle(x, w, 1, 1, 1, shift, 2, b2c.POLICY_MIN_OVERHEAD, ref=ref)
+
+
+# ---- the other entry points -----------------------------------------------------------------------------
+def test_one_shot_device_and_host_calls(lib):
+    for cfg in (CONFIGS[0], CONFIGS[3]):
+        x, w, ref = cfg_reference(cfg)
+        xd, wd = to_dev(x), to_dev(w)
+        y32 = torch.zeros(ref[0].shape, dtype=torch.int32, device="cuda")
+        y8 = torch.zeros(ref[0].shape, dtype=torch.int8, device="cuda")
+        for _ in range(2):  # the second call reuses the cached plan
+            lib.conv2d_int8(xd, wd, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, y32, y8)
+            torch.cuda.synchronize()
+            assert np.array_equal(y32.cpu().numpy(), ref[0])
+            assert np.array_equal(y8.cpu().numpy(), ref[1])
+        h32 = np.zeros(ref[0].shape, dtype=np.int32)
+        h8 = np.zeros(ref[0].shape, dtype=np.int8)
+        lib.conv2d_int8_host(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, h32, h8)
+        assert np.array_equal(h32, ref[0]) and np.array_equal(h8, ref[1])
+        h8[:] = 0
+        lib.conv2d_int8_host(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, None, h8)
+        assert np.array_equal(h8, ref[1])
+
+
+def test_policies(lib):
+    cfg = CONFIGS[0]
+    x, w, ref = cfg_reference(cfg)
+    for policy in (b2c.POLICY_AUTO_TIMED, b2c.POLICY_MIN_OVERHEAD, b2c.POLICY_MIN_WORKSPACE):
+        emb = check_against_oracle(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, cfg.out_mode, policy, ref=ref)
+        if policy == b2c.POLICY_AUTO_TIMED:
+            assert emb.device_us > 0
+        if policy == b2c.POLICY_MIN_WORKSPACE:
+            assert emb.workspace_bytes == 0
+
+
+def test_error_paths_on_device(lib):
+    cfg = CONFIGS[0]
+    d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, out_mode=3)
+    raw = lib.load()
+    plan = lib.Plan(d, b2c.POLICY_MIN_OVERHEAD)
+    x, w = (to_dev(t) for t in cfg.tensors())
+    y32 = torch.zeros((1, 16, 14, 14), dtype=torch.int32, device="cuda")
+    y8 = torch.zeros((1, 16, 14, 14), dtype=torch.int8, device="cuda")
+    ws = torch.zeros(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
+    p = lambda t: ctypes.c_void_p(t.data_ptr()) if t is not None else None
+    assert raw.b2c_conv2d_int8_run(plan._h, p(x), p(y32), p(y8), p(ws), None) == b2c.E_NOT_READY
+    plan.set_weights(w)
+    assert raw.b2c_conv2d_int8_run(plan._h, p(x), None, p(y8), p(ws), None) == b2c.E_INVALID_ARG
+    assert raw.b2c_conv2d_int8_run(plan._h, p(x), p(y32), None, p(ws), None) == b2c.E_INVALID_ARG
+    assert raw.b2c_conv2d_int8_run(plan._h, ctypes.c_void_p(x.data_ptr() + 1), p(y32), p(y8), p(ws), None) == b2c.E_INVALID_ARG
+    h = ctypes.c_void_p()
+    assert raw.b2c_plan_create(ctypes.byref(d), 10 ** 6, None, ctypes.byref(h)) == b2c.E_INVALID_ARG
+    assert raw.b2c_plan_create(ctypes.byref(d), -9, None, ctypes.byref(h)) == b2c.E_INVALID_ARG
+    plan.run(x, y32, y8, ws)
+    torch.cuda.synchronize()
+    assert plan.device_status() == b2c.OK
+    plan.destroy()
