@@ -1,0 +1,464 @@
+#!/usr/bin/env python
+"""Benchmark of the int8 convolution hot path on B200.
+
+One "step" is one pass of the whole path (activation layout rewrite, MMA kernel with fused
+shift/clip epilogue, split-reduction finish when the embedding has one) over a batch of G
+independent instances of the headline convolution shape, each instance with its own input,
+weight, output and scratch buffers, so that every launch reads cold data (G x working set is
+larger than the 126 MB L2).  The G launches of a step are captured once in a CUDA graph.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2104_04731_b200.synth import CONFIGS, ConvShape, int8_uniform  # noqa: E402
+
+METRIC = "int8 conv TOPS (2*N*K*P*Q*C*R*S / device time)"
+UNIT = "TOPS"
+HEADLINE = 4  # index into CONFIGS: the large-batch, compute-bound 3x3 stride-2 shape
+L2_BYTES = 126 * 1024 * 1024
+INT8_TO_BF16_RATIO = 2.0  # nominal dense int8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
+
+# DRAM traffic of the dominant kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
+# per launch), valid only for the kernel source it was taken on; see profiles/.
+NCU_TRAFFIC = {"conv_mma_sha1": None, "bytes_per_launch": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def roofline_time_us(cfg: ConvShape, peaks) -> tuple:
+    """(t_roof_us, bound) with t = max(useful ops / int8 peak, algorithmic bytes / HBM bandwidth)."""
+    t_c = 2.0 * cfg.macs / (peaks["bf16_tflops"] * INT8_TO_BF16_RATIO * 1e12) * 1e6
+    t_m = cfg.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6
+    return (t_c, "tensor") if t_c >= t_m else (t_m, "hbm")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------------
+# GPU arm
+# ----------------------------------------------------------------------------------------------------
+class Instances:
+    """G independent instances of one shape, each with its own plan (own packed weights) and buffers."""
+
+    def __init__(self, b2c, torch, cfg: ConvShape, G: int, policy_or_id: int, in_layout=0, prepacked=None):
+        self.cfg, self.G, self.in_layout = cfg, G, in_layout
+        d = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
+                          in_layout, b2c.LAYOUT_NCHW, cfg.out_mode)
+        first = b2c.Plan(d, policy_or_id)
+        self.emb = first.info()
+        self.plans = [first] + [b2c.Plan(d, self.emb.id) for _ in range(G - 1)]
+        oshape = (cfg.N, cfg.K, cfg.P, cfg.Q)
+        xh, wh = cfg.tensors()
+        if in_layout == 1:
+            xh = np.ascontiguousarray(xh.transpose(0, 2, 3, 1))
+        self.x, self.y32, self.y8, self.ws = [], [], [], []
+        for i, p in enumerate(self.plans):
+            # distinct memory per instance; the values repeat (timing does not depend on them)
+            self.x.append(torch.from_numpy(xh).cuda())
+            p.set_weights(torch.from_numpy(wh).cuda())
+            self.y32.append(torch.empty(oshape, dtype=torch.int32, device="cuda") if cfg.out_mode & 1 else None)
+            self.y8.append(torch.empty(oshape, dtype=torch.int8, device="cuda") if cfg.out_mode & 2 else None)
+            self.ws.append(torch.empty(max(16, p.workspace_bytes()), dtype=torch.uint8, device="cuda"))
+        torch.cuda.synchronize()
+        self.launches_per_instance = self._count_launches()
+        self.graph = None
+
+    def _count_launches(self):
+        """Kernels of this library per call: layout rewrite (if any) + MMA kernel + split finish (if any)."""
+        e, c = self.emb, self.cfg
+        n = 1
+        if e.variant == 1 or (e.variant == 0 and not (self.in_layout == 1 and c.C % 32 == 0)):
+            n += 1
+        if e.split_k > 1 and (c.out_mode & 2):
+            n += 1
+        return n
+
+    def run_all(self):
+        for i, p in enumerate(self.plans):
+            p.run(self.x[i], self.y32[i], self.y8[i], self.ws[i])
+
+    def capture(self, torch):
+        self.run_all()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.run_all()
+        self.graph = g
+
+    def step(self):
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self.run_all()
+
+    def check_status(self, b2c):
+        for p in self.plans:
+            s = p.device_status()
+            if s != 0:
+                raise RuntimeError("device status " + b2c.status_string(s))
+
+    def destroy(self):
+        self.graph = None
+        for p in self.plans:
+            p.destroy()
+
+
+def time_steps(torch, fn, steps, warmup, dist=None):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        ms = float(t.item())
+    return ms
+
+
+def instances_for(cfg, min_bytes=2 * L2_BYTES, lo=8, hi=256):
+    per = cfg.algorithmic_bytes + cfg.N * cfg.C * cfg.H * cfg.W  # plus a packed copy of the input
+    return int(max(lo, min(hi, -(-min_bytes // per))))
+
+
+def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, graph=True):
+    """Combined (whole path, NCHW in), Op (MMA kernel alone on a resident packed operand) and Transf."""
+    G = instances_for(cfg)
+    inst = Instances(b2c, torch, cfg, G, policy)
+    if graph:
+        inst.capture(torch)
+    ms = time_steps(torch, inst.step, steps, warmup, dist)
+    inst.check_status(b2c)
+    per_call_us = ms * 1e3 / (steps * G)
+    emb = inst.emb.as_dict()
+    launches = inst.launches_per_instance
+    inst.destroy()
+    t_roof, bound = roofline_time_us(cfg, peaks)
+    res = {
+        "shape": cfg.name, "instances": G, "cold": bool(G * cfg.algorithmic_bytes >= L2_BYTES), "combined_us": per_call_us, "tops": 2.0 * cfg.macs / (per_call_us * 1e-6) / 1e12,
+        "roofline_us": t_roof, "bound": bound, "roofline_frac": t_roof / per_call_us,
+        "embedding": {k: emb[k] for k in ("id", "variant_name", "tile_n", "split_k", "workspace_bytes", "o_mac", "o_data", "device_us")},
+        "launches_per_call": launches,
+    }
+    return res
+
+
+def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=True):
+    """Device time of the MMA kernel alone: same embedding but with the layout rewrite already done
+    (channel-pack map: NHWC input with padded channels; stencil-unroll in-kernel: unchanged)."""
+    if emb_variant == 0 and cfg.C % 32 == 0:
+        d = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, 1, 0, cfg.out_mode)
+        ids = [e.id for e in b2c.enumerate_embeddings(d) if e.variant == 0 and e.tile_n == tile_n and e.split_k == split_k]
+        if not ids:
+            return None
+        G = instances_for(cfg)
+        inst = Instances(b2c, torch, cfg, G, ids[0], in_layout=1)
+    elif emb_variant == 2:
+        d = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, 0, 0, cfg.out_mode)
+        ids = [e.id for e in b2c.enumerate_embeddings(d) if e.variant == 2 and e.tile_n == tile_n and e.split_k == split_k]
+        G = instances_for(cfg)
+        inst = Instances(b2c, torch, cfg, G, ids[0])
+    else:
+        return None
+    if graph:
+        inst.capture(torch)
+    ms = time_steps(torch, inst.step, steps, warmup)
+    inst.check_status(b2c)
+    us = ms * 1e3 / (steps * G)
+    n = inst.launches_per_instance
+    inst.destroy()
+    return {"us": us, "launches_per_call": n}
+
+
+def e2e_measure(b2c, torch, cfg, steps, warmup, dist=None):
+    """Same metric through the host-buffer C-ABI call: pinned host inputs, H2D + path + D2H every call."""
+    xh, wh = cfg.tensors()
+    x = torch.from_numpy(xh).pin_memory().numpy()
+    w = torch.from_numpy(wh).pin_memory().numpy()
+    oshape = (cfg.N, cfg.K, cfg.P, cfg.Q)
+    y32 = torch.empty(oshape, dtype=torch.int32).pin_memory().numpy() if cfg.out_mode & 1 else None
+    y8 = torch.empty(oshape, dtype=torch.int8).pin_memory().numpy() if cfg.out_mode & 2 else None
+    reps = 8
+
+    def fn():
+        for _ in range(reps):
+            b2c.conv2d_int8_host(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, y32, y8)
+
+    for _ in range(max(1, warmup)):
+        fn()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        fn()
+    torch.cuda.synchronize()
+    sec = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([sec], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        sec = float(t.item())
+    calls = steps * reps
+    h2d = (x.nbytes + w.nbytes) * reps
+    d2h = ((y32.nbytes if y32 is not None else 0) + (y8.nbytes if y8 is not None else 0)) * reps
+    return {"sec": sec, "calls": calls, "h2d": h2d, "d2h": d2h}
+
+
+def cpu_baseline(cfg, budget_s=12.0):
+    """The oracle as it stands on the host cores, on a bounded sample of the workload."""
+    import oracle
+
+    x, w = cfg.tensors()
+    cores = os.cpu_count() or 1
+    n_probe = 1
+    t0 = time.perf_counter()
+    oracle.conv2d_int8(x[:n_probe], w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, True, True)
+    t_probe = time.perf_counter() - t0
+    n = int(max(1, min(cfg.N, budget_s / 3.0 / max(t_probe, 1e-6))))
+    best = None
+    for _ in range(3):
+        t0 = time.perf_counter()
+        oracle.conv2d_int8(x[:n], w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, True, True)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    macs = cfg.macs // cfg.N * n
+    return {"value": 2.0 * macs / best / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d of %d images of %s, best of 3, OpenMP over (n, k)" % (n, cfg.N, cfg.name), "seconds": best}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    cfg = CONFIGS[args.config]
+    import oracle
+
+    x, w = cfg.tensors()
+    cores = os.cpu_count() or 1
+    t0 = time.perf_counter()
+    oracle.conv2d_int8(x[:1], w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, True, True)
+    t_probe = time.perf_counter() - t0
+    total = max(1, args.steps + args.warmup)
+    n = int(max(1, min(cfg.N, 60.0 / total / max(t_probe, 1e-6))))
+    for _ in range(args.warmup):
+        oracle.conv2d_int8(x[:n], w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, True, True)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.conv2d_int8(x[:n], w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, True, True)
+    sec = time.perf_counter() - t0
+    macs = cfg.macs // cfg.N * n
+    value = 2.0 * macs * args.steps / sec / 1e12
+    sample = "%d of %d images of %s per step" % (n, cfg.N, cfg.name)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3 / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8 x int8 -> int64 (range-checked to int32)", "data": "synthetic",
+        "config": {"workload": cfg.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def shard_report(world: int, instances_per_rank: int, ops_per_instance: float, steps: int, ms_max: float) -> float:
+    """Whole-job TOPS: every rank runs its own `instances_per_rank` instances per step (weak scaling,
+    no data-path collective); the job time is the slowest rank's."""
+    return world * instances_per_rank * ops_per_instance * steps / (ms_max * 1e-3) / 1e12
+
+
+def run_ours(args):
+    import torch
+
+    import paper_2104_04731_b200 as b2c
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+    b2c.load()
+    peaks = load_peaks()
+    cfg = CONFIGS[args.config]
+    policy = b2c.POLICY_AUTO_TIMED if args.embedding is None else args.embedding
+    graph = not args.no_graph
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    # ---- headline: whole path, device-resident inputs ------------------------------------------
+    G = instances_for(cfg)
+    inst = Instances(b2c, torch, cfg, G, policy)
+    if graph:
+        inst.capture(torch)
+    ms = time_steps(torch, inst.step, args.steps, args.warmup, dist)
+    inst.check_status(b2c)
+    clocks = sampler.stop() if rank == 0 else None
+    emb = inst.emb
+    launches = inst.launches_per_instance * G * args.steps
+    ops = 2.0 * cfg.macs
+    value = shard_report(world, G, ops, args.steps, ms)
+    per_call_us = ms * 1e3 / (args.steps * G)
+    inst.destroy()
+
+    # ---- the dominant kernel alone (the paper's "Op." column) for the roofline -------------------
+    op = op_only(b2c, torch, cfg, emb.variant, emb.tile_n, emb.split_k, args.steps, args.warmup, graph)
+    t_roof, bound = roofline_time_us(cfg, peaks)
+    op_us = op["us"] if op else per_call_us
+    if bound == "tensor":
+        achieved, peak, runit = ops / (op_us * 1e-6) / 1e12, peaks["bf16_tflops"] * INT8_TO_BF16_RATIO, "TFLOP/s"
+    else:
+        achieved, peak, runit = cfg.algorithmic_bytes / (op_us * 1e-6) / 1e9, peaks["hbm_gbs"], "GB/s"
+    sha = hashlib.sha1(open(os.path.join(ROOT, "paper_2104_04731_b200", "csrc", "conv_mma.cu"), "rb").read()).hexdigest()
+    traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["conv_mma_sha1"] == sha else None
+    roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
+                "traffic": traffic, "kernel": "conv_mma_kernel", "kernel_us": op_us,
+                "peak_source": "%s bf16 burst x %.0f (nominal int8:bf16)" % (peaks["source"], INT8_TO_BF16_RATIO)
+                if bound == "tensor" else peaks["source"] + " copy bandwidth"}
+
+    # ---- end to end through the host-buffer call ----------------------------------------------------
+    e = e2e_measure(b2c, torch, cfg, max(1, min(args.steps, 5)), 1, dist)
+    e2e = {"value": world * e["calls"] * ops / e["sec"] / 1e12, "unit": UNIT,
+           "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"]}
+
+    per_config = None
+    if rank == 0 and not args.headline_only:
+        per_config = []
+        for c in CONFIGS:
+            r = measure_shape(b2c, torch, c, max(2, args.steps // 2), 3, peaks, policy if c is cfg else b2c.POLICY_AUTO_TIMED, None, graph)
+            per_config.append(r)
+    cpu = cpu_baseline(cfg) if (rank == 0 and world == 1 and not args.no_cpu) else None
+
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return 0
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "s8 x s8 -> s32", "data": "synthetic",
+        "config": {"workload": cfg.name, "instances_per_step": G, "per_call_us": per_call_us,
+                   "l2": "inputs larger than L2: %d distinct buffer sets per step (%.0f MB)" % (G, G * (cfg.algorithmic_bytes) / 1e6),
+                   "cuda_graph": graph, "parallelism": "independent instances sharded over ranks, no collective",
+                   "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k,
+                                 "planner_us": emb.device_us}},
+        "roofline": roofline, "roofline_time_us": t_roof, "whole_path_roofline_frac": t_roof / per_call_us,
+        "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+    }
+    if cpu is not None:
+        line["cpu_baseline"] = cpu
+    if per_config is not None:
+        line["per_config"] = per_config
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=HEADLINE, help="index into the five benchmark shapes")
+    ap.add_argument("--embedding", type=int, default=None, help="embedding id; default: timed selection")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--headline-only", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
