@@ -7,7 +7,7 @@
 // rule of Table 2; columns = output channels) and a slice of the reduction.  Warp roles:
 //   warp 0      TMA producer (operand B always; operand A for the tiled and im2col-mode maps)
 //   warp 1      tensor-memory allocation, MMA issue (one elected lane)
-//   warps 2-5   operand-A gather into swizzled shared memory (stencil unroll inside the
+//   warps 2-9   operand-A gather into swizzled shared memory (stencil unroll inside the
 //               kernel), then the epilogue: tcgen05.ld, shift / clip, global stores
 // Shared-memory stages form a ring guarded by full/empty mbarriers.  Every wait is bounded:
 // on expiry the block raises an abort flag, records B2C_E_TIMEOUT in the status word, lets
@@ -18,7 +18,8 @@ namespace b2c {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kGatherWarps = 8;                    // warps 2..9: operand-A gather, then epilogue
+constexpr int kThreads = 64 + 32 * kGatherWarps;  // + warp 0 (TMA producer) and warp 1 (MMA issuer)
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
 
 struct __align__(8) SharedCtl {
@@ -50,6 +51,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "r"(bar), "r"(parity)
       : "memory");
   return done != 0;
+}
+// One lane of a converged warp.  Loops of the single-thread roles (TMA issue, MMA issue) are run
+// by the whole warp with only the issuing instructions predicated on this lane, so that loop
+// counters, barrier addresses and descriptors stay warp-uniform.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "elect.sync _|p, 0xffffffff;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(pred));
+  return pred != 0;
 }
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
@@ -138,6 +151,106 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t* v) {
 
 __device__ __forceinline__ int8_t requant(int v, int shift) { return (int8_t)max(-128, min(127, v >> shift)); }
 
+// Loads NC consecutive accumulator columns of this thread's TMEM lane.
+template <int NC>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, int32_t* v);
+template <>
+__device__ __forceinline__ void tmem_ld<16>(uint32_t taddr, int32_t* v) {
+  tmem_ld16(taddr, v);
+}
+template <>
+__device__ __forceinline__ void tmem_ld<32>(uint32_t taddr, int32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Epilogue for NC accumulator columns starting at output channel `kbase` of one output pixel
+// (one thread = one accumulator row).  Section 5.1's quantisation step (shift, clip) is applied
+// here, and the values go to the NKPQ or NPQK tensor; with a split reduction the partial sums
+// are added into a zeroed int32 buffer instead.
+template <int NC>
+__device__ __forceinline__ void epilogue_columns(const ConvArgs& args, uint32_t taddr, int kbase, bool row_valid,
+                                                 long long base_nkpq, long long base_npqk) {
+  int32_t v[NC];
+  __syncwarp();
+  tmem_ld<NC>(taddr, v);  // warp-collective: executed by all lanes
+  const int K = args.K;
+  if (!row_valid || kbase >= K) return;
+  const bool nhwc = args.out_layout == B2C_LAYOUT_NHWC;
+  if (args.split_k > 1) {
+    // Partial sums of the reduction slices meet in global memory; integer addition is
+    // associative, so the order of arrival does not change the result.
+    int32_t* dst = args.acc + (nhwc ? base_npqk + kbase : base_nkpq + (long long)kbase * args.PQ);
+    const long long step = nhwc ? 1 : args.PQ;
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+      if (kbase + j < K) atomicAdd(dst, v[j]);
+      dst += step;
+    }
+  } else if (!nhwc) {
+    // NKPQ: for a fixed column the 32 lanes of a warp hold 32 consecutive pixels, so every
+    // store instruction writes one contiguous run.
+    const long long o = base_nkpq + (long long)kbase * args.PQ;
+    if (args.out_mode & B2C_OUT_I32) {
+      int32_t* dst = args.y32 + o;
+#pragma unroll
+      for (int j = 0; j < NC; ++j) {
+        if (kbase + j < K) *dst = v[j];
+        dst += args.PQ;
+      }
+    }
+    if (args.out_mode & B2C_OUT_I8) {
+      int8_t* dst = args.y8 + o;
+#pragma unroll
+      for (int j = 0; j < NC; ++j) {
+        if (kbase + j < K) *dst = requant(v[j], args.shift);
+        dst += args.PQ;
+      }
+    }
+  } else {
+    // NPQK: a thread owns NC consecutive channels of one pixel: 16-byte vector stores.
+    const bool full = kbase + NC <= K;
+    if (args.out_mode & B2C_OUT_I32) {
+      int32_t* dst = args.y32 + base_npqk + kbase;
+      if (full && (K & 3) == 0) {
+#pragma unroll
+        for (int j = 0; j < NC; j += 4) *reinterpret_cast<int4*>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < NC; ++j)
+          if (kbase + j < K) dst[j] = v[j];
+      }
+    }
+    if (args.out_mode & B2C_OUT_I8) {
+      int8_t* dst = args.y8 + base_npqk + kbase;
+      if (full && (K & 15) == 0) {
+#pragma unroll
+        for (int g = 0; g < NC; g += 16) {
+          uint32_t w[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            w[j] = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) w[j] |= (uint32_t)(uint8_t)requant(v[g + j * 4 + i], args.shift) << (8 * i);
+          }
+          *reinterpret_cast<uint4*>(dst + g) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < NC; ++j)
+          if (kbase + j < K) dst[j] = requant(v[j], args.shift);
+      }
+    }
+  }
+}
+
 template <int AMODE>
 __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                                              const __grid_constant__ CUtensorMap tmap_b,
@@ -149,8 +262,8 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   const int lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * kTileM;
   const int n0 = blockIdx.y * args.tile_n;
-  const int kb_begin = (int)((long long)blockIdx.z * args.num_kb / args.split_k);
-  const int kb_end = (int)((long long)(blockIdx.z + 1) * args.num_kb / args.split_k);
+  const int kb_begin = (int)((unsigned)blockIdx.z * (unsigned)args.num_kb / (unsigned)args.split_k);
+  const int kb_end = (int)((unsigned)(blockIdx.z + 1) * (unsigned)args.num_kb / (unsigned)args.split_k);
   const int stages = args.stages;
   const int bk = args.bk;
   const uint32_t a_stage_bytes = kTileM * bk;
@@ -163,13 +276,17 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   uint8_t* smem_aligned = smem_raw + (smem_base - smem_u32(smem_raw));
   GatherEntry* s_table = reinterpret_cast<GatherEntry*>(smem_aligned + stages * (a_stage_bytes + b_stage_bytes));
 
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < stages; ++s) {
-      mbar_init(smem_u32(&ctl.full[s]), AMODE == A_GATHER ? 1 + 128 : 1);
-      mbar_init(smem_u32(&ctl.empty[s]), 1);
+  if (warp == 0) {
+    if (lane < stages) {
+      mbar_init(smem_u32(&ctl.full[lane]), AMODE == A_GATHER ? 1 + kGatherWarps : 1);
+      mbar_init(smem_u32(&ctl.empty[lane]), 1);
     }
-    mbar_init(smem_u32(&ctl.tmem_full), 1);
-    ctl.abort_flag = 0;
+    if (lane == 8) {
+      mbar_init(smem_u32(&ctl.tmem_full), 1);
+      ctl.abort_flag = 0;
+    }
+    if (lane == 9 && AMODE != A_GATHER) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+    if (lane == 10) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -186,122 +303,168 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = ctl.tmem_base;
 
+  // The loops below keep stage index, phase bit, tap position and addresses as running
+  // counters: each role is a single thread, so every integer division in a loop body would
+  // cost hundreds of cycles of dependent issue.
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
-    if (lane == 0) {
-      int n_img = 0, h_org = 0, w_org = 0;
+    {
+      int n_img = 0, h_org = 0, w_org = 0, cb = 0, sx = 0, r = 0;
       if (AMODE == A_IM2COL_TMA) {
         n_img = m0 / args.PQ;
         const int rem = m0 - n_img * args.PQ;
         const int p = rem / args.Q, q = rem - p * args.Q;
         h_org = p * args.stride_h - args.pad_h;
         w_org = q * args.stride_w - args.pad_w;
+        const int tap = kb_begin / args.kb_per_tap;
+        cb = kb_begin - tap * args.kb_per_tap;
+        r = tap / args.S;
+        sx = tap - r * args.S;
       }
-      int it = 0;
-      for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
-        const int s = it % stages;
-        const uint32_t ph = (uint32_t)(it / stages) & 1u;
+      int s = 0;
+      uint32_t ph = 0;
+      uint32_t a_dst = a_base, b_dst = b_base;
+      int kcol = kb_begin * bk;  // column of the packed weight matrix = reduction offset in bytes
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
         if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) break;
         const uint32_t full = smem_u32(&ctl.full[s]);
         if (AMODE == A_GATHER) {
-          mbar_arrive_expect_tx(full, b_stage_bytes);
-          tma_load_2d(b_base + s * b_stage_bytes, &tmap_b, kb * bk, n0, full);
+          if (elect_one()) {
+            mbar_arrive_expect_tx(full, b_stage_bytes);
+            tma_load_2d(b_dst, &tmap_b, kcol, n0, full);
+          }
         } else if (AMODE == A_TILED) {
-          mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes);
-          tma_load_2d(a_base + s * a_stage_bytes, &tmap_a, kb * bk, m0, full);
-          tma_load_2d(b_base + s * b_stage_bytes, &tmap_b, kb * bk, n0, full);
+          if (elect_one()) {
+            mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes);
+            tma_load_2d(a_dst, &tmap_a, kcol, m0, full);
+            tma_load_2d(b_dst, &tmap_b, kcol, n0, full);
+          }
         } else {
-          const int tap = kb / args.kb_per_tap;
-          const int cb = kb - tap * args.kb_per_tap;
-          const int r = tap / args.S, sx = tap - r * args.S;
-          mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes);
-          tma_load_im2col_4d(a_base + s * a_stage_bytes, &tmap_a, cb * bk, w_org, h_org, n_img, full,
-                             (uint16_t)(sx * args.dil_w), (uint16_t)(r * args.dil_h));
-          tma_load_2d(b_base + s * b_stage_bytes, &tmap_b, tap * args.tap_cols + cb * bk, n0, full);
+          if (elect_one()) {
+            mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes);
+            tma_load_im2col_4d(a_dst, &tmap_a, cb * bk, w_org, h_org, n_img, full, (uint16_t)(sx * args.dil_w),
+                               (uint16_t)(r * args.dil_h));
+            tma_load_2d(b_dst, &tmap_b, kcol, n0, full);
+          }
+          if (++cb == args.kb_per_tap) {
+            cb = 0;
+            if (++sx == args.S) {
+              sx = 0;
+              ++r;
+            }
+          }
+        }
+        kcol += bk;
+        a_dst += a_stage_bytes;
+        b_dst += b_stage_bytes;
+        if (++s == stages) {
+          s = 0;
+          ph ^= 1u;
+          a_dst = a_base;
+          b_dst = b_base;
         }
       }
     }
     __syncwarp();
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    {
       const uint32_t idesc = make_idesc_i8(args.tile_n);
-      int it = 0;
-      bool ok = true;
-      for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
-        const int s = it % stages;
-        const uint32_t ph = (uint32_t)(it / stages) & 1u;
-        if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status)) {
-          ok = false;
-          break;
-        }
+      const uint64_t adesc0 = make_smem_desc(a_base, bk);
+      const uint64_t bdesc0 = make_smem_desc(b_base, bk);
+      const uint64_t a_step = a_stage_bytes >> 4, b_step = b_stage_bytes >> 4;
+      uint64_t adesc = adesc0, bdesc = bdesc0;
+      int s = 0;
+      uint32_t ph = 0;
+      uint32_t accumulate = 0;
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
+        if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t adesc = make_smem_desc(a_base + s * a_stage_bytes, bk);
-        const uint64_t bdesc = make_smem_desc(b_base + s * b_stage_bytes, bk);
         const int ksteps = (kb == args.num_kb - 1) ? args.ksteps_last : args.ksteps_full;
-        for (int k = 0; k < ksteps; ++k) {
-          // Advancing 32 bytes along the row = 2 units of 16 bytes in the descriptor address.
-          mma_i8(tmem_acc, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (it > 0 || k > 0) ? 1u : 0u);
+        if (elect_one()) {
+          // The same lane issues the MMAs and the commit that tracks them.
+          for (int k = 0; k < ksteps; ++k) {
+            // Advancing 32 bytes along the row = 2 units of 16 bytes in the descriptor address.
+            mma_i8(tmem_acc, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (accumulate | (uint32_t)k));
+          }
+          mma_commit(smem_u32(&ctl.empty[s]));
+          if (kb == kb_end - 1) mma_commit(smem_u32(&ctl.tmem_full));
         }
-        mma_commit(smem_u32(&ctl.empty[s]));
+        accumulate = 1;
+        adesc += a_step;
+        bdesc += b_step;
+        if (++s == stages) {
+          s = 0;
+          ph ^= 1u;
+          adesc = adesc0;
+          bdesc = bdesc0;
+        }
       }
-      if (ok) mma_commit(smem_u32(&ctl.tmem_full));
     }
     __syncwarp();
   } else {
     // ---------------------------------------------------------------- gather + epilogue warps
-    const int quad = warp & 3;               // TMEM lane quadrant this warp may read
-    const int row = quad * 32 + lane;        // accumulator row = A-tile row
-    const long long m = (long long)m0 + row;
-    const bool row_valid = m < args.Mg;
+    const int quad = warp & 3;          // TMEM lane quadrant this warp may read
+    const int half = (warp - 2) >> 2;   // two warps share a quadrant and split the columns / chunks
+    const int row = quad * 32 + lane;   // accumulator row = A-tile row
+    const unsigned m = (unsigned)m0 + (unsigned)row;
+    const bool row_valid = m < (unsigned)args.Mg;
     int n_img = 0, pq = 0;
     if (row_valid) {
-      n_img = (int)(m / args.PQ);
-      pq = (int)(m - (long long)n_img * args.PQ);
+      n_img = (int)(m / (unsigned)args.PQ);
+      pq = (int)(m - (unsigned)n_img * (unsigned)args.PQ);
     }
     bool ok = true;
 
     if (AMODE == A_GATHER) {
-      // Stencil unroll formed in place: this thread writes row `row` of the A tile, 128 bytes
-      // per stage, in the 128-byte swizzled order the MMA descriptor expects (16-byte chunk j
-      // of row r lives at chunk position j ^ (r & 7)).
+      // Stencil unroll formed in place: this thread writes half of row `row` of the A tile (four
+      // 16-byte chunks per stage) in the 128-byte swizzled order the MMA descriptor expects
+      // (chunk j of row r lives at chunk position j ^ (r & 7)).
       const int p = pq / args.Q, q = pq - p * args.Q;
       const int h0 = row_valid ? p * args.stride_h - args.pad_h : -(1 << 29);
       const int w0 = q * args.stride_w - args.pad_w;
-      const int8_t* base =
-          args.x + n_img * args.x_stride_n + (long long)(row_valid ? h0 : 0) * args.x_stride_h + (long long)w0 * args.x_stride_w;
+      const int8_t* base = args.x + n_img * args.x_stride_n + (long long)(row_valid ? h0 : 0) * args.x_stride_h +
+                           (long long)w0 * args.x_stride_w;
       const uint32_t row_off = (uint32_t)row * 128u;
       const uint32_t xr = (uint32_t)(row & 7);
-      int it = 0;
-      for (int kb = kb_begin; kb < kb_end; ++kb, ++it) {
-        const int s = it % stages;
-        const uint32_t ph = (uint32_t)(it / stages) & 1u;
+      int s = 0;
+      uint32_t ph = 0;
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
         if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) {
           ok = false;
           break;
         }
         const uint32_t a_row = a_base + s * a_stage_bytes + row_off;
         const int chunks = (kb == args.num_kb - 1) ? args.ksteps_last * 2 : 8;
-        for (int j = 0; j < chunks; ++j) {
-          uint32_t wv[4] = {0, 0, 0, 0};
-          const GatherEntry* te = s_table + kb * 128 + j * 16;
+        const GatherEntry* te = s_table + kb * 128 + half * 64;
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const GatherEntry g = te[e];
-            const int h = h0 + g.dh, ww = w0 + g.dw;
-            uint32_t v = 0;
-            if (g.off >= 0 && (unsigned)h < (unsigned)args.H && (unsigned)ww < (unsigned)args.W)
-              v = (uint8_t)__ldg(base + g.off);
-            wv[e >> 2] |= v << (8 * (e & 3));
+        for (int jj = 0; jj < 4; ++jj) {
+          const int j = half * 4 + jj;
+          if (j < chunks) {
+            uint32_t wv[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const GatherEntry g = te[jj * 16 + e];
+              const int h = h0 + g.dh, ww = w0 + g.dw;
+              uint32_t v = 0;
+              if (g.off >= 0 && (unsigned)h < (unsigned)args.H && (unsigned)ww < (unsigned)args.W)
+                v = (uint8_t)__ldg(base + g.off);
+              wv[e >> 2] |= v << (8 * (e & 3));
+            }
+            const uint32_t dst = a_row + ((((uint32_t)j) ^ xr) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]),
+                         "r"(wv[3]));
           }
-          const uint32_t dst = a_row + ((((uint32_t)j) ^ xr) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]),
-                       "r"(wv[3])
-                       : "memory");
         }
-        // Make the generic-proxy writes visible to the tensor core's async proxy, then signal.
+        // Make the generic-proxy writes visible to the tensor core's async proxy, then one lane
+        // signals for the whole warp.
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(smem_u32(&ctl.full[s]));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctl.full[s]));
+        if (++s == stages) {
+          s = 0;
+          ph ^= 1u;
+        }
       }
     }
 
@@ -309,72 +472,19 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
     if (ok) ok = mbar_wait(smem_u32(&ctl.tmem_full), 0u, &ctl, args.status);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
-      const uint32_t taddr_row = tmem_acc + ((uint32_t)(quad * 32) << 16);
-      const bool split = args.split_k > 1;
-      const bool nhwc = args.out_layout == B2C_LAYOUT_NHWC;
-      const int K = args.K;
       // Output index of (m, k): NKPQ -> (n*K + k)*PQ + pq ; NPQK -> m*K + k.
-      const long long base_nkpq = (long long)n_img * K * args.PQ + pq;
-      const long long base_npqk = m * K;
-      for (int c0 = 0; c0 < args.tile_n; c0 += 16) {
-        int32_t v[16];
-        __syncwarp();
-        tmem_ld16(taddr_row + (uint32_t)c0, v);  // warp-collective: executed by all lanes
-        if (!row_valid) continue;
-        const int kbase = n0 + c0;
-        if (kbase >= K) continue;
-        if (split) {
-          // Partial sums of the reduction slices meet in global memory; integer addition is
-          // associative, so the order of arrival does not change the result.
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int k = kbase + j;
-            if (k < K) {
-              const long long o = nhwc ? base_npqk + k : base_nkpq + (long long)k * args.PQ;
-              atomicAdd(args.acc + o, v[j]);
-            }
-          }
-        } else if (!nhwc) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int k = kbase + j;
-            if (k < K) {
-              const long long o = base_nkpq + (long long)k * args.PQ;
-              if (args.out_mode & B2C_OUT_I32) args.y32[o] = v[j];
-              if (args.out_mode & B2C_OUT_I8) args.y8[o] = requant(v[j], args.shift);
-            }
-          }
+      const long long base_nkpq = (long long)n_img * args.K * args.PQ + pq;
+      const long long base_npqk = (long long)m * args.K;
+      const int cols = args.tile_n >= 32 ? (args.tile_n >> 1) : 16;  // columns handled by this warp
+      const int c_begin = half * cols;
+      if (c_begin < args.tile_n) {
+        const uint32_t taddr = tmem_acc + ((uint32_t)(quad * 32) << 16) + (uint32_t)c_begin;
+        if ((cols & 31) == 0) {
+          for (int c = 0; c < cols; c += 32)
+            epilogue_columns<32>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk);
         } else {
-          const bool full16 = kbase + 16 <= K;
-          if (args.out_mode & B2C_OUT_I32) {
-            int32_t* dst = args.y32 + base_npqk + kbase;
-            if (full16 && (K & 3) == 0) {
-#pragma unroll
-              for (int j = 0; j < 16; j += 4)
-                *reinterpret_cast<int4*>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (kbase + j < K) dst[j] = v[j];
-            }
-          }
-          if (args.out_mode & B2C_OUT_I8) {
-            int8_t* dst = args.y8 + base_npqk + kbase;
-            if (full16 && (K & 15) == 0) {
-              uint32_t w[4];
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                w[j] = 0;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) w[j] |= (uint32_t)(uint8_t)requant(v[j * 4 + i], args.shift) << (8 * i);
-              }
-              *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (kbase + j < K) dst[j] = requant(v[j], args.shift);
-            }
-          }
+          for (int c = 0; c < cols; c += 16)
+            epilogue_columns<16>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk);
         }
       }
     }
@@ -383,12 +493,14 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   // ---------------------------------------------------------------- teardown
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (ctl.abort_flag && threadIdx.x == 0) {
+  if (ctl.abort_flag) {
     // Give copies that were already issued time to land before the shared memory is released.
-    const unsigned long long t0 = global_ns();
-    while (global_ns() - t0 < 50000ull) __nanosleep(1000);
+    if (threadIdx.x == 0) {
+      const unsigned long long t0 = global_ns();
+      while (global_ns() - t0 < 50000ull) __nanosleep(1000);
+    }
+    __syncthreads();
   }
-  __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(args.tmem_cols)
