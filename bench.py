@@ -174,9 +174,23 @@ class Instances:
             p.destroy()
 
 
-def time_steps(torch, fn, steps, warmup, dist=None):
+def max_over_ranks(torch, dist, value: float, device) -> float:
+    """MAX of a per-rank scalar over the process group (the job is as slow as its slowest rank)."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def time_steps(torch, fn, steps, warmup, dist=None, min_warm_s=0.2):
     for _ in range(warmup):
         fn()
+    # a step is a fraction of a millisecond: keep warming until the clocks have had time to ramp
+    t_end = time.perf_counter() + min_warm_s
+    while time.perf_counter() < t_end:
+        fn()
+        torch.cuda.synchronize()
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
@@ -187,12 +201,9 @@ def time_steps(torch, fn, steps, warmup, dist=None):
         fn()
     e1.record()
     torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
+    ms = max_over_ranks(torch, dist, e0.elapsed_time(e1), "cuda")
     if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.barrier()
-        ms = float(t.item())
     return ms
 
 
@@ -221,6 +232,40 @@ def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, grap
         "launches_per_call": launches,
     }
     return res
+
+
+def scaled_shape(cfg: ConvShape, peaks, target_us=50.0) -> ConvShape:
+    """Same per-image shape with the batch scaled until the roofline time reaches `target_us`."""
+    t, _ = roofline_time_us(cfg, peaks)
+    mult = max(1, int(np.ceil(target_us / t)))
+    return ConvShape(cfg.name + "_xN%d" % (cfg.N * mult), cfg.N * mult, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S,
+                     cfg.stride, cfg.pad, cfg.dilation, cfg.shift, cfg.out_mode)
+
+
+def measure_scaled(b2c, torch, cfg, peaks, steps=10):
+    """Secondary series: one large-batch problem per launch (working set beyond L2), whole path."""
+    big = scaled_shape(cfg, peaks)
+    d = b2c.make_desc(big.N, big.C, big.H, big.W, big.K, big.R, big.S, big.stride, big.pad, big.dilation, big.shift,
+                      0, 0, big.out_mode)
+    plan = b2c.Plan(d, b2c.POLICY_AUTO_TIMED)
+    emb = plan.info()
+    x = torch.randint(-128, 128, (big.N, big.C, big.H, big.W), dtype=torch.int8, device="cuda")
+    w = torch.randint(-128, 128, (big.K, big.C, big.R, big.S), dtype=torch.int8, device="cuda")
+    oshape = (big.N, big.K, big.P, big.Q)
+    y32 = torch.empty(oshape, dtype=torch.int32, device="cuda") if big.out_mode & 1 else None
+    y8 = torch.empty(oshape, dtype=torch.int8, device="cuda") if big.out_mode & 2 else None
+    ws = torch.empty(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
+    plan.set_weights(w)
+    ms = time_steps(torch, lambda: plan.run(x, y32, y8, ws), steps, 3, None, 0.05)
+    st = plan.device_status()
+    plan.destroy()
+    if st != 0:
+        raise RuntimeError("device status " + b2c.status_string(st))
+    us = ms * 1e3 / steps
+    t_roof, bound = roofline_time_us(big, peaks)
+    return {"shape": big.name, "us": us, "tops": 2.0 * big.macs / (us * 1e-6) / 1e12, "roofline_us": t_roof,
+            "bound": bound, "roofline_frac": t_roof / us, "bytes": big.algorithmic_bytes,
+            "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k}}
 
 
 def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=True):
@@ -274,10 +319,7 @@ def e2e_measure(b2c, torch, cfg, steps, warmup, dist=None):
         fn()
     torch.cuda.synchronize()
     sec = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([sec], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        sec = float(t.item())
+    sec = max_over_ranks(torch, dist, sec, "cuda")
     calls = steps * reps
     h2d = (x.nbytes + w.nbytes) * reps
     d2h = ((y32.nbytes if y32 is not None else 0) + (y8.nbytes if y8 is not None else 0)) * reps
@@ -415,6 +457,9 @@ def run_ours(args):
         for c in CONFIGS:
             r = measure_shape(b2c, torch, c, max(2, args.steps // 2), 3, peaks, policy if c is cfg else b2c.POLICY_AUTO_TIMED, None, graph)
             per_config.append(r)
+    scaled = None
+    if rank == 0 and not args.headline_only:
+        scaled = [measure_scaled(b2c, torch, c, peaks) for c in CONFIGS]
     cpu = cpu_baseline(cfg) if (rank == 0 and world == 1 and not args.no_cpu) else None
 
     if dist is not None:
@@ -438,6 +483,8 @@ def run_ours(args):
         line["cpu_baseline"] = cpu
     if per_config is not None:
         line["per_config"] = per_config
+    if scaled is not None:
+        line["scaled"] = scaled
     print(json.dumps(line))
     return 0
 

@@ -101,9 +101,11 @@ int b2c_out_shape(const b2c_conv_desc* desc, int32_t* P, int32_t* Q);
 int b2c_enumerate(const b2c_conv_desc* desc, b2c_embedding* out, int32_t cap, int32_t* count);
 
 /* Creates a plan for `desc` on the current device.  `policy_or_id` is a B2C_POLICY_* value or
- * an embedding id from b2c_enumerate.  AUTO_TIMED allocates temporary device buffers, runs
- * each candidate on `cuda_stream` and synchronises that stream.  The plan owns its packed
- * weights, lookup tables and a device status word; free it with b2c_plan_destroy. */
+ * an embedding id from b2c_enumerate.  AUTO_TIMED allocates temporary device buffers, captures
+ * each candidate's launches in a CUDA graph on a private stream, replays it and keeps the
+ * fastest; it synchronises with the device and must not be called while a stream of the calling
+ * thread is being captured.  `cuda_stream` is used for the buffer initialisation only.  The plan
+ * owns its packed weights, lookup tables and a device status word; free it with b2c_plan_destroy. */
 int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_stream, b2c_plan** out);
 
 /* Copies the chosen embedding (with device_us if it was timed) to *chosen. */

@@ -196,29 +196,53 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
   return B2C_OK;
 }
 
-int time_plan(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, cudaStream_t st, float* us) {
-  cudaEvent_t e0, e1;
-  CUDA_TRY(cudaEventCreate(&e0));
-  CUDA_TRY(cudaEventCreate(&e1));
-  const int warm = 3, iters = 20;
+// Device time of one run of `p`: the launches of `iters` runs are captured into a CUDA graph on a
+// private stream and the graph is replayed, so that host launch cost does not mask the kernels.
+int time_plan(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, float* us) {
+  const int iters = 10, replays = 3;
+  cudaStream_t st = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
   int rc = B2C_OK;
-  for (int i = 0; i < warm && rc == B2C_OK; ++i) rc = b2c_conv2d_int8_run(p, x, y32, y8, ws, st);
-  if (rc == B2C_OK) {
-    cudaEventRecord(e0, st);
-    for (int i = 0; i < iters && rc == B2C_OK; ++i) rc = b2c_conv2d_int8_run(p, x, y32, y8, ws, st);
-    cudaEventRecord(e1, st);
-    cudaError_t e = cudaEventSynchronize(e1);
-    if (e != cudaSuccess) {
-      set_last_cuda_error((int)e);
-      rc = B2C_E_CUDA;
-    } else {
-      float ms = 0;
-      cudaEventElapsedTime(&ms, e0, e1);
-      *us = ms * 1000.0f / iters;
+  cudaError_t e = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  if (e == cudaSuccess) {
+    // plain runs first: first-launch set-up (function attributes) must not happen under capture
+    for (int i = 0; i < 2 && rc == B2C_OK; ++i) rc = b2c_conv2d_int8_run(p, x, y32, y8, ws, st);
+    if (rc == B2C_OK) e = cudaStreamSynchronize(st);
+  }
+  if (e == cudaSuccess && rc == B2C_OK) {
+    e = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal);
+    if (e == cudaSuccess) {
+      for (int i = 0; i < iters && rc == B2C_OK; ++i) rc = b2c_conv2d_int8_run(p, x, y32, y8, ws, st);
+      cudaError_t e2 = cudaStreamEndCapture(st, &graph);
+      if (e2 != cudaSuccess) e = e2;
     }
   }
-  cudaEventDestroy(e0);
-  cudaEventDestroy(e1);
+  if (e == cudaSuccess && rc == B2C_OK) e = cudaGraphInstantiate(&exec, graph, 0);
+  if (e == cudaSuccess && rc == B2C_OK) {
+    e = cudaGraphLaunch(exec, st);  // warm
+    if (e == cudaSuccess) e = cudaEventRecord(e0, st);
+    for (int i = 0; i < replays && e == cudaSuccess; ++i) e = cudaGraphLaunch(exec, st);
+    if (e == cudaSuccess) e = cudaEventRecord(e1, st);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+    if (e == cudaSuccess) {
+      float ms = 0;
+      e = cudaEventElapsedTime(&ms, e0, e1);
+      *us = ms * 1000.0f / (iters * replays);
+    }
+  }
+  if (exec) cudaGraphExecDestroy(exec);
+  if (graph) cudaGraphDestroy(graph);
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (st) cudaStreamDestroy(st);
+  if (e != cudaSuccess) {
+    set_last_cuda_error((int)e);
+    return B2C_E_CUDA;
+  }
   if (rc == B2C_OK) {
     int32_t s = 0;
     rc = b2c_plan_device_status(p, &s);
@@ -324,6 +348,7 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
   }
   cudaMemsetAsync(x, 1, g.x_elems, st);
   cudaMemsetAsync(w, 1, g.w_elems, st);
+  cudaStreamSynchronize(st);
   int best = -1;
   float best_us = 0;
   for (size_t i = 0; i < all.size(); ++i) {
@@ -332,8 +357,9 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
     rc = create_plan_for(g, all[i], &p);
     if (rc != B2C_OK) break;
     rc = b2c_plan_set_weights(p, w, st);
+    if (rc == B2C_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = B2C_E_CUDA;
     float us = -1;
-    if (rc == B2C_OK) rc = time_plan(p, x, y32, y8, ws, st, &us);
+    if (rc == B2C_OK) rc = time_plan(p, x, y32, y8, ws, &us);
     b2c_plan_destroy(p);
     if (rc != B2C_OK) break;
     all[i].device_us = us;

@@ -38,8 +38,26 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+// The issue helpers below take `on`: the instruction is predicated on it instead of sitting in a
+// divergent branch, so the surrounding loop stays straight-line, warp-uniform code.
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes, uint32_t on) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %2, 0;\n"
+      "@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n}" ::"r"(bar),
+      "r"(bytes), "r"(on)
+      : "memory");
+}
+// Non-blocking phase test (never suspends the thread).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t done;
@@ -90,19 +108,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, SharedC
   return mbar_wait_slow(bar, parity, ctl, status);
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
+                                            uint32_t on) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-          dst),
-      "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %5, 0;\n"
+      "@q cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n}" ::
+          "r"(dst),
+      "l"(map), "r"(c0), "r"(c1), "r"(bar), "r"(on)
       : "memory");
 }
 __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n,
-                                                   uint32_t bar, uint16_t off_w, uint16_t off_h) {
+                                                   uint32_t bar, uint16_t off_w, uint16_t off_h, uint32_t on) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, "
-      "%5}], [%6], {%7, %8};" ::"r"(dst),
-      "l"(map), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"(off_w), "h"(off_h)
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %9, 0;\n"
+      "@q cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, "
+      "%5}], [%6], {%7, %8};\n}" ::"r"(dst),
+      "l"(map), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"(off_w), "h"(off_h), "r"(on)
       : "memory");
 }
 
@@ -128,16 +149,21 @@ __device__ __forceinline__ uint32_t make_idesc_i8(int n) {
 }
 
 __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                       uint32_t accumulate) {
+                                       uint32_t accumulate, uint32_t on) {
   asm volatile(
-      "{\n.reg .pred p;\n"
+      "{\n.reg .pred p, q;\n"
       "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      "setp.ne.b32 q, %5, 0;\n"
+      "@q tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(on)
       : "memory");
 }
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+__device__ __forceinline__ void mma_commit(uint32_t bar, uint32_t on) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(bar),
+      "r"(on)
+      : "memory");
 }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t* v) {
   asm volatile(
@@ -325,27 +351,22 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       uint32_t ph = 0;
       uint32_t a_dst = a_base, b_dst = b_base;
       int kcol = kb_begin * bk;  // column of the packed weight matrix = reduction offset in bytes
+      const uint32_t leader = elect_one() ? 1u : 0u;
       for (int kb = kb_begin; kb < kb_end; ++kb) {
         if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) break;
         const uint32_t full = smem_u32(&ctl.full[s]);
         if (AMODE == A_GATHER) {
-          if (elect_one()) {
-            mbar_arrive_expect_tx(full, b_stage_bytes);
-            tma_load_2d(b_dst, &tmap_b, kcol, n0, full);
-          }
+          mbar_arrive_expect_tx(full, b_stage_bytes, leader);
+          tma_load_2d(b_dst, &tmap_b, kcol, n0, full, leader);
         } else if (AMODE == A_TILED) {
-          if (elect_one()) {
-            mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes);
-            tma_load_2d(a_dst, &tmap_a, kcol, m0, full);
-            tma_load_2d(b_dst, &tmap_b, kcol, n0, full);
-          }
+          mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes, leader);
+          tma_load_2d(a_dst, &tmap_a, kcol, m0, full, leader);
+          tma_load_2d(b_dst, &tmap_b, kcol, n0, full, leader);
         } else {
-          if (elect_one()) {
-            mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes);
-            tma_load_im2col_4d(a_dst, &tmap_a, cb * bk, w_org, h_org, n_img, full, (uint16_t)(sx * args.dil_w),
-                               (uint16_t)(r * args.dil_h));
-            tma_load_2d(b_dst, &tmap_b, kcol, n0, full);
-          }
+          mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes, leader);
+          tma_load_im2col_4d(a_dst, &tmap_a, cb * bk, w_org, h_org, n_img, full, (uint16_t)(sx * args.dil_w),
+                             (uint16_t)(r * args.dil_h), leader);
+          tma_load_2d(b_dst, &tmap_b, kcol, n0, full, leader);
           if (++cb == args.kb_per_tap) {
             cb = 0;
             if (++sx == args.S) {
@@ -377,20 +398,15 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       int s = 0;
       uint32_t ph = 0;
       uint32_t accumulate = 0;
+      // The same lane issues every MMA and the commits that track them.
+      const uint32_t leader = elect_one() ? 1u : 0u;
+      bool ready = false;  // result of the look-ahead test of this stage's full barrier
       for (int kb = kb_begin; kb < kb_end; ++kb) {
-        if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status)) break;
+        if (!ready && !mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int ksteps = (kb == args.num_kb - 1) ? args.ksteps_last : args.ksteps_full;
-        if (elect_one()) {
-          // The same lane issues the MMAs and the commit that tracks them.
-          for (int k = 0; k < ksteps; ++k) {
-            // Advancing 32 bytes along the row = 2 units of 16 bytes in the descriptor address.
-            mma_i8(tmem_acc, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (accumulate | (uint32_t)k));
-          }
-          mma_commit(smem_u32(&ctl.empty[s]));
-          if (kb == kb_end - 1) mma_commit(smem_u32(&ctl.tmem_full));
-        }
-        accumulate = 1;
+        const int s_cur = s;
+        const uint64_t a_cur = adesc, b_cur = bdesc;
         adesc += a_step;
         bdesc += b_step;
         if (++s == stages) {
@@ -399,6 +415,16 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
           adesc = adesc0;
           bdesc = bdesc0;
         }
+        // Look ahead: test the next stage's barrier now so that its latency overlaps the MMA issue.
+        ready = (kb + 1 < kb_end) && mbar_test_wait(smem_u32(&ctl.full[s]), ph);
+        for (int k = 0; k < ksteps; ++k) {
+          // Advancing 32 bytes along the row = 2 units of 16 bytes in the descriptor address.
+          mma_i8(tmem_acc, a_cur + (uint64_t)(2 * k), b_cur + (uint64_t)(2 * k), idesc, (accumulate | (uint32_t)k),
+                 leader);
+        }
+        mma_commit(smem_u32(&ctl.empty[s_cur]), leader);
+        if (kb == kb_end - 1) mma_commit(smem_u32(&ctl.tmem_full), leader);
+        accumulate = 1;
       }
     }
     __syncwarp();
