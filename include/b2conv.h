@@ -162,6 +162,23 @@ int b2c_pack_activations(const int8_t* x_nchw_dev, int8_t* out_dev, int N, int C
                          void* cuda_stream);
 int b2c_im2col(const b2c_conv_desc* desc, const int8_t* x_dev, int8_t* a_dev, int K_pad, void* cuda_stream);
 
+/* b2c_im2col for callers that cannot allocate device memory (the paper has no counterpart; this
+ * is a property of the library, not of the method).  b2c_im2col puts its lookup table in a
+ * temporary cudaMalloc buffer; code that runs where allocation is forbidden or impossible - inside
+ * a region a framework has frozen against allocation, in a latency-critical loop that must stay
+ * off the allocator, or in a process that has given all device memory to another pool - can call
+ * this instead.  Same arguments, same output, but the table lives in a fixed 128 KB device array
+ * inside the library (held by every GPU that loads it, until the process exits) and is filled by
+ * a small kernel on `cuda_stream`; the call makes no cudaMalloc / cudaFree and does not
+ * synchronise.  Limits and rules:
+ *   - K_pad <= 16384, else B2C_E_WORKSPACE_TOO_SMALL (nothing is launched);
+ *   - the first call on a device looks up the array's device address (cudaGetSymbolAddress):
+ *     make that first call outside any stream capture;
+ *   - all calls on a device share the one array and each call rewrites the part it uses, so two
+ *     calls whose kernels can overlap on the GPU (different streams, no ordering) race: order
+ *     them on one stream or with events. */
+int b2c_im2col_noalloc(const b2c_conv_desc* desc, const int8_t* x_dev, int8_t* a_dev, int K_pad, void* cuda_stream);
+
 const char* b2c_status_string(int status);
 
 /* The last CUDA error code (cudaError_t or CUresult as int) seen by this thread's failing call. */

@@ -25,7 +25,8 @@ VARIANT_NAMES = {0: "channel_pack_tma_im2col", 1: "im2col_explicit", 2: "im2col_
 EXPORTS = [
     "b2c_out_shape", "b2c_enumerate", "b2c_plan_create", "b2c_plan_info", "b2c_plan_workspace_bytes",
     "b2c_plan_set_weights", "b2c_conv2d_int8_run", "b2c_conv2d_int8", "b2c_conv2d_int8_host",
-    "b2c_plan_device_status", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_status_string",
+    "b2c_plan_device_status", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
+    "b2c_status_string",
     "b2c_last_cuda_error",
 ]
 
@@ -87,6 +88,7 @@ def load():
     lib.b2c_plan_destroy.restype = None
     lib.b2c_pack_activations.argtypes = [vp, vp] + [i32] * 5 + [vp]
     lib.b2c_im2col.argtypes = [pd, vp, vp, i32, vp]
+    lib.b2c_im2col_noalloc.argtypes = [pd, vp, vp, i32, vp]
     lib.b2c_status_string.argtypes = [i32]
     lib.b2c_status_string.restype = ctypes.c_char_p
     lib.b2c_last_cuda_error.argtypes = []
@@ -220,3 +222,11 @@ def pack_activations(x, out, C_pad: int, stream=None):
 
 def im2col(desc: ConvDesc, x, a, K_pad: int, stream=None):
     _check(load().b2c_im2col(ctypes.byref(desc), _dptr(x), _dptr(a), K_pad, _stream_ptr(stream)), "b2c_im2col")
+
+
+def im2col_noalloc(desc: ConvDesc, x, a, K_pad: int, stream=None):
+    """Same result as ``im2col`` without any device allocation inside the library (fixed 128 KB
+    table, K_pad <= 16384); for callers that run where cudaMalloc is off limits.  Calls that may
+    overlap on the GPU must be ordered by the caller."""
+    _check(load().b2c_im2col_noalloc(ctypes.byref(desc), _dptr(x), _dptr(a), K_pad, _stream_ptr(stream)),
+           "b2c_im2col_noalloc")

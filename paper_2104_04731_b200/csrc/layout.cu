@@ -193,3 +193,106 @@ cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, l
 }
 
 }  // namespace b2c
+
+// ---------------------------------------------------------------------------------------------
+// Stencil unroll for callers that cannot allocate device memory.
+//
+// b2c_im2col builds its lookup table on the host and puts it in a temporary cudaMalloc buffer.
+// Some callers cannot do that: code running inside a stream capture or under a framework's
+// "no allocation from here on" rule, real-time loops that must not touch the allocator, or
+// processes whose memory pool was handed to another library in full.  For them the table lives in
+// the fixed device array below (128 KB, resident on every GPU that loads the library until the
+// process exits) and is filled by a small kernel on the caller's stream.
+// ---------------------------------------------------------------------------------------------
+namespace b2c {
+namespace {
+
+constexpr int kStaticTableEntries = 16384;  // largest padded reduction length C*R*S the static table can hold
+static __device__ __align__(256) GatherEntry g_static_table[kStaticTableEntries];
+
+// Writes entries [0, K_pad): (c, r, s) -> element offset and displacement; -1 past C*R*S.  Every
+// entry a later im2col launch reads is rewritten here, so nothing of an earlier call survives.
+__global__ void fill_static_table_kernel(GatherEntry* table, int K_pad, int Kg, int R, int S, int dil_h, int dil_w,
+                                         long long stride_c, long long stride_h, long long stride_w) {
+  for (int kg = blockIdx.x * blockDim.x + threadIdx.x; kg < K_pad; kg += gridDim.x * blockDim.x) {
+    GatherEntry e;
+    if (kg < Kg) {
+      const int s = kg % S;
+      const int cr = kg / S;
+      const int r = cr % R;
+      const int c = cr / R;
+      e.off = (int32_t)(c * stride_c + (long long)r * dil_h * stride_h + (long long)s * dil_w * stride_w);
+      e.dh = (int16_t)(r * dil_h);
+      e.dw = (int16_t)(s * dil_w);
+    } else {
+      e.off = -1;
+      e.dh = 0;
+      e.dw = 0;
+    }
+    table[kg] = e;
+  }
+}
+
+// Device address of g_static_table, looked up once per device.  In host code the array's name is
+// only a handle for the runtime; the address a kernel can use comes from cudaGetSymbolAddress.
+constexpr int kMaxDevices = 64;
+GatherEntry* g_static_table_addr[kMaxDevices] = {};
+
+int static_table_address(GatherEntry** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    set_last_cuda_error((int)(e != cudaSuccess ? e : cudaErrorInvalidDevice));
+    return B2C_E_CUDA;
+  }
+  GatherEntry* p = __atomic_load_n(&g_static_table_addr[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_table);
+    if (e != cudaSuccess || !p) {
+      set_last_cuda_error((int)e);
+      return B2C_E_CUDA;
+    }
+    __atomic_store_n(&g_static_table_addr[dev], p, __ATOMIC_RELEASE);
+  }
+  *out = p;
+  return B2C_OK;
+}
+
+}  // namespace
+}  // namespace b2c
+
+extern "C" int b2c_im2col_noalloc(const b2c_conv_desc* desc, const int8_t* x, int8_t* a, int K_pad, void* cuda_stream) {
+  using namespace b2c;
+  if (!desc || !x || !a) return B2C_E_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(a) & 15)) return B2C_E_INVALID_ARG;
+  b2c_conv_desc d = *desc;
+  if ((d.out_mode & 3) == 0) d.out_mode = B2C_OUT_I32;
+  Geom g;
+  int rc = resolve_geom(&d, &g);
+  if (rc != B2C_OK) return rc;
+  if (K_pad < g.Kg || (K_pad % 16) != 0) return B2C_E_INVALID_ARG;
+  if (K_pad > kStaticTableEntries) return B2C_E_WORKSPACE_TOO_SMALL;
+  if ((long long)(d.R - 1) * d.dil_h >= 32768 || (long long)(d.S - 1) * d.dil_w >= 32768 ||
+      (long long)d.C * d.H * d.W >= 0x7FFFFFFFLL)
+    return B2C_E_UNSUPPORTED;
+  GatherEntry* table = nullptr;
+  rc = static_table_address(&table);
+  if (rc != B2C_OK) return rc;
+  const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
+  const long long sc = nchw ? (long long)d.H * d.W : 1;
+  const long long sh = nchw ? d.W : (long long)d.W * d.C;
+  const long long sw = nchw ? 1 : d.C;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  fill_static_table_kernel<<<(K_pad + 255) / 256, 256, 0, st>>>(table, K_pad, g.Kg, d.R, d.S, d.dil_h, d.dil_w, sc, sh,
+                                                                 sw);
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess)
+    e = launch_im2col(x, a, table, g.Mg, g.PQ, g.Q, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
+                      (long long)d.C * d.H * d.W, (int)sh, (int)sw, K_pad, st);
+  if (e != cudaSuccess) {
+    set_last_cuda_error((int)e);
+    return B2C_E_CUDA;
+  }
+  return B2C_OK;
+}
+
