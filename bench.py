@@ -410,18 +410,25 @@ def run_ours(args):
     b2c.load()
     peaks = load_peaks()
     cfg = CONFIGS[args.config]
+    if args.scaled:
+        cfg = scaled_shape(cfg, peaks)
     policy = b2c.POLICY_AUTO_TIMED if args.embedding is None else args.embedding
+    if args.pick:
+        v, tn, sk = (int(t) for t in args.pick.split(","))
+        d0 = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
+                           0, 0, cfg.out_mode)
+        policy = next(e.id for e in b2c.enumerate_embeddings(d0) if (e.variant, e.tile_n, e.split_k) == (v, tn, sk))
     graph = not args.no_graph
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     # ---- headline: whole path, device-resident inputs ------------------------------------------
-    G = instances_for(cfg)
+    G = args.instances if args.instances else instances_for(cfg)
     inst = Instances(b2c, torch, cfg, G, policy)
     if graph:
         inst.capture(torch)
-    ms = time_steps(torch, inst.step, args.steps, args.warmup, dist)
+    ms = time_steps(torch, inst.step, args.steps, args.warmup, dist, args.min_warm_s)
     inst.check_status(b2c)
     clocks = sampler.stop() if rank == 0 else None
     emb = inst.emb
@@ -432,7 +439,9 @@ def run_ours(args):
     inst.destroy()
 
     # ---- the dominant kernel alone (the paper's "Op." column) for the roofline -------------------
-    op = op_only(b2c, torch, cfg, emb.variant, emb.tile_n, emb.split_k, args.steps, args.warmup, graph)
+    op = None
+    if not args.no_op_pass:
+        op = op_only(b2c, torch, cfg, emb.variant, emb.tile_n, emb.split_k, args.steps, args.warmup, graph)
     t_roof, bound = roofline_time_us(cfg, peaks)
     op_us = op["us"] if op else per_call_us
     if bound == "tensor":
@@ -447,15 +456,18 @@ def run_ours(args):
                 if bound == "tensor" else peaks["source"] + " copy bandwidth"}
 
     # ---- end to end through the host-buffer call ----------------------------------------------------
-    e = e2e_measure(b2c, torch, cfg, max(1, min(args.steps, 5)), 1, dist)
-    e2e = {"value": world * e["calls"] * ops / e["sec"] / 1e12, "unit": UNIT,
-           "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"]}
+    e2e = None
+    if not args.no_e2e:
+        e = e2e_measure(b2c, torch, cfg, max(1, min(args.steps, 5)), 1, dist)
+        e2e = {"value": world * e["calls"] * ops / e["sec"] / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"]}
 
     per_config = None
     if rank == 0 and not args.headline_only:
         per_config = []
         for c in CONFIGS:
-            r = measure_shape(b2c, torch, c, max(2, args.steps // 2), 3, peaks, policy if c is cfg else b2c.POLICY_AUTO_TIMED, None, graph)
+            r = measure_shape(b2c, torch, c, max(2, args.steps // 2), 3, peaks,
+                              policy if c is cfg else b2c.POLICY_AUTO_TIMED, None, graph)
             per_config.append(r)
     scaled = None
     if rank == 0 and not args.headline_only:
@@ -499,7 +511,13 @@ def main():
     ap.add_argument("--embedding", type=int, default=None, help="embedding id; default: timed selection")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--headline-only", action="store_true")
+    ap.add_argument("--headline-only", action="store_true", help="skip the per-shape and scaled-batch series")
+    ap.add_argument("--pick", default=None, help="embedding as variant,tile_n,split_k (instead of an id)")
+    ap.add_argument("--scaled", action="store_true", help="use the batch-scaled version of the shape as the workload")
+    ap.add_argument("--instances", type=int, default=0, help="instances per step (default: enough to exceed L2)")
+    ap.add_argument("--min-warm-s", type=float, default=0.2, help="extra time-based warm-up before the timed steps")
+    ap.add_argument("--no-op-pass", action="store_true", help="skip the separate pass that times the MMA kernel alone")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end pass")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
