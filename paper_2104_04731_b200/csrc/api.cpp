@@ -141,9 +141,16 @@ void fill_common_args(b2c_plan* p) {
     a.kb_per_tap = 1;
   }
   // Pipeline depth: as many stages as the reduction slice has blocks, at most 6, within 160 KB.
+  // When the grid has more blocks than the machine has SMs, stay within 100 KB (but keep at least
+  // two stages) so that two blocks are resident per SM: one block's epilogue and set-up then
+  // overlap the other's main loop.
   int per_cta_kb = (a.num_kb + a.split_k - 1) / a.split_k;
   int stages = std::min(6, std::max(1, per_cta_kb));
-  while (stages > 1 && (size_t)stages * (kTileM + a.tile_n) * a.bk > 160 * 1024) --stages;
+  const long long ctas = ((p->g.Mg + kTileM - 1) / kTileM) * ((d.K + a.tile_n - 1) / a.tile_n) * a.split_k;
+  const size_t budget = ctas > kNumSMs ? 100 * 1024 : 160 * 1024;
+  const size_t stage_bytes = (size_t)(kTileM + a.tile_n) * a.bk;
+  while (stages > 2 && (size_t)stages * stage_bytes > budget) --stages;
+  while (stages > 1 && (size_t)stages * stage_bytes > 160 * 1024) --stages;
   a.stages = stages;
 }
 

@@ -9,68 +9,206 @@ namespace b2c {
 
 namespace {
 
-constexpr int kPackC = 64;   // channels per tile
-constexpr int kPackHW = 64;  // pixels per tile
-constexpr int kPackPitch = kPackHW + 4;
+constexpr int kPackThreads = 256;
+constexpr int kPackMaxC = 128;  // channels per tile (64 when the padded channel count is below 128)
+constexpr int kPackMaxP = 256;  // pixels per tile
+constexpr int kPackSmem = kPackMaxC * (kPackMaxP + 4) + (kPackMaxC / 16) * 16;
 
-// One block moves a [64 channels] x [64 pixels] tile of one image through shared memory:
-// reads run along the pixel axis of NCHW, writes along the channel axis of NHWC in 16-byte
-// vectors.  Channels >= C are written as zeros.
-template <bool kVec4>
-__global__ void __launch_bounds__(256) pack_activations_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ out,
-                                                               int C, int HW, int C_pad, int hw_tiles) {
-  __shared__ __align__(16) uint8_t tile[kPackC * kPackPitch];
+// One block moves a [CT channels] x [PT pixels] tile of one image through shared memory.
+// Reads run along the pixel axis of NCHW in VEC-byte vectors (VEC = 16 or 4 when H*W allows the
+// alignment, else 1) with many loads in flight per thread; the tile is kept as rows of `pitch`
+// bytes (pitch/4 odd) with each group of 16 rows skewed by 16 bytes, which makes the transposing
+// reads below conflict free.  Writes run along the channel axis of NHWC: a thread takes 16
+// channels of 4 consecutive pixels as 16 words, transposes them in registers with byte permutes
+// and stores four 16-byte vectors; the 8 (or 4) threads of one pixel cover 128 (or 64) contiguous
+// bytes.  Channels >= C are written as zeros.
+template <int VEC>
+__global__ void __launch_bounds__(kPackThreads) pack_activations_kernel(const int8_t* __restrict__ x,
+                                                                        int8_t* __restrict__ out, int C, int HW,
+                                                                        int C_pad, int hw_tiles, int CT, int PT) {
+  __shared__ __align__(16) uint8_t tile[kPackSmem];
   const int n = blockIdx.x / hw_tiles;
-  const int c0 = blockIdx.y * kPackC;
-  const int hw0 = (blockIdx.x - n * hw_tiles) * kPackHW;
+  const int c0 = blockIdx.y * CT;
+  const int hw0 = (blockIdx.x - n * hw_tiles) * PT;
   const int t = threadIdx.x;
-  const int8_t* xin = x + (size_t)n * C * HW;
-  if (kVec4) {
-    // 16 threads cover one channel row (4 pixels each), 16 rows per pass.
-    const int hq = (t & 15) * 4;
+  const int pitch = PT + 4;
+  const int8_t* xin = x + ((size_t)n * C + c0) * HW + hw0;
+  const int rows = min(CT, C - c0);  // channels that exist; the rest of the tile is zero padding
+
+  // ---- load ----
+  if constexpr (VEC >= 4) {
+    constexpr int NW = VEC / 4;  // words per vector
+    const int wpr = PT >> 2;     // words per row
+    const int vecs = CT * wpr / NW;
+#pragma unroll 8
+    for (int i = t; i < vecs; i += kPackThreads) {
+      const int wi = i * NW;
+      const int row = wi / wpr;
+      const int hw = (wi - row * wpr) * 4;
+      uint32_t v[NW];
 #pragma unroll
-    for (int pass = 0; pass < kPackC / 16; ++pass) {
-      const int cl = pass * 16 + (t >> 4);
-      const int c = c0 + cl;
-      uint32_t v = 0;
-      if (c < C) {
-        const int hw = hw0 + hq;
-        if (hw + 3 < HW) {
-          v = *reinterpret_cast<const uint32_t*>(xin + (size_t)c * HW + hw);
+      for (int k = 0; k < NW; ++k) v[k] = 0;
+      if (row < rows) {
+        const int8_t* src = xin + (size_t)row * HW + hw;
+        if (hw0 + hw + VEC <= HW) {
+          if constexpr (VEC == 16) {
+            const uint4 q = *reinterpret_cast<const uint4*>(src);
+            v[0] = q.x;
+            v[NW - 3] = q.y;
+            v[NW - 2] = q.z;
+            v[NW - 1] = q.w;
+          } else {
+            v[0] = *reinterpret_cast<const uint32_t*>(src);
+          }
         } else {
-          for (int i = 0; i < 4; ++i)
-            if (hw + i < HW) v |= (uint32_t)(uint8_t)xin[(size_t)c * HW + hw + i] << (8 * i);
+          for (int b = 0; b < VEC; ++b)
+            if (hw0 + hw + b < HW) v[b >> 2] |= (uint32_t)(uint8_t)src[b] << (8 * (b & 3));
         }
       }
-      *reinterpret_cast<uint32_t*>(&tile[cl * kPackPitch + hq]) = v;
+      uint32_t* dst = reinterpret_cast<uint32_t*>(&tile[row * pitch + (row >> 4) * 16 + hw]);
+#pragma unroll
+      for (int k = 0; k < NW; ++k) dst[k] = v[k];
     }
   } else {
-    const int hl = t & 63;
-#pragma unroll
-    for (int pass = 0; pass < kPackC / 4; ++pass) {
-      const int cl = pass * 4 + (t >> 6);
-      const int c = c0 + cl;
+    const int total = CT * PT;
+#pragma unroll 8
+    for (int i = t; i < total; i += kPackThreads) {
+      const int row = i / PT;
+      const int hw = i - row * PT;
       uint8_t v = 0;
-      if (c < C && hw0 + hl < HW) v = (uint8_t)xin[(size_t)c * HW + hw0 + hl];
-      tile[cl * kPackPitch + hl] = v;
+      if (row < rows && hw0 + hw < HW) v = (uint8_t)xin[(size_t)row * HW + hw];
+      tile[row * pitch + (row >> 4) * 16 + hw] = v;
     }
   }
   __syncthreads();
-  // Thread -> (pixel, 16-channel chunk); 4 chunks per pixel.
-  const int pl = t >> 2;
-  const int ch = (t & 3) * 16;
-  const int hw = hw0 + pl;
-  if (hw < HW && c0 + ch < C_pad) {
-    uint32_t w[4];
+
+  // ---- transpose in registers and store ----
+  const int chunks = CT >> 4;            // 16-channel chunks per pixel in this tile
+  const int items = (PT >> 2) * chunks;  // (group of 4 pixels, chunk)
+  for (int it = t; it < items; it += kPackThreads) {
+    const int ch = it % chunks;
+    const int pg = it / chunks;
+    const int hw = hw0 + pg * 4;
+    if (hw >= HW || c0 + ch * 16 >= C_pad) continue;
+    uint32_t w[16];
+    const uint8_t* src = &tile[(ch * 16) * pitch + ch * 16 + pg * 4];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) w[i] = *reinterpret_cast<const uint32_t*>(src + i * pitch);
+    int8_t* dst = out + ((size_t)n * HW + hw) * C_pad + c0 + ch * 16;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      uint32_t v = 0;
+      if (hw + j < HW) {
+        uint32_t o[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) v |= (uint32_t)tile[(ch + j * 4 + i) * kPackPitch + pl] << (8 * i);
-      w[j] = v;
+        for (int k = 0; k < 4; ++k) {
+          const uint32_t lo = __byte_perm(w[4 * k], w[4 * k + 1], j | ((4 + j) << 4));
+          const uint32_t hi = __byte_perm(w[4 * k + 2], w[4 * k + 3], j | ((4 + j) << 4));
+          o[k] = __byte_perm(lo, hi, 0x5410);
+        }
+        *reinterpret_cast<uint4*>(dst + (size_t)j * C_pad) = make_uint4(o[0], o[1], o[2], o[3]);
+      }
     }
-    uint4 o = make_uint4(w[0], w[1], w[2], w[3]);
-    *reinterpret_cast<uint4*>(out + ((size_t)n * HW + hw) * C_pad + c0 + ch) = o;
+  }
+}
+
+// Bulk-copy variant of the activation pack for the common aligned cases.  The tile's rows reach
+// shared memory by asynchronous bulk copies (cp.async.bulk) that complete on an mbarrier, so the
+// load phase costs no per-byte instructions and keeps whole tiles in flight:
+//   group mode (kRowMode = false): the tile spans all H*W pixels of 16-channel groups, and every
+//     group (16*H*W contiguous bytes of NCHW) is fetched by one copy;
+//   row mode (kRowMode = true): H*W is a multiple of 16 and every channel row segment of PT pixels
+//     is fetched by one copy.
+// Groups of 16 rows are spaced 16 bytes further apart than their size, which makes the
+// transposing word reads of the store phase conflict free.  The store phase is the same register
+// transpose as in pack_activations_kernel.
+constexpr int kBulkWaitTries = 1 << 22;
+
+template <bool kRowMode>
+__global__ void __launch_bounds__(kPackThreads) pack_activations_bulk_kernel(const int8_t* __restrict__ x,
+                                                                             int8_t* __restrict__ out, int C, int HW,
+                                                                             int C_pad, int hw_tiles, int CT, int PT) {
+  extern __shared__ __align__(128) uint8_t btile[];
+  __shared__ __align__(8) unsigned long long bar;
+  const int n = blockIdx.x / hw_tiles;
+  const int c0 = blockIdx.y * CT;
+  const int hw0 = (blockIdx.x - n * hw_tiles) * PT;
+  const int t = threadIdx.x;
+  const int npx = min(PT, HW - hw0);        // pixels of this tile
+  const int rows = max(0, min(CT, C - c0));  // channels that exist (a multiple of 16)
+  const int rp = kRowMode ? PT : HW;         // row pitch in shared memory
+  const int gs = 16 * rp + 16;               // group stride
+  const uint32_t bar_a = (uint32_t)__cvta_generic_to_shared(&bar);
+  const uint32_t tile_a = (uint32_t)__cvta_generic_to_shared(btile);
+  if (t == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const uint32_t bytes = (uint32_t)rows * (uint32_t)npx;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"(bytes) : "memory");
+  }
+  __syncthreads();
+  const int8_t* xin = x + ((size_t)n * C + c0) * HW + hw0;
+  if (kRowMode) {
+    if (t < rows) {
+      const uint32_t dst = tile_a + (uint32_t)((t >> 4) * gs + (t & 15) * rp);
+      asm volatile(
+          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+          "l"(xin + (size_t)t * HW), "r"((uint32_t)npx), "r"(bar_a)
+          : "memory");
+    }
+  } else {
+    if (t < (rows >> 4)) {
+      const uint32_t dst = tile_a + (uint32_t)(t * gs);
+      asm volatile(
+          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+          "l"(xin + (size_t)t * 16 * HW), "r"((uint32_t)(16 * HW)), "r"(bar_a)
+          : "memory");
+    }
+  }
+  // Bounded wait for the copies; on expiry the block gives up (its part of the output stays unwritten).
+  bool done = false;
+  for (int tries = 0; tries < kBulkWaitTries && !done; ++tries) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar_a)
+        : "memory");
+    done = ok != 0;
+  }
+  if (!done) return;
+
+  const int chunks = CT >> 4;
+  const int items = ((npx + 3) >> 2) * chunks;
+  for (int it = t; it < items; it += kPackThreads) {
+    const int ch = it % chunks;
+    const int pg = it / chunks;
+    const int hw = hw0 + pg * 4;
+    if (c0 + ch * 16 >= C_pad) continue;
+    uint32_t w[16];
+    if (ch * 16 < rows) {
+      const uint8_t* src = btile + ch * gs + pg * 4;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) w[i] = *reinterpret_cast<const uint32_t*>(src + i * rp);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) w[i] = 0;
+    }
+    int8_t* dst = out + ((size_t)n * HW + hw) * C_pad + c0 + ch * 16;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (hw + j < HW) {
+        uint32_t o[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const uint32_t lo = __byte_perm(w[4 * k], w[4 * k + 1], j | ((4 + j) << 4));
+          const uint32_t hi = __byte_perm(w[4 * k + 2], w[4 * k + 3], j | ((4 + j) << 4));
+          o[k] = __byte_perm(lo, hi, 0x5410);
+        }
+        *reinterpret_cast<uint4*>(dst + (size_t)j * C_pad) = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+    }
   }
 }
 
@@ -154,13 +292,31 @@ int grid_for(long long total, int block) {
 cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, int H, int W, int C_pad,
                                     cudaStream_t st) {
   const int HW = H * W;
-  const int hw_tiles = (HW + kPackHW - 1) / kPackHW;
-  dim3 grid((unsigned)hw_tiles * (unsigned)N, (C_pad + kPackC - 1) / kPackC, 1);
-  const bool vec4 = (HW % 4 == 0) && ((reinterpret_cast<uintptr_t>(x) & 3) == 0);
-  if (vec4)
-    pack_activations_kernel<true><<<grid, 256, 0, st>>>(x, out, C, HW, C_pad, hw_tiles);
+  const int CT = C_pad >= 128 ? 128 : 64;
+  const bool a16 = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+  // Bulk-copy kernels: channels in whole groups of 16 and either the whole image per tile
+  // (H*W <= 256, a multiple of 4) or rows that are multiples of 16 bytes.
+  if (a16 && (C % 16) == 0 && (HW % 4) == 0 && (HW <= 256 || (HW % 16) == 0)) {
+    const bool row_mode = HW > 256;
+    const int PT = row_mode ? 256 : HW;
+    const int hw_tiles = (HW + PT - 1) / PT;
+    const size_t smem = (size_t)(CT / 16) * (16 * PT + 16);
+    dim3 grid((unsigned)hw_tiles * (unsigned)N, (C_pad + CT - 1) / CT, 1);
+    if (row_mode)
+      pack_activations_bulk_kernel<true><<<grid, kPackThreads, smem, st>>>(x, out, C, HW, C_pad, hw_tiles, CT, PT);
+    else
+      pack_activations_bulk_kernel<false><<<grid, kPackThreads, smem, st>>>(x, out, C, HW, C_pad, hw_tiles, CT, PT);
+    return cudaGetLastError();
+  }
+  const int PT = HW > 128 ? 256 : (HW > 64 ? 128 : 64);
+  const int hw_tiles = (HW + PT - 1) / PT;
+  dim3 grid((unsigned)hw_tiles * (unsigned)N, (C_pad + CT - 1) / CT, 1);
+  if ((HW % 16) == 0 && a16)
+    pack_activations_kernel<16><<<grid, kPackThreads, 0, st>>>(x, out, C, HW, C_pad, hw_tiles, CT, PT);
+  else if ((HW % 4) == 0 && a16)
+    pack_activations_kernel<4><<<grid, kPackThreads, 0, st>>>(x, out, C, HW, C_pad, hw_tiles, CT, PT);
   else
-    pack_activations_kernel<false><<<grid, 256, 0, st>>>(x, out, C, HW, C_pad, hw_tiles);
+    pack_activations_kernel<1><<<grid, kPackThreads, 0, st>>>(x, out, C, HW, C_pad, hw_tiles, CT, PT);
   return cudaGetLastError();
 }
 
