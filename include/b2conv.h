@@ -71,6 +71,7 @@ typedef struct {
 #define B2C_VARIANT_CP_TMA 0         /* channel pack: NHWC C-padded activations, im2col-mode TMA */
 #define B2C_VARIANT_IM2COL_EXPLICIT 1 /* stencil unroll materialised as a matrix in scratch memory */
 #define B2C_VARIANT_IM2COL_GATHER 2  /* stencil unroll formed in shared memory inside the conv kernel */
+#define B2C_VARIANT_IM2COL_STAGED 3  /* same, from a zero-padded input window staged in shared memory (low-channel shapes) */
 
 typedef struct {
   int32_t id;       /* index in the enumeration for this descriptor; pass to b2c_plan_create      */

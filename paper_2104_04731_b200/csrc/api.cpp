@@ -19,6 +19,8 @@ struct b2c_plan {
   int8_t* w_packed = nullptr;   // device, plan-owned
   size_t w_packed_bytes = 0;
   GatherEntry* table = nullptr;  // device, plan-owned (stencil lookup table)
+  int32_t* table32 = nullptr;    // device, plan-owned (offsets into the staged window)
+  WindowGeom win = {0, 0, 0, 0, 0};
   int table_len = 0;
   int* status = nullptr;         // device status word
   bool weights_set = false;
@@ -120,6 +122,14 @@ void fill_common_args(b2c_plan* p) {
   a.out_mode = d.out_mode;
   a.out_layout = d.out_layout;
   a.table_len = p->table_len;
+  a.table32 = p->table32;
+  a.C = d.C;
+  a.P = p->g.P;
+  a.win_rows = p->win.rows;
+  a.win_pitch = p->win.pitch;
+  a.win_left = p->win.left;
+  a.win_bytes = p->win.bytes;
+  a.win_tap_span = (d.R - 1) * d.dil_h;
   if (p->emb.variant == B2C_VARIANT_CP_TMA) {
     p->amode = A_IM2COL_TMA;
     p->C_pad = cp_channel_pad(d.C);
@@ -131,7 +141,9 @@ void fill_common_args(b2c_plan* p) {
     a.ksteps_full = p->bk / kMmaK;
     a.ksteps_last = a.ksteps_full;
   } else {
-    p->amode = p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT ? A_TILED : A_GATHER;
+    p->amode = p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT
+                   ? A_TILED
+                   : (p->emb.variant == B2C_VARIANT_IM2COL_STAGED ? A_STAGED : A_GATHER);
     p->K_pad = im2col_k_pad(p->g.Kg);
     p->bk = 128;
     a.bk = 128;
@@ -149,8 +161,11 @@ void fill_common_args(b2c_plan* p) {
   const long long ctas = ((p->g.Mg + kTileM - 1) / kTileM) * ((d.K + a.tile_n - 1) / a.tile_n) * a.split_k;
   const size_t budget = ctas > kNumSMs ? 100 * 1024 : 160 * 1024;
   const size_t stage_bytes = (size_t)(kTileM + a.tile_n) * a.bk;
-  while (stages > 2 && (size_t)stages * stage_bytes > budget) --stages;
-  while (stages > 1 && (size_t)stages * stage_bytes > 160 * 1024) --stages;
+  // lookup table and staged window share the block's shared memory with the stages
+  const size_t extra = p->amode == A_STAGED ? (size_t)p->win.bytes + 4 * (size_t)p->table_len + 64
+                                            : (p->amode == A_GATHER ? 8 * (size_t)p->table_len : 0);
+  while (stages > 2 && (size_t)stages * stage_bytes + extra > budget) --stages;
+  while (stages > 1 && (size_t)stages * stage_bytes + extra > 196 * 1024) --stages;
   a.stages = stages;
 }
 
@@ -179,6 +194,19 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
     if (cudaMalloc(&p->table, t.size() * sizeof(GatherEntry)) != cudaSuccess) return fail(B2C_E_CUDA);
     if (cudaMemcpy(p->table, t.data(), t.size() * sizeof(GatherEntry), cudaMemcpyHostToDevice) != cudaSuccess)
       return fail(B2C_E_CUDA);
+    if (emb.variant == B2C_VARIANT_IM2COL_STAGED) {
+      if (!staged_window(g, &p->win)) return fail(B2C_E_UNSUPPORTED);
+      // reduction index (c, r, s) -> byte offset from the window position of the pixel's first tap
+      std::vector<int32_t> t32(K_pad, -1);
+      int kg = 0;
+      for (int c = 0; c < d.C; ++c)
+        for (int r = 0; r < d.R; ++r)
+          for (int s = 0; s < d.S; ++s, ++kg)
+            t32[kg] = (c * p->win.rows + r * d.dil_h) * p->win.pitch + s * d.dil_w;
+      if (cudaMalloc(&p->table32, t32.size() * sizeof(int32_t)) != cudaSuccess) return fail(B2C_E_CUDA);
+      if (cudaMemcpy(p->table32, t32.data(), t32.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+        return fail(B2C_E_CUDA);
+    }
   }
   // Room for one extra box row block so that a TMA box never starts past the allocation.
   if (cudaMalloc(&p->w_packed, p->w_packed_bytes + 256) != cudaSuccess) return fail(B2C_E_CUDA);
@@ -475,6 +503,7 @@ void b2c_plan_destroy(b2c_plan* p) {
   if (!p) return;
   cudaFree(p->w_packed);
   cudaFree(p->table);
+  cudaFree(p->table32);
   cudaFree(p->status);
   cudaFree(p->own_ws);
   delete p;

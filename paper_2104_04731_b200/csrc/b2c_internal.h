@@ -37,7 +37,7 @@ struct GatherEntry {
   int16_t dw;
 };
 
-enum AMode { A_TILED = 0, A_IM2COL_TMA = 1, A_GATHER = 2 };
+enum AMode { A_TILED = 0, A_IM2COL_TMA = 1, A_GATHER = 2, A_STAGED = 3 };
 
 // Everything the MMA kernel needs besides its two tensor maps.
 struct ConvArgs {
@@ -47,6 +47,7 @@ struct ConvArgs {
   int* status;
   const int8_t* x;
   const GatherEntry* table;
+  const int32_t* table32;  // staged window: reduction index -> byte offset inside the window, -1 for padding
   long long x_stride_n;
   int x_stride_h, x_stride_w;
   int Mg, K, PQ, Q, H, W;
@@ -58,6 +59,9 @@ struct ConvArgs {
   int kb_per_tap;   // channel-pack map: blocks per filter tap
   int tap_cols;     // channel-pack map: columns of the packed weight matrix per tap (C_pad)
   int table_len;    // gather: entries of the lookup table (padded reduction length)
+  // staged window (A_STAGED): per image part, C x win_rows rows of win_pitch bytes; image column 0
+  // sits at byte win_left of a row; win_bytes covers the parts a tile can touch
+  int C, P, win_rows, win_pitch, win_left, win_bytes, win_tap_span;
   int bk;           // bytes of reduction per block: 32, 64 or 128
   int tile_n;
   int tmem_cols;
@@ -81,6 +85,11 @@ int im2col_k_pad(int Kg);            // padded reduction length for the stencil-
 void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out);
 int pick_by_policy(const std::vector<b2c_embedding>& all, int policy);  // index or -1
 size_t workspace_bytes_for(const Geom& g, int variant, int split_k);
+// Geometry of the shared-memory input window of the staged stencil unroll; false if it does not fit.
+struct WindowGeom {
+  int rows, pitch, left, parts, bytes;
+};
+bool staged_window(const Geom& g, WindowGeom* w);
 
 // --- tma.cpp -----------------------------------------------------------------------------------
 // Tensor-map encoders obtained through cudaGetDriverEntryPoint (no link-time libcuda dependency).

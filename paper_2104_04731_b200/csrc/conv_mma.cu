@@ -300,18 +300,22 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   const uint32_t a_base = smem_base;
   const uint32_t b_base = smem_base + stages * a_stage_bytes;
   uint8_t* smem_aligned = smem_raw + (smem_base - smem_u32(smem_raw));
-  GatherEntry* s_table = reinterpret_cast<GatherEntry*>(smem_aligned + stages * (a_stage_bytes + b_stage_bytes));
+  uint8_t* smem_extra = smem_aligned + stages * (a_stage_bytes + b_stage_bytes);
+  GatherEntry* s_table = reinterpret_cast<GatherEntry*>(smem_extra);              // A_GATHER
+  int32_t* s_table32 = reinterpret_cast<int32_t*>(smem_extra);                    // A_STAGED
+  uint8_t* s_window = smem_extra + ((args.table_len * 4 + 15) & ~15);             // A_STAGED
+  constexpr bool kThreadsFormA = (AMODE == A_GATHER || AMODE == A_STAGED);
 
   if (warp == 0) {
     if (lane < stages) {
-      mbar_init(smem_u32(&ctl.full[lane]), AMODE == A_GATHER ? 1 + kGatherWarps : 1);
+      mbar_init(smem_u32(&ctl.full[lane]), kThreadsFormA ? 1 + kGatherWarps : 1);
       mbar_init(smem_u32(&ctl.empty[lane]), 1);
     }
     if (lane == 8) {
       mbar_init(smem_u32(&ctl.tmem_full), 1);
       ctl.abort_flag = 0;
     }
-    if (lane == 9 && AMODE != A_GATHER) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+    if (lane == 9 && !kThreadsFormA) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
     if (lane == 10) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -323,6 +327,9 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   }
   if (AMODE == A_GATHER) {
     for (int i = threadIdx.x; i < args.table_len; i += kThreads) s_table[i] = args.table[i];
+  }
+  if (AMODE == A_STAGED) {
+    for (int i = threadIdx.x; i < args.table_len; i += kThreads) s_table32[i] = args.table32[i];
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -355,7 +362,7 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       for (int kb = kb_begin; kb < kb_end; ++kb) {
         if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) break;
         const uint32_t full = smem_u32(&ctl.full[s]);
-        if (AMODE == A_GATHER) {
+        if (kThreadsFormA) {
           mbar_arrive_expect_tx(full, b_stage_bytes, leader);
           tma_load_2d(b_dst, &tmap_b, kcol, n0, full, leader);
         } else if (AMODE == A_TILED) {
@@ -494,6 +501,97 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       }
     }
 
+    if (AMODE == A_STAGED) {
+      // Stencil unroll from a staged window.  First the 256 threads copy, for every image the tile
+      // touches, the input rows its output pixels need into shared memory as a zero-padded window
+      // (rows outside the image and the left/right margins are zeros, so the gather below needs no
+      // bounds tests); then each thread forms half a row of the A tile per stage from that window.
+      const int tg = (int)threadIdx.x - 64;
+      const unsigned m_last = min((unsigned)m0 + (unsigned)kTileM - 1u, (unsigned)args.Mg - 1u);
+      const int img0 = m0 / args.PQ;
+      const int p_first = (m0 - img0 * args.PQ) / args.Q;
+      const int img1 = (int)(m_last / (unsigned)args.PQ);
+      const int p_last = (int)((m_last - (unsigned)img1 * (unsigned)args.PQ) / (unsigned)args.Q);
+      const int parts = img1 - img0 + 1;
+      const int wp = args.win_pitch, wr = args.win_rows, C = args.C;
+      const int vec_per_row = wp >> 4;
+      const int slots = parts * C * wr;
+      const bool vec_ok = (args.W & 15) == 0 && (reinterpret_cast<uintptr_t>(args.x) & 15) == 0;
+      for (int idx = tg; idx < slots * vec_per_row; idx += kGatherWarps * 32) {
+        const int slot = idx / vec_per_row;
+        const int v16 = idx - slot * vec_per_row;
+        const int part = slot / (C * wr);
+        const int cj = slot - part * (C * wr);
+        const int c = cj / wr;
+        const int j = cj - c * wr;
+        const int pl = part == 0 ? p_first : 0;
+        const int ph_ = part == parts - 1 ? p_last : args.P - 1;
+        const int h = pl * args.stride_h - args.pad_h + j;
+        const bool row_live = j <= (ph_ - pl) * args.stride_h + args.win_tap_span && (unsigned)h < (unsigned)args.H;
+        const int col0 = v16 * 16 - args.win_left;  // image column of the first byte of this vector
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (row_live && col0 < args.W && col0 + 16 > 0) {
+          const int8_t* src = args.x + (size_t)(img0 + part) * args.x_stride_n + ((size_t)c * args.H + h) * args.W + col0;
+          if (vec_ok && col0 >= 0 && col0 + 16 <= args.W) {
+            val = __ldg(reinterpret_cast<const uint4*>(src));
+          } else {
+            uint32_t wv[4] = {0, 0, 0, 0};
+            for (int b = 0; b < 16; ++b)
+              if ((unsigned)(col0 + b) < (unsigned)args.W) wv[b >> 2] |= (uint32_t)(uint8_t)__ldg(src + b) << (8 * (b & 3));
+            val = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+          }
+        }
+        *reinterpret_cast<uint4*>(s_window + (size_t)slot * wp + v16 * 16) = val;
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(kGatherWarps * 32) : "memory");
+
+      // window position of this pixel's first tap (r = s = 0, c = 0)
+      int wbase = -1;
+      if (row_valid) {
+        const int p = pq / args.Q, q = pq - p * args.Q;
+        const int part = n_img - img0;
+        const int pl = part == 0 ? p_first : 0;
+        wbase = (part * C * wr + (p - pl) * args.stride_h) * wp + args.win_left + q * args.stride_w - args.pad_w;
+      }
+      const uint32_t row_off = (uint32_t)row * 128u;
+      const uint32_t xr = (uint32_t)(row & 7);
+      int s = 0;
+      uint32_t ph = 0;
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
+        if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) {
+          ok = false;
+          break;
+        }
+        const uint32_t a_row = a_base + s * a_stage_bytes + row_off;
+        const int chunks = (kb == args.num_kb - 1) ? args.ksteps_last * 2 : 8;
+        const int32_t* te = s_table32 + kb * 128 + half * 64;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          const int j = half * 4 + jj;
+          if (j < chunks) {
+            uint32_t wv[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const int off = te[jj * 16 + e];
+              uint32_t v = 0;
+              if (off >= 0 && wbase >= 0) v = s_window[wbase + off];
+              wv[e >> 2] |= v << (8 * (e & 3));
+            }
+            const uint32_t dst = a_row + ((((uint32_t)j) ^ xr) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]),
+                         "r"(wv[3]));
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctl.full[s]));
+        if (++s == stages) {
+          s = 0;
+          ph ^= 1u;
+        }
+      }
+    }
+
     // ---- epilogue ----
     if (ok) ok = mbar_wait(smem_u32(&ctl.tmem_full), 0u, &ctl, args.status);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -539,6 +637,7 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
 size_t conv_mma_smem_bytes(int amode, const ConvArgs& a) {
   size_t b = 1024 + (size_t)a.stages * (kTileM + a.tile_n) * a.bk;
   if (amode == A_GATHER) b += (size_t)a.table_len * sizeof(GatherEntry);
+  if (amode == A_STAGED) b += (size_t)((a.table_len * 4 + 15) & ~15) + (size_t)a.win_bytes + 16;
   return b;
 }
 
@@ -560,6 +659,7 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
   }
   if (amode == A_TILED) B2C_LAUNCH(A_TILED)
   else if (amode == A_IM2COL_TMA) B2C_LAUNCH(A_IM2COL_TMA)
+  else if (amode == A_STAGED) B2C_LAUNCH(A_STAGED)
   else B2C_LAUNCH(A_GATHER)
 #undef B2C_LAUNCH
   return cudaGetLastError();

@@ -101,6 +101,30 @@ static bool cp_legal(const Geom& g) {
   return true;
 }
 
+// The staged stencil unroll keeps, per image a tile can touch, the zero-padded input rows that
+// feed the tile's 128 output pixels: C x rows x pitch bytes, with the left margin rounded up to 16
+// so that aligned 16-byte copies land on aligned shared-memory addresses.
+bool staged_window(const Geom& g, WindowGeom* w) {
+  const b2c_conv_desc& d = g.d;
+  if (d.in_layout != B2C_LAYOUT_NCHW) return false;  // the window is staged from whole NCHW rows
+  const int rows_out = std::min(g.P, (kTileM - 2) / g.Q + 2);  // output rows 128 consecutive pixels can span
+  const int parts = (int)std::min<long long>(d.N, (kTileM - 2) / g.PQ + 2);
+  const long long rows = (long long)(rows_out - 1) * d.stride_h + (long long)(d.R - 1) * d.dil_h + 1;
+  const long long left = round_up(d.pad_w, 16);
+  // columns read: up to (Q-1)*stride_w - pad_w + (S-1)*dil_w
+  const long long right_edge = (long long)(g.Q - 1) * d.stride_w - d.pad_w + (long long)(d.S - 1) * d.dil_w + 1;
+  const long long width = std::max<long long>(d.W, right_edge);
+  const long long pitch = (left + width + 15) / 16 * 16;
+  const long long bytes = (long long)parts * d.C * rows * pitch;
+  if (bytes > 64 * 1024 || im2col_k_pad(g.Kg) > 4096) return false;
+  w->rows = (int)rows;
+  w->pitch = (int)pitch;
+  w->left = (int)left;
+  w->parts = parts;
+  w->bytes = (int)bytes;
+  return true;
+}
+
 static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int tile_n, int split_k) {
   const b2c_conv_desc& d = g.d;
   b2c_embedding e;
@@ -130,6 +154,8 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
     k_issued = K_pad;
     if (variant == B2C_VARIANT_IM2COL_EXPLICIT)
       moved = g.x_elems + 2 * g.Mg * K_pad + (long long)d.K * K_pad + g.y_elems;
+    else if (variant == B2C_VARIANT_IM2COL_STAGED)
+      moved = g.x_elems + (long long)d.K * K_pad + g.y_elems;
     else
       moved = g.x_elems + (long long)d.K * K_pad + g.y_elems;
   }
@@ -150,8 +176,10 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
     if (t >= d.K) break;
   }
   long long tiles_m = (g.Mg + kTileM - 1) / kTileM;
-  for (int variant = 0; variant < 3; ++variant) {
+  for (int variant = 0; variant < 4; ++variant) {
     if (variant == B2C_VARIANT_CP_TMA && !cp_legal(g)) continue;
+    WindowGeom wg;
+    if (variant == B2C_VARIANT_IM2COL_STAGED && !staged_window(g, &wg)) continue;
     int num_kb;
     if (variant == B2C_VARIANT_CP_TMA) {
       int C_pad = cp_channel_pad(d.C);

@@ -60,7 +60,7 @@ def test_config_every_embedding(lib, cfg):
     d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
                       out_mode=cfg.out_mode)
     embs = lib.enumerate_embeddings(d)
-    assert {e.variant for e in embs} == {0, 1, 2}
+    assert {0, 1, 2} <= {e.variant for e in embs}
     for e in embs:
         check_against_oracle(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, cfg.out_mode, e.id, ref=ref)
 
@@ -69,7 +69,7 @@ def test_config_every_embedding(lib, cfg):
 @pytest.mark.parametrize("in_layout,out_layout", [(1, 1), (0, 1), (1, 0)])
 def test_config_layouts(lib, cfg, in_layout, out_layout):
     x, w, ref = cfg_reference(cfg)
-    for variant in (0, 1, 2):
+    for variant in (0, 1, 2, 3):
         d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
                           in_layout, out_layout, 3)
         ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant]
@@ -105,7 +105,7 @@ def test_random_shapes(lib, case):
     ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
     d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode=3)
     embs = lib.enumerate_embeddings(d)
-    for variant in (0, 1, 2):
+    for variant in (0, 1, 2, 3):
         ids = [e.id for e in embs if e.variant == variant]
         for i in ids[:1] + ids[-1:]:
             check_against_oracle(x, w, stride, pad, dil, shift, 3, i, ref=ref)
@@ -120,7 +120,7 @@ def test_extreme_values_and_shift_clip(lib):
     x = np.full((1, 64, 6, 6), -128, dtype=np.int8)
     w = np.full((16, 64, 3, 3), -128, dtype=np.int8)
     ref = oracle.conv2d_int8(x, w, 1, 1, 1, 16)
-    for variant in (0, 1, 2):
+    for variant in (0, 1, 2, 3):
         d = lib.make_desc(1, 64, 6, 6, 16, 3, 3, 1, 1, 1, 16, out_mode=3)
         i = next(e.id for e in lib.enumerate_embeddings(d) if e.variant == variant)
         check_against_oracle(x, w, 1, 1, 1, 16, 3, i, ref=ref)
