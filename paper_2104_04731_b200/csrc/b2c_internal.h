@@ -76,6 +76,31 @@ struct Schedule {
   int split_k;
 };
 
+// Programmatic dependent launch: a kernel launched through launch_pdl may start while the previous
+// kernel of the stream is still running; it must call pdl_wait() before its first access to global
+// memory that an earlier kernel may write or still read, and calls pdl_launch_dependents() once the
+// next kernel may begin its own set-up.  Every kernel of this library follows that rule, so the
+// stream order of memory effects is unchanged; what overlaps is launch latency and block set-up.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // --- planner.cpp -------------------------------------------------------------------------------
 int resolve_geom(const b2c_conv_desc* d, Geom* g);  // validation + derived sizes; B2C_* code
 int round_up(int v, int m);

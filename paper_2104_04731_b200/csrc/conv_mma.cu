@@ -335,6 +335,11 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = ctl.tmem_base;
+  // Everything above touched only kernel parameters, shared memory and the plan's constant lookup
+  // table.  From here on the block reads tensors earlier kernels of the stream produce and writes
+  // tensors they may still read.
+  pdl_wait();
+  pdl_launch_dependents();
 
   // The loops below keep stage index, phase bit, tap position and addresses as running
   // counters: each role is a single thread, so every integer division in a loop body would
@@ -655,7 +660,8 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
       if (e != cudaSuccess) return e;                                                                     \
       configured = 200 * 1024;                                                                            \
     }                                                                                                     \
-    conv_mma_kernel<MODE><<<grid, kThreads, smem, st>>>(*tmap_a, *tmap_b, args);                          \
+    e = launch_pdl(conv_mma_kernel<MODE>, grid, dim3(kThreads), smem, st, *tmap_a, *tmap_b, args);        \
+    if (e != cudaSuccess) return e;                                                                       \
   }
   if (amode == A_TILED) B2C_LAUNCH(A_TILED)
   else if (amode == A_IM2COL_TMA) B2C_LAUNCH(A_IM2COL_TMA)

@@ -34,6 +34,8 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_kernel(const in
   const int pitch = PT + 4;
   const int8_t* xin = x + ((size_t)n * C + c0) * HW + hw0;
   const int rows = min(CT, C - c0);  // channels that exist; the rest of the tile is zero padding
+  pdl_wait();
+  pdl_launch_dependents();
 
   // ---- load ----
   if constexpr (VEC >= 4) {
@@ -146,6 +148,8 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_bulk_kernel(con
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"(bytes) : "memory");
   }
   __syncthreads();
+  pdl_wait();
+  pdl_launch_dependents();
   const int8_t* xin = x + ((size_t)n * C + c0) * HW + hw0;
   if (kRowMode) {
     if (t < rows) {
@@ -247,6 +251,8 @@ __global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ 
                                                      long long x_stride_n, int x_stride_h, int x_stride_w, int K_pad) {
   const int chunks = K_pad >> 4;
   const long long total = Mg * chunks;
+  pdl_wait();
+  pdl_launch_dependents();
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
     const long long m = i / chunks;
@@ -273,6 +279,8 @@ __global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ 
 // the shift-and-clip requantisation (arithmetic shift = floor division by 2^shift).
 __global__ void splitk_finish_kernel(const int32_t* __restrict__ acc, int32_t* __restrict__ y32,
                                      int8_t* __restrict__ y8, long long elems, int shift, int out_mode) {
+  pdl_wait();
+  pdl_launch_dependents();
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < elems;
        i += (long long)gridDim.x * blockDim.x) {
     const int v = acc[i];
@@ -303,21 +311,21 @@ cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, 
     const size_t smem = (size_t)(CT / 16) * (16 * PT + 16);
     dim3 grid((unsigned)hw_tiles * (unsigned)N, (C_pad + CT - 1) / CT, 1);
     if (row_mode)
-      pack_activations_bulk_kernel<true><<<grid, kPackThreads, smem, st>>>(x, out, C, HW, C_pad, hw_tiles, CT, PT);
-    else
-      pack_activations_bulk_kernel<false><<<grid, kPackThreads, smem, st>>>(x, out, C, HW, C_pad, hw_tiles, CT, PT);
-    return cudaGetLastError();
+      return launch_pdl(pack_activations_bulk_kernel<true>, grid, dim3(kPackThreads), smem, st, x, out, C, HW, C_pad,
+                        hw_tiles, CT, PT);
+    return launch_pdl(pack_activations_bulk_kernel<false>, grid, dim3(kPackThreads), smem, st, x, out, C, HW, C_pad,
+                      hw_tiles, CT, PT);
   }
   const int PT = HW > 128 ? 256 : (HW > 64 ? 128 : 64);
   const int hw_tiles = (HW + PT - 1) / PT;
   dim3 grid((unsigned)hw_tiles * (unsigned)N, (C_pad + CT - 1) / CT, 1);
   if ((HW % 16) == 0 && a16)
-    pack_activations_kernel<16><<<grid, kPackThreads, 0, st>>>(x, out, C, HW, C_pad, hw_tiles, CT, PT);
-  else if ((HW % 4) == 0 && a16)
-    pack_activations_kernel<4><<<grid, kPackThreads, 0, st>>>(x, out, C, HW, C_pad, hw_tiles, CT, PT);
-  else
-    pack_activations_kernel<1><<<grid, kPackThreads, 0, st>>>(x, out, C, HW, C_pad, hw_tiles, CT, PT);
-  return cudaGetLastError();
+    return launch_pdl(pack_activations_kernel<16>, grid, dim3(kPackThreads), 0, st, x, out, C, HW, C_pad, hw_tiles, CT,
+                      PT);
+  if ((HW % 4) == 0 && a16)
+    return launch_pdl(pack_activations_kernel<4>, grid, dim3(kPackThreads), 0, st, x, out, C, HW, C_pad, hw_tiles, CT,
+                      PT);
+  return launch_pdl(pack_activations_kernel<1>, grid, dim3(kPackThreads), 0, st, x, out, C, HW, C_pad, hw_tiles, CT, PT);
 }
 
 cudaError_t launch_pack_weights_cp(const int8_t* w, int8_t* out, int K, int C, int R, int S, int C_pad,
@@ -337,15 +345,14 @@ cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, 
                           int W, int stride_h, int stride_w, int pad_h, int pad_w, long long x_stride_n,
                           int x_stride_h, int x_stride_w, int K_pad, cudaStream_t st) {
   const long long total = Mg * (K_pad / 16);
-  im2col_kernel<<<grid_for(total, 256), 256, 0, st>>>(x, a, table, Mg, PQ, Q, H, W, stride_h, stride_w, pad_h, pad_w,
-                                                      x_stride_n, x_stride_h, x_stride_w, K_pad);
-  return cudaGetLastError();
+  return launch_pdl(im2col_kernel, dim3(grid_for(total, 256)), dim3(256), 0, st, x, a, table, Mg, PQ, Q, H, W, stride_h,
+                    stride_w, pad_h, pad_w, x_stride_n, x_stride_h, x_stride_w, K_pad);
 }
 
 cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, long long elems, int shift,
                                  int out_mode, cudaStream_t st) {
-  splitk_finish_kernel<<<grid_for(elems, 256), 256, 0, st>>>(acc, y32, y8, elems, shift, out_mode);
-  return cudaGetLastError();
+  return launch_pdl(splitk_finish_kernel, dim3(grid_for(elems, 256)), dim3(256), 0, st, acc, y32, y8, elems, shift,
+                    out_mode);
 }
 
 }  // namespace b2c

@@ -185,3 +185,44 @@ def test_error_paths_on_device(lib):
     torch.cuda.synchronize()
     assert plan.device_status() == b2c.OK
     plan.destroy()
+
+
+# ---- kernels of consecutive calls overlap their launch and set-up; memory effects must stay in stream order ----
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
+def test_back_to_back_runs_keep_stream_order(lib, variant):
+    cfg = CONFIGS[0]
+    xa, w = cfg.tensors(0)
+    xb, _ = cfg.tensors(1)
+    refs = [oracle.conv2d_int8(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift) for x in (xa, xb)]
+    d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
+                      out_mode=3)
+    eid = next(e.id for e in lib.enumerate_embeddings(d) if e.variant == variant and e.split_k == 1)
+    plan = lib.Plan(d, eid)
+    xs = [to_dev(xa), to_dev(xb)]
+    plan.set_weights(to_dev(w))
+    ws = torch.zeros(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")  # shared by all calls
+    outs = [(torch.zeros(refs[0][0].shape, dtype=torch.int32, device="cuda"),
+             torch.zeros(refs[0][0].shape, dtype=torch.int8, device="cuda")) for _ in range(40)]
+
+    def enqueue():
+        for i, (y32, y8) in enumerate(outs):
+            plan.run(xs[i & 1], y32, y8, ws)
+
+    enqueue()
+    torch.cuda.synchronize()
+    for i, (y32, y8) in enumerate(outs):
+        assert np.array_equal(y32.cpu().numpy(), refs[i & 1][0]), i
+        assert np.array_equal(y8.cpu().numpy(), refs[i & 1][1]), i
+        y32.zero_()
+        y8.zero_()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        enqueue()
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    for i, (y32, y8) in enumerate(outs):
+        assert np.array_equal(y32.cpu().numpy(), refs[i & 1][0]), i
+        assert np.array_equal(y8.cpu().numpy(), refs[i & 1][1]), i
+    assert plan.device_status() == b2c.OK
+    plan.destroy()
