@@ -130,6 +130,7 @@ void fill_common_args(b2c_plan* p) {
   a.win_left = p->win.left;
   a.win_bytes = p->win.bytes;
   a.win_tap_span = (d.R - 1) * d.dil_h;
+  a.win_word_mode = (p->emb.variant == B2C_VARIANT_IM2COL_STAGED && staged_word_mode(p->g)) ? 1 : 0;
   if (p->emb.variant == B2C_VARIANT_CP_TMA) {
     p->amode = A_IM2COL_TMA;
     p->C_pad = cp_channel_pad(d.C);
@@ -144,7 +145,7 @@ void fill_common_args(b2c_plan* p) {
     p->amode = p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT
                    ? A_TILED
                    : (p->emb.variant == B2C_VARIANT_IM2COL_STAGED ? A_STAGED : A_GATHER);
-    p->K_pad = im2col_k_pad(p->g.Kg);
+    p->K_pad = variant_k_pad(p->g, p->emb.variant);
     p->bk = 128;
     a.bk = 128;
     a.num_kb = (p->K_pad + 127) / 128;
@@ -186,7 +187,7 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
     int C_pad = cp_channel_pad(d.C);
     p->w_packed_bytes = (size_t)d.K * d.R * d.S * C_pad;
   } else {
-    int K_pad = im2col_k_pad(g.Kg);
+    int K_pad = variant_k_pad(g, emb.variant);
     p->w_packed_bytes = (size_t)d.K * K_pad;
     std::vector<GatherEntry> t;
     build_table(g, K_pad, &t);
@@ -197,12 +198,24 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
     if (emb.variant == B2C_VARIANT_IM2COL_STAGED) {
       if (!staged_window(g, &p->win)) return fail(B2C_E_UNSUPPORTED);
       // reduction index (c, r, s) -> byte offset from the window position of the pixel's first tap
-      std::vector<int32_t> t32(K_pad, -1);
-      int kg = 0;
-      for (int c = 0; c < d.C; ++c)
-        for (int r = 0; r < d.R; ++r)
-          for (int s = 0; s < d.S; ++s, ++kg)
-            t32[kg] = (c * p->win.rows + r * d.dil_h) * p->win.pitch + s * d.dil_w;
+      std::vector<int32_t> t32;
+      if (staged_word_mode(g)) {
+        // one entry per 32-bit word of an A row: window offset of the word's first byte
+        const int run = staged_run_len(g);
+        t32.assign(K_pad / 4, -1);
+        for (int wi = 0; wi < K_pad / 4; ++wi) {
+          const int cr = (wi * 4) / run, k4 = (wi * 4) % run;
+          if (cr < d.C * d.R) t32[wi] = ((cr / d.R) * p->win.rows + (cr % d.R) * d.dil_h) * p->win.pitch + k4;
+        }
+      } else {
+        t32.assign(K_pad, -1);
+        int kg = 0;
+        for (int c = 0; c < d.C; ++c)
+          for (int r = 0; r < d.R; ++r)
+            for (int s = 0; s < d.S; ++s, ++kg)
+              t32[kg] = (c * p->win.rows + r * d.dil_h) * p->win.pitch + s * d.dil_w;
+      }
+      p->table_len = (int)t32.size();
       if (cudaMalloc(&p->table32, t32.size() * sizeof(int32_t)) != cudaSuccess) return fail(B2C_E_CUDA);
       if (cudaMemcpy(p->table32, t32.data(), t32.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
         return fail(B2C_E_CUDA);
@@ -429,7 +442,8 @@ int b2c_plan_set_weights(b2c_plan* p, const int8_t* w, void* cuda_stream) {
   if (p->emb.variant == B2C_VARIANT_CP_TMA)
     CUDA_TRY(launch_pack_weights_cp(w, p->w_packed, d.K, d.C, d.R, d.S, p->C_pad, st));
   else
-    CUDA_TRY(launch_pack_weights_rows(w, p->w_packed, d.K, p->g.Kg, p->K_pad, st));
+    CUDA_TRY(launch_pack_weights_rows(w, p->w_packed, d.K, p->g.Kg, p->K_pad, d.S,
+                                      p->emb.variant == B2C_VARIANT_IM2COL_STAGED ? staged_run_len(p->g) : d.S, st));
   p->weights_set = true;
   return B2C_OK;
 }

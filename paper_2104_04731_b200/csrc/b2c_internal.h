@@ -61,7 +61,7 @@ struct ConvArgs {
   int table_len;    // gather: entries of the lookup table (padded reduction length)
   // staged window (A_STAGED): per image part, C x win_rows rows of win_pitch bytes; image column 0
   // sits at byte win_left of a row; win_bytes covers the parts a tile can touch
-  int C, P, win_rows, win_pitch, win_left, win_bytes, win_tap_span;
+  int C, P, win_rows, win_pitch, win_left, win_bytes, win_tap_span, win_word_mode;
   int bk;           // bytes of reduction per block: 32, 64 or 128
   int tile_n;
   int tmem_cols;
@@ -115,6 +115,11 @@ struct WindowGeom {
   int rows, pitch, left, parts, bytes;
 };
 bool staged_window(const Geom& g, WindowGeom* w);
+// Staged stencil unroll with unit horizontal dilation: each (c, r) run of S taps is padded to a
+// multiple of 4 so that the A rows are built from aligned 32-bit words of the window.
+bool staged_word_mode(const Geom& g);
+int staged_run_len(const Geom& g);  // taps per (c, r) run after padding
+int variant_k_pad(const Geom& g, int variant);  // padded reduction length of the stencil-unroll variants
 
 // --- tma.cpp -----------------------------------------------------------------------------------
 // Tensor-map encoders obtained through cudaGetDriverEntryPoint (no link-time libcuda dependency).
@@ -131,7 +136,8 @@ cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, 
                                     cudaStream_t st);
 cudaError_t launch_pack_weights_cp(const int8_t* w, int8_t* out, int K, int C, int R, int S, int C_pad,
                                    cudaStream_t st);
-cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg, int K_pad, cudaStream_t st);
+cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg, int K_pad, int S, int S_run,
+                                     cudaStream_t st);
 cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, long long Mg, int PQ, int Q, int H,
                           int W, int stride_h, int stride_w, int pad_h, int pad_w, long long x_stride_n,
                           int x_stride_h, int x_stride_w, int K_pad, cudaStream_t st);

@@ -569,22 +569,53 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
         }
         const uint32_t a_row = a_base + s * a_stage_bytes + row_off;
         const int chunks = (kb == args.num_kb - 1) ? args.ksteps_last * 2 : 8;
-        const int32_t* te = s_table32 + kb * 128 + half * 64;
+        if (args.win_word_mode) {
+          // Unit horizontal dilation: the S taps of a (c, r) run are consecutive window bytes.  Runs
+          // are padded to a multiple of 4 (the packed weights hold zeros there), so every 32-bit
+          // word of the A row is one unaligned word of the window: two aligned loads and a byte
+          // permute whose selector depends only on this pixel's window alignment.
+          const int32_t* te = s_table32 + kb * 32 + half * 16;
+          const uint32_t sel = 0x3210u + 0x1111u * ((uint32_t)wbase & 3u);
+          const uint8_t* wrow = s_window + (wbase & ~3);
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          const int j = half * 4 + jj;
-          if (j < chunks) {
-            uint32_t wv[4] = {0, 0, 0, 0};
+          for (int jj = 0; jj < 4; ++jj) {
+            const int j = half * 4 + jj;
+            if (j < chunks) {
+              uint32_t wv[4];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const int off = te[jj * 16 + e];
-              uint32_t v = 0;
-              if (off >= 0 && wbase >= 0) v = s_window[wbase + off];
-              wv[e >> 2] |= v << (8 * (e & 3));
+              for (int e = 0; e < 4; ++e) {
+                const int off = te[jj * 4 + e];
+                uint32_t v = 0;
+                if (off >= 0 && wbase >= 0) {
+                  const uint32_t lo = *reinterpret_cast<const uint32_t*>(wrow + off);
+                  const uint32_t hi = *reinterpret_cast<const uint32_t*>(wrow + off + 4);
+                  v = __byte_perm(lo, hi, sel);
+                }
+                wv[e] = v;
+              }
+              const uint32_t dst = a_row + ((((uint32_t)j) ^ xr) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]),
+                           "r"(wv[3]));
             }
-            const uint32_t dst = a_row + ((((uint32_t)j) ^ xr) << 4);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]),
-                         "r"(wv[3]));
+          }
+        } else {
+          const int32_t* te = s_table32 + kb * 128 + half * 64;
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) {
+            const int j = half * 4 + jj;
+            if (j < chunks) {
+              uint32_t wv[4] = {0, 0, 0, 0};
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                const int off = te[jj * 16 + e];
+                uint32_t v = 0;
+                if (off >= 0 && wbase >= 0) v = s_window[wbase + off];
+                wv[e >> 2] |= v << (8 * (e & 3));
+              }
+              const uint32_t dst = a_row + ((((uint32_t)j) ^ xr) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]),
+                           "r"(wv[3]));
+            }
           }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

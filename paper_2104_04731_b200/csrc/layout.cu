@@ -230,15 +230,18 @@ __global__ void pack_weights_cp_kernel(const int8_t* __restrict__ w, int8_t* __r
   }
 }
 
-// Stencil-unroll weights: rows of w[k][(c,r,s)] zero-padded to K_pad.
+// Stencil-unroll weights: rows of w[k][(c,r,s)] with every (c, r) run of S taps padded with zeros
+// to S_run entries (S_run = S for the plain unroll), then the row zero-padded to K_pad.
 __global__ void pack_weights_rows_kernel(const int8_t* __restrict__ w, int8_t* __restrict__ out, int K, int Kg,
-                                         int K_pad) {
+                                         int K_pad, int S, int S_run) {
   const long long total = (long long)K * K_pad;
+  const int runs = Kg / S;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
     const int j = (int)(i % K_pad);
     const long long k = i / K_pad;
-    out[i] = j < Kg ? w[k * Kg + j] : (int8_t)0;
+    const int run = j / S_run, s = j - run * S_run;
+    out[i] = (run < runs && s < S) ? w[k * Kg + run * S + s] : (int8_t)0;
   }
 }
 
@@ -335,9 +338,10 @@ cudaError_t launch_pack_weights_cp(const int8_t* w, int8_t* out, int K, int C, i
   return cudaGetLastError();
 }
 
-cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg, int K_pad, cudaStream_t st) {
+cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg, int K_pad, int S, int S_run,
+                                     cudaStream_t st) {
   const long long total = (long long)K * K_pad;
-  pack_weights_rows_kernel<<<grid_for(total, 256), 256, 0, st>>>(w, out, K, Kg, K_pad);
+  pack_weights_rows_kernel<<<grid_for(total, 256), 256, 0, st>>>(w, out, K, Kg, K_pad, S, S_run);
   return cudaGetLastError();
 }
 

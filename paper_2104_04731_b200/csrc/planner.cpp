@@ -64,6 +64,13 @@ int cp_block_bytes(int C_pad) {
 
 int im2col_k_pad(int Kg) { return round_up(Kg, kMmaK); }
 
+bool staged_word_mode(const Geom& g) { return g.d.dil_w == 1; }
+int staged_run_len(const Geom& g) { return staged_word_mode(g) ? round_up(g.d.S, 4) : g.d.S; }
+int variant_k_pad(const Geom& g, int variant) {
+  if (variant == B2C_VARIANT_IM2COL_STAGED) return round_up(g.d.C * g.d.R * staged_run_len(g), kMmaK);
+  return im2col_k_pad(g.Kg);
+}
+
 static int tmem_pow2(int n) {
   int c = 32;
   while (c < n) c <<= 1;
@@ -116,7 +123,7 @@ bool staged_window(const Geom& g, WindowGeom* w) {
   const long long width = std::max<long long>(d.W, right_edge);
   const long long pitch = (left + width + 15) / 16 * 16;
   const long long bytes = (long long)parts * d.C * rows * pitch;
-  if (bytes > 64 * 1024 || im2col_k_pad(g.Kg) > 4096) return false;
+  if (bytes > 64 * 1024 || variant_k_pad(g, B2C_VARIANT_IM2COL_STAGED) > 4096) return false;
   w->rows = (int)rows;
   w->pitch = (int)pitch;
   w->left = (int)left;
@@ -150,7 +157,7 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
     moved = (direct ? 0 : g.x_elems + packed) + packed + (long long)d.K * k_issued + g.y_elems;
   } else {
     e.map_k = B2C_AXIS_CRS;
-    int K_pad = im2col_k_pad(g.Kg);
+    int K_pad = variant_k_pad(g, variant);
     k_issued = K_pad;
     if (variant == B2C_VARIANT_IM2COL_EXPLICIT)
       moved = g.x_elems + 2 * g.Mg * K_pad + (long long)d.K * K_pad + g.y_elems;
@@ -185,7 +192,7 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
       int C_pad = cp_channel_pad(d.C);
       num_kb = d.R * d.S * (C_pad / cp_block_bytes(C_pad));
     } else {
-      num_kb = (im2col_k_pad(g.Kg) + 127) / 128;
+      num_kb = (variant_k_pad(g, variant) + 127) / 128;
     }
     // The in-kernel gather keeps its lookup table in shared memory.
     if (variant == B2C_VARIANT_IM2COL_GATHER && im2col_k_pad(g.Kg) > 4096) continue;
