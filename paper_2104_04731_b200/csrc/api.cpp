@@ -130,6 +130,11 @@ void fill_common_args(b2c_plan* p) {
   a.win_left = p->win.left;
   a.win_bytes = p->win.bytes;
   a.win_tap_span = (d.R - 1) * d.dil_h;
+  a.div_pq = make_fastdiv((uint32_t)p->g.PQ);
+  a.div_q = make_fastdiv((uint32_t)p->g.Q);
+  a.div_vec_per_row = make_fastdiv((uint32_t)std::max(1, p->win.pitch / 16));
+  a.div_c_rows = make_fastdiv((uint32_t)std::max(1, d.C * p->win.rows));
+  a.div_rows = make_fastdiv((uint32_t)std::max(1, p->win.rows));
   a.win_word_mode = (p->emb.variant == B2C_VARIANT_IM2COL_STAGED && staged_word_mode(p->g)) ? 1 : 0;
   if (p->emb.variant == B2C_VARIANT_CP_TMA) {
     p->amode = A_IM2COL_TMA;

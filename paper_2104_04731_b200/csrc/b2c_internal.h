@@ -37,6 +37,31 @@ struct GatherEntry {
   int16_t dw;
 };
 
+// Division of a non-negative 31-bit integer by a run-time constant as multiply + shift
+// (round-up method: l = ceil(log2 d), m = ceil(2^(31+l) / d), n / d = (n * m) >> (31 + l) for all
+// 0 <= n < 2^31).  Per-thread index arithmetic in the kernels uses it instead of the ~20
+// instruction hardware-less integer division.
+struct FastDiv {
+  uint32_t mul;
+  uint32_t shr;
+  uint32_t d;
+#ifdef __CUDACC__
+  __host__ __device__
+#endif
+  inline uint32_t div(uint32_t n) const {
+    return (uint32_t)(((unsigned long long)n * mul) >> shr);
+  }
+};
+inline FastDiv make_fastdiv(uint32_t d) {
+  FastDiv f;
+  f.d = d;
+  uint32_t l = 0;
+  while ((1ull << l) < d) ++l;
+  f.shr = 31 + l;
+  f.mul = (uint32_t)(((1ull << (31 + l)) + d - 1) / d);
+  return f;
+}
+
 enum AMode { A_TILED = 0, A_IM2COL_TMA = 1, A_GATHER = 2, A_STAGED = 3 };
 
 // Everything the MMA kernel needs besides its two tensor maps.
@@ -61,6 +86,7 @@ struct ConvArgs {
   int table_len;    // gather: entries of the lookup table (padded reduction length)
   // staged window (A_STAGED): per image part, C x win_rows rows of win_pitch bytes; image column 0
   // sits at byte win_left of a row; win_bytes covers the parts a tile can touch
+  FastDiv div_pq, div_q, div_vec_per_row, div_c_rows, div_rows;  // by PQ, Q, win_pitch/16, C*win_rows, win_rows
   int C, P, win_rows, win_pitch, win_left, win_bytes, win_tap_span, win_word_mode;
   int bk;           // bytes of reduction per block: 32, 64 or 128
   int tile_n;

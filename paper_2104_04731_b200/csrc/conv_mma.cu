@@ -349,9 +349,9 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
     {
       int n_img = 0, h_org = 0, w_org = 0, cb = 0, sx = 0, r = 0;
       if (AMODE == A_IM2COL_TMA) {
-        n_img = m0 / args.PQ;
+        n_img = (int)args.div_pq.div((uint32_t)m0);
         const int rem = m0 - n_img * args.PQ;
-        const int p = rem / args.Q, q = rem - p * args.Q;
+        const int p = (int)args.div_q.div((uint32_t)rem), q = rem - p * args.Q;
         h_org = p * args.stride_h - args.pad_h;
         w_org = q * args.stride_w - args.pad_w;
         const int tap = kb_begin / args.kb_per_tap;
@@ -449,7 +449,7 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
     const bool row_valid = m < (unsigned)args.Mg;
     int n_img = 0, pq = 0;
     if (row_valid) {
-      n_img = (int)(m / (unsigned)args.PQ);
+      n_img = (int)args.div_pq.div(m);
       pq = (int)(m - (unsigned)n_img * (unsigned)args.PQ);
     }
     bool ok = true;
@@ -458,7 +458,7 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       // Stencil unroll formed in place: this thread writes half of row `row` of the A tile (four
       // 16-byte chunks per stage) in the 128-byte swizzled order the MMA descriptor expects
       // (chunk j of row r lives at chunk position j ^ (r & 7)).
-      const int p = pq / args.Q, q = pq - p * args.Q;
+      const int p = (int)args.div_q.div((uint32_t)pq), q = pq - p * args.Q;
       const int h0 = row_valid ? p * args.stride_h - args.pad_h : -(1 << 29);
       const int w0 = q * args.stride_w - args.pad_w;
       const int8_t* base = args.x + n_img * args.x_stride_n + (long long)(row_valid ? h0 : 0) * args.x_stride_h +
@@ -513,21 +513,21 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       // bounds tests); then each thread forms half a row of the A tile per stage from that window.
       const int tg = (int)threadIdx.x - 64;
       const unsigned m_last = min((unsigned)m0 + (unsigned)kTileM - 1u, (unsigned)args.Mg - 1u);
-      const int img0 = m0 / args.PQ;
-      const int p_first = (m0 - img0 * args.PQ) / args.Q;
-      const int img1 = (int)(m_last / (unsigned)args.PQ);
-      const int p_last = (int)((m_last - (unsigned)img1 * (unsigned)args.PQ) / (unsigned)args.Q);
+      const int img0 = (int)args.div_pq.div((uint32_t)m0);
+      const int p_first = (int)args.div_q.div((uint32_t)(m0 - img0 * args.PQ));
+      const int img1 = (int)args.div_pq.div(m_last);
+      const int p_last = (int)args.div_q.div(m_last - (unsigned)img1 * (unsigned)args.PQ);
       const int parts = img1 - img0 + 1;
       const int wp = args.win_pitch, wr = args.win_rows, C = args.C;
       const int vec_per_row = wp >> 4;
       const int slots = parts * C * wr;
       const bool vec_ok = (args.W & 15) == 0 && (reinterpret_cast<uintptr_t>(args.x) & 15) == 0;
       for (int idx = tg; idx < slots * vec_per_row; idx += kGatherWarps * 32) {
-        const int slot = idx / vec_per_row;
+        const int slot = (int)args.div_vec_per_row.div((uint32_t)idx);
         const int v16 = idx - slot * vec_per_row;
-        const int part = slot / (C * wr);
+        const int part = (int)args.div_c_rows.div((uint32_t)slot);
         const int cj = slot - part * (C * wr);
-        const int c = cj / wr;
+        const int c = (int)args.div_rows.div((uint32_t)cj);
         const int j = cj - c * wr;
         const int pl = part == 0 ? p_first : 0;
         const int ph_ = part == parts - 1 ? p_last : args.P - 1;
@@ -553,7 +553,7 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       // window position of this pixel's first tap (r = s = 0, c = 0)
       int wbase = -1;
       if (row_valid) {
-        const int p = pq / args.Q, q = pq - p * args.Q;
+        const int p = (int)args.div_q.div((uint32_t)pq), q = pq - p * args.Q;
         const int part = n_img - img0;
         const int pl = part == 0 ? p_first : 0;
         wbase = (part * C * wr + (p - pl) * args.stride_h) * wp + args.win_left + q * args.stride_w - args.pad_w;
