@@ -172,6 +172,11 @@ void fill_common_args(b2c_plan* p) {
                                             : (p->amode == A_GATHER ? 8 * (size_t)p->table_len : 0);
   while (stages > 2 && (size_t)stages * stage_bytes + extra > budget) --stages;
   while (stages > 1 && (size_t)stages * stage_bytes + extra > 196 * 1024) --stages;
+  a.cluster_split = cluster_split_ok(p->emb.variant, a.tile_n, a.split_k) ? 1 : 0;
+  size_t region = (size_t)stages * stage_bytes;
+  // the stage buffers double as the 128 x tile_n int32 exchange tile of the cluster reduction
+  if (a.cluster_split) region = std::max(region, (size_t)kTileM * a.tile_n * 4);
+  a.stage_region = (int)region;
   a.stages = stages;
 }
 
@@ -229,7 +234,7 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
   // Room for one extra box row block so that a TMA box never starts past the allocation.
   if (cudaMalloc(&p->w_packed, p->w_packed_bytes + 256) != cudaSuccess) return fail(B2C_E_CUDA);
   fill_common_args(p);
-  p->ws_total = workspace_bytes_for(g, emb.variant, emb.split_k);
+  p->ws_total = workspace_bytes_for(g, emb.variant, emb.tile_n, emb.split_k);
   if (emb.variant == B2C_VARIANT_CP_TMA) {
     bool direct = d.in_layout == B2C_LAYOUT_NHWC && p->C_pad == d.C;
     p->ws_layout_bytes = direct ? 0 : ((size_t)d.N * d.H * d.W * p->C_pad + 255) / 256 * 256;
@@ -494,7 +499,7 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
 
   // ---- split reduction: partial sums meet in a zeroed int32 buffer ----
   bool need_finish = false;
-  if (a.split_k > 1) {
+  if (a.split_k > 1 && !a.cluster_split) {
     if (d.out_mode == B2C_OUT_I32) {
       a.acc = y32;
     } else {

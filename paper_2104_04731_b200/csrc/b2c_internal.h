@@ -94,6 +94,8 @@ struct ConvArgs {
   int stages;
   int split_k;
   int shift, out_mode, out_layout;
+  int stage_region;   // bytes of shared memory reserved for the stage ring (and the cluster exchange tile)
+  int cluster_split;  // split_k slices form a cluster (1, 1, split_k) and reduce through shared memory
 };
 
 struct Schedule {
@@ -112,18 +114,30 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                               int cluster_z, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (cluster_z > 1) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = (unsigned)cluster_z;
+    cfg.numAttrs = 2;
+  }
+  cfg.attrs = attr;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  return launch_pdl_cluster(kernel, grid, block, smem, st, 1, static_cast<Args&&>(args)...);
 }
 #endif
 
@@ -135,7 +149,16 @@ int cp_block_bytes(int C_pad);       // reduction bytes per block for the channe
 int im2col_k_pad(int Kg);            // padded reduction length for the stencil-unroll maps
 void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out);
 int pick_by_policy(const std::vector<b2c_embedding>& all, int policy);  // index or -1
-size_t workspace_bytes_for(const Geom& g, int variant, int split_k);
+size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k);
+// A split reduction of 2, 4 or 8 slices whose tile is wide enough runs as a thread-block cluster:
+// the slices exchange their partial accumulators through distributed shared memory, so no scratch
+// buffer, zero-fill or finish pass is needed.
+// (The variants that keep a lookup table or an input window in shared memory leave room for a
+// 128-column exchange tile at most.)
+inline bool cluster_split_ok(int variant, int tile_n, int split_k) {
+  const bool table_in_smem = variant == B2C_VARIANT_IM2COL_GATHER || variant == B2C_VARIANT_IM2COL_STAGED;
+  return (split_k == 2 || split_k == 4 || split_k == 8) && tile_n >= 32 * split_k && (!table_in_smem || tile_n <= 128);
+}
 // Geometry of the shared-memory input window of the staged stencil unroll; false if it does not fit.
 struct WindowGeom {
   int rows, pitch, left, parts, bytes;

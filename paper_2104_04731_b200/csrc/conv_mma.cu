@@ -202,15 +202,12 @@ __device__ __forceinline__ void tmem_ld<32>(uint32_t taddr, int32_t* v) {
 // here, and the values go to the NKPQ or NPQK tensor; with a split reduction the partial sums
 // are added into a zeroed int32 buffer instead.
 template <int NC>
-__device__ __forceinline__ void epilogue_columns(const ConvArgs& args, uint32_t taddr, int kbase, bool row_valid,
-                                                 long long base_nkpq, long long base_npqk) {
-  int32_t v[NC];
-  __syncwarp();
-  tmem_ld<NC>(taddr, v);  // warp-collective: executed by all lanes
+__device__ __forceinline__ void store_columns(const ConvArgs& args, const int32_t* v, int kbase, bool row_valid,
+                                              long long base_nkpq, long long base_npqk) {
   const int K = args.K;
   if (!row_valid || kbase >= K) return;
   const bool nhwc = args.out_layout == B2C_LAYOUT_NHWC;
-  if (args.split_k > 1) {
+  if (args.split_k > 1 && !args.cluster_split) {
     // Partial sums of the reduction slices meet in global memory; integer addition is
     // associative, so the order of arrival does not change the result.
     int32_t* dst = args.acc + (nhwc ? base_npqk + kbase : base_nkpq + (long long)kbase * args.PQ);
@@ -277,6 +274,42 @@ __device__ __forceinline__ void epilogue_columns(const ConvArgs& args, uint32_t 
   }
 }
 
+template <int NC>
+__device__ __forceinline__ void epilogue_columns(const ConvArgs& args, uint32_t taddr, int kbase, bool row_valid,
+                                                 long long base_nkpq, long long base_npqk, uint32_t exchange_addr) {
+  int32_t v[NC];
+  __syncwarp();
+  tmem_ld<NC>(taddr, v);  // warp-collective: executed by all lanes
+  if (exchange_addr != 0) {
+    // cluster reduction: the partial sums go to this block's exchange tile [column][row]
+#pragma unroll
+    for (int j = 0; j < NC; ++j)
+      asm volatile("st.shared.b32 [%0], %1;" ::"r"(exchange_addr + (uint32_t)j * (kTileM * 4)), "r"(v[j]) : "memory");
+    return;
+  }
+  store_columns<NC>(args, v, kbase, row_valid, base_nkpq, base_npqk);
+}
+
+// Sum of the cluster's partial tiles for NC columns of one row, read through distributed shared
+// memory (`local_addr` is the row's address in this block's exchange tile; every block of the
+// cluster keeps its tile at the same offset).
+template <int NC>
+__device__ __forceinline__ void cluster_sum_columns(uint32_t local_addr, int split, int32_t* v) {
+#pragma unroll
+  for (int j = 0; j < NC; ++j) v[j] = 0;
+  for (int r = 0; r < split; ++r) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(r));
+    // all loads of a slice are issued before the first use, so that they are in flight together
+    int32_t t[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j)
+      asm volatile("ld.shared::cluster.b32 %0, [%1];" : "=r"(t[j]) : "r"(remote + (uint32_t)j * (kTileM * 4)) : "memory");
+#pragma unroll
+    for (int j = 0; j < NC; ++j) v[j] += t[j];
+  }
+}
+
 template <int AMODE>
 __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                                              const __grid_constant__ CUtensorMap tmap_b,
@@ -300,7 +333,7 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   const uint32_t a_base = smem_base;
   const uint32_t b_base = smem_base + stages * a_stage_bytes;
   uint8_t* smem_aligned = smem_raw + (smem_base - smem_u32(smem_raw));
-  uint8_t* smem_extra = smem_aligned + stages * (a_stage_bytes + b_stage_bytes);
+  uint8_t* smem_extra = smem_aligned + args.stage_region;
   GatherEntry* s_table = reinterpret_cast<GatherEntry*>(smem_extra);              // A_GATHER
   int32_t* s_table32 = reinterpret_cast<int32_t*>(smem_extra);                    // A_STAGED
   uint8_t* s_window = smem_extra + ((args.table_len * 4 + 15) & ~15);             // A_STAGED
@@ -639,15 +672,59 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       const int c_begin = half * cols;
       if (c_begin < args.tile_n) {
         const uint32_t taddr = tmem_acc + ((uint32_t)(quad * 32) << 16) + (uint32_t)c_begin;
+        // cluster reduction: the stage buffers are free once the accumulator is complete
+        const uint32_t xch = args.cluster_split ? a_base + (uint32_t)row * 4u + (uint32_t)c_begin * (kTileM * 4) : 0u;
         if ((cols & 31) == 0) {
           for (int c = 0; c < cols; c += 32)
-            epilogue_columns<32>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk);
+            epilogue_columns<32>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk,
+                                 xch ? xch + (uint32_t)c * (kTileM * 4) : 0u);
         } else {
           for (int c = 0; c < cols; c += 16)
-            epilogue_columns<16>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk);
+            epilogue_columns<16>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk,
+                                 xch ? xch + (uint32_t)c * (kTileM * 4) : 0u);
         }
       }
     }
+  }
+
+  if (args.cluster_split) {
+    // ---------------------------------------------------------------- cluster reduction
+    // Barrier 1: every slice's partial tile is in its block's shared memory.  Then block `rank`
+    // sums columns [rank * tile_n / split, (rank + 1) * tile_n / split) over all slices, applies the
+    // epilogue and stores.  Barrier 2: no block leaves while its tile may still be read.
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+    if (warp >= 2 && !ctl.abort_flag) {
+      const int quad = warp & 3, half = (warp - 2) >> 2;
+      const int row = quad * 32 + lane;
+      const unsigned m = (unsigned)m0 + (unsigned)row;
+      const bool row_valid = m < (unsigned)args.Mg;
+      int n_img = 0, pq = 0;
+      if (row_valid) {
+        n_img = (int)args.div_pq.div(m);
+        pq = (int)(m - (unsigned)n_img * (unsigned)args.PQ);
+      }
+      const long long base_nkpq = (long long)n_img * args.K * args.PQ + pq;
+      const long long base_npqk = (long long)m * args.K;
+      const int w = args.tile_n / (2 * args.split_k);  // columns of this thread's slice (>= 16)
+      const int col0 = (int)blockIdx.z * (args.tile_n / args.split_k) + half * w;
+      const uint32_t xch = a_base + (uint32_t)row * 4u + (uint32_t)col0 * (kTileM * 4);
+      if ((w & 31) == 0) {
+        for (int c = 0; c < w; c += 32) {
+          int32_t v[32];
+          cluster_sum_columns<32>(xch + (uint32_t)c * (kTileM * 4), args.split_k, v);
+          store_columns<32>(args, v, n0 + col0 + c, row_valid, base_nkpq, base_npqk);
+        }
+      } else {
+        for (int c = 0; c < w; c += 16) {
+          int32_t v[16];
+          cluster_sum_columns<16>(xch + (uint32_t)c * (kTileM * 4), args.split_k, v);
+          store_columns<16>(args, v, n0 + col0 + c, row_valid, base_nkpq, base_npqk);
+        }
+      }
+    }
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
   }
 
   // ---------------------------------------------------------------- teardown
@@ -671,7 +748,7 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
 }  // namespace
 
 size_t conv_mma_smem_bytes(int amode, const ConvArgs& a) {
-  size_t b = 1024 + (size_t)a.stages * (kTileM + a.tile_n) * a.bk;
+  size_t b = 1024 + (size_t)a.stage_region;
   if (amode == A_GATHER) b += (size_t)a.table_len * sizeof(GatherEntry);
   if (amode == A_STAGED) b += (size_t)((a.table_len * 4 + 15) & ~15) + (size_t)a.win_bytes + 16;
   return b;
@@ -691,7 +768,8 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
       if (e != cudaSuccess) return e;                                                                     \
       configured = 200 * 1024;                                                                            \
     }                                                                                                     \
-    e = launch_pdl(conv_mma_kernel<MODE>, grid, dim3(kThreads), smem, st, *tmap_a, *tmap_b, args);        \
+    e = launch_pdl_cluster(conv_mma_kernel<MODE>, grid, dim3(kThreads), smem, st,                        \
+                           args.cluster_split ? args.split_k : 1, *tmap_a, *tmap_b, args);                \
     if (e != cudaSuccess) return e;                                                                       \
   }
   if (amode == A_TILED) B2C_LAUNCH(A_TILED)

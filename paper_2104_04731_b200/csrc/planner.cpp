@@ -77,7 +77,7 @@ static int tmem_pow2(int n) {
   return c;
 }
 
-size_t workspace_bytes_for(const Geom& g, int variant, int split_k) {
+size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k) {
   size_t ws = 0;
   const b2c_conv_desc& d = g.d;
   if (variant == B2C_VARIANT_CP_TMA) {
@@ -90,7 +90,7 @@ size_t workspace_bytes_for(const Geom& g, int variant, int split_k) {
   ws = (ws + 255) / 256 * 256;
   // A split reduction accumulates int32 partial sums in scratch unless the int32 output itself
   // can serve (int32-only output in any layout).
-  if (split_k > 1 && (d.out_mode & B2C_OUT_I8)) ws += (size_t)g.y_elems * 4;
+  if (split_k > 1 && !cluster_split_ok(variant, tile_n, split_k) && (d.out_mode & B2C_OUT_I8)) ws += (size_t)g.y_elems * 4;
   return ws;
 }
 
@@ -166,10 +166,10 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
     else
       moved = g.x_elems + (long long)d.K * K_pad + g.y_elems;
   }
-  if (split_k > 1) moved += 2 * g.y_elems;  // partial sums written and read once more
+  if (split_k > 1 && !cluster_split_ok(variant, tile_n, split_k)) moved += 2 * g.y_elems;  // partial sums through memory
   e.o_mac = M_pad * N_pad * k_issued - mac_min;
   e.o_data = moved - data_min;
-  e.workspace_bytes = (int64_t)workspace_bytes_for(g, variant, split_k);
+  e.workspace_bytes = (int64_t)workspace_bytes_for(g, variant, tile_n, split_k);
   out->push_back(e);
 }
 
