@@ -165,7 +165,20 @@ void fill_common_args(b2c_plan* p) {
   int per_cta_kb = (a.num_kb + a.split_k - 1) / a.split_k;
   int stages = std::min(6, std::max(1, per_cta_kb));
   const long long ctas = ((p->g.Mg + kTileM - 1) / kTileM) * ((d.K + a.tile_n - 1) / a.tile_n) * a.split_k;
-  const size_t budget = ctas > kNumSMs ? 100 * 1024 : 160 * 1024;
+  // Large TMA-fed problems run persistently: one block per SM walks the tile list with two
+  // accumulator buffers in tensor memory and the deepest stage ring that fits.
+  const long long tiles_m = (p->g.Mg + kTileM - 1) / kTileM;
+  const int tiles_n = (d.K + a.tile_n - 1) / a.tile_n;
+  a.tiles_n = tiles_n;
+  a.num_tiles = (int)std::min<long long>(tiles_m * tiles_n, 0x7FFFFFFF);
+  a.div_tiles_n = make_fastdiv((uint32_t)tiles_n);
+  // (narrow tiles have short main loops and do better with several small blocks per SM)
+  a.persistent = ((p->amode == A_TILED || p->amode == A_IM2COL_TMA) && a.split_k == 1 && a.tile_n >= 128 &&
+                  tiles_m * tiles_n > 2 * kNumSMs && tiles_m * tiles_n < 0x7FFFFFFF)
+                     ? 1
+                     : 0;
+  a.tmem_bufs = (a.persistent && 2 * a.tmem_cols <= 512) ? 2 : 1;
+  const size_t budget = a.persistent ? 196 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 160 * 1024);
   const size_t stage_bytes = (size_t)(kTileM + a.tile_n) * a.bk;
   // lookup table and staged window share the block's shared memory with the stages
   const size_t extra = p->amode == A_STAGED ? (size_t)p->win.bytes + 4 * (size_t)p->table_len + 64

@@ -94,6 +94,10 @@ struct ConvArgs {
   int stages;
   int split_k;
   int shift, out_mode, out_layout;
+  // persistent mode: gridDim.x blocks walk num_tiles tiles (tiles_n column tiles per row tile);
+  // tmem_bufs accumulator buffers of tmem_cols columns each
+  int persistent, num_tiles, tiles_n, tmem_bufs;
+  FastDiv div_tiles_n;
   int stage_region;   // bytes of shared memory reserved for the stage ring (and the cluster exchange tile)
   int cluster_split;  // split_k slices form a cluster (1, 1, split_k) and reduce through shared memory
 };

@@ -12,6 +12,8 @@
 // Shared-memory stages form a ring guarded by full/empty mbarriers.  Every wait is bounded:
 // on expiry the block raises an abort flag, records B2C_E_TIMEOUT in the status word, lets
 // copies in flight drain, frees its tensor memory and returns.
+#include <algorithm>
+
 #include "b2c_internal.h"
 
 namespace b2c {
@@ -25,7 +27,8 @@ constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s
 struct __align__(8) SharedCtl {
   unsigned long long full[8];
   unsigned long long empty[8];
-  unsigned long long tmem_full;
+  unsigned long long tmem_full[2];   // accumulator buffer b complete (MMA warp -> epilogue warps)
+  unsigned long long tmem_empty[2];  // accumulator buffer b drained (epilogue warps -> MMA warp)
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -319,8 +322,26 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * kTileM;
-  const int n0 = blockIdx.y * args.tile_n;
+  // Tile schedule.  Small grids: one tile per block, (blockIdx.x, blockIdx.y) = (row tile, column
+  // tile).  Persistent mode (large TMA-fed problems): gridDim.x blocks walk the tile list
+  // t = blockIdx.x, blockIdx.x + gridDim.x, ... with the column tile fastest (blocks running at the
+  // same time share the A operand in L2), and the accumulator alternates between two tensor-memory
+  // buffers so that the epilogue of one tile overlaps the main loop of the next.
+  const bool persistent = args.persistent != 0;
+  const int tile_first = persistent ? (int)blockIdx.x : 0;
+  const int tile_step = persistent ? (int)gridDim.x : 1;
+  const int tile_end = persistent ? args.num_tiles : 1;
+  const int nbuf = args.tmem_bufs;
+#define B2C_TILE_ORIGIN(t)                                                          \
+  int m0, n0;                                                                       \
+  if (persistent) {                                                                 \
+    const int mt_ = (int)args.div_tiles_n.div((uint32_t)(t));                       \
+    m0 = mt_ * kTileM;                                                              \
+    n0 = ((t) - mt_ * args.tiles_n) * args.tile_n;                                  \
+  } else {                                                                          \
+    m0 = (int)blockIdx.x * kTileM;                                                  \
+    n0 = (int)blockIdx.y * args.tile_n;                                             \
+  }
   const int kb_begin = (int)((unsigned)blockIdx.z * (unsigned)args.num_kb / (unsigned)args.split_k);
   const int kb_end = (int)((unsigned)(blockIdx.z + 1) * (unsigned)args.num_kb / (unsigned)args.split_k);
   const int stages = args.stages;
@@ -345,7 +366,10 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       mbar_init(smem_u32(&ctl.empty[lane]), 1);
     }
     if (lane == 8) {
-      mbar_init(smem_u32(&ctl.tmem_full), 1);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(smem_u32(&ctl.tmem_full[b]), 1);
+        mbar_init(smem_u32(&ctl.tmem_empty[b]), kGatherWarps);
+      }
       ctl.abort_flag = 0;
     }
     if (lane == 9 && !kThreadsFormA) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
@@ -354,7 +378,7 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
-                 "r"(args.tmem_cols)
+                 "r"(args.tmem_cols * nbuf)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -379,7 +403,13 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   // cost hundreds of cycles of dependent issue.
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
-    {
+    int s = 0;
+    uint32_t ph = 0;
+    uint32_t a_dst = a_base, b_dst = b_base;
+    const uint32_t leader = elect_one() ? 1u : 0u;
+    bool alive = true;
+    for (int t = tile_first; t < tile_end && alive; t += tile_step) {
+      B2C_TILE_ORIGIN(t)
       int n_img = 0, h_org = 0, w_org = 0, cb = 0, sx = 0, r = 0;
       if (AMODE == A_IM2COL_TMA) {
         n_img = (int)args.div_pq.div((uint32_t)m0);
@@ -392,13 +422,12 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
         r = tap / args.S;
         sx = tap - r * args.S;
       }
-      int s = 0;
-      uint32_t ph = 0;
-      uint32_t a_dst = a_base, b_dst = b_base;
       int kcol = kb_begin * bk;  // column of the packed weight matrix = reduction offset in bytes
-      const uint32_t leader = elect_one() ? 1u : 0u;
       for (int kb = kb_begin; kb < kb_end; ++kb) {
-        if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) break;
+        if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) {
+          alive = false;
+          break;
+        }
         const uint32_t full = smem_u32(&ctl.full[s]);
         if (kThreadsFormA) {
           mbar_arrive_expect_tx(full, b_stage_bytes, leader);
@@ -442,12 +471,24 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       uint64_t adesc = adesc0, bdesc = bdesc0;
       int s = 0;
       uint32_t ph = 0;
-      uint32_t accumulate = 0;
       // The same lane issues every MMA and the commits that track them.
       const uint32_t leader = elect_one() ? 1u : 0u;
+      bool alive = true;
+      int ti = 0;
+      for (int t = tile_first; t < tile_end && alive; t += tile_step, ++ti) {
+      const int buf = ti % nbuf;
+      const uint32_t use = (uint32_t)(ti / nbuf);
+      // the epilogue must have drained this accumulator buffer (first use passes at once)
+      if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status)) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t d_tmem = tmem_acc + (uint32_t)(buf * args.tmem_cols);
+      uint32_t accumulate = 0;
       bool ready = false;  // result of the look-ahead test of this stage's full barrier
       for (int kb = kb_begin; kb < kb_end; ++kb) {
-        if (!ready && !mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status)) break;
+        if (!ready && !mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status)) {
+          alive = false;
+          break;
+        }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int ksteps = (kb == args.num_kb - 1) ? args.ksteps_last : args.ksteps_full;
         const int s_cur = s;
@@ -464,12 +505,13 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
         ready = (kb + 1 < kb_end) && mbar_test_wait(smem_u32(&ctl.full[s]), ph);
         for (int k = 0; k < ksteps; ++k) {
           // Advancing 32 bytes along the row = 2 units of 16 bytes in the descriptor address.
-          mma_i8(tmem_acc, a_cur + (uint64_t)(2 * k), b_cur + (uint64_t)(2 * k), idesc, (accumulate | (uint32_t)k),
+          mma_i8(d_tmem, a_cur + (uint64_t)(2 * k), b_cur + (uint64_t)(2 * k), idesc, (accumulate | (uint32_t)k),
                  leader);
         }
         mma_commit(smem_u32(&ctl.empty[s_cur]), leader);
-        if (kb == kb_end - 1) mma_commit(smem_u32(&ctl.tmem_full), leader);
+        if (kb == kb_end - 1) mma_commit(smem_u32(&ctl.tmem_full[buf]), leader);
         accumulate = 1;
+      }
       }
     }
     __syncwarp();
@@ -478,6 +520,10 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
     const int quad = warp & 3;          // TMEM lane quadrant this warp may read
     const int half = (warp - 2) >> 2;   // two warps share a quadrant and split the columns / chunks
     const int row = quad * 32 + lane;   // accumulator row = A-tile row
+    bool ok = true;
+    int ti = 0;
+    for (int t = tile_first; t < tile_end && ok; t += tile_step, ++ti) {
+    B2C_TILE_ORIGIN(t)
     const unsigned m = (unsigned)m0 + (unsigned)row;
     const bool row_valid = m < (unsigned)args.Mg;
     int n_img = 0, pq = 0;
@@ -485,7 +531,6 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       n_img = (int)args.div_pq.div(m);
       pq = (int)(m - (unsigned)n_img * (unsigned)args.PQ);
     }
-    bool ok = true;
 
     if (AMODE == A_GATHER) {
       // Stencil unroll formed in place: this thread writes half of row `row` of the A tile (four
@@ -662,7 +707,9 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
     }
 
     // ---- epilogue ----
-    if (ok) ok = mbar_wait(smem_u32(&ctl.tmem_full), 0u, &ctl, args.status);
+    const int buf = ti % nbuf;
+    const uint32_t use = (uint32_t)(ti / nbuf);
+    if (ok) ok = mbar_wait(smem_u32(&ctl.tmem_full[buf]), use & 1u, &ctl, args.status);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
       // Output index of (m, k): NKPQ -> (n*K + k)*PQ + pq ; NPQK -> m*K + k.
@@ -671,7 +718,8 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       const int cols = args.tile_n >= 32 ? (args.tile_n >> 1) : 16;  // columns handled by this warp
       const int c_begin = half * cols;
       if (c_begin < args.tile_n) {
-        const uint32_t taddr = tmem_acc + ((uint32_t)(quad * 32) << 16) + (uint32_t)c_begin;
+        const uint32_t taddr =
+            tmem_acc + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * args.tmem_cols) + (uint32_t)c_begin;
         // cluster reduction: the stage buffers are free once the accumulator is complete
         const uint32_t xch = args.cluster_split ? a_base + (uint32_t)row * 4u + (uint32_t)c_begin * (kTileM * 4) : 0u;
         if ((cols & 31) == 0) {
@@ -684,10 +732,16 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
                                  xch ? xch + (uint32_t)c * (kTileM * 4) : 0u);
         }
       }
+      // this warp has read its part of the accumulator buffer: hand it back to the MMA warp
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
     }
+    }  // tile loop
   }
 
   if (args.cluster_split) {
+    B2C_TILE_ORIGIN(0)
     // ---------------------------------------------------------------- cluster reduction
     // Barrier 1: every slice's partial tile is in its block's shared memory.  Then block `rank`
     // sums columns [rank * tile_n / split, (rank + 1) * tile_n / split) over all slices, applies the
@@ -740,7 +794,7 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   }
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(args.tmem_cols)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(args.tmem_cols * nbuf)
                  : "memory");
   }
 }
@@ -759,6 +813,7 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
   const size_t smem = conv_mma_smem_bytes(amode, args);
   dim3 grid((unsigned)((args.Mg + kTileM - 1) / kTileM), (unsigned)((args.K + args.tile_n - 1) / args.tile_n),
             (unsigned)args.split_k);
+  if (args.persistent) grid = dim3((unsigned)std::min(args.num_tiles, kNumSMs), 1, 1);
   cudaError_t e;
 #define B2C_LAUNCH(MODE)                                                                                  \
   {                                                                                                       \
@@ -777,6 +832,7 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
   else if (amode == A_STAGED) B2C_LAUNCH(A_STAGED)
   else B2C_LAUNCH(A_GATHER)
 #undef B2C_LAUNCH
+#undef B2C_TILE_ORIGIN
   return cudaGetLastError();
 }
 

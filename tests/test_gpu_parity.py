@@ -226,3 +226,18 @@ def test_back_to_back_runs_keep_stream_order(lib, variant):
         assert np.array_equal(y8.cpu().numpy(), refs[i & 1][1]), i
     assert plan.device_status() == b2c.OK
     plan.destroy()
+
+
+# ---- grids much larger than the machine: persistent blocks, two accumulator buffers --------------------
+@pytest.mark.parametrize("tile_n", [32, 128])
+def test_large_grid_persistent_tiles(lib, tile_n):
+    N, C, H, W, K, R, S = 24, 64, 28, 28, 128, 3, 3   # 18816 output pixels = 147 row tiles
+    x = int8_uniform((N, C, H, W), 701)
+    w = int8_uniform((K, C, R, S), 702)
+    ref = oracle.conv2d_int8(x, w, 1, 1, 1, 9)
+    for in_layout, out_layout in ((0, 0), (1, 1)):
+        d = lib.make_desc(N, C, H, W, K, R, S, 1, 1, 1, 9, in_layout, out_layout, 3)
+        for variant in (0, 1):
+            ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant and e.tile_n == tile_n and e.split_k == 1]
+            assert ids
+            check_against_oracle(x, w, 1, 1, 1, 9, 3, ids[0], ref=ref, in_layout=in_layout, out_layout=out_layout)
