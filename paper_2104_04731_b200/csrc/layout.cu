@@ -303,7 +303,7 @@ int grid_for(long long total, int block) {
 cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, int H, int W, int C_pad,
                                     cudaStream_t st) {
   const int HW = H * W;
-  const int CT = C_pad >= 128 ? 128 : 64;
+  int CT = C_pad >= 128 ? 128 : 64;
   const bool a16 = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
   // Bulk-copy kernels: channels in whole groups of 16 and either the whole image per tile
   // (H*W <= 256, a multiple of 4) or rows that are multiples of 16 bytes.
@@ -311,6 +311,8 @@ cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, 
     const bool row_mode = HW > 256;
     const int PT = row_mode ? 256 : HW;
     const int hw_tiles = (HW + PT - 1) / PT;
+    // small tensors: narrower channel tiles so that the grid still covers the machine
+    while (CT > 32 && (long long)hw_tiles * N * ((C_pad + CT - 1) / CT) < 2 * kNumSMs) CT >>= 1;
     const size_t smem = (size_t)(CT / 16) * (16 * PT + 16);
     dim3 grid((unsigned)hw_tiles * (unsigned)N, (C_pad + CT - 1) / CT, 1);
     if (row_mode)

@@ -231,7 +231,7 @@ def test_back_to_back_runs_keep_stream_order(lib, variant):
 # ---- grids much larger than the machine: persistent blocks, two accumulator buffers --------------------
 @pytest.mark.parametrize("tile_n", [32, 128])
 def test_large_grid_persistent_tiles(lib, tile_n):
-    N, C, H, W, K, R, S = 24, 64, 28, 28, 128, 3, 3   # 18816 output pixels = 147 row tiles
+    N, C, H, W, K, R, S = 56, 64, 28, 28, 128, 3, 3   # 43904 output pixels = 343 row tiles (> 2 per SM)
     x = int8_uniform((N, C, H, W), 701)
     w = int8_uniform((K, C, R, S), 702)
     ref = oracle.conv2d_int8(x, w, 1, 1, 1, 9)
