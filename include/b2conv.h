@@ -149,6 +149,12 @@ int b2c_conv2d_int8_host(int N, int C, int H, int W, int K, int R, int S, int st
  * B2C_E_TIMEOUT if a kernel of this plan gave up on a bounded wait; the word is then cleared. */
 int b2c_plan_device_status(b2c_plan* plan, int32_t* status);
 
+/* Failure-detection self-test (no counterpart in the paper): enqueues a one-block kernel that
+ * waits, with the bounded wait every kernel of this library uses, on a barrier nothing completes.
+ * After the wait's limit (about one second) the kernel records B2C_E_TIMEOUT in the plan's status
+ * word and returns normally; b2c_plan_device_status then reports it and the plan stays usable. */
+int b2c_selftest_bounded_wait(b2c_plan* plan, void* cuda_stream);
+
 void b2c_plan_destroy(b2c_plan* plan);
 
 /* Layout rewrites on their own (the Pad / Reorder / Stencil Unroll rules of Table 2), exposed so

@@ -25,7 +25,7 @@ VARIANT_NAMES = {0: "channel_pack_tma_im2col", 1: "im2col_explicit", 2: "im2col_
 EXPORTS = [
     "b2c_out_shape", "b2c_enumerate", "b2c_plan_create", "b2c_plan_info", "b2c_plan_workspace_bytes",
     "b2c_plan_set_weights", "b2c_conv2d_int8_run", "b2c_conv2d_int8", "b2c_conv2d_int8_host",
-    "b2c_plan_device_status", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
+    "b2c_plan_device_status", "b2c_selftest_bounded_wait", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
     "b2c_status_string",
     "b2c_last_cuda_error",
 ]
@@ -85,6 +85,7 @@ def load():
     lib.b2c_conv2d_int8_host.argtypes = [i32] * 11 + [vp] * 4
     lib.b2c_plan_device_status.argtypes = [vp, pi32]
     lib.b2c_plan_destroy.argtypes = [vp]
+    lib.b2c_selftest_bounded_wait.argtypes = [vp, vp]
     lib.b2c_plan_destroy.restype = None
     lib.b2c_pack_activations.argtypes = [vp, vp] + [i32] * 5 + [vp]
     lib.b2c_im2col.argtypes = [pd, vp, vp, i32, vp]
@@ -181,6 +182,10 @@ class Plan:
         s = ctypes.c_int32()
         _check(self._lib.b2c_plan_device_status(self._h, ctypes.byref(s)), "b2c_plan_device_status")
         return s.value
+
+    def selftest_bounded_wait(self, stream=None):
+        """Enqueues the bounded-wait self-test; afterwards device_status() reports E_TIMEOUT once."""
+        _check(self._lib.b2c_selftest_bounded_wait(self._h, _stream_ptr(stream)), "b2c_selftest_bounded_wait")
 
     def destroy(self):
         if getattr(self, "_h", None):

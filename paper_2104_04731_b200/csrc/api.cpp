@@ -536,6 +536,12 @@ int b2c_plan_device_status(b2c_plan* p, int32_t* status) {
   return B2C_OK;
 }
 
+int b2c_selftest_bounded_wait(b2c_plan* p, void* cuda_stream) {
+  if (!p) return B2C_E_INVALID_ARG;
+  CUDA_TRY(launch_bounded_wait_selftest(p->status, (cudaStream_t)cuda_stream));
+  return B2C_OK;
+}
+
 void b2c_plan_destroy(b2c_plan* p) {
   if (!p) return;
   cudaFree(p->w_packed);

@@ -199,5 +199,6 @@ cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, l
 cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,
                             cudaStream_t st);
 size_t conv_mma_smem_bytes(int amode, const ConvArgs& args);
+cudaError_t launch_bounded_wait_selftest(int* status, cudaStream_t st);
 
 }  // namespace b2c

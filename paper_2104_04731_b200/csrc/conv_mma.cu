@@ -799,7 +799,26 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   }
 }
 
+// One block waits, with the same bounded wait the convolution kernel uses, on a barrier that
+// nothing ever completes.  The wait gives up after its time limit, records B2C_E_TIMEOUT in
+// `status` and the kernel returns normally: the context stays usable.
+__global__ void bounded_wait_selftest_kernel(int* status) {
+  __shared__ SharedCtl ctl;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&ctl.full[0]), 1);
+    ctl.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  mbar_wait(smem_u32(&ctl.full[0]), 0u, &ctl, status);
+}
+
 }  // namespace
+
+cudaError_t launch_bounded_wait_selftest(int* status, cudaStream_t st) {
+  bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(status);
+  return cudaGetLastError();
+}
 
 size_t conv_mma_smem_bytes(int amode, const ConvArgs& a) {
   size_t b = 1024 + (size_t)a.stage_region;

@@ -241,3 +241,25 @@ def test_large_grid_persistent_tiles(lib, tile_n):
             ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant and e.tile_n == tile_n and e.split_k == 1]
             assert ids
             check_against_oracle(x, w, 1, 1, 1, 9, 3, ids[0], ref=ref, in_layout=in_layout, out_layout=out_layout)
+
+
+# ---- failure detection: a wait that cannot complete ends by itself and is reported --------------------
+def test_bounded_wait_reports_timeout_and_plan_stays_usable(lib):
+    cfg = CONFIGS[0]
+    x, w, ref = cfg_reference(cfg)
+    d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
+                      out_mode=3)
+    plan = lib.Plan(d, b2c.POLICY_MIN_OVERHEAD)
+    plan.set_weights(to_dev(w))
+    plan.selftest_bounded_wait()            # waits on a barrier nothing completes: gives up after its limit
+    torch.cuda.synchronize()
+    assert plan.device_status() == b2c.E_TIMEOUT
+    assert plan.device_status() == b2c.OK   # the status word is cleared by the read
+    y32 = torch.zeros(ref[0].shape, dtype=torch.int32, device="cuda")
+    y8 = torch.zeros(ref[0].shape, dtype=torch.int8, device="cuda")
+    ws = torch.zeros(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
+    plan.run(to_dev(x), y32, y8, ws)        # the context and the plan still work
+    torch.cuda.synchronize()
+    assert plan.device_status() == b2c.OK
+    assert np.array_equal(y32.cpu().numpy(), ref[0]) and np.array_equal(y8.cpu().numpy(), ref[1])
+    plan.destroy()
