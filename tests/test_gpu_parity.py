@@ -263,3 +263,37 @@ def test_bounded_wait_reports_timeout_and_plan_stays_usable(lib):
     assert plan.device_status() == b2c.OK
     assert np.array_equal(y32.cpu().numpy(), ref[0]) and np.array_equal(y8.cpu().numpy(), ref[1])
     plan.destroy()
+
+
+# ---- degenerate and extreme shapes ----------------------------------------------------------------------
+_EDGE = [
+    # N, C, H, W, K, R, S, stride, pad, dil, shift
+    (1, 1, 1, 1, 1, 1, 1, 1, 0, 1, 0),            # a single multiply
+    (3, 2, 1, 1, 5, 3, 3, 1, 1, 1, 2),            # 1x1 image, every tap but the centre is padding
+    (2, 4, 5, 7, 3, 5, 7, 1, 0, 1, 4),            # kernel as large as the image: P = Q = 1
+    (40, 3, 3, 3, 9, 2, 2, 1, 0, 1, 3),           # P*Q = 4: one tile spans 32 images
+    (1, 8, 9, 9, 4, 2, 2, (4, 5), 0, 1, 1),       # stride larger than the kernel
+    (1, 2, 20, 20, 6, 3, 3, 1, 6, (7, 5), 5),     # dilation wider than half the image, pad 6
+    (2, 32, 4, 4, 7, 1, 1, 1, 0, 1, 6),           # C*R*S exactly one MMA K step
+    (1, 43, 5, 5, 33, 3, 1, 1, (1, 0), 1, 7),     # C*R*S = 129: one byte into the second 128-byte block
+    (1, 131071, 1, 2, 2, 1, 1, 1, 0, 1, 20),      # the largest reduction length the library accepts
+    (1, 1, 3, 300, 2, 1, 280, 1, 0, 1, 8),        # one very wide run of taps
+]
+
+
+@pytest.mark.parametrize("case", _EDGE, ids=lambda c: "n%dc%dh%dw%dk%dr%ds%d" % c[:7])
+def test_edge_shapes(lib, case):
+    N, C, H, W, K, R, S, stride, pad, dil, shift = case
+    x = int8_uniform((N, C, H, W), 811)
+    w = int8_uniform((K, C, R, S), 812)
+    ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode=3)
+    embs = lib.enumerate_embeddings(d)
+    assert embs
+    done = set()
+    for e in embs:
+        key = (e.variant, e.split_k > 1)
+        if key in done:
+            continue
+        done.add(key)
+        check_against_oracle(x, w, stride, pad, dil, shift, 3, e.id, ref=ref)
