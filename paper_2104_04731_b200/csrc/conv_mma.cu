@@ -313,8 +313,8 @@ __device__ __forceinline__ void cluster_sum_columns(uint32_t local_addr, int spl
   }
 }
 
-template <int AMODE>
-__global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constant__ CUtensorMap tmap_a,
+template <int AMODE, bool PERSIST>
+__global__ void __launch_bounds__(kThreads, PERSIST ? 1 : 3) conv_mma_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                                              const __grid_constant__ CUtensorMap tmap_b,
                                                              const ConvArgs args) {
   extern __shared__ uint8_t smem_raw[];
@@ -327,11 +327,13 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
   // t = blockIdx.x, blockIdx.x + gridDim.x, ... with the column tile fastest (blocks running at the
   // same time share the A operand in L2), and the accumulator alternates between two tensor-memory
   // buffers so that the epilogue of one tile overlaps the main loop of the next.
-  const bool persistent = args.persistent != 0;
+  // (PERSIST is a template parameter so that the one-tile-per-block instantiation carries none of
+  // the loop, buffer-index and hand-back overhead.)
+  constexpr bool persistent = PERSIST;
   const int tile_first = persistent ? (int)blockIdx.x : 0;
   const int tile_step = persistent ? (int)gridDim.x : 1;
   const int tile_end = persistent ? args.num_tiles : 1;
-  const int nbuf = args.tmem_bufs;
+  const int nbuf = persistent ? args.tmem_bufs : 1;
 #define B2C_TILE_ORIGIN(t)                                                          \
   int m0, n0;                                                                       \
   if (persistent) {                                                                 \
@@ -366,9 +368,11 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       mbar_init(smem_u32(&ctl.empty[lane]), 1);
     }
     if (lane == 8) {
-      for (int b = 0; b < 2; ++b) {
-        mbar_init(smem_u32(&ctl.tmem_full[b]), 1);
-        mbar_init(smem_u32(&ctl.tmem_empty[b]), kGatherWarps);
+      mbar_init(smem_u32(&ctl.tmem_full[0]), 1);
+      if (persistent) {
+        mbar_init(smem_u32(&ctl.tmem_full[1]), 1);
+        mbar_init(smem_u32(&ctl.tmem_empty[0]), kGatherWarps);
+        mbar_init(smem_u32(&ctl.tmem_empty[1]), kGatherWarps);
       }
       ctl.abort_flag = 0;
     }
@@ -476,11 +480,13 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
       bool alive = true;
       int ti = 0;
       for (int t = tile_first; t < tile_end && alive; t += tile_step, ++ti) {
-      const int buf = ti % nbuf;
-      const uint32_t use = (uint32_t)(ti / nbuf);
-      // the epilogue must have drained this accumulator buffer (first use passes at once)
-      if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status)) break;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int buf = persistent ? ti % nbuf : 0;
+      const uint32_t use = persistent ? (uint32_t)(ti / nbuf) : 0u;
+      if (persistent) {
+        // the epilogue must have drained this accumulator buffer (first use passes at once)
+        if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status)) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      }
       const uint32_t d_tmem = tmem_acc + (uint32_t)(buf * args.tmem_cols);
       uint32_t accumulate = 0;
       bool ready = false;  // result of the look-ahead test of this stage's full barrier
@@ -707,8 +713,8 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
     }
 
     // ---- epilogue ----
-    const int buf = ti % nbuf;
-    const uint32_t use = (uint32_t)(ti / nbuf);
+    const int buf = persistent ? ti % nbuf : 0;
+    const uint32_t use = persistent ? (uint32_t)(ti / nbuf) : 0u;
     if (ok) ok = mbar_wait(smem_u32(&ctl.tmem_full[buf]), use & 1u, &ctl, args.status);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
@@ -732,10 +738,12 @@ __global__ void __launch_bounds__(kThreads) conv_mma_kernel(const __grid_constan
                                  xch ? xch + (uint32_t)c * (kTileM * 4) : 0u);
         }
       }
-      // this warp has read its part of the accumulator buffer: hand it back to the MMA warp
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+      if (persistent) {
+        // this warp has read its part of the accumulator buffer: hand it back to the MMA warp
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctl.tmem_empty[buf]));
+      }
     }
     }  // tile loop
   }
@@ -834,22 +842,25 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
             (unsigned)args.split_k);
   if (args.persistent) grid = dim3((unsigned)std::min(args.num_tiles, kNumSMs), 1, 1);
   cudaError_t e;
-#define B2C_LAUNCH(MODE)                                                                                  \
+#define B2C_LAUNCH(MODE, PERS)                                                                             \
   {                                                                                                       \
     static size_t configured = 0;                                                                         \
     if (smem > configured) {                                                                              \
-      e = cudaFuncSetAttribute(conv_mma_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); \
+      e = cudaFuncSetAttribute(conv_mma_kernel<MODE, PERS>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
+                               200 * 1024);                                                               \
       if (e != cudaSuccess) return e;                                                                     \
       configured = 200 * 1024;                                                                            \
     }                                                                                                     \
-    e = launch_pdl_cluster(conv_mma_kernel<MODE>, grid, dim3(kThreads), smem, st,                        \
+    e = launch_pdl_cluster(conv_mma_kernel<MODE, PERS>, grid, dim3(kThreads), smem, st,                   \
                            args.cluster_split ? args.split_k : 1, *tmap_a, *tmap_b, args);                \
     if (e != cudaSuccess) return e;                                                                       \
   }
-  if (amode == A_TILED) B2C_LAUNCH(A_TILED)
-  else if (amode == A_IM2COL_TMA) B2C_LAUNCH(A_IM2COL_TMA)
-  else if (amode == A_STAGED) B2C_LAUNCH(A_STAGED)
-  else B2C_LAUNCH(A_GATHER)
+  if (amode == A_TILED && args.persistent) B2C_LAUNCH(A_TILED, true)
+  else if (amode == A_TILED) B2C_LAUNCH(A_TILED, false)
+  else if (amode == A_IM2COL_TMA && args.persistent) B2C_LAUNCH(A_IM2COL_TMA, true)
+  else if (amode == A_IM2COL_TMA) B2C_LAUNCH(A_IM2COL_TMA, false)
+  else if (amode == A_STAGED) B2C_LAUNCH(A_STAGED, false)
+  else B2C_LAUNCH(A_GATHER, false)
 #undef B2C_LAUNCH
 #undef B2C_TILE_ORIGIN
   return cudaGetLastError();
