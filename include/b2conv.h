@@ -67,11 +67,15 @@ typedef struct {
 #define B2C_AXIS_K 2   /* output channels                                                        */
 #define B2C_AXIS_C 3   /* input channels, padded to the intrinsic block (Pad + Split); r, s sequential */
 #define B2C_AXIS_CRS 4 /* fused (c, r, s) (Stencil Unroll + Fuse), padded to the K block         */
+#define B2C_AXIS_SC 5  /* fused (s, c) padded to the K block, r sequential (partial Stencil Unroll) */
+#define B2C_AXIS_C_PHASES 6 /* channels x stride phases (Image Pack of a strided conv), padded; r', s' sequential */
 
 #define B2C_VARIANT_CP_TMA 0         /* channel pack: NHWC C-padded activations, im2col-mode TMA */
 #define B2C_VARIANT_IM2COL_EXPLICIT 1 /* stencil unroll materialised as a matrix in scratch memory */
 #define B2C_VARIANT_IM2COL_GATHER 2  /* stencil unroll formed in shared memory inside the conv kernel */
 #define B2C_VARIANT_IM2COL_STAGED 3  /* same, from a zero-padded input window staged in shared memory (low-channel shapes) */
+#define B2C_VARIANT_ROW_UNROLL 4     /* stencil unroll along the kernel row only: scratch tensor [N][H][Q][(s,c)], im2col-mode TMA over r */
+#define B2C_VARIANT_SPACE_TO_DEPTH 5 /* image pack: stride phases folded into channels, then a stride-1 channel-pack conv */
 
 typedef struct {
   int32_t id;       /* index in the enumeration for this descriptor; pass to b2c_plan_create      */

@@ -21,6 +21,8 @@ struct b2c_plan {
   GatherEntry* table = nullptr;  // device, plan-owned (stencil lookup table)
   int32_t* table32 = nullptr;    // device, plan-owned (offsets into the staged window)
   WindowGeom win = {0, 0, 0, 0, 0};
+  TmaView view = {};             // geometry handed to the im2col-mode-TMA kernel (TMA-view variants)
+  int32_t* wtable = nullptr;     // device, plan-owned: packed weight column -> index into one filter, -1 = zero
   int table_len = 0;
   int* status = nullptr;         // device status word
   bool weights_set = false;
@@ -136,16 +138,25 @@ void fill_common_args(b2c_plan* p) {
   a.div_c_rows = make_fastdiv((uint32_t)std::max(1, d.C * p->win.rows));
   a.div_rows = make_fastdiv((uint32_t)std::max(1, p->win.rows));
   a.win_word_mode = (p->emb.variant == B2C_VARIANT_IM2COL_STAGED && staged_word_mode(p->g)) ? 1 : 0;
-  if (p->emb.variant == B2C_VARIANT_CP_TMA) {
+  if (is_tma_view_variant(p->emb.variant)) {
+    // the kernel walks the view's taps and channel blocks; output extent and order are unchanged
+    const TmaView& v = p->view;
     p->amode = A_IM2COL_TMA;
-    p->C_pad = cp_channel_pad(d.C);
-    p->bk = cp_block_bytes(p->C_pad);
+    p->C_pad = v.C;
+    p->bk = cp_block_bytes(v.C);
     a.bk = p->bk;
-    a.kb_per_tap = p->C_pad / p->bk;
-    a.tap_cols = p->C_pad;
-    a.num_kb = d.R * d.S * a.kb_per_tap;
+    a.kb_per_tap = v.C / p->bk;
+    a.tap_cols = v.C;
+    a.num_kb = v.R * v.S * a.kb_per_tap;
     a.ksteps_full = p->bk / kMmaK;
     a.ksteps_last = a.ksteps_full;
+    a.stride_h = v.stride_h;
+    a.stride_w = v.stride_w;
+    a.pad_h = v.pad_h;
+    a.pad_w = v.pad_w;
+    a.dil_h = v.dil_h;
+    a.dil_w = v.dil_w;
+    a.S = v.S;
   } else {
     p->amode = p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT
                    ? A_TILED
@@ -206,9 +217,47 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
   };
   if (cudaMalloc(&p->status, sizeof(int)) != cudaSuccess) return fail(B2C_E_CUDA);
   if (cudaMemset(p->status, 0, sizeof(int)) != cudaSuccess) return fail(B2C_E_CUDA);
-  if (emb.variant == B2C_VARIANT_CP_TMA) {
-    int C_pad = cp_channel_pad(d.C);
-    p->w_packed_bytes = (size_t)d.K * d.R * d.S * C_pad;
+  if (is_tma_view_variant(emb.variant)) {
+    if (!tma_view_for(g, emb.variant, &p->view)) return fail(B2C_E_UNSUPPORTED);
+    const TmaView& v = p->view;
+    p->w_packed_bytes = (size_t)d.K * v.R * v.S * v.C;
+    if (emb.variant != B2C_VARIANT_CP_TMA) {
+      // Lookup tables of the rewritten maps.  Activations: scratch channel j of scratch pixel
+      // (n, h', w') <- input element, in the form the stencil-unroll kernel takes.  Weights: packed
+      // column (tap, j) <- index into one KCRS filter.
+      const long long sc = d.in_layout == B2C_LAYOUT_NCHW ? (long long)d.H * d.W : 1;
+      const long long sh = d.in_layout == B2C_LAYOUT_NCHW ? d.W : (long long)d.W * d.C;
+      const long long sw = d.in_layout == B2C_LAYOUT_NCHW ? 1 : d.C;
+      std::vector<GatherEntry> t(v.C, GatherEntry{-1, 0, 0});
+      std::vector<int32_t> wt((size_t)v.R * v.S * v.C, -1);
+      if (emb.variant == B2C_VARIANT_ROW_UNROLL) {
+        for (int s = 0; s < d.S; ++s)
+          for (int c = 0; c < d.C; ++c) {
+            const int j = s * d.C + c;
+            t[j] = GatherEntry{(int32_t)(c * sc + (long long)s * d.dil_w * sw), 0, (int16_t)(s * d.dil_w)};
+            for (int r = 0; r < d.R; ++r) wt[(size_t)r * v.C + j] = (c * d.R + r) * d.S + s;
+          }
+      } else {
+        for (int c = 0; c < d.C; ++c)
+          for (int dh = 0; dh < d.stride_h; ++dh)
+            for (int dw = 0; dw < d.stride_w; ++dw) {
+              const int j = (c * d.stride_h + dh) * d.stride_w + dw;
+              t[j] = GatherEntry{(int32_t)(c * sc + dh * sh + dw * sw), (int16_t)dh, (int16_t)dw};
+              for (int rp = 0; rp < v.R; ++rp)
+                for (int sp = 0; sp < v.S; ++sp) {
+                  const int r = rp * d.stride_h + dh, s = sp * d.stride_w + dw;
+                  if (r < d.R && s < d.S) wt[((size_t)rp * v.S + sp) * v.C + j] = (c * d.R + r) * d.S + s;
+                }
+            }
+      }
+      p->table_len = (int)t.size();
+      if (cudaMalloc(&p->table, t.size() * sizeof(GatherEntry)) != cudaSuccess) return fail(B2C_E_CUDA);
+      if (cudaMemcpy(p->table, t.data(), t.size() * sizeof(GatherEntry), cudaMemcpyHostToDevice) != cudaSuccess)
+        return fail(B2C_E_CUDA);
+      if (cudaMalloc(&p->wtable, wt.size() * sizeof(int32_t)) != cudaSuccess) return fail(B2C_E_CUDA);
+      if (cudaMemcpy(p->wtable, wt.data(), wt.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+        return fail(B2C_E_CUDA);
+    }
   } else {
     int K_pad = variant_k_pad(g, emb.variant);
     p->w_packed_bytes = (size_t)d.K * K_pad;
@@ -248,16 +297,16 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
   if (cudaMalloc(&p->w_packed, p->w_packed_bytes + 256) != cudaSuccess) return fail(B2C_E_CUDA);
   fill_common_args(p);
   p->ws_total = workspace_bytes_for(g, emb.variant, emb.tile_n, emb.split_k);
-  if (emb.variant == B2C_VARIANT_CP_TMA) {
-    bool direct = d.in_layout == B2C_LAYOUT_NHWC && p->C_pad == d.C;
-    p->ws_layout_bytes = direct ? 0 : ((size_t)d.N * d.H * d.W * p->C_pad + 255) / 256 * 256;
+  if (is_tma_view_variant(emb.variant)) {
+    bool direct = emb.variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && p->C_pad == d.C;
+    p->ws_layout_bytes = direct ? 0 : ((size_t)p->view.bytes() + 255) / 256 * 256;
   } else if (emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
     p->ws_layout_bytes = ((size_t)g.Mg * p->K_pad + 255) / 256 * 256;
   }
   // Tensor map of the packed weights (plan-owned memory, so it is encoded once).
   int rc;
-  if (emb.variant == B2C_VARIANT_CP_TMA) {
-    uint64_t cols = (uint64_t)d.R * d.S * p->C_pad;
+  if (is_tma_view_variant(emb.variant)) {
+    uint64_t cols = (uint64_t)p->view.R * p->view.S * p->view.C;
     rc = encode_tiled_2d(&p->tmap_b, p->w_packed, cols, d.K, cols, p->bk, emb.tile_n, p->bk);
   } else {
     rc = encode_tiled_2d(&p->tmap_b, p->w_packed, p->K_pad, d.K, p->K_pad, 128, emb.tile_n, 128);
@@ -365,7 +414,7 @@ int b2c_enumerate(const b2c_conv_desc* desc, b2c_embedding* out, int32_t cap, in
   enumerate_embeddings(g, &all);
   if (!table_variant_legal(g))
     all.erase(std::remove_if(all.begin(), all.end(), [](const b2c_embedding& e) { return e.variant != B2C_VARIANT_CP_TMA; }),
-              all.end());
+              all.end());  // every other variant goes through the stencil lookup table
   for (size_t i = 0; i < all.size(); ++i) all[i].id = (int)i;
   *count = (int32_t)all.size();
   for (int i = 0; i < cap && i < (int)all.size(); ++i) out[i] = all[i];
@@ -464,6 +513,8 @@ int b2c_plan_set_weights(b2c_plan* p, const int8_t* w, void* cuda_stream) {
   const b2c_conv_desc& d = p->g.d;
   if (p->emb.variant == B2C_VARIANT_CP_TMA)
     CUDA_TRY(launch_pack_weights_cp(w, p->w_packed, d.K, d.C, d.R, d.S, p->C_pad, st));
+  else if (is_tma_view_variant(p->emb.variant))
+    CUDA_TRY(launch_pack_weights_table(w, p->w_packed, d.K, p->g.Kg, p->view.R * p->view.S * p->view.C, p->wtable, st));
   else
     CUDA_TRY(launch_pack_weights_rows(w, p->w_packed, d.K, p->g.Kg, p->K_pad, d.S,
                                       p->emb.variant == B2C_VARIANT_IM2COL_STAGED ? staged_run_len(p->g) : d.S, st));
@@ -491,14 +542,27 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   int rc = B2C_OK;
 
   // ---- layout rewrite of the activations ----
-  if (p->emb.variant == B2C_VARIANT_CP_TMA) {
+  if (is_tma_view_variant(p->emb.variant)) {
+    const TmaView& v = p->view;
     const int8_t* act = x;
     if (p->ws_layout_bytes) {
-      CUDA_TRY(launch_pack_activations(x, reinterpret_cast<int8_t*>(wsb), d.N, d.C, d.H, d.W, p->C_pad, st));
-      act = reinterpret_cast<int8_t*>(wsb);
+      int8_t* scratch = reinterpret_cast<int8_t*>(wsb);
+      if (p->emb.variant == B2C_VARIANT_CP_TMA) {
+        CUDA_TRY(launch_pack_activations(x, scratch, d.N, d.C, d.H, d.W, p->C_pad, st));
+      } else if (p->emb.variant == B2C_VARIANT_ROW_UNROLL) {
+        // scratch pixel (n, h, q): window origin (h, q*stride_w - pad_w), channels (s, c)
+        CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W, 1,
+                               d.stride_w, 0, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w, v.C, st));
+      } else {
+        // scratch pixel (n, h', w'): window origin (h'*stride_h - pad_h, w'*stride_w - pad_w), channels (c, dh, dw)
+        CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W,
+                               d.stride_h, d.stride_w, d.pad_h, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w,
+                               v.C, st));
+      }
+      act = scratch;
     }
-    rc = encode_im2col_nhwc(&tmap_a, act, p->C_pad, d.W, d.H, d.N, d.pad_w, d.pad_h, d.S, d.R, d.dil_w, d.dil_h,
-                            d.stride_w, d.stride_h, p->bk, kTileM, p->bk);
+    rc = encode_im2col_nhwc(&tmap_a, act, v.C, v.W, v.H, v.N, v.pad_w, v.pad_h, v.S, v.R, v.dil_w, v.dil_h,
+                            v.stride_w, v.stride_h, p->bk, kTileM, p->bk);
     if (rc != B2C_OK) return rc;
   } else if (p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
     int8_t* A = reinterpret_cast<int8_t*>(wsb);
@@ -547,6 +611,7 @@ void b2c_plan_destroy(b2c_plan* p) {
   cudaFree(p->w_packed);
   cudaFree(p->table);
   cudaFree(p->table32);
+  cudaFree(p->wtable);
   cudaFree(p->status);
   cudaFree(p->own_ws);
   delete p;

@@ -145,6 +145,21 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 }
 #endif
 
+// What the im2col-mode-TMA convolution kernel is given: an NHWC int8 tensor whose channel count is
+// a multiple of 32 and a filter geometry over it.  The channel-pack map uses the (padded) input
+// itself; the row-unroll and space-to-depth maps first rewrite the input into a scratch tensor for
+// which the remaining convolution has this simpler geometry.  In every case the output extent and
+// pixel order are those of the original convolution.
+struct TmaView {
+  int N, C, H, W;  // NHWC tensor, C already padded
+  int R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
+  long long bytes() const { return (long long)N * H * W * C; }
+};
+inline bool is_tma_view_variant(int v) {
+  return v == B2C_VARIANT_CP_TMA || v == B2C_VARIANT_ROW_UNROLL || v == B2C_VARIANT_SPACE_TO_DEPTH;
+}
+bool tma_view_for(const Geom& g, int variant, TmaView* v);  // false: the variant is not legal for g
+
 // --- planner.cpp -------------------------------------------------------------------------------
 int resolve_geom(const b2c_conv_desc* d, Geom* g);  // validation + derived sizes; B2C_* code
 int round_up(int v, int m);
@@ -189,6 +204,8 @@ cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, 
                                     cudaStream_t st);
 cudaError_t launch_pack_weights_cp(const int8_t* w, int8_t* out, int K, int C, int R, int S, int C_pad,
                                    cudaStream_t st);
+cudaError_t launch_pack_weights_table(const int8_t* w, int8_t* out, int K, int Kg, int cols, const int32_t* table,
+                                      cudaStream_t st);
 cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg, int K_pad, int S, int S_run,
                                      cudaStream_t st);
 cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, long long Mg, int PQ, int Q, int H,

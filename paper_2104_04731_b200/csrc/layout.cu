@@ -230,6 +230,19 @@ __global__ void pack_weights_cp_kernel(const int8_t* __restrict__ w, int8_t* __r
   }
 }
 
+// Table-driven weight pack for the rewritten maps: out[k][j] = w[k][table[j]], zero where table[j] < 0.
+__global__ void pack_weights_table_kernel(const int8_t* __restrict__ w, int8_t* __restrict__ out, int K, int Kg, int cols,
+                                          const int32_t* __restrict__ table) {
+  const long long total = (long long)K * cols;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int j = (int)(i % cols);
+    const long long k = i / cols;
+    const int src = table[j];
+    out[i] = src >= 0 ? w[k * Kg + src] : (int8_t)0;
+  }
+}
+
 // Stencil-unroll weights: rows of w[k][(c,r,s)] with every (c, r) run of S taps padded with zeros
 // to S_run entries (S_run = S for the plain unroll), then the row zero-padded to K_pad.
 __global__ void pack_weights_rows_kernel(const int8_t* __restrict__ w, int8_t* __restrict__ out, int K, int Kg,
@@ -337,6 +350,13 @@ cudaError_t launch_pack_weights_cp(const int8_t* w, int8_t* out, int K, int C, i
                                    cudaStream_t st) {
   const long long total = (long long)K * R * S * C_pad;
   pack_weights_cp_kernel<<<grid_for(total, 256), 256, 0, st>>>(w, out, K, C, R * S, C_pad);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pack_weights_table(const int8_t* w, int8_t* out, int K, int Kg, int cols, const int32_t* table,
+                                      cudaStream_t st) {
+  const long long total = (long long)K * cols;
+  pack_weights_table_kernel<<<grid_for(total, 256), 256, 0, st>>>(w, out, K, Kg, cols, table);
   return cudaGetLastError();
 }
 

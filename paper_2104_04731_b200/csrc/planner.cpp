@@ -80,10 +80,10 @@ static int tmem_pow2(int n) {
 size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k) {
   size_t ws = 0;
   const b2c_conv_desc& d = g.d;
-  if (variant == B2C_VARIANT_CP_TMA) {
-    int C_pad = cp_channel_pad(d.C);
-    bool direct = d.in_layout == B2C_LAYOUT_NHWC && C_pad == d.C;
-    if (!direct) ws += (size_t)d.N * d.H * d.W * C_pad;
+  TmaView v;
+  if (is_tma_view_variant(variant) && tma_view_for(g, variant, &v)) {
+    bool direct = variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && v.C == d.C;
+    if (!direct) ws += (size_t)v.bytes();
   } else if (variant == B2C_VARIANT_IM2COL_EXPLICIT) {
     ws += (size_t)g.Mg * im2col_k_pad(g.Kg);
   }
@@ -94,18 +94,40 @@ size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k) 
   return ws;
 }
 
-static bool cp_legal(const Geom& g) {
-  const b2c_conv_desc& d = g.d;
-  // Limits of the 4-D im2col-mode tensor map: corners in [-128, 127], tap offsets in [0, 255],
-  // traversal strides in [1, 8], dimensions < 2^32, row pitch a multiple of 16 bytes.
-  int up_w = d.pad_w - (d.S - 1) * d.dil_w, up_h = d.pad_h - (d.R - 1) * d.dil_h;
-  if (d.pad_w > 128 || d.pad_h > 128 || up_w < -128 || up_h < -128 || up_w > 127 || up_h > 127) return false;
-  if ((d.S - 1) * d.dil_w > 255 || (d.R - 1) * d.dil_h > 255) return false;
-  if (d.stride_w > 8 || d.stride_h > 8) return false;
-  // NHWC source that is not already a multiple of 32 channels would need a re-pad kernel that
-  // this build does not have.
-  if (d.in_layout == B2C_LAYOUT_NHWC && cp_channel_pad(d.C) != d.C) return false;
+// Limits of the 4-D im2col-mode tensor map: corners in [-128, 127], tap offsets in [0, 255],
+// traversal strides in [1, 8].
+static bool view_fits_tensor_map(const TmaView& v) {
+  int up_w = v.pad_w - (v.S - 1) * v.dil_w, up_h = v.pad_h - (v.R - 1) * v.dil_h;
+  if (v.pad_w > 128 || v.pad_h > 128 || up_w < -128 || up_h < -128 || up_w > 127 || up_h > 127) return false;
+  if ((v.S - 1) * v.dil_w > 255 || (v.R - 1) * v.dil_h > 255) return false;
+  if (v.stride_w > 8 || v.stride_h > 8) return false;
+  if (v.bytes() > (1LL << 40) || (long long)v.H * v.W * v.C > 0x7FFFFFFFLL) return false;
   return true;
+}
+
+bool tma_view_for(const Geom& g, int variant, TmaView* v) {
+  const b2c_conv_desc& d = g.d;
+  if (variant == B2C_VARIANT_CP_TMA) {
+    // Pad + Split + Reorder of the channel axis (Table 2); an NHWC source must already have a
+    // multiple of 32 channels (there is no NHWC re-pad kernel).
+    if (d.in_layout == B2C_LAYOUT_NHWC && cp_channel_pad(d.C) != d.C) return false;
+    *v = TmaView{d.N, cp_channel_pad(d.C), d.H, d.W, d.R, d.S, d.stride_h, d.stride_w, d.pad_h, d.pad_w, d.dil_h, d.dil_w};
+  } else if (variant == B2C_VARIANT_ROW_UNROLL) {
+    // Stencil Unroll along s only: U[n][h][q][(s, c)] = x[n][c][h][q*stride_w - pad_w + s*dil_w].
+    // What is left is an R x 1 convolution over U with the vertical geometry unchanged.
+    if (d.S == 1) return false;  // nothing to unroll: same as the channel-pack map
+    *v = TmaView{d.N, round_up(d.S * d.C, kMmaK), d.H, g.Q, d.R, 1, d.stride_h, 1, d.pad_h, 0, d.dil_h, 1};
+  } else if (variant == B2C_VARIANT_SPACE_TO_DEPTH) {
+    // Image Pack of a strided convolution: with hp = h + pad_h = (p + r')*stride_h + dh the stride
+    // phases (dh, dw) become channels of X'[n][hp / stride_h][wp / stride_w][(c, dh, dw)], and a
+    // stride-1, unpadded R' x S' convolution over X' remains (R' = ceil(R / stride_h)).
+    if (d.dil_h != 1 || d.dil_w != 1 || (d.stride_h == 1 && d.stride_w == 1)) return false;
+    const int Rp = (d.R + d.stride_h - 1) / d.stride_h, Sp = (d.S + d.stride_w - 1) / d.stride_w;
+    *v = TmaView{d.N, round_up(d.C * d.stride_h * d.stride_w, kMmaK), g.P + Rp - 1, g.Q + Sp - 1, Rp, Sp, 1, 1, 0, 0, 1, 1};
+  } else {
+    return false;
+  }
+  return view_fits_tensor_map(*v);
 }
 
 // The staged stencil unroll keeps, per image a tile can touch, the zero-padded input rows that
@@ -148,12 +170,13 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
   long long k_issued, moved;
   long long mac_min = g.Mg * d.K * g.Kg;
   long long data_min = g.x_elems + g.w_elems + g.y_elems;
-  if (variant == B2C_VARIANT_CP_TMA) {
-    e.map_k = B2C_AXIS_C;
-    int C_pad = cp_channel_pad(d.C);
-    k_issued = (long long)d.R * d.S * C_pad;
-    long long packed = (long long)d.N * d.H * d.W * C_pad;
-    bool direct = d.in_layout == B2C_LAYOUT_NHWC && C_pad == d.C;
+  TmaView v;
+  if (is_tma_view_variant(variant) && tma_view_for(g, variant, &v)) {
+    e.map_k = variant == B2C_VARIANT_CP_TMA ? B2C_AXIS_C
+                                            : (variant == B2C_VARIANT_ROW_UNROLL ? B2C_AXIS_SC : B2C_AXIS_C_PHASES);
+    k_issued = (long long)v.R * v.S * v.C;
+    long long packed = v.bytes();
+    bool direct = variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && v.C == d.C;
     moved = (direct ? 0 : g.x_elems + packed) + packed + (long long)d.K * k_issued + g.y_elems;
   } else {
     e.map_k = B2C_AXIS_CRS;
@@ -183,14 +206,14 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
     if (t >= d.K) break;
   }
   long long tiles_m = (g.Mg + kTileM - 1) / kTileM;
-  for (int variant = 0; variant < 4; ++variant) {
-    if (variant == B2C_VARIANT_CP_TMA && !cp_legal(g)) continue;
+  for (int variant = 0; variant < 6; ++variant) {
+    TmaView view;
+    if (is_tma_view_variant(variant) && !tma_view_for(g, variant, &view)) continue;
     WindowGeom wg;
     if (variant == B2C_VARIANT_IM2COL_STAGED && !staged_window(g, &wg)) continue;
     int num_kb;
-    if (variant == B2C_VARIANT_CP_TMA) {
-      int C_pad = cp_channel_pad(d.C);
-      num_kb = d.R * d.S * (C_pad / cp_block_bytes(C_pad));
+    if (is_tma_view_variant(variant)) {
+      num_kb = view.R * view.S * (view.C / cp_block_bytes(view.C));
     } else {
       num_kb = (variant_k_pad(g, variant) + 127) / 128;
     }

@@ -83,11 +83,11 @@ def test_enumeration_is_sorted_and_covers_variants(lib, cfg):
     assert [e.id for e in embs] == list(range(len(embs)))
     costs = [e.o_mac + e.o_data for e in embs]
     assert costs == sorted(costs)
-    assert {0, 1, 2} <= {e.variant for e in embs} <= {0, 1, 2, 3}
+    assert {0, 1, 2} <= {e.variant for e in embs} <= {0, 1, 2, 3, 4, 5}
     for e in embs:
         assert e.tile_m == 128 and e.tile_n in (16, 32, 64, 128, 256) and e.split_k >= 1
         assert e.map_m == b2c.AXIS_NPQ and e.map_n == b2c.AXIS_K
-        assert e.map_k == (b2c.AXIS_C if e.variant == 0 else b2c.AXIS_CRS)
+        assert e.map_k == {0: b2c.AXIS_C, 4: b2c.AXIS_SC, 5: b2c.AXIS_C_PHASES}.get(e.variant, b2c.AXIS_CRS)
         assert e.o_mac >= 0 and e.o_data >= 0 and e.device_us == -1.0
         if e.variant in (b2c.VARIANT_IM2COL_GATHER, b2c.VARIANT_IM2COL_STAGED) and e.split_k == 1:
             assert e.workspace_bytes == 0
@@ -122,6 +122,13 @@ def test_padding_inflates_weights_and_workspace(lib):
     assert ex.workspace_bytes == cfg.N * cfg.P * cfg.Q * 160
     assert ga.workspace_bytes == 0
     assert ga.o_mac < cp.o_mac and ga.o_data < ex.o_data < cp.o_data + ex.o_data
+    # partial unroll (Table 2: stencil unroll on one axis only) and image pack sit between the two
+    ro = next(e for e in embs if e.variant == 4 and e.split_k == 1)
+    sd = next(e for e in embs if e.variant == 5 and e.split_k == 1)
+    assert ro.workspace_bytes == cfg.N * cfg.H * cfg.Q * 32          # (s, c) = 21 -> 32 channels per (n, h, q)
+    # 3*2*2 = 12 -> 32 channels, R' = S' = 4; scratch sizes are rounded up to 256 bytes
+    assert sd.workspace_bytes == -(-cfg.N * (cfg.P + 3) * (cfg.Q + 3) * 32 // 256) * 256
+    assert ga.o_mac < ro.o_mac < cp.o_mac
     assert embs[0].variant in (2, 3)  # lowest overhead: stencil unroll formed inside the kernel
 
 
