@@ -136,9 +136,10 @@ int b2c_conv2d_int8_run(b2c_plan* plan, const int8_t* x_dev, int32_t* y_i32_dev,
 
 /* One-shot form of the paper's problem statement: NCHW int8 input, KCRS int8 weights, NKPQ
  * outputs (either may be NULL, not both), symmetric stride / pad / dilation.  All four tensor
- * pointers are DEVICE pointers.  Picks the minimum-overhead embedding, keeps plans and scratch
- * in a library-owned cache keyed by shape (so it may allocate on first use of a shape),
- * re-packs the weights on every call, and enqueues on `cuda_stream`. */
+ * pointers are DEVICE pointers.  Keeps plans and scratch in a library-owned cache keyed by
+ * shape: the first call for a shape picks the embedding by timed selection (it allocates and
+ * synchronises with the device, so make it outside any stream capture); later calls only
+ * re-pack the weights and enqueue on `cuda_stream`. */
 int b2c_conv2d_int8(int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int dilation,
                     int shift, const int8_t* x_dev, const int8_t* w_dev, int32_t* y_i32_dev,
                     int8_t* y_i8_dev, void* cuda_stream);

@@ -637,7 +637,8 @@ int b2c_conv2d_int8(int N, int C, int H, int W, int K, int R, int S, int stride,
   b2c_plan* p = nullptr;
   auto it = g_cache.find(key);
   if (it == g_cache.end()) {
-    int rc = b2c_plan_create(&d, B2C_POLICY_MIN_OVERHEAD, cuda_stream, &p);
+    // first use of a shape: timed selection (allocates and synchronises once, then cached)
+    int rc = b2c_plan_create(&d, B2C_POLICY_AUTO_TIMED, cuda_stream, &p);
     if (rc != B2C_OK) return rc;
     if (p->ws_total) {
       if (cudaMalloc(&p->own_ws, p->ws_total) != cudaSuccess) {
