@@ -102,12 +102,6 @@ struct ConvArgs {
   int cluster_split;  // split_k slices form a cluster (1, 1, split_k) and reduce through shared memory
 };
 
-struct Schedule {
-  int variant;
-  int tile_n;
-  int split_k;
-};
-
 // Programmatic dependent launch: a kernel launched through launch_pdl may start while the previous
 // kernel of the stream is still running; it must call pdl_wait() before its first access to global
 // memory that an earlier kernel may write or still read, and calls pdl_launch_dependents() once the

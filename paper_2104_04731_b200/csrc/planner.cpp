@@ -71,12 +71,6 @@ int variant_k_pad(const Geom& g, int variant) {
   return im2col_k_pad(g.Kg);
 }
 
-static int tmem_pow2(int n) {
-  int c = 32;
-  while (c < n) c <<= 1;
-  return c;
-}
-
 size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k) {
   size_t ws = 0;
   const b2c_conv_desc& d = g.d;
@@ -237,7 +231,6 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
     return a.o_mac + a.o_data < b.o_mac + b.o_data;
   });
   for (size_t i = 0; i < out->size(); ++i) (*out)[i].id = (int)i;
-  (void)tmem_pow2;
 }
 
 int pick_by_policy(const std::vector<b2c_embedding>& all, int policy) {
