@@ -151,14 +151,34 @@ __device__ __forceinline__ uint32_t make_idesc_i8(int n) {
   return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 }
 
-__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                       uint32_t accumulate, uint32_t on) {
+// One reduction block: `ksteps` (1..4) MMAs over consecutive 32-byte slices of the stage (each
+// step advances both descriptors by 2 units of 16 bytes).  Issued from one asm block so that the
+// predicates and descriptors are formed once and the instructions go out back to back; the first
+// step overwrites the accumulator when `accumulate` is 0, the others always add.
+__device__ __forceinline__ void mma_i8_block(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate, uint32_t on, int ksteps) {
   asm volatile(
-      "{\n.reg .pred p, q;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "setp.ne.b32 q, %5, 0;\n"
-      "@q tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(on)
+      "{\n"
+      ".reg .pred pacc, ptrue, q0, q1, q2, q3;\n"
+      ".reg .b64 a1, a2, a3, b1, b2, b3;\n"
+      "setp.ne.b32 pacc, %4, 0;\n"
+      "setp.eq.b32 ptrue, 0, 0;\n"
+      "setp.ne.b32 q0, %5, 0;\n"
+      "setp.gt.and.s32 q1, %6, 1, q0;\n"
+      "setp.gt.and.s32 q2, %6, 2, q0;\n"
+      "setp.gt.and.s32 q3, %6, 3, q0;\n"
+      "add.u64 a1, %1, 2;\n"
+      "add.u64 b1, %2, 2;\n"
+      "add.u64 a2, %1, 4;\n"
+      "add.u64 b2, %2, 4;\n"
+      "add.u64 a3, %1, 6;\n"
+      "add.u64 b3, %2, 6;\n"
+      "@q0 tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, pacc;\n"
+      "@q1 tcgen05.mma.cta_group::1.kind::i8 [%0], a1, b1, %3, ptrue;\n"
+      "@q2 tcgen05.mma.cta_group::1.kind::i8 [%0], a2, b2, %3, ptrue;\n"
+      "@q3 tcgen05.mma.cta_group::1.kind::i8 [%0], a3, b3, %3, ptrue;\n"
+      "}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(on), "r"(ksteps)
       : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar, uint32_t on) {
@@ -509,11 +529,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST ? 1 : 3) conv_mma_kernel(con
         }
         // Look ahead: test the next stage's barrier now so that its latency overlaps the MMA issue.
         ready = (kb + 1 < kb_end) && mbar_test_wait(smem_u32(&ctl.full[s]), ph);
-        for (int k = 0; k < ksteps; ++k) {
-          // Advancing 32 bytes along the row = 2 units of 16 bytes in the descriptor address.
-          mma_i8(d_tmem, a_cur + (uint64_t)(2 * k), b_cur + (uint64_t)(2 * k), idesc, (accumulate | (uint32_t)k),
-                 leader);
-        }
+        mma_i8_block(d_tmem, a_cur, b_cur, idesc, accumulate, leader, ksteps);
         mma_commit(smem_u32(&ctl.empty[s_cur]), leader);
         if (kb == kb_end - 1) mma_commit(smem_u32(&ctl.tmem_full[buf]), leader);
         accumulate = 1;
