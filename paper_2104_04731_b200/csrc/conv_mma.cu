@@ -313,26 +313,6 @@ __device__ __forceinline__ void epilogue_columns(const ConvArgs& args, uint32_t 
   store_columns<NC>(args, v, kbase, row_valid, base_nkpq, base_npqk);
 }
 
-// Sum of the cluster's partial tiles for NC columns of one row, read through distributed shared
-// memory (`local_addr` is the row's address in this block's exchange tile; every block of the
-// cluster keeps its tile at the same offset).
-template <int NC>
-__device__ __forceinline__ void cluster_sum_columns(uint32_t local_addr, int split, int32_t* v) {
-#pragma unroll
-  for (int j = 0; j < NC; ++j) v[j] = 0;
-  for (int r = 0; r < split; ++r) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(r));
-    // all loads of a slice are issued before the first use, so that they are in flight together
-    int32_t t[NC];
-#pragma unroll
-    for (int j = 0; j < NC; ++j)
-      asm volatile("ld.shared::cluster.b32 %0, [%1];" : "=r"(t[j]) : "r"(remote + (uint32_t)j * (kTileM * 4)) : "memory");
-#pragma unroll
-    for (int j = 0; j < NC; ++j) v[j] += t[j];
-  }
-}
-
 template <int AMODE, bool PERSIST>
 __global__ void __launch_bounds__(kThreads, PERSIST ? 1 : 3) conv_mma_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                                              const __grid_constant__ CUtensorMap tmap_b,
@@ -773,31 +753,98 @@ __global__ void __launch_bounds__(kThreads, PERSIST ? 1 : 3) conv_mma_kernel(con
     asm volatile("barrier.cluster.arrive.release;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
     if (warp >= 2 && !ctl.abort_flag) {
-      const int quad = warp & 3, half = (warp - 2) >> 2;
-      const int row = quad * 32 + lane;
-      const unsigned m = (unsigned)m0 + (unsigned)row;
-      const bool row_valid = m < (unsigned)args.Mg;
+      // Lane g owns accumulator rows 4g .. 4g+3 (one 16-byte vector of the [column][row] tile);
+      // warp w takes columns w, w + 8, ... of this block's slice.  All vector loads of a batch of
+      // columns (from every slice, starting with the own one) are issued before the first add.
+      const int cols_slice = args.tile_n / args.split_k;
+      const int col_base = (int)blockIdx.z * cols_slice;
+      const uint32_t rank = blockIdx.z;
+      const unsigned mrow = (unsigned)m0 + 4u * (unsigned)lane;
+      // rows of this lane: valid count, image and pixel of the first row, same-image flag
       int n_img = 0, pq = 0;
-      if (row_valid) {
-        n_img = (int)args.div_pq.div(m);
-        pq = (int)(m - (unsigned)n_img * (unsigned)args.PQ);
+      if (mrow < (unsigned)args.Mg) {
+        n_img = (int)args.div_pq.div(mrow);
+        pq = (int)(mrow - (unsigned)n_img * (unsigned)args.PQ);
       }
-      const long long base_nkpq = (long long)n_img * args.K * args.PQ + pq;
-      const long long base_npqk = (long long)m * args.K;
-      const int w = args.tile_n / (2 * args.split_k);  // columns of this thread's slice (>= 16)
-      const int col0 = (int)blockIdx.z * (args.tile_n / args.split_k) + half * w;
-      const uint32_t xch = a_base + (uint32_t)row * 4u + (uint32_t)col0 * (kTileM * 4);
-      if ((w & 31) == 0) {
-        for (int c = 0; c < w; c += 32) {
-          int32_t v[32];
-          cluster_sum_columns<32>(xch + (uint32_t)c * (kTileM * 4), args.split_k, v);
-          store_columns<32>(args, v, n0 + col0 + c, row_valid, base_nkpq, base_npqk);
+      const int rows_valid = (int)min(4u, (unsigned)args.Mg > mrow ? (unsigned)args.Mg - mrow : 0u);
+      const bool one_image = rows_valid == 4 && pq + 3 < args.PQ;
+      const bool nhwc = args.out_layout == B2C_LAYOUT_NHWC;
+      constexpr int kBatch = 4;  // columns in flight per thread: kBatch * split vector loads
+      for (int cb = warp - 2; cb < cols_slice; cb += kGatherWarps * kBatch) {
+        int32_t acc[kBatch][4];
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0;
+        for (int rr = 0; rr < args.split_k; ++rr) {
+          uint32_t r = rank + (uint32_t)rr;
+          if (r >= (uint32_t)args.split_k) r -= (uint32_t)args.split_k;
+          int32_t t[kBatch][4];
+#pragma unroll
+          for (int b = 0; b < kBatch; ++b) {
+            const int c = cb + b * kGatherWarps;
+            if (c < cols_slice) {
+              const uint32_t local = a_base + (uint32_t)(col_base + c) * (kTileM * 4) + (uint32_t)lane * 16u;
+              uint32_t remote;
+              asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(r));
+              asm volatile("ld.shared::cluster.v4.b32 {%0, %1, %2, %3}, [%4];"
+                           : "=r"(t[b][0]), "=r"(t[b][1]), "=r"(t[b][2]), "=r"(t[b][3])
+                           : "r"(remote)
+                           : "memory");
+            } else {
+              t[b][0] = t[b][1] = t[b][2] = t[b][3] = 0;
+            }
+          }
+#pragma unroll
+          for (int b = 0; b < kBatch; ++b) {
+            acc[b][0] += t[b][0];
+            acc[b][1] += t[b][1];
+            acc[b][2] += t[b][2];
+            acc[b][3] += t[b][3];
+          }
         }
-      } else {
-        for (int c = 0; c < w; c += 16) {
-          int32_t v[16];
-          cluster_sum_columns<16>(xch + (uint32_t)c * (kTileM * 4), args.split_k, v);
-          store_columns<16>(args, v, n0 + col0 + c, row_valid, base_nkpq, base_npqk);
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+          const int c = cb + b * kGatherWarps;
+          const int k = n0 + col_base + c;
+          if (c >= cols_slice || k >= args.K || rows_valid == 0) continue;
+          if (!nhwc && one_image) {
+            // four consecutive pixels of one image and one channel: contiguous in NKPQ
+            const long long o = ((long long)n_img * args.K + k) * args.PQ + pq;
+            if (args.out_mode & B2C_OUT_I32) {
+              int32_t* dst = args.y32 + o;
+              if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+                *reinterpret_cast<int4*>(dst) = make_int4(acc[b][0], acc[b][1], acc[b][2], acc[b][3]);
+              } else {
+                dst[0] = acc[b][0]; dst[1] = acc[b][1]; dst[2] = acc[b][2]; dst[3] = acc[b][3];
+              }
+            }
+            if (args.out_mode & B2C_OUT_I8) {
+              int8_t* dst = args.y8 + o;
+              const uint32_t q4 = (uint32_t)(uint8_t)requant(acc[b][0], args.shift) |
+                                  ((uint32_t)(uint8_t)requant(acc[b][1], args.shift) << 8) |
+                                  ((uint32_t)(uint8_t)requant(acc[b][2], args.shift) << 16) |
+                                  ((uint32_t)(uint8_t)requant(acc[b][3], args.shift) << 24);
+              if ((reinterpret_cast<uintptr_t>(dst) & 3) == 0) {
+                *reinterpret_cast<uint32_t*>(dst) = q4;
+              } else {
+                dst[0] = (int8_t)(q4 & 0xff); dst[1] = (int8_t)((q4 >> 8) & 0xff);
+                dst[2] = (int8_t)((q4 >> 16) & 0xff); dst[3] = (int8_t)(q4 >> 24);
+              }
+            }
+          } else {
+            // general case: row by row (image boundary inside the group, tail rows, or NPQK)
+            for (int i = 0; i < rows_valid; ++i) {
+              const unsigned mi = mrow + (unsigned)i;
+              long long o;
+              if (nhwc) {
+                o = (long long)mi * args.K + k;
+              } else {
+                const int ni = (int)args.div_pq.div(mi);
+                o = ((long long)ni * args.K + k) * args.PQ + (int)(mi - (unsigned)ni * (unsigned)args.PQ);
+              }
+              if (args.out_mode & B2C_OUT_I32) args.y32[o] = acc[b][i];
+              if (args.out_mode & B2C_OUT_I8) args.y8[o] = requant(acc[b][i], args.shift);
+            }
+          }
         }
       }
     }
