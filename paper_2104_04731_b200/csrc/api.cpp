@@ -183,13 +183,15 @@ void fill_common_args(b2c_plan* p) {
   a.tiles_n = tiles_n;
   a.num_tiles = (int)std::min<long long>(tiles_m * tiles_n, 0x7FFFFFFF);
   a.div_tiles_n = make_fastdiv((uint32_t)tiles_n);
-  // (narrow tiles have short main loops and do better with several small blocks per SM)
-  a.persistent = ((p->amode == A_TILED || p->amode == A_IM2COL_TMA) && a.split_k == 1 && a.tile_n >= 128 &&
-                  tiles_m * tiles_n > 2 * kNumSMs && tiles_m * tiles_n < 0x7FFFFFFF)
-                     ? 1
-                     : 0;
+  // Wide tiles: one block per SM.  Narrow tiles have short main loops and do better with three
+  // blocks per SM, each still walking several tiles (mode 2) once there are enough tiles.
+  const bool tma_fed = (p->amode == A_TILED || p->amode == A_IM2COL_TMA) && a.split_k == 1 &&
+                       tiles_m * tiles_n < 0x7FFFFFFF;
+  a.persistent = 0;
+  if (tma_fed && a.tile_n >= 128 && tiles_m * tiles_n > 2 * kNumSMs) a.persistent = 1;
+  if (tma_fed && a.tile_n < 128 && tiles_m * tiles_n > 2 * 3 * kNumSMs) a.persistent = 2;
   a.tmem_bufs = (a.persistent && 2 * a.tmem_cols <= 512) ? 2 : 1;
-  const size_t budget = a.persistent ? 196 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 160 * 1024);
+  const size_t budget = a.persistent == 1 ? 196 * 1024 : (a.persistent == 2 ? 68 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 160 * 1024));
   const size_t stage_bytes = (size_t)(kTileM + a.tile_n) * a.bk;
   // lookup table and staged window share the block's shared memory with the stages
   const size_t extra = p->amode == A_STAGED ? (size_t)p->win.bytes + 4 * (size_t)p->table_len + 64

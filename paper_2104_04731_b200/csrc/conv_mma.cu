@@ -313,8 +313,10 @@ __device__ __forceinline__ void epilogue_columns(const ConvArgs& args, uint32_t 
   store_columns<NC>(args, v, kbase, row_valid, base_nkpq, base_npqk);
 }
 
-template <int AMODE, bool PERSIST>
-__global__ void __launch_bounds__(kThreads, PERSIST ? 1 : 3) conv_mma_kernel(const __grid_constant__ CUtensorMap tmap_a,
+// PERSIST: 0 = one tile per block; 1 = persistent, one block per SM (wide tiles, deep stage ring);
+// 2 = persistent, three blocks per SM (narrow tiles: short main loops, several epilogues in flight).
+template <int AMODE, int PERSIST>
+__global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                                              const __grid_constant__ CUtensorMap tmap_b,
                                                              const ConvArgs args) {
   extern __shared__ uint8_t smem_raw[];
@@ -329,7 +331,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST ? 1 : 3) conv_mma_kernel(con
   // buffers so that the epilogue of one tile overlaps the main loop of the next.
   // (PERSIST is a template parameter so that the one-tile-per-block instantiation carries none of
   // the loop, buffer-index and hand-back overhead.)
-  constexpr bool persistent = PERSIST;
+  constexpr bool persistent = PERSIST != 0;
   const int tile_first = persistent ? (int)blockIdx.x : 0;
   const int tile_step = persistent ? (int)gridDim.x : 1;
   const int tile_end = persistent ? args.num_tiles : 1;
@@ -903,7 +905,7 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
   const size_t smem = conv_mma_smem_bytes(amode, args);
   dim3 grid((unsigned)((args.Mg + kTileM - 1) / kTileM), (unsigned)((args.K + args.tile_n - 1) / args.tile_n),
             (unsigned)args.split_k);
-  if (args.persistent) grid = dim3((unsigned)std::min(args.num_tiles, kNumSMs), 1, 1);
+  if (args.persistent) grid = dim3((unsigned)std::min(args.num_tiles, kNumSMs * (args.persistent == 2 ? 3 : 1)), 1, 1);
   cudaError_t e;
 #define B2C_LAUNCH(MODE, PERS)                                                                             \
   {                                                                                                       \
@@ -918,12 +920,14 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
                            args.cluster_split ? args.split_k : 1, *tmap_a, *tmap_b, args);                \
     if (e != cudaSuccess) return e;                                                                       \
   }
-  if (amode == A_TILED && args.persistent) B2C_LAUNCH(A_TILED, true)
-  else if (amode == A_TILED) B2C_LAUNCH(A_TILED, false)
-  else if (amode == A_IM2COL_TMA && args.persistent) B2C_LAUNCH(A_IM2COL_TMA, true)
-  else if (amode == A_IM2COL_TMA) B2C_LAUNCH(A_IM2COL_TMA, false)
-  else if (amode == A_STAGED) B2C_LAUNCH(A_STAGED, false)
-  else B2C_LAUNCH(A_GATHER, false)
+  if (amode == A_TILED && args.persistent == 1) B2C_LAUNCH(A_TILED, 1)
+  else if (amode == A_TILED && args.persistent == 2) B2C_LAUNCH(A_TILED, 2)
+  else if (amode == A_TILED) B2C_LAUNCH(A_TILED, 0)
+  else if (amode == A_IM2COL_TMA && args.persistent == 1) B2C_LAUNCH(A_IM2COL_TMA, 1)
+  else if (amode == A_IM2COL_TMA && args.persistent == 2) B2C_LAUNCH(A_IM2COL_TMA, 2)
+  else if (amode == A_IM2COL_TMA) B2C_LAUNCH(A_IM2COL_TMA, 0)
+  else if (amode == A_STAGED) B2C_LAUNCH(A_STAGED, 0)
+  else B2C_LAUNCH(A_GATHER, 0)
 #undef B2C_LAUNCH
 #undef B2C_TILE_ORIGIN
   return cudaGetLastError();

@@ -35,7 +35,6 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_kernel(const in
   const int8_t* xin = x + ((size_t)n * C + c0) * HW + hw0;
   const int rows = min(CT, C - c0);  // channels that exist; the rest of the tile is zero padding
   pdl_wait();
-  pdl_launch_dependents();
 
   // ---- load ----
   if constexpr (VEC >= 4) {
@@ -83,6 +82,7 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_kernel(const in
     }
   }
   __syncthreads();
+  pdl_launch_dependents();  // after the loads: an earlier start would only take shared memory from this grid
 
   // ---- transpose in registers and store ----
   const int chunks = CT >> 4;            // 16-channel chunks per pixel in this tile
@@ -149,7 +149,6 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_bulk_kernel(con
   }
   __syncthreads();
   pdl_wait();
-  pdl_launch_dependents();
   const int8_t* xin = x + ((size_t)n * C + c0) * HW + hw0;
   if (kRowMode) {
     if (t < rows) {
@@ -182,6 +181,9 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_bulk_kernel(con
     done = ok != 0;
   }
   if (!done) return;
+  // The next kernel may start its set-up once every block of this one has its tile in shared
+  // memory (earlier, its resident blocks would only take shared memory away from this grid).
+  pdl_launch_dependents();
 
   const int chunks = CT >> 4;
   const int items = ((npx + 3) >> 2) * chunks;
@@ -268,7 +270,6 @@ __global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ 
   const int chunks = K_pad >> 4;
   const long long total = Mg * chunks;
   pdl_wait();
-  pdl_launch_dependents();
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
     const long long m = i / chunks;
@@ -289,6 +290,7 @@ __global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ 
     }
     *reinterpret_cast<uint4*>(a + m * K_pad + ck * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
   }
+  pdl_launch_dependents();
 }
 
 // Finish of a split reduction: the int32 sums are complete in `acc`; copy them out and/or apply
