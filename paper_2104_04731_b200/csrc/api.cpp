@@ -190,6 +190,10 @@ void fill_common_args(b2c_plan* p) {
   a.persistent = 0;
   if (tma_fed && a.tile_n >= 128 && tiles_m * tiles_n > 2 * kNumSMs) a.persistent = 1;
   if (tma_fed && a.tile_n < 128 && tiles_m * tiles_n > 2 * 3 * kNumSMs) a.persistent = 2;
+  // the staged-window kernel walks tiles the same way (window restaged per tile)
+  if (p->amode == A_STAGED && a.split_k == 1 && tiles_m * tiles_n > 2 * 3 * kNumSMs &&
+      tiles_m * tiles_n < 0x7FFFFFFF)
+    a.persistent = 2;
   a.tmem_bufs = (a.persistent && 2 * a.tmem_cols <= 512) ? 2 : 1;
   const size_t budget = a.persistent == 1 ? 196 * 1024 : (a.persistent == 2 ? 68 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 160 * 1024));
   const size_t stage_bytes = (size_t)(kTileM + a.tile_n) * a.bk;

@@ -526,6 +526,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     const int row = quad * 32 + lane;   // accumulator row = A-tile row
     bool ok = true;
     int ti = 0;
+    int s = 0;         // stage ring position of the A-forming threads (runs on across tiles)
+    uint32_t ph = 0;
     for (int t = tile_first; t < tile_end && ok; t += tile_step, ++ti) {
     B2C_TILE_ORIGIN(t)
     const unsigned m = (unsigned)m0 + (unsigned)row;
@@ -547,8 +549,6 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
                            (long long)w0 * args.x_stride_w;
       const uint32_t row_off = (uint32_t)row * 128u;
       const uint32_t xr = (uint32_t)(row & 7);
-      int s = 0;
-      uint32_t ph = 0;
       for (int kb = kb_begin; kb < kb_end; ++kb) {
         if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) {
           ok = false;
@@ -594,6 +594,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       // (rows outside the image and the left/right margins are zeros, so the gather below needs no
       // bounds tests); then each thread forms half a row of the A tile per stage from that window.
       const int tg = (int)threadIdx.x - 64;
+      // (persistent blocks: every thread must be done reading the previous tile's window)
+      if (ti > 0) asm volatile("bar.sync 1, %0;" ::"n"(kGatherWarps * 32) : "memory");
       const unsigned m_last = min((unsigned)m0 + (unsigned)kTileM - 1u, (unsigned)args.Mg - 1u);
       const int img0 = (int)args.div_pq.div((uint32_t)m0);
       const int p_first = (int)args.div_q.div((uint32_t)(m0 - img0 * args.PQ));
@@ -642,8 +644,6 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       }
       const uint32_t row_off = (uint32_t)row * 128u;
       const uint32_t xr = (uint32_t)(row & 7);
-      int s = 0;
-      uint32_t ph = 0;
       for (int kb = kb_begin; kb < kb_end; ++kb) {
         if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) {
           ok = false;
@@ -926,6 +926,7 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
   else if (amode == A_IM2COL_TMA && args.persistent == 1) B2C_LAUNCH(A_IM2COL_TMA, 1)
   else if (amode == A_IM2COL_TMA && args.persistent == 2) B2C_LAUNCH(A_IM2COL_TMA, 2)
   else if (amode == A_IM2COL_TMA) B2C_LAUNCH(A_IM2COL_TMA, 0)
+  else if (amode == A_STAGED && args.persistent == 2) B2C_LAUNCH(A_STAGED, 2)
   else if (amode == A_STAGED) B2C_LAUNCH(A_STAGED, 0)
   else B2C_LAUNCH(A_GATHER, 0)
 #undef B2C_LAUNCH

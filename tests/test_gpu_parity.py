@@ -298,3 +298,16 @@ def test_edge_shapes(lib, case):
             continue
         done.add(key)
         check_against_oracle(x, w, stride, pad, dil, shift, 3, e.id, ref=ref)
+
+
+def test_large_grid_staged_window_walks_tiles(lib):
+    # 980 tiles of a low-channel strided shape: the staged-window kernel runs persistently
+    N, C, H, W, K, R, S = 10, 3, 224, 224, 64, 7, 7
+    x = int8_uniform((N, C, H, W), 711)
+    w = int8_uniform((K, C, R, S), 712)
+    ref = oracle.conv2d_int8(x, w, 2, 3, 1, 7)
+    d = lib.make_desc(N, C, H, W, K, R, S, 2, 3, 1, 7, out_mode=3)
+    for tile_n in (32, 64):
+        ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == 3 and e.tile_n == tile_n and e.split_k == 1]
+        assert ids
+        check_against_oracle(x, w, 2, 3, 1, 7, 3, ids[0], ref=ref)
