@@ -5,7 +5,11 @@ One "step" is one pass of the whole path (activation layout rewrite, MMA kernel 
 shift/clip epilogue, split-reduction finish when the embedding has one) over a batch of G
 independent instances of the headline convolution shape, each instance with its own input,
 weight, output and scratch buffers, so that every launch reads cold data (G x working set is
-larger than the 126 MB L2).  The G launches of a step are captured once in a CUDA graph.
+larger than the 126 MB L2).  The G launches of a step are captured once in a CUDA graph; since
+the instances share nothing, they are dealt onto `--streams` branches of that graph so that kernels
+of different instances overlap on the GPU (throughput of the batch is what `value` reports), and the
+embedding is chosen by the planner's concurrent timed selection.  `--streams 1` runs one call after
+the other; `per_config` reports both series for every shape.
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 """
@@ -133,6 +137,8 @@ class Instances:
         torch.cuda.synchronize()
         self.launches_per_instance = self._count_launches()
         self.graph = None
+        self.side = None
+        self.streams = 1
 
     def _count_launches(self):
         """Kernels of this library per call: layout rewrite (if any) + MMA kernel + split finish (if any)."""
@@ -145,18 +151,37 @@ class Instances:
             n += 1  # a split reduction that is not a cluster goes through memory and needs the finish kernel
         return n
 
-    def run_all(self):
+    def run_all(self, torch=None, streams=1):
+        """Enqueues every instance once.  With streams > 1 the instances (which share no buffer and no
+        plan) are dealt round-robin onto that many side streams forked from, and joined back into, the
+        current stream, so that kernels of different instances may run side by side on the GPU."""
+        if streams <= 1:
+            for i, p in enumerate(self.plans):
+                p.run(self.x[i], self.y32[i], self.y8[i], self.ws[i])
+            return
+        if self.side is None or len(self.side) != streams:
+            self.side = [torch.cuda.Stream() for _ in range(streams)]
+        cur = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(cur)
+        for s in self.side:
+            s.wait_event(fork)
         for i, p in enumerate(self.plans):
-            p.run(self.x[i], self.y32[i], self.y8[i], self.ws[i])
+            p.run(self.x[i], self.y32[i], self.y8[i], self.ws[i], stream=self.side[i % streams])
+        for s in self.side:
+            join = torch.cuda.Event()
+            join.record(s)
+            cur.wait_event(join)
 
-    def capture(self, torch, repeat=1):
-        self.run_all()
+    def capture(self, torch, repeat=1, streams=1):
+        self.run_all(torch, streams)
         torch.cuda.synchronize()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             for _ in range(repeat):
-                self.run_all()
+                self.run_all(torch, streams)
         self.graph = g
+        self.streams = streams
 
     def step(self):
         if self.graph is not None:
@@ -214,8 +239,10 @@ def instances_for(cfg, min_bytes=2 * L2_BYTES, lo=8, hi=256):
     return int(max(lo, min(hi, -(-min_bytes // per))))
 
 
-def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, graph=True):
-    """Combined (whole path, NCHW in), Op (MMA kernel alone on a resident packed operand) and Transf."""
+def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, graph=True, streams=1):
+    """Combined (whole path, NCHW in), Op (MMA kernel alone on a resident packed operand) and Transf.,
+    one call after the other on one stream (latency series); and the same batch of instances dealt
+    onto `streams` graph branches with the embedding chosen for throughput (concurrent series)."""
     G = instances_for(cfg)
     inst = Instances(b2c, torch, cfg, G, policy)
     if graph:
@@ -234,13 +261,24 @@ def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, grap
     warm.destroy()
     op = op_only(b2c, torch, cfg, emb["variant"], emb["tile_n"], emb["split_k"], steps, warmup, graph)
     t_roof, bound = roofline_time_us(cfg, peaks)
+    keys = ("id", "variant_name", "tile_n", "split_k", "workspace_bytes", "o_mac", "o_data", "device_us")
     res = {
         "shape": cfg.name, "instances": G, "warm_us": ms_w * 1e3 / (10 * 20),
         "op_us": op["us"] if op else None, "transf_us": max(0.0, per_call_us - op["us"]) if op else None, "cold": bool(G * cfg.algorithmic_bytes >= L2_BYTES), "combined_us": per_call_us, "tops": 2.0 * cfg.macs / (per_call_us * 1e-6) / 1e12,
         "roofline_us": t_roof, "bound": bound, "roofline_frac": t_roof / per_call_us,
-        "embedding": {k: emb[k] for k in ("id", "variant_name", "tile_n", "split_k", "workspace_bytes", "o_mac", "o_data", "device_us")},
+        "embedding": {k: emb[k] for k in keys},
         "launches_per_call": launches,
     }
+    if graph and streams > 1:
+        conc = Instances(b2c, torch, cfg, G, b2c.POLICY_AUTO_TIMED_CONCURRENT)
+        conc.capture(torch, streams=streams)
+        ms_c = time_steps(torch, conc.step, steps, warmup, dist)
+        conc.check_status(b2c)
+        us_c = ms_c * 1e3 / (steps * G)
+        emb_c = conc.emb.as_dict()
+        conc.destroy()
+        res["concurrent"] = {"streams": streams, "us_per_call": us_c, "tops": 2.0 * cfg.macs / (us_c * 1e-6) / 1e12,
+                             "roofline_frac": t_roof / us_c, "embedding": {k: emb_c[k] for k in keys}}
     return res
 
 
@@ -278,7 +316,7 @@ def measure_scaled(b2c, torch, cfg, peaks, steps=10):
             "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k}}
 
 
-def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=True):
+def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=True, streams=1):
     """Device time of the MMA kernel alone: same embedding but with the layout rewrite already done
     (channel-pack map: NHWC input with padded channels; stencil-unroll in-kernel: unchanged)."""
     if emb_variant == 0 and cfg.C % 32 == 0:
@@ -297,7 +335,7 @@ def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=
     else:
         return None
     if graph:
-        inst.capture(torch)
+        inst.capture(torch, streams=streams)
     ms = time_steps(torch, inst.step, steps, warmup)
     inst.check_status(b2c)
     us = ms * 1e3 / (steps * G)
@@ -447,7 +485,8 @@ def run_ours(args):
     cfg = CONFIGS[args.config]
     if args.scaled:
         cfg = scaled_shape(cfg, peaks)
-    policy = b2c.POLICY_AUTO_TIMED if args.embedding is None else args.embedding
+    auto = b2c.POLICY_AUTO_TIMED_CONCURRENT if args.streams > 1 else b2c.POLICY_AUTO_TIMED
+    policy = auto if args.embedding is None else args.embedding
     if args.pick:
         v, tn, sk = (int(t) for t in args.pick.split(","))
         d0 = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
@@ -462,7 +501,7 @@ def run_ours(args):
     G = args.instances if args.instances else instances_for(cfg)
     inst = Instances(b2c, torch, cfg, G, policy)
     if graph:
-        inst.capture(torch)
+        inst.capture(torch, streams=args.streams)
     ms = time_steps(torch, inst.step, args.steps, args.warmup, dist, args.min_warm_s)
     inst.check_status(b2c)
     clocks = sampler.stop() if rank == 0 else None
@@ -476,7 +515,7 @@ def run_ours(args):
     # ---- the dominant kernel alone (the paper's "Op." column) for the roofline -------------------
     op = None
     if not args.no_op_pass:
-        op = op_only(b2c, torch, cfg, emb.variant, emb.tile_n, emb.split_k, args.steps, args.warmup, graph)
+        op = op_only(b2c, torch, cfg, emb.variant, emb.tile_n, emb.split_k, args.steps, args.warmup, graph, args.streams)
     t_roof, bound = roofline_time_us(cfg, peaks)
     op_us = op["us"] if op else per_call_us
     if bound == "tensor":
@@ -487,6 +526,7 @@ def run_ours(args):
     traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["conv_mma_sha1"] == sha else None
     roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
                 "traffic": traffic, "kernel": "conv_mma_kernel", "kernel_us": op_us,
+                "kernel_us_note": "timed region / launches, %d launches in flight" % (args.streams if graph else 1),
                 "peak_source": "%s bf16 burst x %.0f (nominal int8:bf16)" % (peaks["source"], INT8_TO_BF16_RATIO)
                 if bound == "tensor" else peaks["source"] + " copy bandwidth"}
 
@@ -501,8 +541,8 @@ def run_ours(args):
     if rank == 0 and not args.headline_only:
         per_config = []
         for c in CONFIGS:
-            r = measure_shape(b2c, torch, c, max(2, args.steps // 2), 3, peaks,
-                              policy if c is cfg else b2c.POLICY_AUTO_TIMED, None, graph)
+            r = measure_shape(b2c, torch, c, max(2, args.steps // 2), 3, peaks, b2c.POLICY_AUTO_TIMED, None, graph,
+                              args.streams)
             per_config.append(r)
     scaled = None
     if rank == 0 and not args.headline_only:
@@ -520,7 +560,8 @@ def run_ours(args):
         "dtype": "s8 x s8 -> s32", "data": "synthetic",
         "config": {"workload": cfg.name, "instances_per_step": G, "per_call_us": per_call_us,
                    "l2": "inputs larger than L2: %d distinct buffer sets per step (%.0f MB)" % (G, G * (cfg.algorithmic_bytes) / 1e6),
-                   "cuda_graph": graph, "parallelism": "independent instances sharded over ranks, no collective",
+                   "cuda_graph": graph, "streams": args.streams if graph else 1,
+                   "parallelism": "independent instances sharded over ranks, no collective",
                    "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k,
                                  "planner_us": emb.device_us}},
         "roofline": roofline, "roofline_time_us": t_roof, "whole_path_roofline_frac": t_roof / per_call_us,
@@ -552,6 +593,8 @@ def main():
     ap.add_argument("--scaled", action="store_true", help="use the batch-scaled version of the shape as the workload")
     ap.add_argument("--instances", type=int, default=0, help="instances per step (default: enough to exceed L2)")
     ap.add_argument("--min-warm-s", type=float, default=0.2, help="extra time-based warm-up before the timed steps")
+    ap.add_argument("--streams", type=int, default=16,
+                    help="graph branches the independent instances of a step are dealt onto (1 = one call after the other)")
     ap.add_argument("--no-op-pass", action="store_true", help="skip the separate pass that times the MMA kernel alone")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end pass")
     args = ap.parse_args()

@@ -324,47 +324,74 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
 
 // Device time of one run of `p`: the launches of `iters` runs are captured into a CUDA graph on a
 // private stream and the graph is replayed, so that host launch cost does not mask the kernels.
-int time_plan(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, float* us) {
+// With lanes > 1 every iteration enqueues one run per lane, each lane on a stream of its own
+// (forked from and joined back into the first) with its own outputs and scratch, so that kernels
+// of different lanes may overlap on the GPU; *us is then the time per run at that concurrency.
+constexpr int kMaxLanes = 8;
+struct LaneBuffers {
+  int32_t* y32;
+  int8_t* y8;
+  void* ws;
+};
+int time_plan(b2c_plan* p, const int8_t* x, const LaneBuffers* lane, int lanes, float* us) {
   const int iters = 10, replays = 3;
-  cudaStream_t st = nullptr;
-  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaStream_t st[kMaxLanes] = {};
+  cudaEvent_t e0 = nullptr, e1 = nullptr, fork = nullptr, join[kMaxLanes] = {};
   cudaGraph_t graph = nullptr;
   cudaGraphExec_t exec = nullptr;
   int rc = B2C_OK;
-  cudaError_t e = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking);
+  cudaError_t e = cudaSuccess;
+  for (int l = 0; l < lanes && e == cudaSuccess; ++l) e = cudaStreamCreateWithFlags(&st[l], cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaEventCreate(&e0);
   if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&fork, cudaEventDisableTiming);
+  for (int l = 1; l < lanes && e == cudaSuccess; ++l) e = cudaEventCreateWithFlags(&join[l], cudaEventDisableTiming);
   if (e == cudaSuccess) {
     // plain runs first: first-launch set-up (function attributes) must not happen under capture
-    for (int i = 0; i < 2 && rc == B2C_OK; ++i) rc = b2c_conv2d_int8_run(p, x, y32, y8, ws, st);
-    if (rc == B2C_OK) e = cudaStreamSynchronize(st);
+    for (int i = 0; i < 2 && rc == B2C_OK; ++i)
+      rc = b2c_conv2d_int8_run(p, x, lane[0].y32, lane[0].y8, lane[0].ws, st[0]);
+    if (rc == B2C_OK) e = cudaStreamSynchronize(st[0]);
   }
   if (e == cudaSuccess && rc == B2C_OK) {
-    e = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal);
+    e = cudaStreamBeginCapture(st[0], cudaStreamCaptureModeThreadLocal);
     if (e == cudaSuccess) {
-      for (int i = 0; i < iters && rc == B2C_OK; ++i) rc = b2c_conv2d_int8_run(p, x, y32, y8, ws, st);
-      cudaError_t e2 = cudaStreamEndCapture(st, &graph);
-      if (e2 != cudaSuccess) e = e2;
+      if (lanes > 1) {
+        e = cudaEventRecord(fork, st[0]);
+        for (int l = 1; l < lanes && e == cudaSuccess; ++l) e = cudaStreamWaitEvent(st[l], fork, 0);
+      }
+      for (int i = 0; i < iters && rc == B2C_OK && e == cudaSuccess; ++i)
+        for (int l = 0; l < lanes && rc == B2C_OK; ++l)
+          rc = b2c_conv2d_int8_run(p, x, lane[l].y32, lane[l].y8, lane[l].ws, st[l]);
+      for (int l = 1; l < lanes && e == cudaSuccess; ++l) {
+        e = cudaEventRecord(join[l], st[l]);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st[0], join[l], 0);
+      }
+      cudaError_t e2 = cudaStreamEndCapture(st[0], &graph);
+      if (e == cudaSuccess && e2 != cudaSuccess) e = e2;
     }
   }
   if (e == cudaSuccess && rc == B2C_OK) e = cudaGraphInstantiate(&exec, graph, 0);
   if (e == cudaSuccess && rc == B2C_OK) {
-    e = cudaGraphLaunch(exec, st);  // warm
-    if (e == cudaSuccess) e = cudaEventRecord(e0, st);
-    for (int i = 0; i < replays && e == cudaSuccess; ++i) e = cudaGraphLaunch(exec, st);
-    if (e == cudaSuccess) e = cudaEventRecord(e1, st);
+    e = cudaGraphLaunch(exec, st[0]);  // warm
+    if (e == cudaSuccess) e = cudaEventRecord(e0, st[0]);
+    for (int i = 0; i < replays && e == cudaSuccess; ++i) e = cudaGraphLaunch(exec, st[0]);
+    if (e == cudaSuccess) e = cudaEventRecord(e1, st[0]);
     if (e == cudaSuccess) e = cudaEventSynchronize(e1);
     if (e == cudaSuccess) {
       float ms = 0;
       e = cudaEventElapsedTime(&ms, e0, e1);
-      *us = ms * 1000.0f / (iters * replays);
+      *us = ms * 1000.0f / (iters * replays * lanes);
     }
   }
   if (exec) cudaGraphExecDestroy(exec);
   if (graph) cudaGraphDestroy(graph);
   if (e0) cudaEventDestroy(e0);
   if (e1) cudaEventDestroy(e1);
-  if (st) cudaStreamDestroy(st);
+  if (fork) cudaEventDestroy(fork);
+  for (int l = 0; l < kMaxLanes; ++l) {
+    if (join[l]) cudaEventDestroy(join[l]);
+    if (st[l]) cudaStreamDestroy(st[l]);
+  }
   if (e != cudaSuccess) {
     set_last_cuda_error((int)e);
     return B2C_E_CUDA;
@@ -439,8 +466,9 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
   std::vector<b2c_embedding> all(count);
   rc = b2c_enumerate(desc, all.data(), count, &count);
   if (rc != B2C_OK) return rc;
-  if (policy_or_id < B2C_POLICY_MIN_WORKSPACE) return B2C_E_INVALID_ARG;
-  if (policy_or_id != B2C_POLICY_AUTO_TIMED) {
+  if (policy_or_id < B2C_POLICY_AUTO_TIMED_CONCURRENT) return B2C_E_INVALID_ARG;
+  const int lanes = policy_or_id == B2C_POLICY_AUTO_TIMED_CONCURRENT ? kMaxLanes : 1;
+  if (policy_or_id != B2C_POLICY_AUTO_TIMED && policy_or_id != B2C_POLICY_AUTO_TIMED_CONCURRENT) {
     int idx = pick_by_policy(all, policy_or_id);
     if (idx < 0) return B2C_E_INVALID_ARG;
     return create_plan_for(g, all[idx], out);
@@ -455,19 +483,23 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
       groups.push_back(e.variant);
   size_t ws_max = 0;
   for (const b2c_embedding& e : all) ws_max = std::max(ws_max, (size_t)e.workspace_bytes);
-  int8_t *x = nullptr, *w = nullptr, *y8 = nullptr;
-  int32_t* y32 = nullptr;
-  void* ws = nullptr;
+  int8_t *x = nullptr, *w = nullptr;
+  LaneBuffers lane[kMaxLanes] = {};
   auto cleanup = [&]() {
     cudaFree(x);
     cudaFree(w);
-    cudaFree(y8);
-    cudaFree(y32);
-    cudaFree(ws);
+    for (int l = 0; l < kMaxLanes; ++l) {
+      cudaFree(lane[l].y8);
+      cudaFree(lane[l].y32);
+      cudaFree(lane[l].ws);
+    }
   };
-  if (cudaMalloc(&x, g.x_elems + 256) != cudaSuccess || cudaMalloc(&w, g.w_elems + 256) != cudaSuccess ||
-      cudaMalloc(&y8, g.y_elems + 256) != cudaSuccess || cudaMalloc(&y32, g.y_elems * 4 + 256) != cudaSuccess ||
-      cudaMalloc(&ws, ws_max + 256) != cudaSuccess) {
+  bool alloc_ok = cudaMalloc(&x, g.x_elems + 256) == cudaSuccess && cudaMalloc(&w, g.w_elems + 256) == cudaSuccess;
+  for (int l = 0; l < lanes && alloc_ok; ++l)
+    alloc_ok = cudaMalloc(&lane[l].y8, g.y_elems + 256) == cudaSuccess &&
+               cudaMalloc(&lane[l].y32, g.y_elems * 4 + 256) == cudaSuccess &&
+               cudaMalloc(&lane[l].ws, ws_max + 256) == cudaSuccess;
+  if (!alloc_ok) {
     set_last_cuda_error((int)cudaGetLastError());
     cleanup();
     return B2C_E_CUDA;
@@ -485,7 +517,7 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
     rc = b2c_plan_set_weights(p, w, st);
     if (rc == B2C_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = B2C_E_CUDA;
     float us = -1;
-    if (rc == B2C_OK) rc = time_plan(p, x, y32, y8, ws, &us);
+    if (rc == B2C_OK) rc = time_plan(p, x, lane, lanes, &us);
     b2c_plan_destroy(p);
     if (rc != B2C_OK) break;
     all[i].device_us = us;

@@ -156,9 +156,10 @@ def test_one_shot_device_and_host_calls(lib):
 def test_policies(lib):
     cfg = CONFIGS[0]
     x, w, ref = cfg_reference(cfg)
-    for policy in (b2c.POLICY_AUTO_TIMED, b2c.POLICY_MIN_OVERHEAD, b2c.POLICY_MIN_WORKSPACE):
+    for policy in (b2c.POLICY_AUTO_TIMED, b2c.POLICY_AUTO_TIMED_CONCURRENT, b2c.POLICY_MIN_OVERHEAD,
+                   b2c.POLICY_MIN_WORKSPACE):
         emb = check_against_oracle(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, cfg.out_mode, policy, ref=ref)
-        if policy == b2c.POLICY_AUTO_TIMED:
+        if policy in (b2c.POLICY_AUTO_TIMED, b2c.POLICY_AUTO_TIMED_CONCURRENT):
             assert emb.device_us > 0
         if policy == b2c.POLICY_MIN_WORKSPACE:
             assert emb.workspace_bytes == 0
