@@ -3,6 +3,7 @@
 // the timed candidate selection.  See include/b2conv.h for the contract of each entry point.
 #include <algorithm>
 #include <cstring>
+#include <cstdlib>
 #include <map>
 #include <mutex>
 #include <new>
@@ -125,6 +126,7 @@ void fill_common_args(b2c_plan* p) {
   a.out_layout = d.out_layout;
   a.table_len = p->table_len;
   a.table32 = p->table32;
+  a.swap = is_swapped(p->emb) ? 1 : 0;
   a.C = d.C;
   a.P = p->g.P;
   a.win_rows = p->win.rows;
@@ -175,7 +177,8 @@ void fill_common_args(b2c_plan* p) {
   // overlap the other's main loop.
   int per_cta_kb = (a.num_kb + a.split_k - 1) / a.split_k;
   int stages = std::min(6, std::max(1, per_cta_kb));
-  const long long ctas = ((p->g.Mg + kTileM - 1) / kTileM) * ((d.K + a.tile_n - 1) / a.tile_n) * a.split_k;
+  const long long ctas = a.swap ? ((p->g.Mg + a.tile_n - 1) / a.tile_n) * ((d.K + kTileM - 1) / kTileM) * a.split_k
+                                : ((p->g.Mg + kTileM - 1) / kTileM) * ((d.K + a.tile_n - 1) / a.tile_n) * a.split_k;
   // Large TMA-fed problems run persistently: one block per SM walks the tile list with two
   // accumulator buffers in tensor memory and the deepest stage ring that fits.
   const long long tiles_m = (p->g.Mg + kTileM - 1) / kTileM;
@@ -185,7 +188,7 @@ void fill_common_args(b2c_plan* p) {
   a.div_tiles_n = make_fastdiv((uint32_t)tiles_n);
   // Wide tiles: one block per SM.  Narrow tiles have short main loops and do better with three
   // blocks per SM, each still walking several tiles (mode 2) once there are enough tiles.
-  const bool tma_fed = (p->amode == A_TILED || p->amode == A_IM2COL_TMA) && a.split_k == 1 &&
+  const bool tma_fed = (p->amode == A_TILED || p->amode == A_IM2COL_TMA) && a.split_k == 1 && !a.swap &&
                        tiles_m * tiles_n < 0x7FFFFFFF;
   a.persistent = 0;
   if (tma_fed && a.tile_n >= 128 && tiles_m * tiles_n > 2 * kNumSMs) a.persistent = 1;
@@ -195,14 +198,15 @@ void fill_common_args(b2c_plan* p) {
       tiles_m * tiles_n < 0x7FFFFFFF)
     a.persistent = 2;
   a.tmem_bufs = (a.persistent && 2 * a.tmem_cols <= 512) ? 2 : 1;
-  const size_t budget = a.persistent == 1 ? 196 * 1024 : (a.persistent == 2 ? 68 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 160 * 1024));
+  size_t budget = a.persistent == 1 ? 196 * 1024 : (a.persistent == 2 ? 68 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 160 * 1024));
+  if (getenv("B2C_XBUDGET") && !a.persistent) budget = (size_t)atoi(getenv("B2C_XBUDGET")) * 1024;
   const size_t stage_bytes = (size_t)(kTileM + a.tile_n) * a.bk;
   // lookup table and staged window share the block's shared memory with the stages
   const size_t extra = p->amode == A_STAGED ? (size_t)p->win.bytes + 4 * (size_t)p->table_len + 64
                                             : (p->amode == A_GATHER ? 8 * (size_t)p->table_len : 0);
   while (stages > 2 && (size_t)stages * stage_bytes + extra > budget) --stages;
   while (stages > 1 && (size_t)stages * stage_bytes + extra > 196 * 1024) --stages;
-  a.cluster_split = cluster_split_ok(p->emb.variant, a.tile_n, a.split_k) ? 1 : 0;
+  a.cluster_split = cluster_split_ok(p->emb.variant, a.tile_n, a.split_k, a.swap != 0) ? 1 : 0;
   size_t region = (size_t)stages * stage_bytes;
   // the stage buffers double as the 128 x tile_n int32 exchange tile of the cluster reduction
   if (a.cluster_split) region = std::max(region, (size_t)kTileM * a.tile_n * 4);
@@ -302,7 +306,7 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
   // Room for one extra box row block so that a TMA box never starts past the allocation.
   if (cudaMalloc(&p->w_packed, p->w_packed_bytes + 256) != cudaSuccess) return fail(B2C_E_CUDA);
   fill_common_args(p);
-  p->ws_total = workspace_bytes_for(g, emb.variant, emb.tile_n, emb.split_k);
+  p->ws_total = workspace_bytes_for(g, emb.variant, emb.tile_n, emb.split_k, is_swapped(emb));
   if (is_tma_view_variant(emb.variant)) {
     bool direct = emb.variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && p->C_pad == d.C;
     p->ws_layout_bytes = direct ? 0 : ((size_t)p->view.bytes() + 255) / 256 * 256;
@@ -310,12 +314,14 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
     p->ws_layout_bytes = ((size_t)g.Mg * p->K_pad + 255) / 256 * 256;
   }
   // Tensor map of the packed weights (plan-owned memory, so it is encoded once).
+  // (Swapped map: the weights are the 128-row operand, so their box is 128 rows high.)
   int rc;
+  const int w_box_rows = is_swapped(emb) ? kTileM : emb.tile_n;
   if (is_tma_view_variant(emb.variant)) {
     uint64_t cols = (uint64_t)p->view.R * p->view.S * p->view.C;
-    rc = encode_tiled_2d(&p->tmap_b, p->w_packed, cols, d.K, cols, p->bk, emb.tile_n, p->bk);
+    rc = encode_tiled_2d(&p->tmap_b, p->w_packed, cols, d.K, cols, p->bk, w_box_rows, p->bk);
   } else {
-    rc = encode_tiled_2d(&p->tmap_b, p->w_packed, p->K_pad, d.K, p->K_pad, 128, emb.tile_n, 128);
+    rc = encode_tiled_2d(&p->tmap_b, p->w_packed, p->K_pad, d.K, p->K_pad, 128, w_box_rows, 128);
   }
   if (rc != B2C_OK) return fail(rc);
   *out = p;
@@ -600,13 +606,13 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
       act = scratch;
     }
     rc = encode_im2col_nhwc(&tmap_a, act, v.C, v.W, v.H, v.N, v.pad_w, v.pad_h, v.S, v.R, v.dil_w, v.dil_h,
-                            v.stride_w, v.stride_h, p->bk, kTileM, p->bk);
+                            v.stride_w, v.stride_h, p->bk, a.swap ? a.tile_n : kTileM, p->bk);
     if (rc != B2C_OK) return rc;
   } else if (p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
     int8_t* A = reinterpret_cast<int8_t*>(wsb);
     CUDA_TRY(launch_im2col(x, A, p->table, g.Mg, g.PQ, g.Q, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
                            a.x_stride_n, a.x_stride_h, a.x_stride_w, p->K_pad, st));
-    rc = encode_tiled_2d(&tmap_a, A, p->K_pad, (uint64_t)g.Mg, p->K_pad, 128, kTileM, 128);
+    rc = encode_tiled_2d(&tmap_a, A, p->K_pad, (uint64_t)g.Mg, p->K_pad, 128, a.swap ? a.tile_n : kTileM, 128);
     if (rc != B2C_OK) return rc;
   } else {
     tmap_a = p->tmap_b;  // unused by the gather kernel; any valid map

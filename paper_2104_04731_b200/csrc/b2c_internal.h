@@ -100,6 +100,9 @@ struct ConvArgs {
   FastDiv div_tiles_n;
   int stage_region;   // bytes of shared memory reserved for the stage ring (and the cluster exchange tile)
   int cluster_split;  // split_k slices form a cluster (1, 1, split_k) and reduce through shared memory
+  // swapped axis map: accumulator rows = output channels (the 128-row MMA operand is the packed
+  // weights), accumulator columns = tile_n fused (n, p, q) pixels (the N operand is the activations)
+  int swap;
 };
 
 // Programmatic dependent launch: a kernel launched through launch_pdl may start while the previous
@@ -162,13 +165,15 @@ int cp_block_bytes(int C_pad);       // reduction bytes per block for the channe
 int im2col_k_pad(int Kg);            // padded reduction length for the stencil-unroll maps
 void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out);
 int pick_by_policy(const std::vector<b2c_embedding>& all, int policy);  // index or -1
-size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k);
+size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k, bool swap = false);
+inline bool is_swapped(const b2c_embedding& e) { return e.map_m == B2C_AXIS_K; }
 // A split reduction of 2, 4 or 8 slices whose tile is wide enough runs as a thread-block cluster:
 // the slices exchange their partial accumulators through distributed shared memory, so no scratch
 // buffer, zero-fill or finish pass is needed.
 // (The variants that keep a lookup table or an input window in shared memory leave room for a
 // 128-column exchange tile at most.)
-inline bool cluster_split_ok(int variant, int tile_n, int split_k) {
+inline bool cluster_split_ok(int variant, int tile_n, int split_k, bool swap = false) {
+  if (swap) return false;  // the swapped map meets its partial sums in global memory
   const bool table_in_smem = variant == B2C_VARIANT_IM2COL_GATHER || variant == B2C_VARIANT_IM2COL_STAGED;
   return (split_k == 2 || split_k == 4 || split_k == 8) && tile_n >= 32 * split_k && (!table_in_smem || tile_n <= 128);
 }

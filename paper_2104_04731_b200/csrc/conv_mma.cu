@@ -297,6 +297,87 @@ __device__ __forceinline__ void store_columns(const ConvArgs& args, const int32_
   }
 }
 
+// Swapped axis map: this thread's accumulator row is output channel k, and v holds 16 consecutive
+// fused pixels m_first .. m_first + 15.  NPQK: for a fixed pixel the 32 lanes of a warp hold 32
+// consecutive channels, so every store instruction writes one contiguous run.  NKPQ: the 16 pixels
+// of a thread are contiguous while they stay inside one image, and go out as 16-byte vectors when
+// the run is complete and aligned.
+__device__ __forceinline__ void store_columns_swapped(const ConvArgs& args, const int32_t* v, int k, bool row_valid,
+                                                      int m_first) {
+  if (!row_valid || m_first >= args.Mg) return;
+  const int count = min(16, args.Mg - m_first);
+  const int n_img = (int)args.div_pq.div((uint32_t)m_first);
+  int pq = m_first - n_img * args.PQ;
+  const bool nhwc = args.out_layout == B2C_LAYOUT_NHWC;
+  const bool split = args.split_k > 1;
+  if (nhwc) {
+    long long o = (long long)m_first * args.K + k;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      if (j < count) {
+        if (split) {
+          atomicAdd(args.acc + o, v[j]);
+        } else {
+          if (args.out_mode & B2C_OUT_I32) args.y32[o] = v[j];
+          if (args.out_mode & B2C_OUT_I8) args.y8[o] = requant(v[j], args.shift);
+        }
+      }
+      o += args.K;
+    }
+    return;
+  }
+  long long o = ((long long)n_img * args.K + k) * args.PQ + pq;
+  if (!split && count == 16 && pq + 16 <= args.PQ) {
+    if (args.out_mode & B2C_OUT_I32) {
+      int32_t* dst = args.y32 + o;
+      if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+        for (int j = 0; j < 16; j += 4) *reinterpret_cast<int4*>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) dst[j] = v[j];
+      }
+    }
+    if (args.out_mode & B2C_OUT_I8) {
+      int8_t* dst = args.y8 + o;
+      uint32_t w[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        w[j] = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) w[j] |= (uint32_t)(uint8_t)requant(v[j * 4 + i], args.shift) << (8 * i);
+      }
+      if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+        *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+      } else if ((reinterpret_cast<uintptr_t>(dst) & 3) == 0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) reinterpret_cast<uint32_t*>(dst)[j] = w[j];
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) dst[j] = (int8_t)((w[j >> 2] >> (8 * (j & 3))) & 0xff);
+      }
+    }
+    return;
+  }
+  // general case: the run crosses an image boundary, is a tail, or adds into the split buffer
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    if (j < count) {
+      if (split) {
+        atomicAdd(args.acc + o, v[j]);
+      } else {
+        if (args.out_mode & B2C_OUT_I32) args.y32[o] = v[j];
+        if (args.out_mode & B2C_OUT_I8) args.y8[o] = requant(v[j], args.shift);
+      }
+      ++o;
+      if (++pq == args.PQ) {
+        pq = 0;
+        o += (long long)(args.K - 1) * args.PQ;  // same channel of the next image
+      }
+    }
+  }
+}
+
 template <int NC>
 __device__ __forceinline__ void epilogue_columns(const ConvArgs& args, uint32_t taddr, int kbase, bool row_valid,
                                                  long long base_nkpq, long long base_npqk, uint32_t exchange_addr) {
@@ -342,6 +423,9 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     const int mt_ = (int)args.div_tiles_n.div((uint32_t)(t));                       \
     m0 = mt_ * kTileM;                                                              \
     n0 = ((t) - mt_ * args.tiles_n) * args.tile_n;                                  \
+  } else if (args.swap) {                                                           \
+    m0 = (int)blockIdx.y * kTileM;     /* accumulator rows: output channels */      \
+    n0 = (int)blockIdx.x * args.tile_n; /* accumulator columns: fused pixels */     \
   } else {                                                                          \
     m0 = (int)blockIdx.x * kTileM;                                                  \
     n0 = (int)blockIdx.y * args.tile_n;                                             \
@@ -417,9 +501,14 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     for (int t = tile_first; t < tile_end && alive; t += tile_step) {
       B2C_TILE_ORIGIN(t)
       int n_img = 0, h_org = 0, w_org = 0, cb = 0, sx = 0, r = 0;
+      // Swapped axis map: the activations are the N operand (tile_n pixels from n0 on, into the B
+      // region) and the packed weights the 128-row operand (rows m0 .., into the A region).
+      const bool swap = args.swap != 0;
+      const int pix0 = swap ? n0 : m0;
+      const int wrow0 = swap ? m0 : n0;
       if (AMODE == A_IM2COL_TMA) {
-        n_img = (int)args.div_pq.div((uint32_t)m0);
-        const int rem = m0 - n_img * args.PQ;
+        n_img = (int)args.div_pq.div((uint32_t)pix0);
+        const int rem = pix0 - n_img * args.PQ;
         const int p = (int)args.div_q.div((uint32_t)rem), q = rem - p * args.Q;
         h_org = p * args.stride_h - args.pad_h;
         w_org = q * args.stride_w - args.pad_w;
@@ -440,13 +529,13 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
           tma_load_2d(b_dst, &tmap_b, kcol, n0, full, leader);
         } else if (AMODE == A_TILED) {
           mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes, leader);
-          tma_load_2d(a_dst, &tmap_a, kcol, m0, full, leader);
-          tma_load_2d(b_dst, &tmap_b, kcol, n0, full, leader);
+          tma_load_2d(swap ? b_dst : a_dst, &tmap_a, kcol, pix0, full, leader);
+          tma_load_2d(swap ? a_dst : b_dst, &tmap_b, kcol, wrow0, full, leader);
         } else {
           mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes, leader);
-          tma_load_im2col_4d(a_dst, &tmap_a, cb * bk, w_org, h_org, n_img, full, (uint16_t)(sx * args.dil_w),
-                             (uint16_t)(r * args.dil_h), leader);
-          tma_load_2d(b_dst, &tmap_b, kcol, n0, full, leader);
+          tma_load_im2col_4d(swap ? b_dst : a_dst, &tmap_a, cb * bk, w_org, h_org, n_img, full,
+                             (uint16_t)(sx * args.dil_w), (uint16_t)(r * args.dil_h), leader);
+          tma_load_2d(swap ? a_dst : b_dst, &tmap_b, kcol, wrow0, full, leader);
           if (++cb == args.kb_per_tap) {
             cb = 0;
             if (++sx == args.S) {
@@ -531,9 +620,9 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     for (int t = tile_first; t < tile_end && ok; t += tile_step, ++ti) {
     B2C_TILE_ORIGIN(t)
     const unsigned m = (unsigned)m0 + (unsigned)row;
-    const bool row_valid = m < (unsigned)args.Mg;
+    const bool row_valid = m < (unsigned)(args.swap ? args.K : args.Mg);
     int n_img = 0, pq = 0;
-    if (row_valid) {
+    if (row_valid && !args.swap) {
       n_img = (int)args.div_pq.div(m);
       pq = (int)(m - (unsigned)n_img * (unsigned)args.PQ);
     }
@@ -726,7 +815,15 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
             tmem_acc + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * args.tmem_cols) + (uint32_t)c_begin;
         // cluster reduction: the stage buffers are free once the accumulator is complete
         const uint32_t xch = args.cluster_split ? a_base + (uint32_t)row * 4u + (uint32_t)c_begin * (kTileM * 4) : 0u;
-        if ((cols & 31) == 0) {
+        if (args.swap) {
+          // accumulator row = output channel m, columns = pixels n0 + c_begin ..
+          for (int c = 0; c < cols; c += 16) {
+            int32_t v[16];
+            __syncwarp();
+            tmem_ld<16>(taddr + (uint32_t)c, v);
+            store_columns_swapped(args, v, (int)m, row_valid, n0 + c_begin + c);
+          }
+        } else if ((cols & 31) == 0) {
           for (int c = 0; c < cols; c += 32)
             epilogue_columns<32>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk,
                                  xch ? xch + (uint32_t)c * (kTileM * 4) : 0u);
@@ -905,6 +1002,9 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
   const size_t smem = conv_mma_smem_bytes(amode, args);
   dim3 grid((unsigned)((args.Mg + kTileM - 1) / kTileM), (unsigned)((args.K + args.tile_n - 1) / args.tile_n),
             (unsigned)args.split_k);
+  if (args.swap)
+    grid = dim3((unsigned)((args.Mg + args.tile_n - 1) / args.tile_n), (unsigned)((args.K + kTileM - 1) / kTileM),
+                (unsigned)args.split_k);
   if (args.persistent) grid = dim3((unsigned)std::min(args.num_tiles, kNumSMs * (args.persistent == 2 ? 3 : 1)), 1, 1);
   cudaError_t e;
 #define B2C_LAUNCH(MODE, PERS)                                                                             \

@@ -71,7 +71,7 @@ int variant_k_pad(const Geom& g, int variant) {
   return im2col_k_pad(g.Kg);
 }
 
-size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k) {
+size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k, bool swap) {
   size_t ws = 0;
   const b2c_conv_desc& d = g.d;
   TmaView v;
@@ -84,7 +84,8 @@ size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k) 
   ws = (ws + 255) / 256 * 256;
   // A split reduction accumulates int32 partial sums in scratch unless the int32 output itself
   // can serve (int32-only output in any layout).
-  if (split_k > 1 && !cluster_split_ok(variant, tile_n, split_k) && (d.out_mode & B2C_OUT_I8)) ws += (size_t)g.y_elems * 4;
+  if (split_k > 1 && !cluster_split_ok(variant, tile_n, split_k, swap) && (d.out_mode & B2C_OUT_I8))
+    ws += (size_t)g.y_elems * 4;
   return ws;
 }
 
@@ -148,12 +149,13 @@ bool staged_window(const Geom& g, WindowGeom* w) {
   return true;
 }
 
-static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int tile_n, int split_k) {
+static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int tile_n, int split_k,
+                bool swap = false) {
   const b2c_conv_desc& d = g.d;
   b2c_embedding e;
   std::memset(&e, 0, sizeof(e));
-  e.map_m = B2C_AXIS_NPQ;
-  e.map_n = B2C_AXIS_K;
+  e.map_m = swap ? B2C_AXIS_K : B2C_AXIS_NPQ;
+  e.map_n = swap ? B2C_AXIS_NPQ : B2C_AXIS_K;
   e.variant = variant;
   e.tile_m = kTileM;
   e.tile_n = tile_n;
@@ -161,6 +163,10 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
   e.device_us = -1.0f;
   long long M_pad = (g.Mg + kTileM - 1) / kTileM * kTileM;
   long long N_pad = (long long)round_up(d.K, tile_n);
+  if (swap) {
+    M_pad = (long long)round_up(d.K, kTileM);
+    N_pad = (g.Mg + tile_n - 1) / tile_n * tile_n;
+  }
   long long k_issued, moved;
   long long mac_min = g.Mg * d.K * g.Kg;
   long long data_min = g.x_elems + g.w_elems + g.y_elems;
@@ -183,10 +189,10 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
     else
       moved = g.x_elems + (long long)d.K * K_pad + g.y_elems;
   }
-  if (split_k > 1 && !cluster_split_ok(variant, tile_n, split_k)) moved += 2 * g.y_elems;  // partial sums through memory
+  if (split_k > 1 && !cluster_split_ok(variant, tile_n, split_k, swap)) moved += 2 * g.y_elems;  // partial sums through memory
   e.o_mac = M_pad * N_pad * k_issued - mac_min;
   e.o_data = moved - data_min;
-  e.workspace_bytes = (int64_t)workspace_bytes_for(g, variant, tile_n, split_k);
+  e.workspace_bytes = (int64_t)workspace_bytes_for(g, variant, tile_n, split_k, swap);
   out->push_back(e);
 }
 
@@ -224,6 +230,24 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
         // A split reduction only helps while the grid is smaller than the machine.
         if (split > 1 && ctas * (split / 2) >= kNumSMs) break;
         add(out, g, variant, t, split);
+      }
+    }
+    // Swapped axis map (M <- k, N <- fused pixels) for the TMA-fed variants: the 128 accumulator rows
+    // are output channels, so it is only listed when K fills at least half of them; the pixel tile
+    // widths are those that waste less than a quarter of their columns (or the covering one).
+    if ((is_tma_view_variant(variant) || variant == B2C_VARIANT_IM2COL_EXPLICIT) && d.K >= kTileM / 2) {
+      const long long tiles_k = (d.K + kTileM - 1) / kTileM;
+      for (int t = 32; t <= 256; t <<= 1) {
+        const long long n_pad = (g.Mg + t - 1) / t * t;
+        const bool covering = t >= g.Mg || t == 256;
+        if (!covering && (n_pad - g.Mg) * 4 > n_pad) continue;
+        const long long ctas = tiles_k * (n_pad / t);
+        for (int split = 1; split <= 32; split <<= 1) {
+          if (split > num_kb) break;
+          if (split > 1 && ctas * (split / 2) >= kNumSMs) break;
+          add(out, g, variant, t, split, true);
+        }
+        if (t >= g.Mg) break;
       }
     }
   }

@@ -115,6 +115,38 @@ def test_random_shapes(lib, case):
     check_against_oracle(x, w, stride, pad, dil, shift, 3, e2.id, ref=ref, in_layout=1, out_layout=1)
 
 
+# ---- swapped axis map (M <- k, N <- fused pixels) -------------------------------------------------------
+@pytest.mark.parametrize("case", [
+    # N, C, H, W, K, R, S, stride, pad, dil, shift
+    (2, 32, 9, 11, 64, 3, 3, 1, 1, 1, 8),          # one channel tile half full
+    (3, 40, 7, 7, 129, 3, 2, (2, 1), (1, 0), 1, 9),   # two channel tiles, the second with one row; images of 12 pixels
+    (1, 256, 14, 14, 200, 3, 3, 2, 1, 1, 10),      # 49 pixels: runs cross no image boundary, ragged channel tile
+    (5, 3, 20, 21, 96, 5, 5, 2, 2, (1, 2), 6),     # low channel count: row-unroll / space-to-depth / explicit views
+    (2, 64, 30, 30, 128, 1, 1, 1, 0, 1, 7),        # 1x1, 1800 pixels: several 256-pixel tiles and a tail
+])
+@pytest.mark.parametrize("out_layout", [0, 1])
+def test_swapped_axis_map(lib, case, out_layout):
+    N, C, H, W, K, R, S, stride, pad, dil, shift = case
+    x = int8_uniform((N, C, H, W), 611)
+    w = int8_uniform((K, C, R, S), 612)
+    ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, 0, out_layout, 3)
+    swapped = [e for e in lib.enumerate_embeddings(d) if e.map_m == b2c.AXIS_K]
+    assert swapped and all(e.map_n == b2c.AXIS_NPQ and e.tile_m == 128 for e in swapped)
+    seen = set()
+    for e in swapped:
+        key = (e.variant, e.tile_n, min(e.split_k, 2))
+        if key in seen:
+            continue
+        seen.add(key)
+        check_against_oracle(x, w, stride, pad, dil, shift, 3, e.id, ref=ref, out_layout=out_layout)
+    # int8-only output through a split reduction goes through the scratch buffer and the finish kernel
+    d8 = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, 0, out_layout, 2)
+    split = [e for e in lib.enumerate_embeddings(d8) if e.map_m == b2c.AXIS_K and e.split_k > 1]
+    if split:
+        check_against_oracle(x, w, stride, pad, dil, shift, 2, split[0].id, ref=ref, out_layout=out_layout)
+
+
 def test_extreme_values_and_shift_clip(lib):
     # -128 * -128 is the largest product; all-(-128) tensors with 9*64 taps reach 9437184.
     x = np.full((1, 64, 6, 6), -128, dtype=np.int8)

@@ -86,7 +86,9 @@ def test_enumeration_is_sorted_and_covers_variants(lib, cfg):
     assert {0, 1, 2} <= {e.variant for e in embs} <= {0, 1, 2, 3, 4, 5}
     for e in embs:
         assert e.tile_m == 128 and e.tile_n in (16, 32, 64, 128, 256) and e.split_k >= 1
-        assert e.map_m == b2c.AXIS_NPQ and e.map_n == b2c.AXIS_K
+        assert (e.map_m, e.map_n) in ((b2c.AXIS_NPQ, b2c.AXIS_K), (b2c.AXIS_K, b2c.AXIS_NPQ))
+        if e.map_m == b2c.AXIS_K:  # swapped map: TMA-fed variants only, and only when K fills half a tile
+            assert e.variant in (0, 1, 4, 5) and cfg.K >= 64 and e.tile_n >= 32
         assert e.map_k == {0: b2c.AXIS_C, 4: b2c.AXIS_SC, 5: b2c.AXIS_C_PHASES}.get(e.variant, b2c.AXIS_CRS)
         assert e.o_mac >= 0 and e.o_data >= 0 and e.device_us == -1.0
         if e.variant in (b2c.VARIANT_IM2COL_GATHER, b2c.VARIANT_IM2COL_STAGED) and e.split_k == 1:
@@ -100,13 +102,19 @@ def test_channel_pack_utilisation_law(lib):
         N, H, W, K, R, S = 2, 16, 16, 64, 3, 3  # pad 1 stride 1 -> P = Q = 16, M = 512
         d = b2c.make_desc(N, C, H, W, K, R, S, 1, 1, 1)
         mac_min = N * K * 16 * 16 * C * R * S
-        cp = [e for e in b2c.enumerate_embeddings(d) if e.variant == 0 and e.tile_n == 64 and e.split_k == 1]
+        cp = [e for e in b2c.enumerate_embeddings(d)
+              if e.variant == 0 and e.tile_n == 64 and e.split_k == 1 and e.map_m == b2c.AXIS_NPQ]
         assert len(cp) == 1
         assert (cp[0].o_mac + mac_min) * C == mac_min * C_pad
         # the stencil-unroll maps pad the fused (c, r, s) axis to 32 instead
         kp = -(-C * R * S // 32) * 32
         un = [e for e in b2c.enumerate_embeddings(d) if e.variant == 2 and e.tile_n == 64 and e.split_k == 1]
         assert (un[0].o_mac + mac_min) * (C * R * S) == mac_min * kp
+        # swapped map (M <- k, N <- pixels): K = 64 fills half of the 128 accumulator rows, so the
+        # issued MACs double on top of the channel padding; M = 512 pixels is a multiple of every tile
+        for e in b2c.enumerate_embeddings(d):
+            if e.variant == 0 and e.map_m == b2c.AXIS_K and e.split_k == 1:
+                assert (e.o_mac + mac_min) * C == 2 * mac_min * C_pad
 
 
 def test_padding_inflates_weights_and_workspace(lib):
@@ -114,7 +122,7 @@ def test_padding_inflates_weights_and_workspace(lib):
     # the scratch size of the channel-pack map.
     cfg = CONFIGS[2]  # C = 3
     d = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad)
-    embs = b2c.enumerate_embeddings(d)
+    embs = [e for e in b2c.enumerate_embeddings(d) if e.map_m == b2c.AXIS_NPQ]
     cp = next(e for e in embs if e.variant == 0 and e.split_k == 1)
     ga = next(e for e in embs if e.variant == 2 and e.split_k == 1)
     ex = next(e for e in embs if e.variant == 1 and e.split_k == 1)
@@ -138,3 +146,22 @@ def test_nhwc_input_channel_pack_needs_multiple_of_32(lib):
     d = b2c.make_desc(1, 64, 8, 8, 16, 3, 3, 1, 1, in_layout=b2c.LAYOUT_NHWC)
     cp = [e for e in b2c.enumerate_embeddings(d) if e.variant == 0 and e.split_k == 1]
     assert cp and all(e.workspace_bytes == 0 for e in cp)
+
+
+def test_swapped_map_is_listed_only_when_k_fills_half_a_tile(lib):
+    for K, listed in [(16, False), (63, False), (64, True), (129, True), (512, True)]:
+        d = b2c.make_desc(2, 32, 12, 12, K, 3, 3, 1, 1)
+        swapped = [e for e in b2c.enumerate_embeddings(d) if e.map_m == b2c.AXIS_K]
+        assert bool(swapped) == listed, K
+        for e in swapped:
+            assert e.map_n == b2c.AXIS_NPQ and e.variant in (0, 1, 4, 5)
+            # pixel tile: covering width or less than a quarter of its columns wasted
+            M = 2 * 12 * 12
+            n_pad = -(-M // e.tile_n) * e.tile_n
+            assert e.tile_n >= M or e.tile_n == 256 or (n_pad - M) * 4 <= n_pad
+            # a swapped split reduction meets in memory: int8 output needs the int32 scratch
+            if e.split_k > 1:
+                d8 = b2c.make_desc(2, 32, 12, 12, K, 3, 3, 1, 1, out_mode=2)
+                e8 = next(c for c in b2c.enumerate_embeddings(d8)
+                          if (c.map_m, c.variant, c.tile_n, c.split_k) == (e.map_m, e.variant, e.tile_n, e.split_k))
+                assert e8.workspace_bytes >= 4 * M * K
