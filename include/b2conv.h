@@ -76,6 +76,8 @@ typedef struct {
 #define B2C_VARIANT_IM2COL_STAGED 3  /* same, from a zero-padded input window staged in shared memory (low-channel shapes) */
 #define B2C_VARIANT_ROW_UNROLL 4     /* stencil unroll along the kernel row only: scratch tensor [N][H][Q][(s,c)], im2col-mode TMA over r */
 #define B2C_VARIANT_SPACE_TO_DEPTH 5 /* image pack: stride phases folded into channels, then a stride-1 channel-pack conv */
+#define B2C_VARIANT_DILATION_PACK 6  /* image pack of a dilated conv (Section 6.1): the dil_h*dil_w phase sub-images are fused
+                                      * into the batch, convolved densely, and the epilogue interleaves the results back */
 
 typedef struct {
   int32_t id;       /* index in the enumeration for this descriptor; pass to b2c_plan_create      */

@@ -127,6 +127,9 @@ void fill_common_args(b2c_plan* p) {
   a.table_len = p->table_len;
   a.table32 = p->table32;
   a.swap = is_swapped(p->emb) ? 1 : 0;
+  a.out_PQ = p->g.PQ;
+  a.out_P = p->g.P;
+  a.out_Q = p->g.Q;
   a.C = d.C;
   a.P = p->g.P;
   a.win_rows = p->win.rows;
@@ -159,6 +162,23 @@ void fill_common_args(b2c_plan* p) {
     a.dil_h = v.dil_h;
     a.dil_w = v.dil_w;
     a.S = v.S;
+    if (p->emb.variant == B2C_VARIANT_DILATION_PACK) {
+      // the kernel's rows are the pixels of the phase sub-image convolutions
+      const int Pv = v.H + 2 * v.pad_h - v.R + 1, Qv = v.W + 2 * v.pad_w - v.S + 1;
+      a.Mg = (int)view_rows(p->g, p->emb.variant, v);
+      a.PQ = Pv * Qv;
+      a.Q = Qv;
+      a.P = Pv;
+      a.div_pq = make_fastdiv((uint32_t)a.PQ);
+      a.div_q = make_fastdiv((uint32_t)a.Q);
+      a.remap = 1;
+      a.ph_dh = d.dil_h;
+      a.ph_dw = d.dil_w;
+      a.ph_pad_h = v.pad_h;
+      a.ph_pad_w = v.pad_w;
+      a.out_pad_h = d.pad_h;
+      a.out_pad_w = d.pad_w;
+    }
   } else {
     p->amode = p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT
                    ? A_TILED
@@ -178,10 +198,10 @@ void fill_common_args(b2c_plan* p) {
   int per_cta_kb = (a.num_kb + a.split_k - 1) / a.split_k;
   int stages = std::min(6, std::max(1, per_cta_kb));
   const long long ctas = a.swap ? ((p->g.Mg + a.tile_n - 1) / a.tile_n) * ((d.K + kTileM - 1) / kTileM) * a.split_k
-                                : ((p->g.Mg + kTileM - 1) / kTileM) * ((d.K + a.tile_n - 1) / a.tile_n) * a.split_k;
+                                : (((long long)a.Mg + kTileM - 1) / kTileM) * ((d.K + a.tile_n - 1) / a.tile_n) * a.split_k;
   // Large TMA-fed problems run persistently: one block per SM walks the tile list with two
   // accumulator buffers in tensor memory and the deepest stage ring that fits.
-  const long long tiles_m = (p->g.Mg + kTileM - 1) / kTileM;
+  const long long tiles_m = ((long long)a.Mg + kTileM - 1) / kTileM;
   const int tiles_n = (d.K + a.tile_n - 1) / a.tile_n;
   a.tiles_n = tiles_n;
   a.num_tiles = (int)std::min<long long>(tiles_m * tiles_n, 0x7FFFFFFF);
@@ -231,7 +251,7 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
     if (!tma_view_for(g, emb.variant, &p->view)) return fail(B2C_E_UNSUPPORTED);
     const TmaView& v = p->view;
     p->w_packed_bytes = (size_t)d.K * v.R * v.S * v.C;
-    if (emb.variant != B2C_VARIANT_CP_TMA) {
+    if (emb.variant != B2C_VARIANT_CP_TMA && emb.variant != B2C_VARIANT_DILATION_PACK) {
       // Lookup tables of the rewritten maps.  Activations: scratch channel j of scratch pixel
       // (n, h', w') <- input element, in the form the stencil-unroll kernel takes.  Weights: packed
       // column (tap, j) <- index into one KCRS filter.
@@ -555,7 +575,7 @@ int b2c_plan_set_weights(b2c_plan* p, const int8_t* w, void* cuda_stream) {
   if (!aligned16(w)) return B2C_E_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const b2c_conv_desc& d = p->g.d;
-  if (p->emb.variant == B2C_VARIANT_CP_TMA)
+  if (p->emb.variant == B2C_VARIANT_CP_TMA || p->emb.variant == B2C_VARIANT_DILATION_PACK)
     CUDA_TRY(launch_pack_weights_cp(w, p->w_packed, d.K, d.C, d.R, d.S, p->C_pad, st));
   else if (is_tma_view_variant(p->emb.variant))
     CUDA_TRY(launch_pack_weights_table(w, p->w_packed, d.K, p->g.Kg, p->view.R * p->view.S * p->view.C, p->wtable, st));
@@ -593,6 +613,10 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
       int8_t* scratch = reinterpret_cast<int8_t*>(wsb);
       if (p->emb.variant == B2C_VARIANT_CP_TMA) {
         CUDA_TRY(launch_pack_activations(x, scratch, d.N, d.C, d.H, d.W, p->C_pad, st));
+      } else if (p->emb.variant == B2C_VARIANT_DILATION_PACK) {
+        const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
+        CUDA_TRY(launch_phase_split(x, scratch, d.N, d.C, d.H, d.W, d.dil_h, d.dil_w, v.H, v.W, v.C, a.x_stride_n,
+                                    nchw ? (long long)d.H * d.W : 1, a.x_stride_h, a.x_stride_w, st));
       } else if (p->emb.variant == B2C_VARIANT_ROW_UNROLL) {
         // scratch pixel (n, h, q): window origin (h, q*stride_w - pad_w), channels (s, c)
         CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W, 1,

@@ -103,6 +103,12 @@ struct ConvArgs {
   // swapped axis map: accumulator rows = output channels (the 128-row MMA operand is the packed
   // weights), accumulator columns = tile_n fused (n, p, q) pixels (the N operand is the activations)
   int swap;
+  // Output geometry.  out_PQ is the channel stride of the NKPQ tensor (always the convolution's own
+  // P*Q).  remap != 0 (dilation phase pack): accumulator row m' = (n', p', q') of the phase
+  // sub-image convolution belongs to image n = n' / (ph_dh*ph_dw), phase (a, b) = the remainder,
+  // output pixel p = (p' - ph_pad_h)*ph_dh + a + out_pad_h (q likewise), and is dropped when that
+  // pixel lies outside the out_P x out_Q output.
+  int out_PQ, remap, ph_dh, ph_dw, ph_pad_h, ph_pad_w, out_pad_h, out_pad_w, out_P, out_Q;
 };
 
 // Programmatic dependent launch: a kernel launched through launch_pdl may start while the previous
@@ -153,8 +159,13 @@ struct TmaView {
   long long bytes() const { return (long long)N * H * W * C; }
 };
 inline bool is_tma_view_variant(int v) {
-  return v == B2C_VARIANT_CP_TMA || v == B2C_VARIANT_ROW_UNROLL || v == B2C_VARIANT_SPACE_TO_DEPTH;
+  return v == B2C_VARIANT_CP_TMA || v == B2C_VARIANT_ROW_UNROLL || v == B2C_VARIANT_SPACE_TO_DEPTH ||
+         v == B2C_VARIANT_DILATION_PACK;
 }
+constexpr int kNumVariants = 7;
+// Output pixels of the convolution a view describes: the original N*P*Q, except for the dilation
+// phase pack, whose sub-image convolutions also produce rows that map outside the output.
+long long view_rows(const Geom& g, int variant, const TmaView& v);
 bool tma_view_for(const Geom& g, int variant, TmaView* v);  // false: the variant is not legal for g
 
 // --- planner.cpp -------------------------------------------------------------------------------
@@ -173,7 +184,8 @@ inline bool is_swapped(const b2c_embedding& e) { return e.map_m == B2C_AXIS_K; }
 // (The variants that keep a lookup table or an input window in shared memory leave room for a
 // 128-column exchange tile at most.)
 inline bool cluster_split_ok(int variant, int tile_n, int split_k, bool swap = false) {
-  if (swap) return false;  // the swapped map meets its partial sums in global memory
+  // the swapped map and the phase pack (scattered output rows) meet their partial sums in global memory
+  if (swap || variant == B2C_VARIANT_DILATION_PACK) return false;
   const bool table_in_smem = variant == B2C_VARIANT_IM2COL_GATHER || variant == B2C_VARIANT_IM2COL_STAGED;
   return (split_k == 2 || split_k == 4 || split_k == 8) && tile_n >= 32 * split_k && (!table_in_smem || tile_n <= 128);
 }
@@ -210,6 +222,9 @@ cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg
 cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, long long Mg, int PQ, int Q, int H,
                           int W, int stride_h, int stride_w, int pad_h, int pad_w, long long x_stride_n,
                           int x_stride_h, int x_stride_w, int K_pad, cudaStream_t st);
+cudaError_t launch_phase_split(const int8_t* x, int8_t* out, int N, int C, int H, int W, int dh, int dw, int Hs, int Ws,
+                               int C_pad, long long stride_n, long long stride_c, int stride_h, int stride_w,
+                               cudaStream_t st);
 cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, long long elems, int shift,
                                  int out_mode, cudaStream_t st);
 cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,

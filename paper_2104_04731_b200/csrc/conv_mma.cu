@@ -233,8 +233,8 @@ __device__ __forceinline__ void store_columns(const ConvArgs& args, const int32_
   if (args.split_k > 1 && !args.cluster_split) {
     // Partial sums of the reduction slices meet in global memory; integer addition is
     // associative, so the order of arrival does not change the result.
-    int32_t* dst = args.acc + (nhwc ? base_npqk + kbase : base_nkpq + (long long)kbase * args.PQ);
-    const long long step = nhwc ? 1 : args.PQ;
+    int32_t* dst = args.acc + (nhwc ? base_npqk + kbase : base_nkpq + (long long)kbase * args.out_PQ);
+    const long long step = nhwc ? 1 : args.out_PQ;
 #pragma unroll
     for (int j = 0; j < NC; ++j) {
       if (kbase + j < K) atomicAdd(dst, v[j]);
@@ -243,13 +243,13 @@ __device__ __forceinline__ void store_columns(const ConvArgs& args, const int32_
   } else if (!nhwc) {
     // NKPQ: for a fixed column the 32 lanes of a warp hold 32 consecutive pixels, so every
     // store instruction writes one contiguous run.
-    const long long o = base_nkpq + (long long)kbase * args.PQ;
+    const long long o = base_nkpq + (long long)kbase * args.out_PQ;
     if (args.out_mode & B2C_OUT_I32) {
       int32_t* dst = args.y32 + o;
 #pragma unroll
       for (int j = 0; j < NC; ++j) {
         if (kbase + j < K) *dst = v[j];
-        dst += args.PQ;
+        dst += args.out_PQ;
       }
     }
     if (args.out_mode & B2C_OUT_I8) {
@@ -257,7 +257,7 @@ __device__ __forceinline__ void store_columns(const ConvArgs& args, const int32_
 #pragma unroll
       for (int j = 0; j < NC; ++j) {
         if (kbase + j < K) *dst = requant(v[j], args.shift);
-        dst += args.PQ;
+        dst += args.out_PQ;
       }
     }
   } else {
@@ -620,11 +620,25 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     for (int t = tile_first; t < tile_end && ok; t += tile_step, ++ti) {
     B2C_TILE_ORIGIN(t)
     const unsigned m = (unsigned)m0 + (unsigned)row;
-    const bool row_valid = m < (unsigned)(args.swap ? args.K : args.Mg);
+    bool row_valid = m < (unsigned)(args.swap ? args.K : args.Mg);
     int n_img = 0, pq = 0;
     if (row_valid && !args.swap) {
       n_img = (int)args.div_pq.div(m);
       pq = (int)(m - (unsigned)n_img * (unsigned)args.PQ);
+    }
+    // Where this row's results go: (out_img, out_pq) in the convolution's own output.  The phase
+    // pack interleaves the sub-image results back and drops rows that fall outside the output.
+    int out_img = n_img, out_pq = pq;
+    if (args.remap && row_valid) {
+      const int ps = (int)args.div_q.div((uint32_t)pq), qs = pq - ps * args.Q;
+      const int phases = args.ph_dh * args.ph_dw;
+      out_img = n_img / phases;
+      const int ph = n_img - out_img * phases;
+      const int a = ph / args.ph_dw, b = ph - a * args.ph_dw;
+      const int po = (ps - args.ph_pad_h) * args.ph_dh + a + args.out_pad_h;
+      const int qo = (qs - args.ph_pad_w) * args.ph_dw + b + args.out_pad_w;
+      row_valid = (unsigned)po < (unsigned)args.out_P && (unsigned)qo < (unsigned)args.out_Q;
+      out_pq = po * args.out_Q + qo;
     }
 
     if (AMODE == A_GATHER) {
@@ -806,8 +820,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
       // Output index of (m, k): NKPQ -> (n*K + k)*PQ + pq ; NPQK -> m*K + k.
-      const long long base_nkpq = (long long)n_img * args.K * args.PQ + pq;
-      const long long base_npqk = (long long)m * args.K;
+      const long long base_nkpq = (long long)out_img * args.K * args.out_PQ + out_pq;
+      const long long base_npqk = args.remap ? ((long long)out_img * args.out_PQ + out_pq) * args.K : (long long)m * args.K;
       const int cols = args.tile_n >= 32 ? (args.tile_n >> 1) : 16;  // columns handled by this warp
       const int c_begin = half * cols;
       if (c_begin < args.tile_n) {

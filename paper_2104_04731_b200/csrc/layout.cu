@@ -293,6 +293,43 @@ __global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ 
   pdl_launch_dependents();
 }
 
+// Image Pack of a dilated convolution: sub-image (n, a, b) holds phase (a, b) of image n,
+// out[n'][hs][ws][c] = x[n][c][hs*dh + a][ws*dw + b] with n' = (n*dh + a)*dw + b, zeros past the
+// image and in the padded channels; NHWC with C_pad channels.  One thread writes 16 channels of one
+// sub-image pixel as a 16-byte vector.
+__global__ void __launch_bounds__(256) phase_split_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ out, int N,
+                                                          int C, int H, int W, int dh, int dw, int Hs, int Ws, int C_pad,
+                                                          long long stride_n, long long stride_c, int stride_h,
+                                                          int stride_w) {
+  const int chunks = C_pad >> 4;
+  const long long total = (long long)N * dh * dw * Hs * Ws * chunks;
+  pdl_wait();
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long pix = i / chunks;
+    const int ck = (int)(i - pix * chunks);
+    const int ws = (int)(pix % Ws);
+    const long long t = pix / Ws;
+    const int hs = (int)(t % Hs);
+    const long long nsub = t / Hs;
+    const int b = (int)(nsub % dw);
+    const int a = (int)((nsub / dw) % dh);
+    const long long n = nsub / ((long long)dw * dh);
+    const int h = hs * dh + a, w = ws * dw + b;
+    uint32_t wv[4] = {0, 0, 0, 0};
+    if (h < H && w < W) {
+      const int8_t* src = x + n * stride_n + (long long)h * stride_h + (long long)w * stride_w;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const int c = ck * 16 + e;
+        if (c < C) wv[e >> 2] |= (uint32_t)(uint8_t)src[c * stride_c] << (8 * (e & 3));
+      }
+    }
+    *reinterpret_cast<uint4*>(out + pix * C_pad + ck * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+  }
+  pdl_launch_dependents();
+}
+
 // Finish of a split reduction: the int32 sums are complete in `acc`; copy them out and/or apply
 // the shift-and-clip requantisation (arithmetic shift = floor division by 2^shift).
 __global__ void splitk_finish_kernel(const int32_t* __restrict__ acc, int32_t* __restrict__ y32,
@@ -375,6 +412,14 @@ cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, 
   const long long total = Mg * (K_pad / 16);
   return launch_pdl(im2col_kernel, dim3(grid_for(total, 256)), dim3(256), 0, st, x, a, table, Mg, PQ, Q, H, W, stride_h,
                     stride_w, pad_h, pad_w, x_stride_n, x_stride_h, x_stride_w, K_pad);
+}
+
+cudaError_t launch_phase_split(const int8_t* x, int8_t* out, int N, int C, int H, int W, int dh, int dw, int Hs, int Ws,
+                               int C_pad, long long stride_n, long long stride_c, int stride_h, int stride_w,
+                               cudaStream_t st) {
+  const long long total = (long long)N * dh * dw * Hs * Ws * (C_pad / 16);
+  return launch_pdl(phase_split_kernel, dim3(grid_for(total, 256)), dim3(256), 0, st, x, out, N, C, H, W, dh, dw, Hs, Ws,
+                    C_pad, stride_n, stride_c, stride_h, stride_w);
 }
 
 cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, long long elems, int shift,

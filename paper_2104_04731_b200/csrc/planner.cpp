@@ -119,10 +119,27 @@ bool tma_view_for(const Geom& g, int variant, TmaView* v) {
     if (d.dil_h != 1 || d.dil_w != 1 || (d.stride_h == 1 && d.stride_w == 1)) return false;
     const int Rp = (d.R + d.stride_h - 1) / d.stride_h, Sp = (d.S + d.stride_w - 1) / d.stride_w;
     *v = TmaView{d.N, round_up(d.C * d.stride_h * d.stride_w, kMmaK), g.P + Rp - 1, g.Q + Sp - 1, Rp, Sp, 1, 1, 0, 0, 1, 1};
+  } else if (variant == B2C_VARIANT_DILATION_PACK) {
+    // Image Pack of a dilated convolution (Section 6.1): with h - pad_h = i*dil_h + a every tap of an
+    // output pixel reads phase a of the image, X_a[j] = x[j*dil_h + a], at j = i + r.  The dil_h*dil_w
+    // phase sub-images (extent ceil(H / dil_h), zeros past the image) are fused into the batch and a
+    // dense, stride-1 R x S convolution with padding ceil(pad / dil) remains.
+    if ((d.dil_h == 1 && d.dil_w == 1) || d.stride_h != 1 || d.stride_w != 1) return false;
+    const long long n_sub = (long long)d.N * d.dil_h * d.dil_w;
+    if (n_sub > 0x7FFFFFFF) return false;
+    *v = TmaView{(int)n_sub, cp_channel_pad(d.C), (d.H + d.dil_h - 1) / d.dil_h, (d.W + d.dil_w - 1) / d.dil_w, d.R, d.S,
+                 1, 1, (d.pad_h + d.dil_h - 1) / d.dil_h, (d.pad_w + d.dil_w - 1) / d.dil_w, 1, 1};
+    const long long rows = (long long)v->N * (v->H + 2 * v->pad_h - v->R + 1) * (v->W + 2 * v->pad_w - v->S + 1);
+    if (rows > 0x7FFFFF00LL) return false;
   } else {
     return false;
   }
   return view_fits_tensor_map(*v);
+}
+
+long long view_rows(const Geom& g, int variant, const TmaView& v) {
+  if (variant != B2C_VARIANT_DILATION_PACK) return g.Mg;
+  return (long long)v.N * (v.H + 2 * v.pad_h - v.R + 1) * (v.W + 2 * v.pad_w - v.S + 1);
 }
 
 // The staged stencil unroll keeps, per image a tile can touch, the zero-padded input rows that
@@ -172,8 +189,10 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
   long long data_min = g.x_elems + g.w_elems + g.y_elems;
   TmaView v;
   if (is_tma_view_variant(variant) && tma_view_for(g, variant, &v)) {
-    e.map_k = variant == B2C_VARIANT_CP_TMA ? B2C_AXIS_C
-                                            : (variant == B2C_VARIANT_ROW_UNROLL ? B2C_AXIS_SC : B2C_AXIS_C_PHASES);
+    e.map_k = (variant == B2C_VARIANT_CP_TMA || variant == B2C_VARIANT_DILATION_PACK)
+                  ? B2C_AXIS_C
+                  : (variant == B2C_VARIANT_ROW_UNROLL ? B2C_AXIS_SC : B2C_AXIS_C_PHASES);
+    if (!swap) M_pad = (view_rows(g, variant, v) + kTileM - 1) / kTileM * kTileM;
     k_issued = (long long)v.R * v.S * v.C;
     long long packed = v.bytes();
     bool direct = variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && v.C == d.C;
@@ -205,10 +224,11 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
     tiles.push_back(t);
     if (t >= d.K) break;
   }
-  long long tiles_m = (g.Mg + kTileM - 1) / kTileM;
-  for (int variant = 0; variant < 6; ++variant) {
+  for (int variant = 0; variant < kNumVariants; ++variant) {
     TmaView view;
     if (is_tma_view_variant(variant) && !tma_view_for(g, variant, &view)) continue;
+    const long long tiles_m =
+        ((is_tma_view_variant(variant) ? view_rows(g, variant, view) : g.Mg) + kTileM - 1) / kTileM;
     WindowGeom wg;
     if (variant == B2C_VARIANT_IM2COL_STAGED && !staged_window(g, &wg)) continue;
     int num_kb;
@@ -235,7 +255,8 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
     // Swapped axis map (M <- k, N <- fused pixels) for the TMA-fed variants: the 128 accumulator rows
     // are output channels, so it is only listed when K fills at least half of them; the pixel tile
     // widths are those that waste less than a quarter of their columns (or the covering one).
-    if ((is_tma_view_variant(variant) || variant == B2C_VARIANT_IM2COL_EXPLICIT) && d.K >= kTileM / 2) {
+    if ((is_tma_view_variant(variant) || variant == B2C_VARIANT_IM2COL_EXPLICIT) && d.K >= kTileM / 2 &&
+        variant != B2C_VARIANT_DILATION_PACK) {
       const long long tiles_k = (d.K + kTileM - 1) / kTileM;
       for (int t = 32; t <= 256; t <<= 1) {
         const long long n_pad = (g.Mg + t - 1) / t * t;

@@ -69,7 +69,7 @@ def test_config_every_embedding(lib, cfg):
 @pytest.mark.parametrize("in_layout,out_layout", [(1, 1), (0, 1), (1, 0)])
 def test_config_layouts(lib, cfg, in_layout, out_layout):
     x, w, ref = cfg_reference(cfg)
-    for variant in (0, 1, 2, 3, 4, 5):
+    for variant in (0, 1, 2, 3, 4, 5, 6):
         d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
                           in_layout, out_layout, 3)
         ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant]
@@ -105,7 +105,7 @@ def test_random_shapes(lib, case):
     ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
     d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode=3)
     embs = lib.enumerate_embeddings(d)
-    for variant in (0, 1, 2, 3, 4, 5):
+    for variant in (0, 1, 2, 3, 4, 5, 6):
         ids = [e.id for e in embs if e.variant == variant]
         for i in ids[:1] + ids[-1:]:
             check_against_oracle(x, w, stride, pad, dil, shift, 3, i, ref=ref)
@@ -147,12 +147,44 @@ def test_swapped_axis_map(lib, case, out_layout):
         check_against_oracle(x, w, stride, pad, dil, shift, 2, split[0].id, ref=ref, out_layout=out_layout)
 
 
+# ---- dilation phase pack (Image Pack of a dilated conv: phases fused into the batch) ---------------------
+@pytest.mark.parametrize("case", [
+    # N, C, H, W, K, R, S, pad, dil, shift
+    (1, 16, 20, 20, 24, 3, 3, 2, 2, 8),             # "same" dilated 3x3, even image
+    (2, 3, 17, 23, 16, 3, 3, (4, 4), (4, 4), 6),    # dilation 4, odd image: phase sub-images of unequal size
+    (2, 5, 19, 14, 40, 3, 2, (1, 0), (2, 3), 7),    # pad not a multiple of the dilation; mixed dilation
+    (1, 32, 13, 13, 8, 2, 4, (0, 5), (3, 1), 5),    # only the vertical axis dilated, wide horizontal padding
+    (3, 64, 9, 31, 130, 3, 3, (3, 1), (3, 2), 9),   # several column tiles, ragged rows
+])
+@pytest.mark.parametrize("layouts", [(0, 0), (1, 1)])
+def test_dilation_phase_pack(lib, case, layouts):
+    N, C, H, W, K, R, S, pad, dil, shift = case
+    in_layout, out_layout = layouts
+    x = int8_uniform((N, C, H, W), 621)
+    w = int8_uniform((K, C, R, S), 622)
+    ref = oracle.conv2d_int8(x, w, 1, pad, dil, shift)
+    d = lib.make_desc(N, C, H, W, K, R, S, 1, pad, dil, shift, in_layout, out_layout, 3)
+    packs = [e for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_DILATION_PACK]
+    assert packs and all(e.map_k == b2c.AXIS_C and e.workspace_bytes > 0 for e in packs)
+    seen = set()
+    for e in packs:
+        key = (e.tile_n, min(e.split_k, 2))
+        if key in seen:
+            continue
+        seen.add(key)
+        check_against_oracle(x, w, 1, pad, dil, shift, 3, e.id, ref=ref, in_layout=in_layout, out_layout=out_layout)
+    # not listed without dilation or with a stride
+    for (st, dl) in [(1, 1), (2, 2)]:
+        d2 = lib.make_desc(N, C, H + 8, W + 8, K, R, S, st, pad, dl, shift)
+        assert all(e.variant != b2c.VARIANT_DILATION_PACK for e in lib.enumerate_embeddings(d2))
+
+
 def test_extreme_values_and_shift_clip(lib):
     # -128 * -128 is the largest product; all-(-128) tensors with 9*64 taps reach 9437184.
     x = np.full((1, 64, 6, 6), -128, dtype=np.int8)
     w = np.full((16, 64, 3, 3), -128, dtype=np.int8)
     ref = oracle.conv2d_int8(x, w, 1, 1, 1, 16)
-    for variant in (0, 1, 2, 3, 4, 5):
+    for variant in (0, 1, 2, 3, 4, 5, 6):
         d = lib.make_desc(1, 64, 6, 6, 16, 3, 3, 1, 1, 1, 16, out_mode=3)
         ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant]
         if ids:

@@ -243,3 +243,19 @@ def test_config_samples_against_python(cfg):
                     acc += int(np.dot(xi[n, :, h, ww], wi[k, :, r, s]))
         assert int(y32[n, k, p, q]) == acc
         assert int(y8[n, k, p, q]) == max(-128, min(127, acc >> cfg.shift))  # Python >> on int is floor
+
+
+@pytest.mark.parametrize("geom", [((2, 2), (2, 2)), ((4, 4), (4, 4)), ((2, 3), (1, 0)), ((3, 1), (0, 5))])
+def test_dilated_conv_is_blown_up_stencil(geom):
+    """Section 6.1 describes the reference for a dilated convolution as the same stencil "blown up
+    with zeros": an undilated convolution whose kernel has the taps at (r*dil_h, s*dil_w) and zeros
+    in between.  Pins the oracle's dilation handling against its own undilated path."""
+    dil, pad = geom
+    x = int8_uniform((2, 3, 15, 17), 71)
+    w = int8_uniform((4, 3, 3, 2), 72)
+    R, S = w.shape[2:]
+    big = np.zeros((4, 3, dil[0] * (R - 1) + 1, dil[1] * (S - 1) + 1), dtype=np.int8)
+    big[:, :, ::dil[0], ::dil[1]] = w
+    got, _ = oracle.conv2d_int8(x, w, 1, pad, dil, 0)
+    want, _ = oracle.conv2d_int8(x, big, 1, pad, 1, 0)
+    assert got.shape == want.shape and np.array_equal(got, want)
