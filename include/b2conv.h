@@ -141,6 +141,23 @@ int b2c_plan_set_weights(b2c_plan* plan, const int8_t* w_kcrs_dev, void* cuda_st
 int b2c_conv2d_int8_run(b2c_plan* plan, const int8_t* x_dev, int32_t* y_i32_dev, int8_t* y_i8_dev,
                         void* workspace_dev, void* cuda_stream);
 
+/* The two halves of b2c_conv2d_int8_run on their own, matching the "Transf." and "Op." columns of
+ * Tables 3 to 5: b2c_plan_rewrite_activations enqueues only the layout rewrite of x into the start
+ * of workspace_dev (nothing is enqueued for embeddings without a rewrite), and
+ * b2c_conv2d_int8_run_rewritten enqueues only the MMA kernel, epilogue and split finish on a
+ * workspace an earlier b2c_plan_rewrite_activations (or b2c_conv2d_int8_run) of the same plan filled,
+ * e.g. to convolve one rewritten input again after b2c_plan_set_weights.  x_dev may be NULL in
+ * run_rewritten when the plan has a rewrite; embeddings without one read x_dev there.  Same
+ * argument rules, stream semantics and error codes as b2c_conv2d_int8_run. */
+int b2c_plan_rewrite_activations(b2c_plan* plan, const int8_t* x_dev, void* workspace_dev, void* cuda_stream);
+int b2c_conv2d_int8_run_rewritten(b2c_plan* plan, const int8_t* x_dev, int32_t* y_i32_dev, int8_t* y_i8_dev,
+                                  void* workspace_dev, void* cuda_stream);
+
+/* Memory footprint of the chosen embedding (the "Memory" columns of Tables 3 to 5): bytes of the
+ * rewritten activation operand in the workspace (0 without a rewrite) and of the plan's packed
+ * weights.  Host only. */
+int b2c_plan_footprint(const b2c_plan* plan, size_t* rewritten_bytes, size_t* packed_weight_bytes);
+
 /* One-shot form of the paper's problem statement: NCHW int8 input, KCRS int8 weights, NKPQ
  * outputs (either may be NULL, not both), symmetric stride / pad / dilation.  All four tensor
  * pointers are DEVICE pointers.  Keeps plans and scratch in a library-owned cache keyed by

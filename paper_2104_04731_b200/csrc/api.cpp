@@ -586,15 +586,43 @@ int b2c_plan_set_weights(b2c_plan* p, const int8_t* w, void* cuda_stream) {
   return B2C_OK;
 }
 
-int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, void* cuda_stream) {
-  if (!p || !x) return B2C_E_INVALID_ARG;
-  if (!p->weights_set) return B2C_E_NOT_READY;
+// The two halves of the path.  run_rewrite is the layout rewrite of the activations (the paper's
+// "Transf." column): it fills the start of the workspace.  run_convolve is the MMA kernel with its
+// epilogue and the split-reduction finish (the "Op." column): it reads the rewritten operand from
+// the workspace (or x itself when the embedding has no rewrite).
+static int run_rewrite(b2c_plan* p, const int8_t* x, void* ws, cudaStream_t st) {
   const b2c_conv_desc& d = p->g.d;
-  if ((d.out_mode & B2C_OUT_I32) && !y32) return B2C_E_INVALID_ARG;
-  if ((d.out_mode & B2C_OUT_I8) && !y8) return B2C_E_INVALID_ARG;
-  if (p->ws_total > 0 && !ws) return B2C_E_INVALID_ARG;
-  if (!aligned16(x) || !aligned16(y32) || !aligned16(y8) || !aligned16(ws)) return B2C_E_INVALID_ARG;
-  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const Geom& g = p->g;
+  const ConvArgs& a = p->args;
+  if (!p->ws_layout_bytes) return B2C_OK;
+  int8_t* scratch = static_cast<int8_t*>(ws);
+  if (is_tma_view_variant(p->emb.variant)) {
+    const TmaView& v = p->view;
+    if (p->emb.variant == B2C_VARIANT_CP_TMA) {
+      CUDA_TRY(launch_pack_activations(x, scratch, d.N, d.C, d.H, d.W, p->C_pad, st));
+    } else if (p->emb.variant == B2C_VARIANT_DILATION_PACK) {
+      const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
+      CUDA_TRY(launch_phase_split(x, scratch, d.N, d.C, d.H, d.W, d.dil_h, d.dil_w, v.H, v.W, v.C, a.x_stride_n,
+                                  nchw ? (long long)d.H * d.W : 1, a.x_stride_h, a.x_stride_w, st));
+    } else if (p->emb.variant == B2C_VARIANT_ROW_UNROLL) {
+      // scratch pixel (n, h, q): window origin (h, q*stride_w - pad_w), channels (s, c)
+      CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W, 1,
+                             d.stride_w, 0, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w, v.C, st));
+    } else {
+      // scratch pixel (n, h', w'): window origin (h'*stride_h - pad_h, w'*stride_w - pad_w), channels (c, dh, dw)
+      CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W,
+                             d.stride_h, d.stride_w, d.pad_h, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w,
+                             v.C, st));
+    }
+  } else if (p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
+    CUDA_TRY(launch_im2col(x, scratch, p->table, g.Mg, g.PQ, g.Q, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
+                           a.x_stride_n, a.x_stride_h, a.x_stride_w, p->K_pad, st));
+  }
+  return B2C_OK;
+}
+
+static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, cudaStream_t st) {
+  const b2c_conv_desc& d = p->g.d;
   const Geom& g = p->g;
   ConvArgs a = p->args;
   a.x = x;
@@ -604,39 +632,14 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   std::memset(&tmap_a, 0, sizeof(tmap_a));
   uint8_t* wsb = static_cast<uint8_t*>(ws);
   int rc = B2C_OK;
-
-  // ---- layout rewrite of the activations ----
   if (is_tma_view_variant(p->emb.variant)) {
     const TmaView& v = p->view;
-    const int8_t* act = x;
-    if (p->ws_layout_bytes) {
-      int8_t* scratch = reinterpret_cast<int8_t*>(wsb);
-      if (p->emb.variant == B2C_VARIANT_CP_TMA) {
-        CUDA_TRY(launch_pack_activations(x, scratch, d.N, d.C, d.H, d.W, p->C_pad, st));
-      } else if (p->emb.variant == B2C_VARIANT_DILATION_PACK) {
-        const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
-        CUDA_TRY(launch_phase_split(x, scratch, d.N, d.C, d.H, d.W, d.dil_h, d.dil_w, v.H, v.W, v.C, a.x_stride_n,
-                                    nchw ? (long long)d.H * d.W : 1, a.x_stride_h, a.x_stride_w, st));
-      } else if (p->emb.variant == B2C_VARIANT_ROW_UNROLL) {
-        // scratch pixel (n, h, q): window origin (h, q*stride_w - pad_w), channels (s, c)
-        CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W, 1,
-                               d.stride_w, 0, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w, v.C, st));
-      } else {
-        // scratch pixel (n, h', w'): window origin (h'*stride_h - pad_h, w'*stride_w - pad_w), channels (c, dh, dw)
-        CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W,
-                               d.stride_h, d.stride_w, d.pad_h, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w,
-                               v.C, st));
-      }
-      act = scratch;
-    }
+    const int8_t* act = p->ws_layout_bytes ? reinterpret_cast<const int8_t*>(wsb) : x;
     rc = encode_im2col_nhwc(&tmap_a, act, v.C, v.W, v.H, v.N, v.pad_w, v.pad_h, v.S, v.R, v.dil_w, v.dil_h,
                             v.stride_w, v.stride_h, p->bk, a.swap ? a.tile_n : kTileM, p->bk);
     if (rc != B2C_OK) return rc;
   } else if (p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
-    int8_t* A = reinterpret_cast<int8_t*>(wsb);
-    CUDA_TRY(launch_im2col(x, A, p->table, g.Mg, g.PQ, g.Q, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
-                           a.x_stride_n, a.x_stride_h, a.x_stride_w, p->K_pad, st));
-    rc = encode_tiled_2d(&tmap_a, A, p->K_pad, (uint64_t)g.Mg, p->K_pad, 128, a.swap ? a.tile_n : kTileM, 128);
+    rc = encode_tiled_2d(&tmap_a, wsb, p->K_pad, (uint64_t)g.Mg, p->K_pad, 128, a.swap ? a.tile_n : kTileM, 128);
     if (rc != B2C_OK) return rc;
   } else {
     tmap_a = p->tmap_b;  // unused by the gather kernel; any valid map
@@ -656,6 +659,46 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
 
   CUDA_TRY(launch_conv_mma(p->amode, &tmap_a, &p->tmap_b, a, st));
   if (need_finish) CUDA_TRY(launch_splitk_finish(a.acc, y32, y8, g.y_elems, d.shift, d.out_mode, st));
+  return B2C_OK;
+}
+
+static int check_run_args(b2c_plan* p, const int8_t* x, bool need_x, int32_t* y32, int8_t* y8, bool need_y, void* ws) {
+  if (!p || (need_x && !x)) return B2C_E_INVALID_ARG;
+  const b2c_conv_desc& d = p->g.d;
+  if (need_y && !p->weights_set) return B2C_E_NOT_READY;
+  if (need_y && (d.out_mode & B2C_OUT_I32) && !y32) return B2C_E_INVALID_ARG;
+  if (need_y && (d.out_mode & B2C_OUT_I8) && !y8) return B2C_E_INVALID_ARG;
+  if (p->ws_total > 0 && !ws) return B2C_E_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(y32) || !aligned16(y8) || !aligned16(ws)) return B2C_E_INVALID_ARG;
+  return B2C_OK;
+}
+
+int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, void* cuda_stream) {
+  int rc = check_run_args(p, x, true, y32, y8, true, ws);
+  if (rc != B2C_OK) return rc;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  rc = run_rewrite(p, x, ws, st);
+  if (rc != B2C_OK) return rc;
+  return run_convolve(p, x, y32, y8, ws, st);
+}
+
+int b2c_plan_rewrite_activations(b2c_plan* p, const int8_t* x, void* ws, void* cuda_stream) {
+  int rc = check_run_args(p, x, true, nullptr, nullptr, false, ws);
+  if (rc != B2C_OK) return rc;
+  return run_rewrite(p, x, ws, (cudaStream_t)cuda_stream);
+}
+
+int b2c_conv2d_int8_run_rewritten(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, void* cuda_stream) {
+  // x is still needed by the embeddings that have no rewrite (they read the input directly)
+  int rc = check_run_args(p, x, p && p->ws_layout_bytes == 0, y32, y8, true, ws);
+  if (rc != B2C_OK) return rc;
+  return run_convolve(p, x, y32, y8, ws, (cudaStream_t)cuda_stream);
+}
+
+int b2c_plan_footprint(const b2c_plan* p, size_t* rewritten_bytes, size_t* packed_weight_bytes) {
+  if (!p || !rewritten_bytes || !packed_weight_bytes) return B2C_E_INVALID_ARG;
+  *rewritten_bytes = p->ws_layout_bytes;
+  *packed_weight_bytes = p->w_packed_bytes;
   return B2C_OK;
 }
 

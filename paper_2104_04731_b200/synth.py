@@ -84,3 +84,14 @@ CONFIGS = [
     ConvShape("cfg4_c1_96x480_k32_9x21s2", 2, 1, 96, 480, 32, 9, 21, 2, 0, 1, 0, 1),
     ConvShape("cfg5_n32_c256_14x14_k512_3x3s2", 32, 256, 14, 14, 512, 3, 3, 2, 1, 1, 10, 2),
 ]
+
+# Extra shapes for the candidate report: the shape classes of the paper's dilated rows (Table 3:
+# dilation 2 and 4) and of its batch-1 rows on the 8x8x8 intrinsic (Table 5: data (1, C, H, W),
+# weights (K, C, R, S), pad, stride), int32 output.
+REPORT_EXTRA = [
+    ConvShape("dil2_c16_64x64_k32_3x3", 1, 16, 64, 64, 32, 3, 3, 1, 2, 2, 0, 1),
+    ConvShape("dil4_c3_96x96_k16_3x3", 1, 3, 96, 96, 16, 3, 3, 1, 4, 4, 0, 1),
+    ConvShape("t5_c32_16x16_k64_3x3", 1, 32, 16, 16, 64, 3, 3, 1, 1, 1, 0, 1),
+    ConvShape("t5_c72_56x56_k96_1x1", 1, 72, 56, 56, 96, 1, 1, 1, 0, 1, 0, 1),
+    ConvShape("t5_c8_224x224_k24_3x3s2", 1, 8, 224, 224, 24, 3, 3, 2, 1, 1, 0, 1),
+]

@@ -179,6 +179,36 @@ def test_dilation_phase_pack(lib, case, layouts):
         assert all(e.variant != b2c.VARIANT_DILATION_PACK for e in lib.enumerate_embeddings(d2))
 
 
+def test_rewrite_and_convolve_halves(lib):
+    # b2c_plan_rewrite_activations + b2c_conv2d_int8_run_rewritten = b2c_conv2d_int8_run, for every variant
+    cfg = CONFIGS[0]
+    x, w, ref = cfg_reference(cfg)
+    x2 = int8_uniform(x.shape, 631)
+    d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
+                      out_mode=3)
+    seen = set()
+    for e in lib.enumerate_embeddings(d):
+        if e.variant in seen:
+            continue
+        seen.add(e.variant)
+        plan = lib.Plan(d, e.id)
+        data_b, weight_b = plan.footprint()
+        assert weight_b >= w.size and (data_b > 0) == (e.variant in (0, 1, 4, 5))
+        assert data_b <= plan.workspace_bytes()
+        ws = torch.zeros(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
+        y32 = torch.zeros(ref[0].shape, dtype=torch.int32, device="cuda")
+        y8 = torch.zeros(ref[1].shape, dtype=torch.int8, device="cuda")
+        plan.set_weights(to_dev(w))
+        plan.rewrite_activations(to_dev(x), ws)
+        # a different tensor as x: variants with a rewrite must read the workspace, not x
+        xin = to_dev(x2) if data_b else to_dev(x)
+        plan.run_rewritten(xin, y32, y8, ws)
+        torch.cuda.synchronize()
+        assert plan.device_status() == b2c.OK
+        assert np.array_equal(y32.cpu().numpy(), ref[0]) and np.array_equal(y8.cpu().numpy(), ref[1]), e.variant
+        plan.destroy()
+
+
 def test_extreme_values_and_shift_clip(lib):
     # -128 * -128 is the largest product; all-(-128) tensors with 9*64 taps reach 9437184.
     x = np.full((1, 64, 6, 6), -128, dtype=np.int8)
