@@ -41,6 +41,8 @@ def _load():
         lib.oracle_requant.restype = ctypes.c_int8
         lib.oracle_conv2d_int8.argtypes = [vp, vp] + [i32] * 14 + [vp, vp, i32]
         lib.oracle_conv2d_int8.restype = i32
+        lib.oracle_conv2d_int8_act.argtypes = [vp, vp, vp, i32] + [i32] * 14 + [vp, vp, i32]
+        lib.oracle_conv2d_int8_act.restype = i32
         lib.oracle_im2col.argtypes = [vp] + [i32] * 12 + [vp]
         lib.oracle_im2col.restype = None
         lib.oracle_gemm_abt.argtypes = [vp, vp, i64, i64, i64, vp]
@@ -76,10 +78,12 @@ def requant(acc: int, shift: int) -> int:
     return int(_load().oracle_requant(int(acc), int(shift)))
 
 
-def conv2d_int8(x, w, stride=1, pad=0, dilation=1, shift=0, want_i32=True, want_i8=True, threads=0):
+def conv2d_int8(x, w, stride=1, pad=0, dilation=1, shift=0, want_i32=True, want_i8=True, threads=0, bias=None,
+                relu=False):
     """x: int8 [N,C,H,W]; w: int8 [K,C,R,S] -> (y32 int32 [N,K,P,Q] or None, y8 int8 or None).
 
-    Raises OverflowError when an accumulator leaves the int32 range.
+    Optional activation step before the outputs are written: per-output-channel int32 `bias` [K]
+    added to the exact sum, then ReLU.  Raises OverflowError when a value leaves the int32 range.
     """
     x = np.ascontiguousarray(x, dtype=np.int8)
     w = np.ascontiguousarray(w, dtype=np.int8)
@@ -92,8 +96,12 @@ def conv2d_int8(x, w, stride=1, pad=0, dilation=1, shift=0, want_i32=True, want_
     P, Q = out_shape(H, W, R, S, (sh, sw), (ph, pw), (dh, dw))
     y32 = np.empty((N, K, P, Q), dtype=np.int32) if want_i32 else None
     y8 = np.empty((N, K, P, Q), dtype=np.int8) if want_i8 else None
-    rc = _load().oracle_conv2d_int8(
-        _ptr(x), _ptr(w), N, C, H, W, K, R, S, sh, sw, ph, pw, dh, dw, int(shift), _ptr(y32), _ptr(y8), int(threads)
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.int32)
+        assert bias.shape == (K,)
+    rc = _load().oracle_conv2d_int8_act(
+        _ptr(x), _ptr(w), _ptr(bias), int(bool(relu)), N, C, H, W, K, R, S, sh, sw, ph, pw, dh, dw, int(shift),
+        _ptr(y32), _ptr(y8), int(threads)
     )
     if rc != 0:
         raise OverflowError("an accumulator left the int32 range")

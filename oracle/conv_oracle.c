@@ -53,17 +53,26 @@ int8_t oracle_requant(int64_t acc, int shift) {
 }
 
 /*
- * The definition (Figure 5 step 1; Table 2 access [n, i + k]):
+ * The definition (Figure 5 step 1; Table 2 access [n, i + k]), followed by the vector unit's
+ * "activation and quantization operations" (Section 5.1; the micro-benchmark of Section 5.2 runs
+ * pack -> conv -> activation -> unpack).  The paper does not say which activation; the reading
+ * taken here is an optional per-output-channel int32 bias and an optional ReLU, both applied to
+ * the exact sum before the outputs are written:
+ *   t = acc + bias[k]   (bias == NULL: t = acc);   relu != 0: t = max(t, 0);
+ *   y32 = t;   y8 = clip(floor(t / 2^shift)).
+ * t outside the int32 range is reported like an accumulator overflow.
+ *
+ * The convolution itself:
  *   y[n][k][p][q] = sum_{c,r,s} x[n][c][p*stride_h - pad_h + r*dil_h][q*stride_w - pad_w + s*dil_w]
  *                               * w[k][c][r][s]        (terms outside the image are zero)
  * x is NCHW, w is KCRS, y32/y8 are NKPQ; either output pointer may be NULL.
  * Returns 0, or 1 if some accumulator left the int32 range (outputs then undefined there).
  * `threads` > 0 sets the OpenMP team size used over the (n, k) loops; <= 0 keeps the default.
  */
-int oracle_conv2d_int8(const int8_t* x, const int8_t* w,
-                       int N, int C, int H, int W, int K, int R, int S,
-                       int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
-                       int shift, int32_t* y32, int8_t* y8, int threads) {
+int oracle_conv2d_int8_act(const int8_t* x, const int8_t* w, const int32_t* bias, int relu,
+                           int N, int C, int H, int W, int K, int R, int S,
+                           int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                           int shift, int32_t* y32, int8_t* y8, int threads) {
   const int P = oracle_out_extent(H, R, stride_h, pad_h, dil_h);
   const int Q = oracle_out_extent(W, S, stride_w, pad_w, dil_w);
   int overflow = 0;
@@ -92,6 +101,9 @@ int oracle_conv2d_int8(const int8_t* x, const int8_t* w,
             }
           }
           if (acc > INT32_MAX || acc < INT32_MIN) overflow |= 1;
+          if (bias) acc += (int64_t)bias[k];
+          if (relu && acc < 0) acc = 0;
+          if (acc > INT32_MAX || acc < INT32_MIN) overflow |= 1;
           size_t o = (((size_t)n * K + k) * P + p) * Q + q;
           if (y32) y32[o] = (int32_t)acc;
           if (y8) y8[o] = oracle_requant(acc, shift);
@@ -100,6 +112,15 @@ int oracle_conv2d_int8(const int8_t* x, const int8_t* w,
     }
   }
   return overflow;
+}
+
+/* The convolution with the plain quantisation step only (no bias, no ReLU). */
+int oracle_conv2d_int8(const int8_t* x, const int8_t* w,
+                       int N, int C, int H, int W, int K, int R, int S,
+                       int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                       int shift, int32_t* y32, int8_t* y8, int threads) {
+  return oracle_conv2d_int8_act(x, w, NULL, 0, N, C, H, W, K, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                                shift, y32, y8, threads);
 }
 
 /*

@@ -259,3 +259,32 @@ def test_dilated_conv_is_blown_up_stencil(geom):
     got, _ = oracle.conv2d_int8(x, w, 1, pad, dil, 0)
     want, _ = oracle.conv2d_int8(x, big, 1, pad, 1, 0)
     assert got.shape == want.shape and np.array_equal(got, want)
+
+
+def test_bias_and_relu_step():
+    """Activation step (Section 5.1's vector unit; reading: per-channel int32 bias, then ReLU):
+    pinned against numpy arithmetic on the plain convolution's int32 output, Python floor shift."""
+    x = int8_uniform((2, 5, 9, 8), 81)
+    w = int8_uniform((6, 5, 3, 3), 82)
+    bias = np.array([0, 1, -1, 70000, -70000, 2 ** 20], dtype=np.int32)
+    plain, _ = oracle.conv2d_int8(x, w, 1, 1, 1, 0)
+    for relu in (False, True):
+        for shift in (0, 4, 9):
+            y32, y8 = oracle.conv2d_int8(x, w, 1, 1, 1, shift, bias=bias, relu=relu)
+            t = plain.astype(np.int64) + bias.astype(np.int64)[None, :, None, None]
+            if relu:
+                t = np.maximum(t, 0)
+            assert np.array_equal(y32, t)
+            want8 = np.array([max(-128, min(127, int(v) >> shift)) for v in t.ravel()], dtype=np.int64).reshape(t.shape)
+            assert np.array_equal(y8, want8)
+            if relu:
+                assert y32.min() == 0 and (plain + bias[None, :, None, None] < 0).any() and y8.min() >= 0
+    # no bias, no ReLU is the plain convolution; a zero bias changes nothing
+    a = oracle.conv2d_int8(x, w, 2, 0, 1, 3, bias=np.zeros(6, dtype=np.int32))
+    b = oracle.conv2d_int8(x, w, 2, 0, 1, 3)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    # a bias that pushes a value past int32 is an error, not a wrap
+    big = np.full(6, 2 ** 31 - 1, dtype=np.int32)
+    xp, wp = np.full((1, 5, 3, 3), 127, dtype=np.int8), np.full((6, 5, 3, 3), 127, dtype=np.int8)
+    with pytest.raises(OverflowError):
+        oracle.conv2d_int8(xp, wp, 1, 0, 1, 0, bias=big)
