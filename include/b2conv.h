@@ -131,6 +131,18 @@ int b2c_plan_workspace_bytes(const b2c_plan* plan, size_t* bytes);
  * asynchronously on `cuda_stream`.  Call once per weight tensor, before run. */
 int b2c_plan_set_weights(b2c_plan* plan, const int8_t* w_kcrs_dev, void* cuda_stream);
 
+/* Activation step between accumulation and output (Section 5.1: the vector unit after the GEMM core
+ * performs "activation and quantization"; the paper does not name the activation, the reading here
+ * is bias + ReLU).  With a plan so configured every complete sum becomes
+ *   t = acc + bias[k]  (bias_dev != NULL),  then  t = max(t, 0)  (relu == 1),
+ * the int32 output is t and the int8 output clip(floor(t / 2^shift)).  bias_dev: K int32 values in
+ * device memory (4-byte aligned), copied into the plan asynchronously on `cuda_stream`; NULL removes
+ * the bias.  relu: 0 or 1.  The caller keeps acc + bias inside int32 (|acc| <= C*R*S*2^14); the
+ * addition wraps otherwise.  Applies to later b2c_conv2d_int8_run / run_rewritten calls of this
+ * plan; a new plan has no bias and no ReLU.  INVALID_ARG on a null plan, misaligned bias or relu
+ * outside {0, 1}; B2C_E_CUDA if the copy or its buffer fails. */
+int b2c_plan_set_activation(b2c_plan* plan, const int32_t* bias_dev, int relu, void* cuda_stream);
+
 /* Enqueues the whole path on `cuda_stream` and returns without waiting: activation layout
  * rewrite (if the embedding has one), the MMA kernel with fused shift/clip epilogue, stores in
  * desc.out_layout.  x_dev: int8 input in desc.in_layout.  y_i32_dev / y_i8_dev: outputs

@@ -27,7 +27,7 @@ VARIANT_NAMES = {0: "channel_pack_tma_im2col", 1: "im2col_explicit", 2: "im2col_
 EXPORTS = [
     "b2c_out_shape", "b2c_enumerate", "b2c_plan_create", "b2c_plan_info", "b2c_plan_workspace_bytes",
     "b2c_plan_set_weights", "b2c_conv2d_int8_run", "b2c_conv2d_int8", "b2c_conv2d_int8_host",
-    "b2c_plan_rewrite_activations", "b2c_conv2d_int8_run_rewritten", "b2c_plan_footprint",
+    "b2c_plan_rewrite_activations", "b2c_conv2d_int8_run_rewritten", "b2c_plan_footprint", "b2c_plan_set_activation",
     "b2c_plan_device_status", "b2c_selftest_bounded_wait", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
     "b2c_status_string",
     "b2c_last_cuda_error",
@@ -86,6 +86,7 @@ def load():
     lib.b2c_conv2d_int8_run.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.b2c_plan_rewrite_activations.argtypes = [vp, vp, vp, vp]
     lib.b2c_conv2d_int8_run_rewritten.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.b2c_plan_set_activation.argtypes = [vp, vp, i32, vp]
     lib.b2c_plan_footprint.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
     lib.b2c_conv2d_int8.argtypes = [i32] * 11 + [vp] * 5
     lib.b2c_conv2d_int8_host.argtypes = [i32] * 11 + [vp] * 4
@@ -183,6 +184,11 @@ class Plan:
     def run(self, x, y32=None, y8=None, workspace=None, stream=None):
         _check(self._lib.b2c_conv2d_int8_run(self._h, _dptr(x), _dptr(y32), _dptr(y8), _dptr(workspace),
                                               _stream_ptr(stream)), "b2c_conv2d_int8_run")
+
+    def set_activation(self, bias=None, relu=False, stream=None):
+        """Activation step before the outputs are written: int32 CUDA tensor `bias` [K] (or None), ReLU flag."""
+        _check(self._lib.b2c_plan_set_activation(self._h, _dptr(bias), int(bool(relu)), _stream_ptr(stream)),
+               "b2c_plan_set_activation")
 
     def rewrite_activations(self, x, workspace=None, stream=None):
         """Only the layout rewrite of x into the workspace (the "Transf." half of run)."""

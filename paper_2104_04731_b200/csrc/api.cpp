@@ -26,6 +26,9 @@ struct b2c_plan {
   int32_t* wtable = nullptr;     // device, plan-owned: packed weight column -> index into one filter, -1 = zero
   int table_len = 0;
   int* status = nullptr;         // device status word
+  int32_t* bias_buf = nullptr;   // device, plan-owned copy of the per-channel bias (activation step)
+  int32_t* bias = nullptr;       // bias_buf while a bias is set, else null
+  int relu = 0;
   bool weights_set = false;
   // derived launch parameters
   int amode = 0;
@@ -628,6 +631,9 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   a.x = x;
   a.y32 = y32;
   a.y8 = y8;
+  a.bias = p->bias;
+  a.relu = p->relu;
+  const bool act = p->bias != nullptr || p->relu != 0;
   CUtensorMap tmap_a;
   std::memset(&tmap_a, 0, sizeof(tmap_a));
   uint8_t* wsb = static_cast<uint8_t*>(ws);
@@ -649,7 +655,8 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   bool need_finish = false;
   if (a.split_k > 1 && !a.cluster_split) {
     if (d.out_mode == B2C_OUT_I32) {
-      a.acc = y32;
+      a.acc = y32;           // the partial sums meet in the output itself ...
+      need_finish = act;     // ... and the activation step, if any, is applied to it in place afterwards
     } else {
       a.acc = reinterpret_cast<int32_t*>(wsb + p->ws_layout_bytes);
       need_finish = true;
@@ -658,7 +665,9 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   }
 
   CUDA_TRY(launch_conv_mma(p->amode, &tmap_a, &p->tmap_b, a, st));
-  if (need_finish) CUDA_TRY(launch_splitk_finish(a.acc, y32, y8, g.y_elems, d.shift, d.out_mode, st));
+  if (need_finish)
+    CUDA_TRY(launch_splitk_finish(a.acc, y32, y8, g.y_elems, d.shift, d.out_mode, p->bias, p->relu, d.K, g.PQ,
+                                  d.out_layout == B2C_LAYOUT_NHWC ? 1 : 0, st));
   return B2C_OK;
 }
 
@@ -695,6 +704,21 @@ int b2c_conv2d_int8_run_rewritten(b2c_plan* p, const int8_t* x, int32_t* y32, in
   return run_convolve(p, x, y32, y8, ws, (cudaStream_t)cuda_stream);
 }
 
+int b2c_plan_set_activation(b2c_plan* p, const int32_t* bias_dev, int relu, void* cuda_stream) {
+  if (!p || (relu != 0 && relu != 1)) return B2C_E_INVALID_ARG;
+  if (bias_dev && (reinterpret_cast<uintptr_t>(bias_dev) & 3) != 0) return B2C_E_INVALID_ARG;
+  const size_t bytes = (size_t)p->g.d.K * sizeof(int32_t);
+  if (bias_dev) {
+    if (!p->bias_buf) CUDA_TRY(cudaMalloc(&p->bias_buf, bytes));
+    CUDA_TRY(cudaMemcpyAsync(p->bias_buf, bias_dev, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)cuda_stream));
+    p->bias = p->bias_buf;
+  } else {
+    p->bias = nullptr;  // the buffer is kept for a later call
+  }
+  p->relu = relu;
+  return B2C_OK;
+}
+
 int b2c_plan_footprint(const b2c_plan* p, size_t* rewritten_bytes, size_t* packed_weight_bytes) {
   if (!p || !rewritten_bytes || !packed_weight_bytes) return B2C_E_INVALID_ARG;
   *rewritten_bytes = p->ws_layout_bytes;
@@ -724,6 +748,7 @@ void b2c_plan_destroy(b2c_plan* p) {
   cudaFree(p->table32);
   cudaFree(p->wtable);
   cudaFree(p->status);
+  cudaFree(p->bias_buf);
   cudaFree(p->own_ws);
   delete p;
 }

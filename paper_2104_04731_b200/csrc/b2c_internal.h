@@ -109,6 +109,10 @@ struct ConvArgs {
   // output pixel p = (p' - ph_pad_h)*ph_dh + a + out_pad_h (q likewise), and is dropped when that
   // pixel lies outside the out_P x out_Q output.
   int out_PQ, remap, ph_dh, ph_dw, ph_pad_h, ph_pad_w, out_pad_h, out_pad_w, out_P, out_Q;
+  // activation step applied to the complete sums before they are written: + bias[k] (nullptr: none),
+  // then max(., 0) when relu != 0
+  const int32_t* bias;
+  int relu;
 };
 
 // Programmatic dependent launch: a kernel launched through launch_pdl may start while the previous
@@ -226,7 +230,7 @@ cudaError_t launch_phase_split(const int8_t* x, int8_t* out, int N, int C, int H
                                int C_pad, long long stride_n, long long stride_c, int stride_h, int stride_w,
                                cudaStream_t st);
 cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, long long elems, int shift,
-                                 int out_mode, cudaStream_t st);
+                                 int out_mode, const int32_t* bias, int relu, int K, int PQ, int nhwc, cudaStream_t st);
 cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,
                             cudaStream_t st);
 size_t conv_mma_smem_bytes(int amode, const ConvArgs& args);

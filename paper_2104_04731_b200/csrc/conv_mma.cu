@@ -200,6 +200,14 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t* v) {
 
 __device__ __forceinline__ int8_t requant(int v, int shift) { return (int8_t)max(-128, min(127, v >> shift)); }
 
+// Activation step of Section 5.1's vector unit on a complete sum of output channel k: optional
+// per-channel bias, optional ReLU.  (Partial sums of a split reduction are never passed here.)
+__device__ __forceinline__ int activate(const ConvArgs& args, int v, int k) {
+  if (args.bias != nullptr) v += __ldg(args.bias + k);
+  if (args.relu) v = max(v, 0);
+  return v;
+}
+
 // Loads NC consecutive accumulator columns of this thread's TMEM lane.
 template <int NC>
 __device__ __forceinline__ void tmem_ld(uint32_t taddr, int32_t* v);
@@ -225,7 +233,7 @@ __device__ __forceinline__ void tmem_ld<32>(uint32_t taddr, int32_t* v) {
 // here, and the values go to the NKPQ or NPQK tensor; with a split reduction the partial sums
 // are added into a zeroed int32 buffer instead.
 template <int NC>
-__device__ __forceinline__ void store_columns(const ConvArgs& args, const int32_t* v, int kbase, bool row_valid,
+__device__ __forceinline__ void store_columns(const ConvArgs& args, int32_t* v, int kbase, bool row_valid,
                                               long long base_nkpq, long long base_npqk) {
   const int K = args.K;
   if (!row_valid || kbase >= K) return;
@@ -240,7 +248,14 @@ __device__ __forceinline__ void store_columns(const ConvArgs& args, const int32_
       if (kbase + j < K) atomicAdd(dst, v[j]);
       dst += step;
     }
-  } else if (!nhwc) {
+    return;
+  }
+  if (args.bias != nullptr || args.relu) {
+#pragma unroll
+    for (int j = 0; j < NC; ++j)
+      if (kbase + j < K) v[j] = activate(args, v[j], kbase + j);
+  }
+  if (!nhwc) {
     // NKPQ: for a fixed column the 32 lanes of a warp hold 32 consecutive pixels, so every
     // store instruction writes one contiguous run.
     const long long o = base_nkpq + (long long)kbase * args.out_PQ;
@@ -302,7 +317,7 @@ __device__ __forceinline__ void store_columns(const ConvArgs& args, const int32_
 // consecutive channels, so every store instruction writes one contiguous run.  NKPQ: the 16 pixels
 // of a thread are contiguous while they stay inside one image, and go out as 16-byte vectors when
 // the run is complete and aligned.
-__device__ __forceinline__ void store_columns_swapped(const ConvArgs& args, const int32_t* v, int k, bool row_valid,
+__device__ __forceinline__ void store_columns_swapped(const ConvArgs& args, int32_t* v, int k, bool row_valid,
                                                       int m_first) {
   if (!row_valid || m_first >= args.Mg) return;
   const int count = min(16, args.Mg - m_first);
@@ -310,6 +325,10 @@ __device__ __forceinline__ void store_columns_swapped(const ConvArgs& args, cons
   int pq = m_first - n_img * args.PQ;
   const bool nhwc = args.out_layout == B2C_LAYOUT_NHWC;
   const bool split = args.split_k > 1;
+  if (!split && (args.bias != nullptr || args.relu)) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = activate(args, v[j], k);
+  }
   if (nhwc) {
     long long o = (long long)m_first * args.K + k;
 #pragma unroll
@@ -919,6 +938,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
           const int c = cb + b * kGatherWarps;
           const int k = n0 + col_base + c;
           if (c >= cols_slice || k >= args.K || rows_valid == 0) continue;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) acc[b][i] = activate(args, acc[b][i], k);
           if (!nhwc && one_image) {
             // four consecutive pixels of one image and one channel: contiguous in NKPQ
             const long long o = ((long long)n_img * args.K + k) * args.PQ + pq;

@@ -333,13 +333,17 @@ __global__ void __launch_bounds__(256) phase_split_kernel(const int8_t* __restri
 // Finish of a split reduction: the int32 sums are complete in `acc`; copy them out and/or apply
 // the shift-and-clip requantisation (arithmetic shift = floor division by 2^shift).
 __global__ void splitk_finish_kernel(const int32_t* __restrict__ acc, int32_t* __restrict__ y32,
-                                     int8_t* __restrict__ y8, long long elems, int shift, int out_mode) {
+                                     int8_t* __restrict__ y8, long long elems, int shift, int out_mode,
+                                     const int32_t* __restrict__ bias, int relu, int K, int PQ, int nhwc) {
   pdl_wait();
   pdl_launch_dependents();
+  const bool act = bias != nullptr || relu != 0;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < elems;
        i += (long long)gridDim.x * blockDim.x) {
-    const int v = acc[i];
-    if ((out_mode & B2C_OUT_I32) && y32 != acc) y32[i] = v;
+    int v = acc[i];
+    if (bias != nullptr) v += bias[nhwc ? (int)(i % K) : (int)((i / PQ) % K)];  // output channel of element i
+    if (relu) v = max(v, 0);
+    if ((out_mode & B2C_OUT_I32) && (y32 != acc || act)) y32[i] = v;
     if (out_mode & B2C_OUT_I8) y8[i] = (int8_t)max(-128, min(127, v >> shift));
   }
 }
@@ -423,9 +427,9 @@ cudaError_t launch_phase_split(const int8_t* x, int8_t* out, int N, int C, int H
 }
 
 cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, long long elems, int shift,
-                                 int out_mode, cudaStream_t st) {
+                                 int out_mode, const int32_t* bias, int relu, int K, int PQ, int nhwc, cudaStream_t st) {
   return launch_pdl(splitk_finish_kernel, dim3(grid_for(elems, 256)), dim3(256), 0, st, acc, y32, y8, elems, shift,
-                    out_mode);
+                    out_mode, bias, relu, K, PQ, nhwc);
 }
 
 }  // namespace b2c

@@ -209,6 +209,54 @@ def test_rewrite_and_convolve_halves(lib):
         plan.destroy()
 
 
+# ---- activation step (bias + ReLU) fused into every epilogue ---------------------------------------------
+@pytest.mark.parametrize("case", [
+    # N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode
+    (1, 16, 14, 14, 16, 3, 3, 1, 1, 1, 8, 3),      # small: every variant, split reductions through memory
+    (2, 64, 12, 12, 136, 3, 3, 1, 1, 1, 9, 3),     # cluster reductions, swapped map, two channel tiles
+    (1, 256, 7, 7, 64, 3, 3, 1, 1, 1, 10, 2),      # int8 only: split goes through the scratch and the finish kernel
+    (2, 8, 20, 20, 24, 3, 3, 1, 2, 2, 6, 1),       # dilated (phase pack), int32 only: split meets in the output itself
+])
+@pytest.mark.parametrize("out_layout", [0, 1])
+def test_bias_and_relu(lib, case, out_layout):
+    N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode = case
+    x = int8_uniform((N, C, H, W), 641)
+    w = int8_uniform((K, C, R, S), 642)
+    bias = (int8_uniform((K,), 643).astype(np.int32) * 3001)
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, 0, out_layout, out_mode)
+    P, Q = lib.out_shape(d)
+    oshape = (N, K, P, Q) if out_layout == 0 else (N, P, Q, K)
+    refs = {(b, r): oracle.conv2d_int8(x, w, stride, pad, dil, shift, bias=bias if b else None, relu=r)
+            for b in (0, 1) for r in (False, True)}
+    assert (refs[(1, False)][0] < 0).any()  # the ReLU has something to clip
+    seen = set()
+    xd, wd, bd = to_dev(x), to_dev(w), to_dev(bias)
+    for e in lib.enumerate_embeddings(d):
+        key = (e.variant, e.map_m, min(e.split_k, 2), e.tile_n >= 32 * e.split_k)
+        if key in seen:
+            continue
+        seen.add(key)
+        plan = lib.Plan(d, e.id)
+        ws = torch.zeros(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
+        plan.set_weights(wd)
+        for (b, r) in [(1, True), (1, False), (0, True), (0, False)]:  # the last pair removes the step again
+            plan.set_activation(bd if b else None, r)
+            y32 = torch.full(oshape, -7777777, dtype=torch.int32, device="cuda") if out_mode & 1 else None
+            y8 = torch.full(oshape, 77, dtype=torch.int8, device="cuda") if out_mode & 2 else None
+            plan.run(xd, y32, y8, ws)
+            torch.cuda.synchronize()
+            tag = "variant %d map_m %d tile %d split %d bias %d relu %d" % (e.variant, e.map_m, e.tile_n, e.split_k, b, r)
+            for got, want in ((y32, refs[(b, r)][0]), (y8, refs[(b, r)][1])):
+                if got is None:
+                    continue
+                g = got.cpu().numpy()
+                g = g if out_layout == 0 else g.transpose(0, 3, 1, 2)
+                assert np.array_equal(g, want), tag
+        assert plan.device_status() == b2c.OK
+        plan.destroy()
+    assert len(seen) >= 6
+
+
 def test_extreme_values_and_shift_clip(lib):
     # -128 * -128 is the largest product; all-(-128) tensors with 9*64 taps reach 9437184.
     x = np.full((1, 64, 6, 6), -128, dtype=np.int8)
