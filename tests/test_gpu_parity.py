@@ -257,6 +257,53 @@ def test_bias_and_relu(lib, case, out_layout):
     assert len(seen) >= 6
 
 
+def test_chained_layers_skip_the_activation_pack(lib):
+    # Layout coordination between layers: an int8 NHWC output with a multiple of 32 channels is the
+    # channel-pack operand of the next layer as it stands, so the second plan has no rewrite at all.
+    x = int8_uniform((2, 24, 18, 18), 651)
+    w1 = int8_uniform((64, 24, 3, 3), 652)
+    w2 = int8_uniform((40, 64, 3, 3), 653)
+    bias1 = int8_uniform((64,), 654).astype(np.int32) * 500
+    _, h_ref = oracle.conv2d_int8(x, w1, 1, 1, 1, 7, bias=bias1, relu=True)
+    ref = oracle.conv2d_int8(h_ref, w2, 2, 1, 1, 9)
+    d1 = lib.make_desc(2, 24, 18, 18, 64, 3, 3, 1, 1, 1, 7, b2c.LAYOUT_NCHW, b2c.LAYOUT_NHWC, b2c.OUT_I8)
+    d2 = lib.make_desc(2, 64, 18, 18, 40, 3, 3, 2, 1, 1, 9, b2c.LAYOUT_NHWC, b2c.LAYOUT_NCHW, 3)
+    p1 = lib.Plan(d1, b2c.POLICY_MIN_OVERHEAD)
+    cp = [e for e in lib.enumerate_embeddings(d2) if e.variant == b2c.VARIANT_CP_TMA and e.split_k == 1]
+    p2 = lib.Plan(d2, cp[0].id)
+    assert p2.workspace_bytes() == 0 and p2.footprint()[0] == 0
+    h = torch.zeros((2, 18, 18, 64), dtype=torch.int8, device="cuda")
+    y32 = torch.zeros(ref[0].shape, dtype=torch.int32, device="cuda")
+    y8 = torch.zeros(ref[1].shape, dtype=torch.int8, device="cuda")
+    ws1 = torch.zeros(max(16, p1.workspace_bytes()), dtype=torch.uint8, device="cuda")
+    p1.set_weights(to_dev(w1))
+    p1.set_activation(to_dev(bias1), True)
+    p2.set_weights(to_dev(w2))
+    p1.run(to_dev(x), None, h, ws1)
+    p2.run(h, y32, y8, None)
+    torch.cuda.synchronize()
+    assert np.array_equal(h.cpu().numpy().transpose(0, 3, 1, 2), h_ref)
+    assert np.array_equal(y32.cpu().numpy(), ref[0]) and np.array_equal(y8.cpu().numpy(), ref[1])
+    p1.destroy()
+    p2.destroy()
+
+
+@pytest.mark.parametrize("batch,cin,cout", [(1, 256, 512), (37, 72, 96), (300, 33, 17)])
+def test_dense_layer_is_a_1x1_convolution(lib, batch, cin, cout):
+    # A fully connected layer y = x W^T is the 1x1 convolution of a 1x1 image: M = batch, K = cout.
+    x = int8_uniform((batch, cin, 1, 1), 661)
+    w = int8_uniform((cout, cin, 1, 1), 662)
+    want = x.reshape(batch, cin).astype(np.int64) @ w.reshape(cout, cin).astype(np.int64).T
+    d = lib.make_desc(batch, cin, 1, 1, cout, 1, 1, out_mode=1)
+    seen = set()
+    for e in lib.enumerate_embeddings(d):
+        if (e.variant, e.map_m) in seen:
+            continue
+        seen.add((e.variant, e.map_m))
+        y32, _, _ = run_embedding(x, w, 1, 0, 1, 0, 1, e.id)
+        assert np.array_equal(y32.reshape(batch, cout), want), (e.variant, e.map_m)
+
+
 def test_extreme_values_and_shift_clip(lib):
     # -128 * -128 is the largest product; all-(-128) tensors with 9*64 taps reach 9437184.
     x = np.full((1, 64, 6, 6), -128, dtype=np.int8)
