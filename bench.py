@@ -260,9 +260,9 @@ def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, grap
     warm.capture(torch, repeat=20)
     ms_w = time_steps(torch, warm.step, 10, 3, None, 0.0)
     warm.destroy()
-    op = op_only(b2c, torch, cfg, emb["variant"], emb["tile_n"], emb["split_k"], steps, warmup, graph)
+    op = op_only(b2c, torch, cfg, emb["variant"], emb["tile_n"], emb["split_k"], steps, warmup, graph, 1, emb["map_m"])
     t_roof, bound = roofline_time_us(cfg, peaks)
-    keys = ("id", "variant_name", "tile_n", "split_k", "workspace_bytes", "o_mac", "o_data", "device_us")
+    keys = ("id", "variant_name", "map_m", "tile_n", "split_k", "workspace_bytes", "o_mac", "o_data", "device_us")
     res = {
         "shape": cfg.name, "instances": G, "warm_us": ms_w * 1e3 / (10 * 20),
         "op_us": op["us"] if op else None, "transf_us": max(0.0, per_call_us - op["us"]) if op else None, "cold": bool(G * cfg.algorithmic_bytes >= L2_BYTES), "combined_us": per_call_us, "tops": 2.0 * cfg.macs / (per_call_us * 1e-6) / 1e12,
@@ -317,12 +317,13 @@ def measure_scaled(b2c, torch, cfg, peaks, steps=10):
             "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k}}
 
 
-def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=True, streams=1):
+def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=True, streams=1, map_m=1):
     """Device time of the MMA kernel alone: same embedding but with the layout rewrite already done
     (channel-pack map: NHWC input with padded channels; stencil-unroll in-kernel: unchanged)."""
     if emb_variant == 0 and cfg.C % 32 == 0:
         d = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, 1, 0, cfg.out_mode)
-        ids = [e.id for e in b2c.enumerate_embeddings(d) if e.variant == 0 and e.tile_n == tile_n and e.split_k == split_k]
+        ids = [e.id for e in b2c.enumerate_embeddings(d)
+               if e.variant == 0 and e.tile_n == tile_n and e.split_k == split_k and e.map_m == map_m]
         if not ids:
             return None
         G = instances_for(cfg)
@@ -330,7 +331,8 @@ def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=
     elif emb_variant in (2, 3):
         # stencil unroll inside the kernel: there is no separate rewrite, the kernel is the whole path
         d = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, 0, 0, cfg.out_mode)
-        ids = [e.id for e in b2c.enumerate_embeddings(d) if e.variant == emb_variant and e.tile_n == tile_n and e.split_k == split_k]
+        ids = [e.id for e in b2c.enumerate_embeddings(d)
+               if e.variant == emb_variant and e.tile_n == tile_n and e.split_k == split_k and e.map_m == map_m]
         G = instances_for(cfg)
         inst = Instances(b2c, torch, cfg, G, ids[0])
     else:
@@ -568,7 +570,8 @@ def run_ours(args):
         v, tn, sk = (int(t) for t in args.pick.split(","))
         d0 = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
                            0, 0, cfg.out_mode)
-        policy = next(e.id for e in b2c.enumerate_embeddings(d0) if (e.variant, e.tile_n, e.split_k) == (v, tn, sk))
+        policy = next(e.id for e in b2c.enumerate_embeddings(d0)
+                      if (e.variant, e.tile_n, e.split_k) == (v, tn, sk) and e.map_m == b2c.AXIS_NPQ)
     graph = not args.no_graph
     if args.report == "candidates":
         rep = candidates_report(b2c, torch, CONFIGS + REPORT_EXTRA)
@@ -597,7 +600,8 @@ def run_ours(args):
     # ---- the dominant kernel alone (the paper's "Op." column) for the roofline -------------------
     op = None
     if not args.no_op_pass:
-        op = op_only(b2c, torch, cfg, emb.variant, emb.tile_n, emb.split_k, args.steps, args.warmup, graph, args.streams)
+        op = op_only(b2c, torch, cfg, emb.variant, emb.tile_n, emb.split_k, args.steps, args.warmup, graph, args.streams,
+                     emb.map_m)
     t_roof, bound = roofline_time_us(cfg, peaks)
     op_us = op["us"] if op else per_call_us
     if bound == "tensor":
@@ -645,7 +649,7 @@ def run_ours(args):
                    "cuda_graph": graph, "streams": args.streams if graph else 1,
                    "parallelism": "independent instances sharded over ranks, no collective",
                    "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k,
-                                 "planner_us": emb.device_us}},
+                                 "swapped": emb.map_m == b2c.AXIS_K, "planner_us": emb.device_us}},
         "roofline": roofline, "roofline_time_us": t_roof, "whole_path_roofline_frac": t_roof / per_call_us,
         "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
     }

@@ -3,7 +3,6 @@
 // the timed candidate selection.  See include/b2conv.h for the contract of each entry point.
 #include <algorithm>
 #include <cstring>
-#include <cstdlib>
 #include <map>
 #include <mutex>
 #include <new>
@@ -221,8 +220,7 @@ void fill_common_args(b2c_plan* p) {
       tiles_m * tiles_n < 0x7FFFFFFF)
     a.persistent = 2;
   a.tmem_bufs = (a.persistent && 2 * a.tmem_cols <= 512) ? 2 : 1;
-  size_t budget = a.persistent == 1 ? 196 * 1024 : (a.persistent == 2 ? 68 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 160 * 1024));
-  if (getenv("B2C_XBUDGET") && !a.persistent) budget = (size_t)atoi(getenv("B2C_XBUDGET")) * 1024;
+  const size_t budget = a.persistent == 1 ? 196 * 1024 : (a.persistent == 2 ? 68 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 160 * 1024));
   const size_t stage_bytes = (size_t)(kTileM + a.tile_n) * a.bk;
   // lookup table and staged window share the block's shared memory with the stages
   const size_t extra = p->amode == A_STAGED ? (size_t)p->win.bytes + 4 * (size_t)p->table_len + 64
