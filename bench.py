@@ -292,29 +292,40 @@ def scaled_shape(cfg: ConvShape, peaks, target_us=50.0) -> ConvShape:
 
 
 def measure_scaled(b2c, torch, cfg, peaks, steps=10):
-    """Secondary series: one large-batch problem per launch (working set beyond L2), whole path."""
+    """Secondary series: one large-batch problem per launch (working set beyond L2), whole path; and,
+    where the channel count allows it, the same problem with NHWC input (the layout a previous int8
+    layer of this library leaves behind), for which the channel-pack map needs no rewrite."""
     big = scaled_shape(cfg, peaks)
-    d = b2c.make_desc(big.N, big.C, big.H, big.W, big.K, big.R, big.S, big.stride, big.pad, big.dilation, big.shift,
-                      0, 0, big.out_mode)
-    plan = b2c.Plan(d, b2c.POLICY_AUTO_TIMED)
-    emb = plan.info()
-    x = torch.randint(-128, 128, (big.N, big.C, big.H, big.W), dtype=torch.int8, device="cuda")
-    w = torch.randint(-128, 128, (big.K, big.C, big.R, big.S), dtype=torch.int8, device="cuda")
-    oshape = (big.N, big.K, big.P, big.Q)
-    y32 = torch.empty(oshape, dtype=torch.int32, device="cuda") if big.out_mode & 1 else None
-    y8 = torch.empty(oshape, dtype=torch.int8, device="cuda") if big.out_mode & 2 else None
-    ws = torch.empty(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
-    plan.set_weights(w)
-    ms = time_steps(torch, lambda: plan.run(x, y32, y8, ws), steps, 3, None, 0.05)
-    st = plan.device_status()
-    plan.destroy()
-    if st != 0:
-        raise RuntimeError("device status " + b2c.status_string(st))
-    us = ms * 1e3 / steps
     t_roof, bound = roofline_time_us(big, peaks)
-    return {"shape": big.name, "us": us, "tops": 2.0 * big.macs / (us * 1e-6) / 1e12, "roofline_us": t_roof,
-            "bound": bound, "roofline_frac": t_roof / us, "bytes": big.algorithmic_bytes,
-            "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k}}
+
+    def one(in_layout):
+        d = b2c.make_desc(big.N, big.C, big.H, big.W, big.K, big.R, big.S, big.stride, big.pad, big.dilation, big.shift,
+                          in_layout, 0, big.out_mode)
+        plan = b2c.Plan(d, b2c.POLICY_AUTO_TIMED)
+        emb = plan.info()
+        shape = (big.N, big.C, big.H, big.W) if in_layout == 0 else (big.N, big.H, big.W, big.C)
+        x = torch.randint(-128, 128, shape, dtype=torch.int8, device="cuda")
+        w = torch.randint(-128, 128, (big.K, big.C, big.R, big.S), dtype=torch.int8, device="cuda")
+        oshape = (big.N, big.K, big.P, big.Q)
+        y32 = torch.empty(oshape, dtype=torch.int32, device="cuda") if big.out_mode & 1 else None
+        y8 = torch.empty(oshape, dtype=torch.int8, device="cuda") if big.out_mode & 2 else None
+        ws = torch.empty(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
+        plan.set_weights(w)
+        ms = time_steps(torch, lambda: plan.run(x, y32, y8, ws), steps, 3, None, 0.05)
+        st = plan.device_status()
+        plan.destroy()
+        if st != 0:
+            raise RuntimeError("device status " + b2c.status_string(st))
+        us = ms * 1e3 / steps
+        return {"us": us, "tops": 2.0 * big.macs / (us * 1e-6) / 1e12, "roofline_frac": t_roof / us,
+                "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k,
+                              "swapped": emb.map_m == b2c.AXIS_K}}
+
+    res = {"shape": big.name, "roofline_us": t_roof, "bound": bound, "bytes": big.algorithmic_bytes}
+    res.update(one(0))
+    if big.C % 32 == 0:
+        res["nhwc_input"] = one(1)
+    return res
 
 
 def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=True, streams=1, map_m=1):
