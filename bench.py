@@ -144,9 +144,9 @@ class Instances:
         """Kernels of this library per call: layout rewrite (if any) + MMA kernel + split finish (if any)."""
         e, c = self.emb, self.cfg
         n = 1
-        if e.variant in (1, 4, 5, 6) or (e.variant == 0 and not (self.in_layout == 1 and c.C % 32 == 0)):
+        if e.variant in (1, 4, 5, 6, 8) or (e.variant in (0, 7) and not (self.in_layout == 1 and c.C % 32 == 0)):
             n += 1
-        cluster = (e.map_m != 2 and e.variant != 6 and e.split_k in (2, 4, 8) and e.tile_n >= 32 * e.split_k
+        cluster = (e.map_m != 2 and e.variant not in (6, 7, 8) and e.split_k in (2, 4, 8) and e.tile_n >= 32 * e.split_k
                    and (e.variant in (0, 1, 4, 5) or e.tile_n <= 128))  # the swapped map (map_m = k) and the phase pack never cluster
         if e.split_k > 1 and not cluster and (c.out_mode & 2):
             n += 1  # a split reduction that is not a cluster goes through memory and needs the finish kernel
@@ -331,10 +331,10 @@ def measure_scaled(b2c, torch, cfg, peaks, steps=10):
 def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=True, streams=1, map_m=1):
     """Device time of the MMA kernel alone: same embedding but with the layout rewrite already done
     (channel-pack map: NHWC input with padded channels; stencil-unroll in-kernel: unchanged)."""
-    if emb_variant == 0 and cfg.C % 32 == 0:
+    if emb_variant in (0, 7) and cfg.C % 32 == 0:
         d = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, 1, 0, cfg.out_mode)
         ids = [e.id for e in b2c.enumerate_embeddings(d)
-               if e.variant == 0 and e.tile_n == tile_n and e.split_k == split_k and e.map_m == map_m]
+               if e.variant == emb_variant and e.tile_n == tile_n and e.split_k == split_k and e.map_m == map_m]
         if not ids:
             return None
         G = instances_for(cfg)

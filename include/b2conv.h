@@ -79,6 +79,11 @@ typedef struct {
 #define B2C_VARIANT_DILATION_PACK 6  /* image pack of a dilated conv (Section 6.1): the dil_h*dil_w phase sub-images are fused
                                       * into the batch, convolved densely, and the epilogue interleaves the results back */
 
+#define B2C_VARIANT_CP_SHIFT 7       /* channel pack with the stencil as operand shifts (stride 1): every tile stages the padded
+                                      * image rows it needs once, tap (r, s) is the same shared-memory tile read (r*dil_h rows +
+                                      * s*dil_w pixels) further on, and the packed weights stay resident in shared memory */
+#define B2C_VARIANT_S2D_SHIFT 8      /* image pack (space to depth) of a strided conv, then the stride-1 remainder as operand shifts */
+
 typedef struct {
   int32_t id;       /* index in the enumeration for this descriptor; pass to b2c_plan_create      */
   int32_t map_m, map_n, map_k; /* B2C_AXIS_*                                                      */

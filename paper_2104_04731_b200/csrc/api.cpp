@@ -164,6 +164,25 @@ void fill_common_args(b2c_plan* p) {
     a.dil_h = v.dil_h;
     a.dil_w = v.dil_w;
     a.S = v.S;
+    if (is_shift_variant(p->emb.variant)) {
+      ShiftGeom sg;
+      shift_geom(p->g, v, &sg);  // legal: checked when the plan was created
+      p->amode = A_SHIFT;
+      a.Mg = (int)sg.mtot;
+      a.sh_mtot = (int)sg.mtot;
+      a.sh_wps = sg.wps;
+      a.sh_hp = sg.hp;
+      a.sh_rows = sg.rows;
+      a.sh_row_bytes = sg.row_bytes;
+      a.sh_ncb = sg.ncb;
+      a.sh_R = v.R;
+      a.sh_cblk_bytes = sg.cblk_bytes;
+      a.sh_win_bytes = sg.win_bytes;
+      a.sh_w_bytes = sg.w_bytes;
+      a.div_wps = make_fastdiv((uint32_t)sg.wps);
+      a.div_hp = make_fastdiv((uint32_t)sg.hp);
+      a.remap = 2;
+    }
     if (p->emb.variant == B2C_VARIANT_DILATION_PACK) {
       // the kernel's rows are the pixels of the phase sub-image convolutions
       const int Pv = v.H + 2 * v.pad_h - v.R + 1, Qv = v.W + 2 * v.pad_w - v.S + 1;
@@ -228,6 +247,21 @@ void fill_common_args(b2c_plan* p) {
   while (stages > 2 && (size_t)stages * stage_bytes + extra > budget) --stages;
   while (stages > 1 && (size_t)stages * stage_bytes + extra > 196 * 1024) --stages;
   a.cluster_split = cluster_split_ok(p->emb.variant, a.tile_n, a.split_k, a.swap != 0) ? 1 : 0;
+  if (p->amode == A_SHIFT) {
+    // two window buffers form the stage ring; the resident weights follow them
+    ShiftGeom sg;
+    shift_geom(p->g, p->view, &sg);
+    a.persistent = 2;
+    a.tmem_bufs = 2 * a.tmem_cols <= 512 ? 2 : 1;
+    a.tiles_n = 1;
+    a.num_tiles = (int)((sg.mtot + kTileM - 1) / kTileM);
+    a.div_tiles_n = make_fastdiv(1);
+    a.num_kb = 1;
+    a.stages = 2;
+    a.stage_region = 2 * sg.win_bytes + sg.w_bytes;
+    a.persistent_blocks_per_sm = sg.blocks_per_sm;
+    return;
+  }
   size_t region = (size_t)stages * stage_bytes;
   // the stage buffers double as the 128 x tile_n int32 exchange tile of the cluster reduction
   if (a.cluster_split) region = std::max(region, (size_t)kTileM * a.tile_n * 4);
@@ -252,7 +286,8 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
     if (!tma_view_for(g, emb.variant, &p->view)) return fail(B2C_E_UNSUPPORTED);
     const TmaView& v = p->view;
     p->w_packed_bytes = (size_t)d.K * v.R * v.S * v.C;
-    if (emb.variant != B2C_VARIANT_CP_TMA && emb.variant != B2C_VARIANT_DILATION_PACK) {
+    if (emb.variant != B2C_VARIANT_CP_TMA && emb.variant != B2C_VARIANT_DILATION_PACK &&
+        emb.variant != B2C_VARIANT_CP_SHIFT) {
       // Lookup tables of the rewritten maps.  Activations: scratch channel j of scratch pixel
       // (n, h', w') <- input element, in the form the stencil-unroll kernel takes.  Weights: packed
       // column (tap, j) <- index into one KCRS filter.
@@ -329,7 +364,7 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
   fill_common_args(p);
   p->ws_total = workspace_bytes_for(g, emb.variant, emb.tile_n, emb.split_k, is_swapped(emb));
   if (is_tma_view_variant(emb.variant)) {
-    bool direct = emb.variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && p->C_pad == d.C;
+    bool direct = shift_base_variant(emb.variant) == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && p->C_pad == d.C;
     p->ws_layout_bytes = direct ? 0 : ((size_t)p->view.bytes() + 255) / 256 * 256;
   } else if (emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
     p->ws_layout_bytes = ((size_t)g.Mg * p->K_pad + 255) / 256 * 256;
@@ -504,10 +539,11 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
   // fastest is kept).  All schedules of the five lowest-overhead (axis map, layout variant)
   // groups are run on scratch tensors.
   cudaStream_t st = (cudaStream_t)cuda_stream;
+  // (A shift variant belongs to the group of the view it executes: same rewrite, same weights.)
   std::vector<int> groups;
   for (const b2c_embedding& e : all)
-    if (std::find(groups.begin(), groups.end(), e.variant) == groups.end() && groups.size() < 5)
-      groups.push_back(e.variant);
+    if (std::find(groups.begin(), groups.end(), shift_base_variant(e.variant)) == groups.end() && groups.size() < 5)
+      groups.push_back(shift_base_variant(e.variant));
   size_t ws_max = 0;
   for (const b2c_embedding& e : all) ws_max = std::max(ws_max, (size_t)e.workspace_bytes);
   int8_t *x = nullptr, *w = nullptr;
@@ -537,7 +573,7 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
   int best = -1;
   float best_us = 0;
   for (size_t i = 0; i < all.size(); ++i) {
-    if (std::find(groups.begin(), groups.end(), all[i].variant) == groups.end()) continue;
+    if (std::find(groups.begin(), groups.end(), shift_base_variant(all[i].variant)) == groups.end()) continue;
     b2c_plan* p = nullptr;
     rc = create_plan_for(g, all[i], &p);
     if (rc != B2C_OK) break;
@@ -576,7 +612,8 @@ int b2c_plan_set_weights(b2c_plan* p, const int8_t* w, void* cuda_stream) {
   if (!aligned16(w)) return B2C_E_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const b2c_conv_desc& d = p->g.d;
-  if (p->emb.variant == B2C_VARIANT_CP_TMA || p->emb.variant == B2C_VARIANT_DILATION_PACK)
+  if (p->emb.variant == B2C_VARIANT_CP_TMA || p->emb.variant == B2C_VARIANT_DILATION_PACK ||
+      p->emb.variant == B2C_VARIANT_CP_SHIFT)
     CUDA_TRY(launch_pack_weights_cp(w, p->w_packed, d.K, d.C, d.R, d.S, p->C_pad, st));
   else if (is_tma_view_variant(p->emb.variant))
     CUDA_TRY(launch_pack_weights_table(w, p->w_packed, d.K, p->g.Kg, p->view.R * p->view.S * p->view.C, p->wtable, st));
@@ -599,13 +636,14 @@ static int run_rewrite(b2c_plan* p, const int8_t* x, void* ws, cudaStream_t st) 
   int8_t* scratch = static_cast<int8_t*>(ws);
   if (is_tma_view_variant(p->emb.variant)) {
     const TmaView& v = p->view;
-    if (p->emb.variant == B2C_VARIANT_CP_TMA) {
+    const int base_variant = shift_base_variant(p->emb.variant);
+    if (base_variant == B2C_VARIANT_CP_TMA) {
       CUDA_TRY(launch_pack_activations(x, scratch, d.N, d.C, d.H, d.W, p->C_pad, st));
-    } else if (p->emb.variant == B2C_VARIANT_DILATION_PACK) {
+    } else if (base_variant == B2C_VARIANT_DILATION_PACK) {
       const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
       CUDA_TRY(launch_phase_split(x, scratch, d.N, d.C, d.H, d.W, d.dil_h, d.dil_w, v.H, v.W, v.C, a.x_stride_n,
                                   nchw ? (long long)d.H * d.W : 1, a.x_stride_h, a.x_stride_w, st));
-    } else if (p->emb.variant == B2C_VARIANT_ROW_UNROLL) {
+    } else if (base_variant == B2C_VARIANT_ROW_UNROLL) {
       // scratch pixel (n, h, q): window origin (h, q*stride_w - pad_w), channels (s, c)
       CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W, 1,
                              d.stride_w, 0, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w, v.C, st));
@@ -639,7 +677,10 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   if (is_tma_view_variant(p->emb.variant)) {
     const TmaView& v = p->view;
     const int8_t* act = p->ws_layout_bytes ? reinterpret_cast<const int8_t*>(wsb) : x;
-    rc = encode_im2col_nhwc(&tmap_a, act, v.C, v.W, v.H, v.N, v.pad_w, v.pad_h, v.S, v.R, v.dil_w, v.dil_h,
+    if (p->amode == A_SHIFT)
+      rc = encode_tiled_nhwc_rows(&tmap_a, act, v.C, v.W, v.H, v.N, p->bk, a.sh_wps, p->bk);
+    else
+      rc = encode_im2col_nhwc(&tmap_a, act, v.C, v.W, v.H, v.N, v.pad_w, v.pad_h, v.S, v.R, v.dil_w, v.dil_h,
                             v.stride_w, v.stride_h, p->bk, a.swap ? a.tile_n : kTileM, p->bk);
     if (rc != B2C_OK) return rc;
   } else if (p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {

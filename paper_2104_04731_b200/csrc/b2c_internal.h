@@ -62,7 +62,7 @@ inline FastDiv make_fastdiv(uint32_t d) {
   return f;
 }
 
-enum AMode { A_TILED = 0, A_IM2COL_TMA = 1, A_GATHER = 2, A_STAGED = 3 };
+enum AMode { A_TILED = 0, A_IM2COL_TMA = 1, A_GATHER = 2, A_STAGED = 3, A_SHIFT = 4 };
 
 // Everything the MMA kernel needs besides its two tensor maps.
 struct ConvArgs {
@@ -109,6 +109,15 @@ struct ConvArgs {
   // output pixel p = (p' - ph_pad_h)*ph_dh + a + out_pad_h (q likewise), and is dropped when that
   // pixel lies outside the out_P x out_Q output.
   int out_PQ, remap, ph_dh, ph_dw, ph_pad_h, ph_pad_w, out_pad_h, out_pad_w, out_P, out_Q;
+  // Stencil as operand shift (A_SHIFT; stride-1 geometry over an NHWC tensor with padded channels).
+  // Accumulator rows enumerate window origins on a grid of sh_hp x sh_wps positions per image
+  // (sh_wps = padded width rounded up to 8, so that every staged image row starts on a swizzle
+  // atom); a tile's 128 consecutive positions read, for tap (r, s), the 128 consecutive staged
+  // pixels that start (r*dil_h*sh_wps + s*dil_w) pixels further on.  One stage holds sh_rows padded
+  // image rows per channel block; the packed weights stay resident in shared memory.
+  int sh_wps, sh_hp, sh_rows, sh_row_bytes, sh_ncb, sh_R, sh_cblk_bytes, sh_win_bytes, sh_w_bytes, sh_mtot;
+  int persistent_blocks_per_sm;  // blocks per SM the persistent grid is sized for (0: the mode's default)
+  FastDiv div_wps, div_hp;
   // activation step applied to the complete sums before they are written: + bias[k] (nullptr: none),
   // then max(., 0) when relu != 0
   const int32_t* bias;
@@ -164,9 +173,23 @@ struct TmaView {
 };
 inline bool is_tma_view_variant(int v) {
   return v == B2C_VARIANT_CP_TMA || v == B2C_VARIANT_ROW_UNROLL || v == B2C_VARIANT_SPACE_TO_DEPTH ||
-         v == B2C_VARIANT_DILATION_PACK;
+         v == B2C_VARIANT_DILATION_PACK || v == B2C_VARIANT_CP_SHIFT || v == B2C_VARIANT_S2D_SHIFT;
 }
-constexpr int kNumVariants = 7;
+// The two shift variants execute the channel-pack and space-to-depth views (same rewrite, same
+// packed weights) with the stencil as operand shifts over a staged window instead of one
+// im2col-mode copy per tap.
+inline bool is_shift_variant(int v) { return v == B2C_VARIANT_CP_SHIFT || v == B2C_VARIANT_S2D_SHIFT; }
+inline int shift_base_variant(int v) {
+  return v == B2C_VARIANT_CP_SHIFT ? B2C_VARIANT_CP_TMA : (v == B2C_VARIANT_S2D_SHIFT ? B2C_VARIANT_SPACE_TO_DEPTH : v);
+}
+constexpr int kNumVariants = 9;
+// Shared-memory geometry of the shift execution of a view; false if it does not apply (stride,
+// more than 256 output channels, rows wider than one copy, or window + weights beyond shared memory).
+struct ShiftGeom {
+  int wps, hp, rows, row_bytes, ncb, cb, cblk_bytes, win_bytes, w_bytes, tile_n, blocks_per_sm;
+  long long mtot;
+};
+bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg);
 // Output pixels of the convolution a view describes: the original N*P*Q, except for the dilation
 // phase pack, whose sub-image convolutions also produce rows that map outside the output.
 long long view_rows(const Geom& g, int variant, const TmaView& v);
@@ -189,7 +212,7 @@ inline bool is_swapped(const b2c_embedding& e) { return e.map_m == B2C_AXIS_K; }
 // 128-column exchange tile at most.)
 inline bool cluster_split_ok(int variant, int tile_n, int split_k, bool swap = false) {
   // the swapped map and the phase pack (scattered output rows) meet their partial sums in global memory
-  if (swap || variant == B2C_VARIANT_DILATION_PACK) return false;
+  if (swap || variant == B2C_VARIANT_DILATION_PACK || is_shift_variant(variant)) return false;
   const bool table_in_smem = variant == B2C_VARIANT_IM2COL_GATHER || variant == B2C_VARIANT_IM2COL_STAGED;
   return (split_k == 2 || split_k == 4 || split_k == 8) && tile_n >= 32 * split_k && (!table_in_smem || tile_n <= 128);
 }
@@ -208,6 +231,8 @@ int variant_k_pad(const Geom& g, int variant);  // padded reduction length of th
 // Tensor-map encoders obtained through cudaGetDriverEntryPoint (no link-time libcuda dependency).
 int encode_tiled_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
                     uint32_t box_inner, uint32_t box_outer, int swizzle_bytes);
+int encode_tiled_nhwc_rows(CUtensorMap* map, const void* base, int C_pad, int W, int H, int N, int box_c, int box_w,
+                           int swizzle_bytes);
 int encode_im2col_nhwc(CUtensorMap* map, const void* base, int C_pad, int W, int H, int N, int pad_w, int pad_h,
                        int S, int R, int dil_w, int dil_h, int stride_w, int stride_h, int channels_per_pixel,
                        int pixels_per_column, int swizzle_bytes);

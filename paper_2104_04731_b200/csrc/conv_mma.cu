@@ -130,6 +130,16 @@ __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorM
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_tiled_4d(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n,
+                                                  uint32_t bar, uint32_t on) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %7, 0;\n"
+      "@q cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], "
+      "[%6];\n}" ::"r"(dst),
+      "l"(map), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "r"(on)
+      : "memory");
+}
+
 // Shared-memory operand descriptor for a K-major tile whose rows are `bk` bytes long and stored
 // with the matching 32/64/128-byte swizzle: start address (16-byte units), leading-dimension
 // offset unused for swizzled K-major layouts (set to 1), stride between 8-row groups = 8 * bk
@@ -144,6 +154,13 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, int bk) {
   d |= swz << 61;
   return d;
 }
+
+// A tile may also start at any row of a buffer that TMA filled with the pattern anchored at its
+// natural boundary (1024 / 512 / 256 bytes for the 128 / 64 / 32-byte swizzle): the swizzle is a
+// function of the shared-memory address bits, applied after the row and chunk offsets have been
+// added to the start address, so the same descriptor (base offset 0) with a start address moved by
+// whole rows reads the rows further on.  The shift execution relies on this; its parity tests
+// cover all three swizzle widths.
 
 // Instruction descriptor for kind::i8: D = s32 (code 2 at bit 4), A = B = signed 8-bit (code 1
 // at bits 7 and 10), both operands K-major (no transpose bits), N/8 at bit 17, M/16 at bit 24.
@@ -453,7 +470,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
   const int kb_end = (int)((unsigned)(blockIdx.z + 1) * (unsigned)args.num_kb / (unsigned)args.split_k);
   const int stages = args.stages;
   const int bk = args.bk;
-  const uint32_t a_stage_bytes = kTileM * bk;
+  const uint32_t a_stage_bytes = AMODE == A_SHIFT ? (uint32_t)args.sh_win_bytes : (uint32_t)(kTileM * bk);
   const uint32_t b_stage_bytes = args.tile_n * bk;
 
   // Stage buffers start on a 1024-byte boundary (the 128-byte swizzle repeats every 1024 bytes).
@@ -481,6 +498,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       }
       ctl.abort_flag = 0;
     }
+    if (lane == 11 && AMODE == A_SHIFT) mbar_init(smem_u32(&ctl.full[7]), 1);  // resident weights have landed
     if (lane == 9 && !kThreadsFormA) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
     if (lane == 10) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -517,6 +535,46 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     uint32_t a_dst = a_base, b_dst = b_base;
     const uint32_t leader = elect_one() ? 1u : 0u;
     bool alive = true;
+    if (AMODE == A_SHIFT) {
+      // Resident weights: one box [bk bytes x tile_n channels] per (tap, channel block), once.
+      const uint32_t wfull = smem_u32(&ctl.full[7]);
+      const int taps = args.sh_R * args.S;
+      mbar_arrive_expect_tx(wfull, (uint32_t)args.sh_w_bytes, leader);
+      uint32_t w_dst = b_base;
+      for (int tap = 0; tap < taps; ++tap)
+        for (int cblk = 0; cblk < args.sh_ncb; ++cblk) {
+          tma_load_2d(w_dst, &tmap_b, tap * args.tap_cols + cblk * bk, 0, wfull, leader);
+          w_dst += b_stage_bytes;
+        }
+      // One window per tile: the sh_rows padded image rows from the row that holds the tile's first
+      // position on, each row by one copy per channel block (zeros outside the image).
+      const uint32_t win_tx = (uint32_t)(args.sh_ncb * args.sh_rows * args.sh_row_bytes);
+      for (int t = tile_first; t < tile_end; t += tile_step) {
+        const uint32_t pos0 = (uint32_t)t * kTileM;
+        const uint32_t row0 = args.div_wps.div(pos0);
+        int n = (int)args.div_hp.div(row0);
+        int hp = (int)row0 - n * args.sh_hp;
+        if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) break;
+        const uint32_t full = smem_u32(&ctl.full[s]);
+        mbar_arrive_expect_tx(full, win_tx, leader);
+        uint32_t dst = a_base + s * a_stage_bytes;
+        for (int j = 0; j < args.sh_rows; ++j) {
+          for (int cblk = 0; cblk < args.sh_ncb; ++cblk)
+            tma_load_tiled_4d(dst + cblk * args.sh_cblk_bytes, &tmap_a, cblk * bk, -args.pad_w, hp - args.pad_h, n, full,
+                              leader);
+          dst += args.sh_row_bytes;
+          if (++hp == args.sh_hp) {
+            hp = 0;
+            ++n;
+          }
+        }
+        if (++s == stages) {
+          s = 0;
+          ph ^= 1u;
+        }
+      }
+      alive = false;  // the generic stage loop below is not used
+    }
     for (int t = tile_first; t < tile_end && alive; t += tile_step) {
       B2C_TILE_ORIGIN(t)
       int n_img = 0, h_org = 0, w_org = 0, cb = 0, sx = 0, r = 0;
@@ -589,6 +647,45 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       const uint32_t leader = elect_one() ? 1u : 0u;
       bool alive = true;
       int ti = 0;
+      if (AMODE == A_SHIFT) {
+        // Stencil as operand shift: all taps of a tile are issued from one staged window, the A
+        // descriptor moving (r*dil_h*sh_wps + s*dil_w) pixels per tap, the B descriptor walking the
+        // resident weight tiles.
+        alive = mbar_wait(smem_u32(&ctl.full[7]), 0u, &ctl, args.status);
+        const uint32_t cblk_steps = (uint32_t)(bk / kMmaK);
+        for (int t = tile_first; t < tile_end && alive; t += tile_step, ++ti) {
+          const int buf = ti % nbuf;
+          const uint32_t use = (uint32_t)(ti / nbuf);
+          if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status)) break;
+          if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status)) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t d_tmem = tmem_acc + (uint32_t)(buf * args.tmem_cols);
+          const uint32_t pos0 = (uint32_t)t * kTileM;
+          const uint32_t rel = pos0 - args.div_wps.div(pos0) * (uint32_t)args.sh_wps;
+          const uint32_t a_win = a_base + s * a_stage_bytes + rel * (uint32_t)bk;
+          uint32_t accumulate = 0;
+          uint32_t b_addr = b_base;
+          for (int r = 0; r < args.sh_R; ++r) {
+            uint32_t a_tap = a_win + (uint32_t)(r * args.dil_h * args.sh_wps) * (uint32_t)bk;
+            for (int sx = 0; sx < args.S; ++sx) {
+              for (int cblk = 0; cblk < args.sh_ncb; ++cblk) {
+                mma_i8_block(d_tmem, make_smem_desc(a_tap + (uint32_t)(cblk * args.sh_cblk_bytes), bk),
+                             make_smem_desc(b_addr, bk), idesc, accumulate, leader, (int)cblk_steps);
+                accumulate = 1;
+                b_addr += b_stage_bytes;
+              }
+              a_tap += (uint32_t)(args.dil_w * bk);
+            }
+          }
+          mma_commit(smem_u32(&ctl.empty[s]), leader);
+          mma_commit(smem_u32(&ctl.tmem_full[buf]), leader);
+          if (++s == stages) {
+            s = 0;
+            ph ^= 1u;
+          }
+        }
+        alive = false;  // the generic stage loop below is not used
+      }
       for (int t = tile_first; t < tile_end && alive; t += tile_step, ++ti) {
       const int buf = persistent ? ti % nbuf : 0;
       const uint32_t use = persistent ? (uint32_t)(ti / nbuf) : 0u;
@@ -648,7 +745,15 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     // Where this row's results go: (out_img, out_pq) in the convolution's own output.  The phase
     // pack interleaves the sub-image results back and drops rows that fall outside the output.
     int out_img = n_img, out_pq = pq;
-    if (args.remap && row_valid) {
+    if (args.remap == 2 && row_valid) {
+      // shift execution: row m is window origin (n, hp, wp) on the padded grid of sh_hp x sh_wps positions
+      const uint32_t rowi = args.div_wps.div(m);
+      const int wp = (int)(m - rowi * (uint32_t)args.sh_wps);
+      out_img = (int)args.div_hp.div(rowi);
+      const int hp = (int)rowi - out_img * args.sh_hp;
+      row_valid = hp < args.out_P && wp < args.out_Q;
+      out_pq = hp * args.out_Q + wp;
+    } else if (args.remap && row_valid) {
       const int ps = (int)args.div_q.div((uint32_t)pq), qs = pq - ps * args.Q;
       const int phases = args.ph_dh * args.ph_dw;
       out_img = n_img / phases;
@@ -1040,7 +1145,10 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
   if (args.swap)
     grid = dim3((unsigned)((args.Mg + args.tile_n - 1) / args.tile_n), (unsigned)((args.K + kTileM - 1) / kTileM),
                 (unsigned)args.split_k);
-  if (args.persistent) grid = dim3((unsigned)std::min(args.num_tiles, kNumSMs * (args.persistent == 2 ? 3 : 1)), 1, 1);
+  if (args.persistent) {
+    const int per_sm = args.persistent_blocks_per_sm > 0 ? args.persistent_blocks_per_sm : (args.persistent == 2 ? 3 : 1);
+    grid = dim3((unsigned)std::min(args.num_tiles, kNumSMs * per_sm), 1, 1);
+  }
   cudaError_t e;
 #define B2C_LAUNCH(MODE, PERS)                                                                             \
   {                                                                                                       \
@@ -1061,6 +1169,7 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
   else if (amode == A_IM2COL_TMA && args.persistent == 1) B2C_LAUNCH(A_IM2COL_TMA, 1)
   else if (amode == A_IM2COL_TMA && args.persistent == 2) B2C_LAUNCH(A_IM2COL_TMA, 2)
   else if (amode == A_IM2COL_TMA) B2C_LAUNCH(A_IM2COL_TMA, 0)
+  else if (amode == A_SHIFT) B2C_LAUNCH(A_SHIFT, 2)
   else if (amode == A_STAGED && args.persistent == 2) B2C_LAUNCH(A_STAGED, 2)
   else if (amode == A_STAGED) B2C_LAUNCH(A_STAGED, 0)
   else B2C_LAUNCH(A_GATHER, 0)

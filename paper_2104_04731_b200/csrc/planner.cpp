@@ -76,7 +76,7 @@ size_t workspace_bytes_for(const Geom& g, int variant, int tile_n, int split_k, 
   const b2c_conv_desc& d = g.d;
   TmaView v;
   if (is_tma_view_variant(variant) && tma_view_for(g, variant, &v)) {
-    bool direct = variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && v.C == d.C;
+    bool direct = shift_base_variant(variant) == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && v.C == d.C;
     if (!direct) ws += (size_t)v.bytes();
   } else if (variant == B2C_VARIANT_IM2COL_EXPLICIT) {
     ws += (size_t)g.Mg * im2col_k_pad(g.Kg);
@@ -100,8 +100,42 @@ static bool view_fits_tensor_map(const TmaView& v) {
   return true;
 }
 
+bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg) {
+  if (v.stride_h != 1 || v.stride_w != 1 || g.d.K > 256) return false;
+  const int wp = v.W + 2 * v.pad_w;
+  sg->wps = round_up(wp, 8);
+  sg->hp = v.H + 2 * v.pad_h;
+  if (sg->wps > 256) return false;  // one copy per staged image row
+  sg->cb = cp_block_bytes(v.C);
+  sg->ncb = v.C / sg->cb;
+  const long long shift_max = (long long)(v.R - 1) * v.dil_h * sg->wps + (long long)(v.S - 1) * v.dil_w;
+  // a tile starts anywhere inside its first staged row and reads 128 positions plus the largest shift
+  const long long rows = (sg->wps - 1 + kTileM - 1 + shift_max) / sg->wps + 1;
+  if (rows > 4096) return false;
+  sg->rows = (int)rows;
+  sg->row_bytes = sg->wps * sg->cb;
+  const long long cblk = rows * sg->row_bytes;
+  const long long win = (cblk * sg->ncb + 1023) / 1024 * 1024;
+  int tile_n = 16;
+  while (tile_n < g.d.K) tile_n <<= 1;
+  const long long wbytes = (long long)v.R * v.S * sg->ncb * tile_n * sg->cb;
+  const long long total = 2 * win + wbytes + 2048;
+  if (total > 200 * 1024) return false;
+  sg->cblk_bytes = (int)cblk;
+  sg->win_bytes = (int)win;
+  sg->w_bytes = (int)wbytes;
+  sg->tile_n = tile_n;
+  sg->blocks_per_sm = (int)std::max<long long>(1, std::min<long long>(3, (220 * 1024) / total));
+  sg->mtot = (long long)v.N * sg->hp * sg->wps;
+  return sg->mtot <= 0x7FFFFF00LL;
+}
+
 bool tma_view_for(const Geom& g, int variant, TmaView* v) {
   const b2c_conv_desc& d = g.d;
+  if (is_shift_variant(variant)) {
+    ShiftGeom sg;
+    return tma_view_for(g, shift_base_variant(variant), v) && shift_geom(g, *v, &sg);
+  }
   if (variant == B2C_VARIANT_CP_TMA) {
     // Pad + Split + Reorder of the channel axis (Table 2); an NHWC source must already have a
     // multiple of 32 channels (there is no NHWC re-pad kernel).
@@ -138,6 +172,11 @@ bool tma_view_for(const Geom& g, int variant, TmaView* v) {
 }
 
 long long view_rows(const Geom& g, int variant, const TmaView& v) {
+  if (is_shift_variant(variant)) {
+    // window origins on the padded grid (width rounded up to 8), not only the valid output pixels
+    ShiftGeom sg;
+    return shift_geom(g, v, &sg) ? sg.mtot : g.Mg;
+  }
   if (variant != B2C_VARIANT_DILATION_PACK) return g.Mg;
   return (long long)v.N * (v.H + 2 * v.pad_h - v.R + 1) * (v.W + 2 * v.pad_w - v.S + 1);
 }
@@ -189,13 +228,13 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
   long long data_min = g.x_elems + g.w_elems + g.y_elems;
   TmaView v;
   if (is_tma_view_variant(variant) && tma_view_for(g, variant, &v)) {
-    e.map_k = (variant == B2C_VARIANT_CP_TMA || variant == B2C_VARIANT_DILATION_PACK)
+    e.map_k = (variant == B2C_VARIANT_CP_TMA || variant == B2C_VARIANT_DILATION_PACK || variant == B2C_VARIANT_CP_SHIFT)
                   ? B2C_AXIS_C
                   : (variant == B2C_VARIANT_ROW_UNROLL ? B2C_AXIS_SC : B2C_AXIS_C_PHASES);
     if (!swap) M_pad = (view_rows(g, variant, v) + kTileM - 1) / kTileM * kTileM;
     k_issued = (long long)v.R * v.S * v.C;
     long long packed = v.bytes();
-    bool direct = variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && v.C == d.C;
+    bool direct = shift_base_variant(variant) == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && v.C == d.C;
     moved = (direct ? 0 : g.x_elems + packed) + packed + (long long)d.K * k_issued + g.y_elems;
   } else {
     e.map_k = B2C_AXIS_CRS;
@@ -239,6 +278,12 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
     }
     // The in-kernel gather keeps its lookup table in shared memory.
     if (variant == B2C_VARIANT_IM2COL_GATHER && im2col_k_pad(g.Kg) > 4096) continue;
+    if (is_shift_variant(variant)) {
+      // one schedule: all output channels in one column tile (the weights are resident), no split
+      ShiftGeom sg;
+      if (shift_geom(g, view, &sg)) add(out, g, variant, sg.tile_n, 1);
+      continue;
+    }
     for (int t : tiles) {
       // Skip widths that only add padding: keep t if it is the covering width or K % t == 0
       // or it wastes less than a quarter of the columns.
@@ -256,7 +301,7 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
     // are output channels, so it is only listed when K fills at least half of them; the pixel tile
     // widths are those that waste less than a quarter of their columns (or the covering one).
     if ((is_tma_view_variant(variant) || variant == B2C_VARIANT_IM2COL_EXPLICIT) && d.K >= kTileM / 2 &&
-        variant != B2C_VARIANT_DILATION_PACK) {
+        variant != B2C_VARIANT_DILATION_PACK && !is_shift_variant(variant)) {
       const long long tiles_k = (d.K + kTileM - 1) / kTileM;
       for (int t = 32; t <= 256; t <<= 1) {
         const long long n_pad = (g.Mg + t - 1) / t * t;

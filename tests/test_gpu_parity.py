@@ -69,7 +69,7 @@ def test_config_every_embedding(lib, cfg):
 @pytest.mark.parametrize("in_layout,out_layout", [(1, 1), (0, 1), (1, 0)])
 def test_config_layouts(lib, cfg, in_layout, out_layout):
     x, w, ref = cfg_reference(cfg)
-    for variant in (0, 1, 2, 3, 4, 5, 6):
+    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8):
         d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
                           in_layout, out_layout, 3)
         ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant]
@@ -105,7 +105,7 @@ def test_random_shapes(lib, case):
     ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
     d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode=3)
     embs = lib.enumerate_embeddings(d)
-    for variant in (0, 1, 2, 3, 4, 5, 6):
+    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8):
         ids = [e.id for e in embs if e.variant == variant]
         for i in ids[:1] + ids[-1:]:
             check_against_oracle(x, w, stride, pad, dil, shift, 3, i, ref=ref)
@@ -193,7 +193,7 @@ def test_rewrite_and_convolve_halves(lib):
         seen.add(e.variant)
         plan = lib.Plan(d, e.id)
         data_b, weight_b = plan.footprint()
-        assert weight_b >= w.size and (data_b > 0) == (e.variant in (0, 1, 4, 5))
+        assert weight_b >= w.size and (data_b > 0) == (e.variant in (0, 1, 4, 5, 7, 8))
         assert data_b <= plan.workspace_bytes()
         ws = torch.zeros(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
         y32 = torch.zeros(ref[0].shape, dtype=torch.int32, device="cuda")
@@ -304,12 +304,54 @@ def test_dense_layer_is_a_1x1_convolution(lib, batch, cin, cout):
         assert np.array_equal(y32.reshape(batch, cout), want), (e.variant, e.map_m)
 
 
+# ---- stencil as operand shift (stride-1 views: staged window, resident weights) -------------------------
+@pytest.mark.parametrize("case", [
+    # N, C, H, W, K, R, S, stride, pad, dil, shift
+    (1, 16, 14, 14, 16, 3, 3, 1, 1, 1, 8),           # 32-byte channel block, padded width 16
+    (2, 64, 20, 27, 64, 3, 3, 1, 1, 1, 9),           # 64-byte block, padded width 29 -> 32, tiles cross images
+    (3, 128, 9, 9, 40, 3, 3, 1, 1, 1, 10),           # 128-byte block
+    (1, 160, 11, 13, 24, 3, 2, 1, (2, 0), 1, 10),    # C_pad 160: five 32-byte blocks; asymmetric padding
+    (2, 256, 8, 8, 16, 1, 1, 1, 0, 1, 9),            # 1x1: a single tap, two 128-byte blocks
+    (2, 24, 19, 17, 48, 3, 3, 1, 2, 2, 7),           # dilated: shifts of two rows / two pixels
+    (1, 8, 30, 250, 32, 5, 3, 1, (2, 1), 1, 6),      # wide rows (padded width 252 -> 256): windows of several rows
+    (4, 3, 40, 40, 64, 7, 7, 2, 3, 1, 6),            # stride 2: only through space to depth
+    (2, 1, 33, 61, 32, 9, 21, 2, 0, 1, 5),           # single channel, wide kernel, stride 2
+    (2, 5, 21, 23, 20, 4, 5, (3, 2), (1, 2), 1, 5),  # stride 3 x 2
+])
+@pytest.mark.parametrize("layouts", [(0, 0), (1, 1)])
+def test_shift_execution(lib, case, layouts):
+    N, C, H, W, K, R, S, stride, pad, dil, shift = case
+    in_layout, out_layout = layouts
+    x = int8_uniform((N, C, H, W), 671)
+    w = int8_uniform((K, C, R, S), 672)
+    ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, in_layout, out_layout, 3)
+    shifts = [e for e in lib.enumerate_embeddings(d) if e.variant in (b2c.VARIANT_CP_SHIFT, b2c.VARIANT_S2D_SHIFT)]
+    want = {b2c.VARIANT_S2D_SHIFT} if stride != 1 else {b2c.VARIANT_CP_SHIFT}
+    if in_layout == 1 and C % 32 != 0 and stride == 1:
+        want = set()  # an NHWC source needs padded channels for the channel-pack view
+    assert {e.variant for e in shifts} == want
+    for e in shifts:
+        assert e.split_k == 1 and e.tile_n >= K and e.map_m == b2c.AXIS_NPQ
+        check_against_oracle(x, w, stride, pad, dil, shift, 3, e.id, ref=ref, in_layout=in_layout, out_layout=out_layout)
+
+
+def test_shift_execution_many_tiles(lib):
+    # enough tiles for every block of the persistent grid to walk several, both accumulator buffers in use
+    x = int8_uniform((40, 32, 28, 28), 673)
+    w = int8_uniform((32, 32, 3, 3), 674)
+    ref = oracle.conv2d_int8(x, w, 1, 1, 1, 9)
+    d = lib.make_desc(40, 32, 28, 28, 32, 3, 3, 1, 1, 1, 9, out_mode=3)
+    e = next(e for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_CP_SHIFT)
+    check_against_oracle(x, w, 1, 1, 1, 9, 3, e.id, ref=ref)
+
+
 def test_extreme_values_and_shift_clip(lib):
     # -128 * -128 is the largest product; all-(-128) tensors with 9*64 taps reach 9437184.
     x = np.full((1, 64, 6, 6), -128, dtype=np.int8)
     w = np.full((16, 64, 3, 3), -128, dtype=np.int8)
     ref = oracle.conv2d_int8(x, w, 1, 1, 1, 16)
-    for variant in (0, 1, 2, 3, 4, 5, 6):
+    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8):
         d = lib.make_desc(1, 64, 6, 6, 16, 3, 3, 1, 1, 1, 16, out_mode=3)
         ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant]
         if ids:
