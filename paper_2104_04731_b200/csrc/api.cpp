@@ -248,7 +248,7 @@ void fill_common_args(b2c_plan* p) {
   while (stages > 1 && (size_t)stages * stage_bytes + extra > 196 * 1024) --stages;
   a.cluster_split = cluster_split_ok(p->emb.variant, a.tile_n, a.split_k, a.swap != 0) ? 1 : 0;
   if (p->amode == A_SHIFT) {
-    // two window buffers form the stage ring; the resident weights follow them
+    // the window buffers form the stage ring; the resident weights follow them
     ShiftGeom sg;
     shift_geom(p->g, p->view, &sg);
     a.persistent = 2;
@@ -257,8 +257,8 @@ void fill_common_args(b2c_plan* p) {
     a.num_tiles = (int)((sg.mtot + kTileM - 1) / kTileM);
     a.div_tiles_n = make_fastdiv(1);
     a.num_kb = 1;
-    a.stages = 2;
-    a.stage_region = 2 * sg.win_bytes + sg.w_bytes;
+    a.stages = sg.stages;
+    a.stage_region = sg.stages * sg.win_bytes + sg.w_bytes;
     a.persistent_blocks_per_sm = sg.blocks_per_sm;
     return;
   }

@@ -186,7 +186,7 @@ constexpr int kNumVariants = 9;
 // Shared-memory geometry of the shift execution of a view; false if it does not apply (stride,
 // more than 256 output channels, rows wider than one copy, or window + weights beyond shared memory).
 struct ShiftGeom {
-  int wps, hp, rows, row_bytes, ncb, cb, cblk_bytes, win_bytes, w_bytes, tile_n, blocks_per_sm;
+  int wps, hp, rows, row_bytes, ncb, cb, cblk_bytes, win_bytes, w_bytes, tile_n, stages, blocks_per_sm;
   long long mtot;
 };
 bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg);

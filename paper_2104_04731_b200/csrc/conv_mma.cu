@@ -198,6 +198,37 @@ __device__ __forceinline__ void mma_i8_block(uint32_t d_tmem, uint64_t adesc, ui
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(on), "r"(ksteps)
       : "memory");
 }
+// Up to four MMAs whose descriptors advance by constant steps (one 32-byte slice per tap: the A
+// descriptor moves by the tap's pixel shift, the B descriptor to the next resident weight tile).
+// One asm block, so that predicates and descriptors are formed once and the instructions go out
+// back to back.
+__device__ __forceinline__ void mma_i8_run4(uint32_t d_tmem, uint64_t adesc, uint64_t a_step, uint64_t bdesc,
+                                            uint64_t b_step, uint32_t idesc, uint32_t accumulate, uint32_t on,
+                                            int count) {
+  asm volatile(
+      "{\n"
+      ".reg .pred pacc, ptrue, q0, q1, q2, q3;\n"
+      ".reg .b64 a1, a2, a3, b1, b2, b3;\n"
+      "setp.ne.b32 pacc, %6, 0;\n"
+      "setp.eq.b32 ptrue, 0, 0;\n"
+      "setp.ne.b32 q0, %7, 0;\n"
+      "setp.gt.and.s32 q1, %8, 1, q0;\n"
+      "setp.gt.and.s32 q2, %8, 2, q0;\n"
+      "setp.gt.and.s32 q3, %8, 3, q0;\n"
+      "add.u64 a1, %1, %2;\n"
+      "add.u64 b1, %3, %4;\n"
+      "add.u64 a2, a1, %2;\n"
+      "add.u64 b2, b1, %4;\n"
+      "add.u64 a3, a2, %2;\n"
+      "add.u64 b3, b2, %4;\n"
+      "@q0 tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %3, %5, pacc;\n"
+      "@q1 tcgen05.mma.cta_group::1.kind::i8 [%0], a1, b1, %5, ptrue;\n"
+      "@q2 tcgen05.mma.cta_group::1.kind::i8 [%0], a2, b2, %5, ptrue;\n"
+      "@q3 tcgen05.mma.cta_group::1.kind::i8 [%0], a3, b3, %5, ptrue;\n"
+      "}" ::"r"(d_tmem),
+      "l"(adesc), "l"(a_step), "l"(bdesc), "l"(b_step), "r"(idesc), "r"(accumulate), "r"(on), "r"(count)
+      : "memory");
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar, uint32_t on) {
   asm volatile(
       "{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n"
@@ -653,6 +684,10 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         // resident weight tiles.
         alive = mbar_wait(smem_u32(&ctl.full[7]), 0u, &ctl, args.status);
         const uint32_t cblk_steps = (uint32_t)(bk / kMmaK);
+        const uint64_t a_r_step = (uint64_t)((uint32_t)(args.dil_h * args.sh_wps * bk) >> 4);
+        const uint64_t a_s_step = (uint64_t)((uint32_t)(args.dil_w * bk) >> 4);
+        const uint64_t a_c_step = (uint64_t)((uint32_t)args.sh_cblk_bytes >> 4);
+        const int sh_R = args.sh_R, sh_S = args.S, sh_ncb = args.sh_ncb;  // in registers: the loops below are one thread's dependent chain
         for (int t = tile_first; t < tile_end && alive; t += tile_step, ++ti) {
           const int buf = ti % nbuf;
           const uint32_t use = (uint32_t)(ti / nbuf);
@@ -662,19 +697,39 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
           const uint32_t d_tmem = tmem_acc + (uint32_t)(buf * args.tmem_cols);
           const uint32_t pos0 = (uint32_t)t * kTileM;
           const uint32_t rel = pos0 - args.div_wps.div(pos0) * (uint32_t)args.sh_wps;
-          const uint32_t a_win = a_base + s * a_stage_bytes + rel * (uint32_t)bk;
+          // descriptors advance by address deltas in 16-byte units: per filter row, per tap, per
+          // channel block, per 32-byte slice
+          uint64_t a_row = make_smem_desc(a_base + s * a_stage_bytes + rel * (uint32_t)bk, bk);
+          uint64_t bdesc = bdesc0;
           uint32_t accumulate = 0;
-          uint32_t b_addr = b_base;
-          for (int r = 0; r < args.sh_R; ++r) {
-            uint32_t a_tap = a_win + (uint32_t)(r * args.dil_h * args.sh_wps) * (uint32_t)bk;
-            for (int sx = 0; sx < args.S; ++sx) {
-              for (int cblk = 0; cblk < args.sh_ncb; ++cblk) {
-                mma_i8_block(d_tmem, make_smem_desc(a_tap + (uint32_t)(cblk * args.sh_cblk_bytes), bk),
-                             make_smem_desc(b_addr, bk), idesc, accumulate, leader, (int)cblk_steps);
+          if (sh_ncb == 1 && cblk_steps == 1) {
+            // one MMA per tap: runs of up to four taps of a filter row per asm block
+            for (int r = 0; r < sh_R; ++r) {
+              uint64_t a_tap = a_row;
+              for (int sx = 0; sx < sh_S; sx += 4) {
+                mma_i8_run4(d_tmem, a_tap, a_s_step, bdesc, b_step, idesc, accumulate, leader, sh_S - sx);
                 accumulate = 1;
-                b_addr += b_stage_bytes;
+                a_tap += 4 * a_s_step;
+                bdesc += 4 * b_step;
               }
-              a_tap += (uint32_t)(args.dil_w * bk);
+              bdesc -= (uint64_t)((4 - (sh_S & 3)) & 3) * b_step;  // the last run of a row may be short
+              a_row += a_r_step;
+            }
+          } else {
+            // per tap and channel block: the 32-byte slices of one swizzle row as one asm block
+            for (int r = 0; r < sh_R; ++r) {
+              uint64_t a_tap = a_row;
+              for (int sx = 0; sx < sh_S; ++sx) {
+                uint64_t a_c = a_tap;
+                for (int cblk = 0; cblk < sh_ncb; ++cblk) {
+                  mma_i8_block(d_tmem, a_c, bdesc, idesc, accumulate, leader, (int)cblk_steps);
+                  accumulate = 1;
+                  a_c += a_c_step;
+                  bdesc += b_step;
+                }
+                a_tap += a_s_step;
+              }
+              a_row += a_r_step;
             }
           }
           mma_commit(smem_u32(&ctl.empty[s]), leader);

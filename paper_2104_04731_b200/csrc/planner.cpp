@@ -119,13 +119,23 @@ bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg) {
   int tile_n = 16;
   while (tile_n < g.d.K) tile_n <<= 1;
   const long long wbytes = (long long)v.R * v.S * sg->ncb * tile_n * sg->cb;
-  const long long total = 2 * win + wbytes + 2048;
-  if (total > 200 * 1024) return false;
+  if (2 * win + wbytes + 2048 > 200 * 1024) return false;
   sg->cblk_bytes = (int)cblk;
   sg->win_bytes = (int)win;
   sg->w_bytes = (int)wbytes;
   sg->tile_n = tile_n;
-  sg->blocks_per_sm = (int)std::max<long long>(1, std::min<long long>(3, (220 * 1024) / total));
+  // Window buffers per block and blocks per SM: as many windows in flight per SM as fit (each block
+  // at least two, at most six), preferring more resident blocks on a tie.
+  sg->stages = 2;
+  sg->blocks_per_sm = 1;
+  for (int bps = 3; bps >= 1; --bps) {
+    const long long room = (220 * 1024) / bps - wbytes - 2048;
+    const int st = (int)std::min<long long>(6, std::min<long long>(room, 198 * 1024 - wbytes) / win);
+    if (st >= 2 && st * bps > sg->stages * sg->blocks_per_sm) {
+      sg->stages = st;
+      sg->blocks_per_sm = bps;
+    }
+  }
   sg->mtot = (long long)v.N * sg->hp * sg->wps;
   return sg->mtot <= 0x7FFFFF00LL;
 }
