@@ -470,7 +470,10 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
   extern __shared__ uint8_t smem_raw[];
   __shared__ SharedCtl ctl;
 
-  const int warp = threadIdx.x >> 5;
+  // The warp index is broadcast from lane 0 so that the compiler can prove the role branches below
+  // warp-uniform: inside them, loop counters, barrier addresses and above all the MMA descriptors
+  // can then live in the uniform datapath that the MMA instruction takes its operands from.
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
   // Tile schedule.  Small grids: one tile per block, (blockIdx.x, blockIdx.y) = (row tile, column
   // tile).  Persistent mode (large TMA-fed problems): gridDim.x blocks walk the tile list
@@ -549,7 +552,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_acc = ctl.tmem_base;
+  const uint32_t tmem_acc = __shfl_sync(0xffffffffu, ctl.tmem_base, 0);  // same value in every lane, provably
   // Everything above touched only kernel parameters, shared memory and the plan's constant lookup
   // table.  From here on the block reads tensors earlier kernels of the stream produce and writes
   // tensors they may still read.
@@ -682,7 +685,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         // Stencil as operand shift: all taps of a tile are issued from one staged window, the A
         // descriptor moving (r*dil_h*sh_wps + s*dil_w) pixels per tap, the B descriptor walking the
         // resident weight tiles.
-        alive = mbar_wait(smem_u32(&ctl.full[7]), 0u, &ctl, args.status);
+        alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.full[7]), 0u, &ctl, args.status));
         const uint32_t cblk_steps = (uint32_t)(bk / kMmaK);
         const uint64_t a_r_step = (uint64_t)((uint32_t)(args.dil_h * args.sh_wps * bk) >> 4);
         const uint64_t a_s_step = (uint64_t)((uint32_t)(args.dil_w * bk) >> 4);
@@ -691,8 +694,10 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         for (int t = tile_first; t < tile_end && alive; t += tile_step, ++ti) {
           const int buf = ti % nbuf;
           const uint32_t use = (uint32_t)(ti / nbuf);
-          if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status)) break;
-          if (!mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status)) break;
+          // (votes: the outcome of a wait is the same for all lanes, and saying so keeps the loop's
+          // control flow, and with it the descriptor arithmetic, warp-uniform for the compiler)
+          if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status))) break;
+          if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status))) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t d_tmem = tmem_acc + (uint32_t)(buf * args.tmem_cols);
           const uint32_t pos0 = (uint32_t)t * kTileM;
