@@ -588,7 +588,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         const uint32_t row0 = args.div_wps.div(pos0);
         int n = (int)args.div_hp.div(row0);
         int hp = (int)row0 - n * args.sh_hp;
-        if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) break;
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status))) break;
         const uint32_t full = smem_u32(&ctl.full[s]);
         mbar_arrive_expect_tx(full, win_tx, leader);
         uint32_t dst = a_base + s * a_stage_bytes;
@@ -630,7 +630,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       }
       int kcol = kb_begin * bk;  // column of the packed weight matrix = reduction offset in bytes
       for (int kb = kb_begin; kb < kb_end; ++kb) {
-        if (!mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status)) {
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status))) {
           alive = false;
           break;
         }
@@ -751,14 +751,14 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       const uint32_t use = persistent ? (uint32_t)(ti / nbuf) : 0u;
       if (persistent) {
         // the epilogue must have drained this accumulator buffer (first use passes at once)
-        if (!mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status)) break;
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status))) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       }
       const uint32_t d_tmem = tmem_acc + (uint32_t)(buf * args.tmem_cols);
       uint32_t accumulate = 0;
       bool ready = false;  // result of the look-ahead test of this stage's full barrier
       for (int kb = kb_begin; kb < kb_end; ++kb) {
-        if (!ready && !mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status)) {
+        if (!ready && !__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status))) {
           alive = false;
           break;
         }
@@ -775,7 +775,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
           bdesc = bdesc0;
         }
         // Look ahead: test the next stage's barrier now so that its latency overlaps the MMA issue.
-        ready = (kb + 1 < kb_end) && mbar_test_wait(smem_u32(&ctl.full[s]), ph);
+        ready = (kb + 1 < kb_end) && __all_sync(0xffffffffu, mbar_test_wait(smem_u32(&ctl.full[s]), ph));
         mma_i8_block(d_tmem, a_cur, b_cur, idesc, accumulate, leader, ksteps);
         mma_commit(smem_u32(&ctl.empty[s_cur]), leader);
         if (kb == kb_end - 1) mma_commit(smem_u32(&ctl.tmem_full[buf]), leader);
