@@ -648,10 +648,11 @@ static int run_rewrite(b2c_plan* p, const int8_t* x, void* ws, cudaStream_t st) 
       CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W, 1,
                              d.stride_w, 0, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w, v.C, st));
     } else {
-      // scratch pixel (n, h', w'): window origin (h'*stride_h - pad_h, w'*stride_w - pad_w), channels (c, dh, dw)
-      CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W,
-                             d.stride_h, d.stride_w, d.pad_h, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w,
-                             v.C, st));
+      // space to depth: scratch pixel (n, h', w') holds the stride phases (c, dh, dw) of its window
+      const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
+      CUDA_TRY(launch_space_to_depth(x, scratch, v.N, v.H, v.W, d.C, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
+                                     v.C, a.x_stride_n, nchw ? (long long)d.H * d.W : 1, a.x_stride_h, a.x_stride_w,
+                                     st));
     }
   } else if (p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
     CUDA_TRY(launch_im2col(x, scratch, p->table, g.Mg, g.PQ, g.Q, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,

@@ -251,6 +251,9 @@ cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg
 cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, long long Mg, int PQ, int Q, int H,
                           int W, int stride_h, int stride_w, int pad_h, int pad_w, long long x_stride_n,
                           int x_stride_h, int x_stride_w, int K_pad, cudaStream_t st);
+cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, int Ws, int C, int H, int W, int sh,
+                                  int sw, int pad_h, int pad_w, int C_pad, long long stride_n, long long stride_c,
+                                  int stride_h, int stride_w, cudaStream_t st);
 cudaError_t launch_phase_split(const int8_t* x, int8_t* out, int N, int C, int H, int W, int dh, int dw, int Hs, int Ws,
                                int C_pad, long long stride_n, long long stride_c, int stride_h, int stride_w,
                                cudaStream_t st);

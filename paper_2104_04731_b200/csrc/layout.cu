@@ -3,6 +3,8 @@
 // (reduction index made contiguous, Section 5.1: the B operand is held transposed), the
 // explicit Stencil Unroll (im2col matrix, formed by direct indexing rather than the index-list
 // gather the paper found slow in Section 6.1), and the finish pass of a split reduction.
+#include <algorithm>
+
 #include "b2c_internal.h"
 
 namespace b2c {
@@ -330,6 +332,118 @@ __global__ void __launch_bounds__(256) phase_split_kernel(const int8_t* __restri
   pdl_launch_dependents();
 }
 
+// Image Pack of a strided convolution (space to depth): scratch pixel (n, hs, ws) holds the
+// stride_h x stride_w phases of every channel, out[n][hs][ws][(c*stride_h + dh)*stride_w + dw] =
+// x[n][c][hs*stride_h + dh - pad_h][ws*stride_w + dw - pad_w], zeros outside the image and in the
+// padded channels.  One thread forms 16 consecutive scratch channels of one pixel by direct indexing
+// (running (c, dh, dw) counters, no lookup table) and stores them as one 16-byte vector.
+__global__ void __launch_bounds__(256) space_to_depth_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ out,
+                                                             unsigned total, FastDiv div_chunks, FastDiv div_ws,
+                                                             FastDiv div_hs, int C, int H, int W, int sh, int sw,
+                                                             int pad_h, int pad_w, int C_pad, long long stride_n,
+                                                             int stride_c, int stride_h, int stride_w) {
+  // (32-bit indices and multiply-shift divisions: a 64-bit division costs more than the 16 bytes moved)
+  const int chunks = (int)div_chunks.d, Ws = (int)div_ws.d, Hs = (int)div_hs.d;
+  const int creal = C * sh * sw;
+  const int phases = sh * sw;
+  pdl_wait();
+  for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    const unsigned pix = div_chunks.div(i);
+    const int ck = (int)(i - pix * (unsigned)chunks);
+    uint32_t wv[4] = {0, 0, 0, 0};
+    const int j0 = ck * 16;
+    if (j0 < creal) {
+      const unsigned t = div_ws.div(pix);
+      const int ws = (int)(pix - t * (unsigned)Ws);
+      const unsigned n = div_hs.div(t);
+      const int hs = (int)(t - n * (unsigned)Hs);
+      const int h0 = hs * sh - pad_h, w0 = ws * sw - pad_w;
+      int c = j0 / phases;
+      int rem = j0 - c * phases;
+      int dh = rem / sw, dw = rem - dh * sw;
+      const int8_t* base = x + (long long)n * stride_n;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const int h = h0 + dh, w = w0 + dw;
+        if (c < C && (unsigned)h < (unsigned)H && (unsigned)w < (unsigned)W)
+          wv[e >> 2] |= (uint32_t)(uint8_t)base[c * stride_c + h * stride_h + w * stride_w] << (8 * (e & 3));
+        if (++dw == sw) {
+          dw = 0;
+          if (++dh == sh) {
+            dh = 0;
+            ++c;
+          }
+        }
+      }
+    }
+    *reinterpret_cast<uint4*>(out + (size_t)i * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+  }
+  pdl_launch_dependents();
+}
+
+// Space to depth for NCHW input whose rows are multiples of 16 bytes: one block forms kS2dTile
+// consecutive scratch pixels of one scratch row.  The C*stride_h input row segments those pixels
+// read are first copied to shared memory with aligned 16-byte loads (zeros outside the image), then
+// each thread assembles the bytes of its pixel from shared memory and stores 16-byte vectors.
+constexpr int kS2dTile = 128;
+__global__ void __launch_bounds__(kS2dTile) space_to_depth_rows_kernel(const int8_t* __restrict__ x,
+                                                                       int8_t* __restrict__ out, int Hs, int Ws, int C,
+                                                                       int H, int W, int sh, int sw, int pad_h,
+                                                                       int pad_w, int C_pad, int seg, int ws_tiles) {
+  extern __shared__ __align__(16) uint8_t s2d_rows[];
+  const int tile = blockIdx.x % ws_tiles;
+  const int rowi = blockIdx.x / ws_tiles;  // (n, hs)
+  const int n = rowi / Hs, hs = rowi - n * Hs;
+  const int ws0 = tile * kS2dTile;
+  const int wbeg = ws0 * sw - pad_w;        // first input column of the tile
+  const int walign = wbeg & ~15;            // (two's complement: rounds toward minus infinity)
+  const int rows = C * sh;
+  const int vecs = seg >> 4;
+  pdl_wait();
+  for (int i = threadIdx.x; i < rows * vecs; i += kS2dTile) {
+    const int r = i / vecs, v = i - r * vecs;
+    const int c = r / sh, dh = r - c * sh;
+    const int h = hs * sh + dh - pad_h;
+    const int w = walign + v * 16;
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if ((unsigned)h < (unsigned)H && w >= 0 && w + 16 <= W)
+      val = __ldg(reinterpret_cast<const uint4*>(x + (((size_t)n * C + c) * H + h) * W + w));
+    else if ((unsigned)h < (unsigned)H && w + 16 > 0 && w < W) {
+      uint32_t wv[4] = {0, 0, 0, 0};
+      const int8_t* src = x + (((size_t)n * C + c) * H + h) * W;
+      for (int b = 0; b < 16; ++b)
+        if ((unsigned)(w + b) < (unsigned)W) wv[b >> 2] |= (uint32_t)(uint8_t)src[w + b] << (8 * (b & 3));
+      val = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+    }
+    *reinterpret_cast<uint4*>(s2d_rows + (size_t)r * seg + v * 16) = val;
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+  const int ws = ws0 + threadIdx.x;
+  if (ws >= Ws) return;
+  const int off0 = threadIdx.x * sw + (wbeg - walign);
+  const int creal = C * sh * sw;
+  int8_t* dst = out + (((size_t)n * Hs + hs) * Ws + ws) * C_pad;
+  int c = 0, dh = 0, dw = 0;
+  for (int j0 = 0; j0 < C_pad; j0 += 16) {
+    uint32_t wv[4] = {0, 0, 0, 0};
+    if (j0 < creal) {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        if (c < C) wv[e >> 2] |= (uint32_t)s2d_rows[(c * sh + dh) * seg + off0 + dw] << (8 * (e & 3));
+        if (++dw == sw) {
+          dw = 0;
+          if (++dh == sh) {
+            dh = 0;
+            ++c;
+          }
+        }
+      }
+    }
+    *reinterpret_cast<uint4*>(dst + j0) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+  }
+}
+
 // Finish of a split reduction: the int32 sums are complete in `acc`; copy them out and/or apply
 // the shift-and-clip requantisation (arithmetic shift = floor division by 2^shift).
 __global__ void splitk_finish_kernel(const int32_t* __restrict__ acc, int32_t* __restrict__ y32,
@@ -416,6 +530,33 @@ cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, 
   const long long total = Mg * (K_pad / 16);
   return launch_pdl(im2col_kernel, dim3(grid_for(total, 256)), dim3(256), 0, st, x, a, table, Mg, PQ, Q, H, W, stride_h,
                     stride_w, pad_h, pad_w, x_stride_n, x_stride_h, x_stride_w, K_pad);
+}
+
+cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, int Ws, int C, int H, int W, int sh,
+                                  int sw, int pad_h, int pad_w, int C_pad, long long stride_n, long long stride_c,
+                                  int stride_h, int stride_w, cudaStream_t st) {
+  // Fast path: NCHW rows that are multiples of 16 bytes, row segments of a tile within 48 KB.
+  const int seg = ((kS2dTile * sw + sw + 15 + 15) / 16) * 16;  // bytes of one input row a tile reads, from a 16-byte boundary
+  const long long smem = (long long)C * sh * seg;
+  const long long blocks = (long long)N * Hs * ((Ws + kS2dTile - 1) / kS2dTile);
+  if (stride_w == 1 && stride_h == W && stride_c == (long long)H * W && (W % 16) == 0 &&
+      (reinterpret_cast<uintptr_t>(x) & 15) == 0 && smem <= 48 * 1024 && blocks < 0x7FFFFFFFLL && Ws >= 32)
+    return launch_pdl(space_to_depth_rows_kernel, dim3((unsigned)blocks), dim3(kS2dTile), (size_t)smem, st, x, out, Hs, Ws, C,
+                      H, W, sh, sw, pad_h, pad_w, C_pad, seg, (Ws + kS2dTile - 1) / kS2dTile);
+  // total 16-byte chunks of the scratch tensor; the planner keeps N*Hs*Ws*C_pad below 2^40 and one
+  // image below 2^31 bytes, and the launch below is split so that each part's chunk count fits 32 bits
+  const long long per_image = (long long)Hs * Ws * (C_pad / 16);
+  const int images_per_launch = (int)std::max<long long>(1, std::min<long long>(N, 0x7FFFFFFFLL / per_image));
+  for (int n0 = 0; n0 < N; n0 += images_per_launch) {
+    const int nn = std::min(images_per_launch, N - n0);
+    const long long total = per_image * nn;
+    cudaError_t e = launch_pdl(space_to_depth_kernel, dim3(grid_for(total, 256)), dim3(256), 0, st,
+                               x + (long long)n0 * stride_n, out + (long long)n0 * per_image * 16, (unsigned)total,
+                               make_fastdiv((uint32_t)(C_pad / 16)), make_fastdiv((uint32_t)Ws), make_fastdiv((uint32_t)Hs),
+                               C, H, W, sh, sw, pad_h, pad_w, C_pad, stride_n, (int)stride_c, stride_h, stride_w);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 cudaError_t launch_phase_split(const int8_t* x, int8_t* out, int N, int C, int H, int W, int dh, int dw, int Hs, int Ws,
