@@ -336,6 +336,17 @@ def test_shift_execution(lib, case, layouts):
         check_against_oracle(x, w, stride, pad, dil, shift, 3, e.id, ref=ref, in_layout=in_layout, out_layout=out_layout)
 
 
+def test_shift_execution_long_tile_walk(lib):
+    # about twelve tiles per block of the persistent grid: the window ring and both accumulator
+    # buffers wrap several times (cfg 1's layer at batch 1800)
+    x = int8_uniform((1800, 16, 14, 14), 675)
+    w = int8_uniform((16, 16, 3, 3), 676)
+    ref = oracle.conv2d_int8(x, w, 1, 1, 1, 8)
+    d = lib.make_desc(1800, 16, 14, 14, 16, 3, 3, 1, 1, 1, 8, out_mode=3)
+    e = next(e for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_CP_SHIFT)
+    check_against_oracle(x, w, 1, 1, 1, 8, 3, e.id, ref=ref)
+
+
 def test_shift_execution_many_tiles(lib):
     # enough tiles for every block of the persistent grid to walk several, both accumulator buffers in use
     x = int8_uniform((40, 32, 28, 28), 673)
