@@ -229,6 +229,33 @@ __device__ __forceinline__ void mma_i8_run4(uint32_t d_tmem, uint64_t adesc, uin
       "l"(adesc), "l"(a_step), "l"(bdesc), "l"(b_step), "r"(idesc), "r"(accumulate), "r"(on), "r"(count)
       : "memory");
 }
+// Two taps of a filter row with two 32-byte slices each (64-byte channel blocks): four MMAs in one
+// asm block.  The second tap's descriptors lie a_step / b_step further on; `taps` is 1 or 2.
+__device__ __forceinline__ void mma_i8_pair2(uint32_t d_tmem, uint64_t adesc, uint64_t a_step, uint64_t bdesc,
+                                             uint64_t b_step, uint32_t idesc, uint32_t accumulate, uint32_t on,
+                                             int taps) {
+  asm volatile(
+      "{\n"
+      ".reg .pred pacc, ptrue, q0, q1;\n"
+      ".reg .b64 a1, a2, a3, b1, b2, b3;\n"
+      "setp.ne.b32 pacc, %6, 0;\n"
+      "setp.eq.b32 ptrue, 0, 0;\n"
+      "setp.ne.b32 q0, %7, 0;\n"
+      "setp.gt.and.s32 q1, %8, 1, q0;\n"
+      "add.u64 a1, %1, 2;\n"
+      "add.u64 b1, %3, 2;\n"
+      "add.u64 a2, %1, %2;\n"
+      "add.u64 b2, %3, %4;\n"
+      "add.u64 a3, a2, 2;\n"
+      "add.u64 b3, b2, 2;\n"
+      "@q0 tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %3, %5, pacc;\n"
+      "@q0 tcgen05.mma.cta_group::1.kind::i8 [%0], a1, b1, %5, ptrue;\n"
+      "@q1 tcgen05.mma.cta_group::1.kind::i8 [%0], a2, b2, %5, ptrue;\n"
+      "@q1 tcgen05.mma.cta_group::1.kind::i8 [%0], a3, b3, %5, ptrue;\n"
+      "}" ::"r"(d_tmem),
+      "l"(adesc), "l"(a_step), "l"(bdesc), "l"(b_step), "r"(idesc), "r"(accumulate), "r"(on), "r"(taps)
+      : "memory");
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar, uint32_t on) {
   asm volatile(
       "{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n"
@@ -718,6 +745,19 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
                 bdesc += 4 * b_step;
               }
               bdesc -= (uint64_t)((4 - (sh_S & 3)) & 3) * b_step;  // the last run of a row may be short
+              a_row += a_r_step;
+            }
+          } else if (sh_ncb == 1 && cblk_steps == 2) {
+            // two MMAs per tap: two taps of a filter row per asm block
+            for (int r = 0; r < sh_R; ++r) {
+              uint64_t a_tap = a_row;
+              for (int sx = 0; sx < sh_S; sx += 2) {
+                mma_i8_pair2(d_tmem, a_tap, a_s_step, bdesc, b_step, idesc, accumulate, leader, sh_S - sx);
+                accumulate = 1;
+                a_tap += 2 * a_s_step;
+                bdesc += 2 * b_step;
+              }
+              bdesc -= (uint64_t)(sh_S & 1) * b_step;  // the last pair of a row may be a single tap
               a_row += a_r_step;
             }
           } else {
