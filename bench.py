@@ -144,9 +144,9 @@ class Instances:
         """Kernels of this library per call: layout rewrite (if any) + MMA kernel + split finish (if any)."""
         e, c = self.emb, self.cfg
         n = 1
-        if e.variant in (1, 4, 5, 6, 8) or (e.variant in (0, 7) and not (self.in_layout == 1 and c.C % 32 == 0)):
+        if e.variant in (1, 4, 5, 6, 8, 9) or (e.variant in (0, 7) and not (self.in_layout == 1 and c.C % 32 == 0)):
             n += 1
-        cluster = (e.map_m != 2 and e.variant not in (6, 7, 8) and e.split_k in (2, 4, 8) and e.tile_n >= 32 * e.split_k
+        cluster = (e.map_m != 2 and e.variant not in (6, 7, 8, 9) and e.split_k in (2, 4, 8) and e.tile_n >= 32 * e.split_k
                    and (e.variant in (0, 1, 4, 5) or e.tile_n <= 128))  # the swapped map (map_m = k) and the phase pack never cluster
         if e.split_k > 1 and not cluster and (c.out_mode & 2):
             n += 1  # a split reduction that is not a cluster goes through memory and needs the finish kernel

@@ -83,6 +83,9 @@ typedef struct {
                                       * image rows it needs once, tap (r, s) is the same shared-memory tile read (r*dil_h rows +
                                       * s*dil_w pixels) further on, and the packed weights stay resident in shared memory */
 #define B2C_VARIANT_S2D_SHIFT 8      /* image pack (space to depth) of a strided conv, then the stride-1 remainder as operand shifts */
+#define B2C_VARIANT_ROWPHASE_SHIFT 9 /* low-channel shapes: the kernel row is unrolled into channels together with the vertical
+                                      * stride phases (scratch [N][P + R' - 1][Q][(dh, s, c)], R' = ceil(R / stride_h)); what remains
+                                      * is an R' x 1 stride-1 convolution, executed as operand shifts over 8 x 16-pixel tiles */
 
 typedef struct {
   int32_t id;       /* index in the enumeration for this descriptor; pass to b2c_plan_create      */

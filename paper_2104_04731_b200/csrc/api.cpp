@@ -166,7 +166,7 @@ void fill_common_args(b2c_plan* p) {
     a.S = v.S;
     if (is_shift_variant(p->emb.variant)) {
       ShiftGeom sg;
-      shift_geom(p->g, v, &sg);  // legal: checked when the plan was created
+      shift_geom(p->g, v, &sg, shift_tiles_2d(p->emb.variant));  // legal: checked when the plan was created
       p->amode = A_SHIFT;
       a.Mg = (int)sg.mtot;
       a.sh_mtot = (int)sg.mtot;
@@ -182,6 +182,13 @@ void fill_common_args(b2c_plan* p) {
       a.div_wps = make_fastdiv((uint32_t)sg.wps);
       a.div_hp = make_fastdiv((uint32_t)sg.hp);
       a.remap = 2;
+      if (shift_tiles_2d(p->emb.variant)) {
+        a.remap = 3;
+        a.sh_tiles_h = sg.tiles_h;
+        a.sh_tiles_w = sg.tiles_w;
+        a.div_tiles_hw = make_fastdiv((uint32_t)(sg.tiles_h * sg.tiles_w));
+        a.div_tiles_w = make_fastdiv((uint32_t)sg.tiles_w);
+      }
     }
     if (p->emb.variant == B2C_VARIANT_DILATION_PACK) {
       // the kernel's rows are the pixels of the phase sub-image convolutions
@@ -250,7 +257,7 @@ void fill_common_args(b2c_plan* p) {
   if (p->amode == A_SHIFT) {
     // the window buffers form the stage ring; the resident weights follow them
     ShiftGeom sg;
-    shift_geom(p->g, p->view, &sg);
+    shift_geom(p->g, p->view, &sg, shift_tiles_2d(p->emb.variant));
     a.persistent = 2;
     a.tmem_bufs = 2 * a.tmem_cols <= 512 ? 2 : 1;
     a.tiles_n = 1;
@@ -296,7 +303,19 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
       const long long sw = d.in_layout == B2C_LAYOUT_NCHW ? 1 : d.C;
       std::vector<GatherEntry> t(v.C, GatherEntry{-1, 0, 0});
       std::vector<int32_t> wt((size_t)v.R * v.S * v.C, -1);
-      if (emb.variant == B2C_VARIANT_ROW_UNROLL) {
+      if (emb.variant == B2C_VARIANT_ROWPHASE_SHIFT) {
+        // scratch channel j = (dh*S + s)*C + c; packed weight column (r', j) <- filter tap r = r'*stride_h + dh
+        // (the activation rewrite has a kernel of its own and needs no table)
+        for (int dh = 0; dh < d.stride_h; ++dh)
+          for (int s = 0; s < d.S; ++s)
+            for (int c = 0; c < d.C; ++c) {
+              const int j = (dh * d.S + s) * d.C + c;
+              for (int rp = 0; rp < v.R; ++rp) {
+                const int r = rp * d.stride_h + dh;
+                if (r < d.R) wt[(size_t)rp * v.C + j] = (c * d.R + r) * d.S + s;
+              }
+            }
+      } else if (emb.variant == B2C_VARIANT_ROW_UNROLL) {
         for (int s = 0; s < d.S; ++s)
           for (int c = 0; c < d.C; ++c) {
             const int j = s * d.C + c;
@@ -643,6 +662,11 @@ static int run_rewrite(b2c_plan* p, const int8_t* x, void* ws, cudaStream_t st) 
       const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
       CUDA_TRY(launch_phase_split(x, scratch, d.N, d.C, d.H, d.W, d.dil_h, d.dil_w, v.H, v.W, v.C, a.x_stride_n,
                                   nchw ? (long long)d.H * d.W : 1, a.x_stride_h, a.x_stride_w, st));
+    } else if (base_variant == B2C_VARIANT_ROWPHASE_SHIFT) {
+      const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
+      CUDA_TRY(launch_row_phase_unroll(x, scratch, v.N, v.H, v.W, d.C, d.H, d.W, d.S, d.stride_h, d.stride_w, d.pad_h,
+                                       d.pad_w, d.dil_w, v.C, a.x_stride_n, nchw ? (long long)d.H * d.W : 1,
+                                       a.x_stride_h, a.x_stride_w, st));
     } else if (base_variant == B2C_VARIANT_ROW_UNROLL) {
       // scratch pixel (n, h, q): window origin (h, q*stride_w - pad_w), channels (s, c)
       CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W, 1,
@@ -679,7 +703,7 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
     const TmaView& v = p->view;
     const int8_t* act = p->ws_layout_bytes ? reinterpret_cast<const int8_t*>(wsb) : x;
     if (p->amode == A_SHIFT)
-      rc = encode_tiled_nhwc_rows(&tmap_a, act, v.C, v.W, v.H, v.N, p->bk, a.sh_wps, p->bk);
+      rc = encode_tiled_nhwc_rows(&tmap_a, act, v.C, v.W, v.H, v.N, p->bk, a.sh_wps, p->bk, a.remap == 3 ? a.sh_rows : 1);
     else
       rc = encode_im2col_nhwc(&tmap_a, act, v.C, v.W, v.H, v.N, v.pad_w, v.pad_h, v.S, v.R, v.dil_w, v.dil_h,
                             v.stride_w, v.stride_h, p->bk, a.swap ? a.tile_n : kTileM, p->bk);

@@ -116,6 +116,10 @@ struct ConvArgs {
   // pixels that start (r*dil_h*sh_wps + s*dil_w) pixels further on.  One stage holds sh_rows padded
   // image rows per channel block; the packed weights stay resident in shared memory.
   int sh_wps, sh_hp, sh_rows, sh_row_bytes, sh_ncb, sh_R, sh_cblk_bytes, sh_win_bytes, sh_w_bytes, sh_mtot;
+  // two-dimensional tiles (remap == 3): tile t = (image, tile row, tile column); accumulator row m of
+  // a tile is pixel (m / kShiftTileW, m % kShiftTileW) of it; the window is one box per channel block
+  int sh_tiles_h, sh_tiles_w;
+  FastDiv div_tiles_hw, div_tiles_w;
   int persistent_blocks_per_sm;  // blocks per SM the persistent grid is sized for (0: the mode's default)
   FastDiv div_wps, div_hp;
   // activation step applied to the complete sums before they are written: + bias[k] (nullptr: none),
@@ -173,23 +177,37 @@ struct TmaView {
 };
 inline bool is_tma_view_variant(int v) {
   return v == B2C_VARIANT_CP_TMA || v == B2C_VARIANT_ROW_UNROLL || v == B2C_VARIANT_SPACE_TO_DEPTH ||
-         v == B2C_VARIANT_DILATION_PACK || v == B2C_VARIANT_CP_SHIFT || v == B2C_VARIANT_S2D_SHIFT;
+         v == B2C_VARIANT_DILATION_PACK || v == B2C_VARIANT_CP_SHIFT || v == B2C_VARIANT_S2D_SHIFT ||
+         v == B2C_VARIANT_ROWPHASE_SHIFT;
 }
 // The two shift variants execute the channel-pack and space-to-depth views (same rewrite, same
 // packed weights) with the stencil as operand shifts over a staged window instead of one
 // im2col-mode copy per tap.
-inline bool is_shift_variant(int v) { return v == B2C_VARIANT_CP_SHIFT || v == B2C_VARIANT_S2D_SHIFT; }
+inline bool is_shift_variant(int v) {
+  return v == B2C_VARIANT_CP_SHIFT || v == B2C_VARIANT_S2D_SHIFT || v == B2C_VARIANT_ROWPHASE_SHIFT;
+}
+// The row-phase view has a single tap per filter row, so its tiles can be two-dimensional
+// (kShiftTileH x kShiftTileW output pixels): the window is then one box of
+// (kShiftTileH + R' - 1) x kShiftTileW pixels, tap r' the same tile read r' * kShiftTileW pixels on.
+constexpr int kShiftTileH = 8, kShiftTileW = 16;
+// Row-phase unroll kernel: pixels per block and bytes of one input row segment a block stages
+// (counted from a 16-byte boundary); the C*stride_h segments of a block must fit in shared memory.
+constexpr int kRowPhaseTile = 128;
+constexpr int kRowPhaseSmemMax = 160 * 1024;
+inline int row_phase_seg(int sw, int S, int dil_w) { return ((kRowPhaseTile * sw + (S - 1) * dil_w + 1 + 15 + 15) / 16) * 16; }
+inline bool shift_tiles_2d(int v) { return v == B2C_VARIANT_ROWPHASE_SHIFT; }
 inline int shift_base_variant(int v) {
   return v == B2C_VARIANT_CP_SHIFT ? B2C_VARIANT_CP_TMA : (v == B2C_VARIANT_S2D_SHIFT ? B2C_VARIANT_SPACE_TO_DEPTH : v);
 }
-constexpr int kNumVariants = 9;
+constexpr int kNumVariants = 10;
 // Shared-memory geometry of the shift execution of a view; false if it does not apply (stride,
 // more than 256 output channels, rows wider than one copy, or window + weights beyond shared memory).
 struct ShiftGeom {
   int wps, hp, rows, row_bytes, ncb, cb, cblk_bytes, win_bytes, w_bytes, tile_n, stages, blocks_per_sm;
+  int tiles_h, tiles_w;  // two-dimensional tiles only
   long long mtot;
 };
-bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg);
+bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg, bool tiles_2d = false);
 // Output pixels of the convolution a view describes: the original N*P*Q, except for the dilation
 // phase pack, whose sub-image convolutions also produce rows that map outside the output.
 long long view_rows(const Geom& g, int variant, const TmaView& v);
@@ -232,7 +250,7 @@ int variant_k_pad(const Geom& g, int variant);  // padded reduction length of th
 int encode_tiled_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
                     uint32_t box_inner, uint32_t box_outer, int swizzle_bytes);
 int encode_tiled_nhwc_rows(CUtensorMap* map, const void* base, int C_pad, int W, int H, int N, int box_c, int box_w,
-                           int swizzle_bytes);
+                           int swizzle_bytes, int box_h = 1);
 int encode_im2col_nhwc(CUtensorMap* map, const void* base, int C_pad, int W, int H, int N, int pad_w, int pad_h,
                        int S, int R, int dil_w, int dil_h, int stride_w, int stride_h, int channels_per_pixel,
                        int pixels_per_column, int swizzle_bytes);
@@ -254,6 +272,9 @@ cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, 
 cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, int Ws, int C, int H, int W, int sh,
                                   int sw, int pad_h, int pad_w, int C_pad, long long stride_n, long long stride_c,
                                   int stride_h, int stride_w, cudaStream_t st);
+cudaError_t launch_row_phase_unroll(const int8_t* x, int8_t* out, int N, int Hs, int Q, int C, int H, int W, int S, int sh,
+                                    int sw, int pad_h, int pad_w, int dil_w, int C_pad, long long stride_n,
+                                    long long stride_c, int stride_h, int stride_w, cudaStream_t st);
 cudaError_t launch_phase_split(const int8_t* x, int8_t* out, int N, int C, int H, int W, int dh, int dw, int Hs, int Ws,
                                int C_pad, long long stride_n, long long stride_c, int stride_h, int stride_w,
                                cudaStream_t st);

@@ -619,6 +619,16 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         const uint32_t full = smem_u32(&ctl.full[s]);
         mbar_arrive_expect_tx(full, win_tx, leader);
         uint32_t dst = a_base + s * a_stage_bytes;
+        if (args.remap == 3) {
+          // two-dimensional tile (image, tile row, tile column): the window is one box of sh_rows rows
+          // of 16 pixels per channel block
+          const int img = (int)args.div_tiles_hw.div((uint32_t)t);
+          const int rem = t - img * (args.sh_tiles_h * args.sh_tiles_w);
+          const int th = (int)args.div_tiles_w.div((uint32_t)rem), tw = rem - th * args.sh_tiles_w;
+          for (int cblk = 0; cblk < args.sh_ncb; ++cblk)
+            tma_load_tiled_4d(dst + cblk * args.sh_cblk_bytes, &tmap_a, cblk * bk, tw * kShiftTileW, th * kShiftTileH, img,
+                              full, leader);
+        } else
         for (int j = 0; j < args.sh_rows; ++j) {
           for (int cblk = 0; cblk < args.sh_ncb; ++cblk)
             tma_load_tiled_4d(dst + cblk * args.sh_cblk_bytes, &tmap_a, cblk * bk, -args.pad_w, hp - args.pad_h, n, full,
@@ -715,9 +725,12 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.full[7]), 0u, &ctl, args.status));
         const uint32_t cblk_steps = (uint32_t)(bk / kMmaK);
         const uint64_t a_r_step = (uint64_t)((uint32_t)(args.dil_h * args.sh_wps * bk) >> 4);
-        const uint64_t a_s_step = (uint64_t)((uint32_t)(args.dil_w * bk) >> 4);
+        const uint64_t a_s_step = args.S == 1 ? a_r_step : (uint64_t)((uint32_t)(args.dil_w * bk) >> 4);
         const uint64_t a_c_step = (uint64_t)((uint32_t)args.sh_cblk_bytes >> 4);
-        const int sh_R = args.sh_R, sh_S = args.S, sh_ncb = args.sh_ncb;  // in registers: the loops below are one thread's dependent chain
+        // (in registers: the loops below are one thread's dependent chain.  A view with one tap per
+        // filter row walks its rows as the taps of a single run, so that they share asm blocks.)
+        const bool rows_as_taps = args.S == 1;
+        const int sh_R = rows_as_taps ? 1 : args.sh_R, sh_S = rows_as_taps ? args.sh_R : args.S, sh_ncb = args.sh_ncb;
         for (int t = tile_first; t < tile_end && alive; t += tile_step, ++ti) {
           const int buf = ti % nbuf;
           const uint32_t use = (uint32_t)(ti / nbuf);
@@ -845,7 +858,16 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     // Where this row's results go: (out_img, out_pq) in the convolution's own output.  The phase
     // pack interleaves the sub-image results back and drops rows that fall outside the output.
     int out_img = n_img, out_pq = pq;
-    if (args.remap == 2 && row_valid) {
+    if (args.remap == 3 && row_valid) {
+      // two-dimensional tiles: tile (image, tile row, tile column), row = pixel (row / 16, row % 16) of it
+      const uint32_t tile = (uint32_t)m0 / kTileM;
+      out_img = (int)args.div_tiles_hw.div(tile);
+      const int rem = (int)tile - out_img * (args.sh_tiles_h * args.sh_tiles_w);
+      const int th = (int)args.div_tiles_w.div((uint32_t)rem), tw = rem - th * args.sh_tiles_w;
+      const int po = th * kShiftTileH + row / kShiftTileW, qo = tw * kShiftTileW + row % kShiftTileW;
+      row_valid = po < args.out_P && qo < args.out_Q;
+      out_pq = po * args.out_Q + qo;
+    } else if (args.remap == 2 && row_valid) {
       // shift execution: row m is window origin (n, hp, wp) on the padded grid of sh_hp x sh_wps positions
       const uint32_t rowi = args.div_wps.div(m);
       const int wp = (int)(m - rowi * (uint32_t)args.sh_wps);

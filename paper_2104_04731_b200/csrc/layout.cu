@@ -444,6 +444,86 @@ __global__ void __launch_bounds__(kS2dTile) space_to_depth_rows_kernel(const int
   }
 }
 
+// Row-phase unroll: scratch pixel (n, hs, q) holds, for every vertical stride phase dh, tap s and
+// channel c, out[n][hs][q][(dh*S + s)*C + c] = x[n][c][hs*stride_h + dh - pad_h][q*stride_w - pad_w + s*dil_w]
+// (zeros outside the image and in the padded channels).  One block forms kS2dTile consecutive pixels
+// of one scratch row: the C*stride_h input row segments they read are staged in shared memory
+// (aligned 16-byte loads where the layout allows, byte loads otherwise), then each thread assembles
+// its pixel's bytes from there and stores 16-byte vectors.
+__global__ void __launch_bounds__(kS2dTile) row_phase_unroll_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ out,
+                                                                    int Hs, int Q, int C, int H, int W, int S, int sh,
+                                                                    int sw, int pad_h, int pad_w, int dil_w, int C_pad,
+                                                                    int seg, int q_tiles, long long stride_n,
+                                                                    long long stride_c, int stride_h, int stride_w,
+                                                                    int vec_ok) {
+  extern __shared__ __align__(16) uint8_t rp_rows[];
+  const int tile = blockIdx.x % q_tiles;
+  const int rowi = blockIdx.x / q_tiles;  // (n, hs)
+  const int n = rowi / Hs, hs = rowi - n * Hs;
+  const int q0 = tile * kS2dTile;
+  const int wbeg = q0 * sw - pad_w;  // first input column the tile reads
+  const int walign = wbeg & ~15;     // rounds toward minus infinity
+  const int rows = C * sh;
+  const int8_t* xn = x + (size_t)n * stride_n;
+  pdl_wait();
+  if (vec_ok) {
+    const int vecs = seg >> 4;
+    for (int i = threadIdx.x; i < rows * vecs; i += kS2dTile) {
+      const int r = i / vecs, v = i - r * vecs;
+      const int c = r / sh, dh = r - c * sh;
+      const int h = hs * sh + dh - pad_h;
+      const int w = walign + v * 16;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if ((unsigned)h < (unsigned)H && w >= 0 && w + 16 <= W) {
+        val = __ldg(reinterpret_cast<const uint4*>(xn + c * stride_c + (long long)h * stride_h + w));
+      } else if ((unsigned)h < (unsigned)H && w + 16 > 0 && w < W) {
+        uint32_t wv[4] = {0, 0, 0, 0};
+        const int8_t* src = xn + c * stride_c + (long long)h * stride_h;
+        for (int b = 0; b < 16; ++b)
+          if ((unsigned)(w + b) < (unsigned)W) wv[b >> 2] |= (uint32_t)(uint8_t)src[w + b] << (8 * (b & 3));
+        val = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+      }
+      *reinterpret_cast<uint4*>(rp_rows + (size_t)r * seg + v * 16) = val;
+    }
+  } else {
+    for (int i = threadIdx.x; i < rows * seg; i += kS2dTile) {
+      const int r = i / seg, b = i - r * seg;
+      const int c = r / sh, dh = r - c * sh;
+      const int h = hs * sh + dh - pad_h;
+      const int w = walign + b;
+      uint8_t val = 0;
+      if ((unsigned)h < (unsigned)H && (unsigned)w < (unsigned)W)
+        val = (uint8_t)xn[c * stride_c + (long long)h * stride_h + (long long)w * stride_w];
+      rp_rows[(size_t)r * seg + b] = val;
+    }
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+  const int q = q0 + threadIdx.x;
+  if (q >= Q) return;
+  const int off0 = threadIdx.x * sw + (wbeg - walign);
+  const int creal = sh * S * C;
+  int8_t* dst = out + (((size_t)n * Hs + hs) * Q + q) * C_pad;
+  int dh = 0, s = 0, c = 0;
+  for (int j0 = 0; j0 < C_pad; j0 += 16) {
+    uint32_t wv[4] = {0, 0, 0, 0};
+    if (j0 < creal) {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        if (dh < sh) wv[e >> 2] |= (uint32_t)rp_rows[(c * sh + dh) * seg + off0 + s * dil_w] << (8 * (e & 3));
+        if (++c == C) {
+          c = 0;
+          if (++s == S) {
+            s = 0;
+            ++dh;
+          }
+        }
+      }
+    }
+    *reinterpret_cast<uint4*>(dst + j0) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+  }
+}
+
 // Finish of a split reduction: the int32 sums are complete in `acc`; copy them out and/or apply
 // the shift-and-clip requantisation (arithmetic shift = floor division by 2^shift).
 __global__ void splitk_finish_kernel(const int32_t* __restrict__ acc, int32_t* __restrict__ y32,
@@ -557,6 +637,30 @@ cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, i
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
+}
+
+cudaError_t launch_row_phase_unroll(const int8_t* x, int8_t* out, int N, int Hs, int Q, int C, int H, int W, int S, int sh,
+                                    int sw, int pad_h, int pad_w, int dil_w, int C_pad, long long stride_n,
+                                    long long stride_c, int stride_h, int stride_w, cudaStream_t st) {
+  // bytes of one input row a tile of kS2dTile pixels reads, counted from a 16-byte boundary
+  static_assert(kRowPhaseTile == kS2dTile, "one pixel per thread");
+  const int seg = row_phase_seg(sw, S, dil_w);
+  const long long smem = (long long)C * sh * seg;
+  const int q_tiles = (Q + kS2dTile - 1) / kS2dTile;
+  const long long blocks = (long long)N * Hs * q_tiles;
+  if (smem > kRowPhaseSmemMax || blocks >= 0x7FFFFFFFLL) return cudaErrorInvalidValue;
+  const int vec_ok = (stride_w == 1 && (stride_h % 16) == 0 && (stride_c % 16) == 0 && (stride_n % 16) == 0 &&
+                      (reinterpret_cast<uintptr_t>(x) & 15) == 0)
+                         ? 1
+                         : 0;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(row_phase_unroll_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowPhaseSmemMax);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  return launch_pdl(row_phase_unroll_kernel, dim3((unsigned)blocks), dim3(kS2dTile), (size_t)smem, st, x, out, Hs, Q, C, H,
+                    W, S, sh, sw, pad_h, pad_w, dil_w, C_pad, seg, q_tiles, stride_n, stride_c, stride_h, stride_w, vec_ok);
 }
 
 cudaError_t launch_phase_split(const int8_t* x, int8_t* out, int N, int C, int H, int W, int dh, int dw, int Hs, int Ws,

@@ -100,18 +100,32 @@ static bool view_fits_tensor_map(const TmaView& v) {
   return true;
 }
 
-bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg) {
+bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg, bool tiles_2d) {
   if (v.stride_h != 1 || v.stride_w != 1 || g.d.K > 256) return false;
-  const int wp = v.W + 2 * v.pad_w;
-  sg->wps = round_up(wp, 8);
-  sg->hp = v.H + 2 * v.pad_h;
-  if (sg->wps > 256) return false;  // one copy per staged image row
   sg->cb = cp_block_bytes(v.C);
   sg->ncb = v.C / sg->cb;
-  const long long shift_max = (long long)(v.R - 1) * v.dil_h * sg->wps + (long long)(v.S - 1) * v.dil_w;
-  // a tile starts anywhere inside its first staged row and reads 128 positions plus the largest shift
-  const long long rows = (sg->wps - 1 + kTileM - 1 + shift_max) / sg->wps + 1;
-  if (rows > 4096) return false;
+  sg->tiles_h = sg->tiles_w = 0;
+  long long rows;
+  if (tiles_2d) {
+    // 8 x 16-pixel tiles over an unpadded view with one tap per filter row: the window is one box of
+    // (8 + R - 1) rows of 16 pixels, and a tap moves the tile by one row of 16 pixels
+    if (v.S != 1 || v.pad_h != 0 || v.pad_w != 0 || v.dil_h != 1) return false;
+    sg->wps = kShiftTileW;
+    sg->hp = v.H;
+    rows = kShiftTileH + v.R - 1;
+    if (rows > 256) return false;
+    sg->tiles_h = (g.P + kShiftTileH - 1) / kShiftTileH;
+    sg->tiles_w = (g.Q + kShiftTileW - 1) / kShiftTileW;
+  } else {
+    const int wp = v.W + 2 * v.pad_w;
+    sg->wps = round_up(wp, 8);
+    sg->hp = v.H + 2 * v.pad_h;
+    if (sg->wps > 256) return false;  // one copy per staged image row
+    const long long shift_max = (long long)(v.R - 1) * v.dil_h * sg->wps + (long long)(v.S - 1) * v.dil_w;
+    // a tile starts anywhere inside its first staged row and reads 128 positions plus the largest shift
+    rows = (sg->wps - 1 + kTileM - 1 + shift_max) / sg->wps + 1;
+    if (rows > 4096) return false;
+  }
   sg->rows = (int)rows;
   sg->row_bytes = sg->wps * sg->cb;
   const long long cblk = rows * sg->row_bytes;
@@ -136,12 +150,25 @@ bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg) {
       sg->blocks_per_sm = bps;
     }
   }
-  sg->mtot = (long long)v.N * sg->hp * sg->wps;
+  sg->mtot = tiles_2d ? (long long)v.N * sg->tiles_h * sg->tiles_w * kTileM : (long long)v.N * sg->hp * sg->wps;
   return sg->mtot <= 0x7FFFFF00LL;
 }
 
 bool tma_view_for(const Geom& g, int variant, TmaView* v) {
   const b2c_conv_desc& d = g.d;
+  if (variant == B2C_VARIANT_ROWPHASE_SHIFT) {
+    // Stencil Unroll along s and Image Pack of the vertical stride in one rewrite:
+    // U[n][h'][q][(dh, s, c)] = x[n][c][h'*stride_h + dh - pad_h][q*stride_w - pad_w + s*dil_w], and an
+    // R' x 1, stride-1, unpadded convolution over U remains (r = r'*stride_h + dh).
+    if (d.dil_h != 1) return false;
+    const int Rp = (d.R + d.stride_h - 1) / d.stride_h;
+    const long long cq = (long long)d.stride_h * d.S * d.C;
+    if (cq > 4096) return false;
+    if ((long long)d.C * d.stride_h * row_phase_seg(d.stride_w, d.S, d.dil_w) > kRowPhaseSmemMax) return false;
+    *v = TmaView{d.N, round_up((int)cq, kMmaK), g.P + Rp - 1, g.Q, Rp, 1, 1, 1, 0, 0, 1, 1};
+    ShiftGeom sg;
+    return view_fits_tensor_map(*v) && shift_geom(g, *v, &sg, true);
+  }
   if (is_shift_variant(variant)) {
     ShiftGeom sg;
     return tma_view_for(g, shift_base_variant(variant), v) && shift_geom(g, *v, &sg);
@@ -185,7 +212,7 @@ long long view_rows(const Geom& g, int variant, const TmaView& v) {
   if (is_shift_variant(variant)) {
     // window origins on the padded grid (width rounded up to 8), not only the valid output pixels
     ShiftGeom sg;
-    return shift_geom(g, v, &sg) ? sg.mtot : g.Mg;
+    return shift_geom(g, v, &sg, shift_tiles_2d(variant)) ? sg.mtot : g.Mg;
   }
   if (variant != B2C_VARIANT_DILATION_PACK) return g.Mg;
   return (long long)v.N * (v.H + 2 * v.pad_h - v.R + 1) * (v.W + 2 * v.pad_w - v.S + 1);
@@ -240,7 +267,8 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
   if (is_tma_view_variant(variant) && tma_view_for(g, variant, &v)) {
     e.map_k = (variant == B2C_VARIANT_CP_TMA || variant == B2C_VARIANT_DILATION_PACK || variant == B2C_VARIANT_CP_SHIFT)
                   ? B2C_AXIS_C
-                  : (variant == B2C_VARIANT_ROW_UNROLL ? B2C_AXIS_SC : B2C_AXIS_C_PHASES);
+                  : ((variant == B2C_VARIANT_ROW_UNROLL || variant == B2C_VARIANT_ROWPHASE_SHIFT) ? B2C_AXIS_SC
+                                                                                                  : B2C_AXIS_C_PHASES);
     if (!swap) M_pad = (view_rows(g, variant, v) + kTileM - 1) / kTileM * kTileM;
     k_issued = (long long)v.R * v.S * v.C;
     long long packed = v.bytes();
@@ -291,7 +319,7 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
     if (is_shift_variant(variant)) {
       // one schedule: all output channels in one column tile (the weights are resident), no split
       ShiftGeom sg;
-      if (shift_geom(g, view, &sg)) add(out, g, variant, sg.tile_n, 1);
+      if (shift_geom(g, view, &sg, shift_tiles_2d(variant))) add(out, g, variant, sg.tile_n, 1);
       continue;
     }
     for (int t : tiles) {

@@ -98,7 +98,7 @@ int encode_im2col_nhwc(CUtensorMap* map, const void* base, int C_pad, int W, int
 // copy fetches `box_c` channel bytes of `box_w` consecutive pixels of one image row; pixels left or
 // right of the row, rows above or below the image and images past the batch read as zeros.
 int encode_tiled_nhwc_rows(CUtensorMap* map, const void* base, int C_pad, int W, int H, int N, int box_c, int box_w,
-                           int swizzle_bytes) {
+                           int swizzle_bytes, int box_h) {
   std::call_once(g_once, resolve);
   if (!g_tiled) {
     set_last_cuda_error((int)CUDA_ERROR_NOT_FOUND);
@@ -106,7 +106,7 @@ int encode_tiled_nhwc_rows(CUtensorMap* map, const void* base, int C_pad, int W,
   }
   cuuint64_t dims[4] = {(cuuint64_t)C_pad, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
   cuuint64_t strides[3] = {(cuuint64_t)C_pad, (cuuint64_t)C_pad * W, (cuuint64_t)C_pad * W * H};
-  cuuint32_t box[4] = {(cuuint32_t)box_c, (cuuint32_t)box_w, 1, 1};
+  cuuint32_t box[4] = {(cuuint32_t)box_c, (cuuint32_t)box_w, (cuuint32_t)box_h, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = g_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(swizzle_bytes), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,

@@ -69,7 +69,7 @@ def test_config_every_embedding(lib, cfg):
 @pytest.mark.parametrize("in_layout,out_layout", [(1, 1), (0, 1), (1, 0)])
 def test_config_layouts(lib, cfg, in_layout, out_layout):
     x, w, ref = cfg_reference(cfg)
-    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8):
+    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8, 9):
         d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
                           in_layout, out_layout, 3)
         ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant]
@@ -105,7 +105,7 @@ def test_random_shapes(lib, case):
     ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
     d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode=3)
     embs = lib.enumerate_embeddings(d)
-    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8):
+    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8, 9):
         ids = [e.id for e in embs if e.variant == variant]
         for i in ids[:1] + ids[-1:]:
             check_against_oracle(x, w, stride, pad, dil, shift, 3, i, ref=ref)
@@ -193,7 +193,7 @@ def test_rewrite_and_convolve_halves(lib):
         seen.add(e.variant)
         plan = lib.Plan(d, e.id)
         data_b, weight_b = plan.footprint()
-        assert weight_b >= w.size and (data_b > 0) == (e.variant in (0, 1, 4, 5, 7, 8))
+        assert weight_b >= w.size and (data_b > 0) == (e.variant in (0, 1, 4, 5, 7, 8, 9))
         assert data_b <= plan.workspace_bytes()
         ws = torch.zeros(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
         y32 = torch.zeros(ref[0].shape, dtype=torch.int32, device="cuda")
@@ -336,6 +336,32 @@ def test_shift_execution(lib, case, layouts):
         check_against_oracle(x, w, stride, pad, dil, shift, 3, e.id, ref=ref, in_layout=in_layout, out_layout=out_layout)
 
 
+@pytest.mark.parametrize("case", [
+    # N, C, H, W, K, R, S, stride, pad, dil, shift
+    (4, 3, 40, 48, 64, 7, 7, 2, 3, 1, 6),              # the low-channel 7x7 stride-2 class: (dh, s, c) = 42 -> 64 channels
+    (2, 1, 33, 64, 32, 9, 21, 2, 0, 1, 5),             # single channel, wide kernel: 42 -> 64, five filter rows left
+    (2, 1, 30, 61, 32, 9, 21, (2, 2), (1, 3), 1, 5),   # rows not a multiple of 16 bytes: byte staging
+    (3, 5, 21, 23, 20, 4, 5, (3, 2), (1, 2), (1, 2), 5),   # stride 3 x 2, horizontal dilation 2, ragged tiles
+    (1, 16, 14, 14, 16, 3, 3, 1, 1, 1, 8),             # stride 1: plain row unroll, 48 -> 64 channels
+    (2, 40, 12, 12, 24, 3, 3, (2, 1), 1, 1, 8),        # 2 * 3 * 40 = 240 -> 256 channels: two 128-byte blocks
+    (1, 2, 70, 9, 8, 5, 2, (1, 1), (2, 0), 1, 4),      # tall image: many tile rows, one tile column
+])
+@pytest.mark.parametrize("layouts", [(0, 0), (1, 1)])
+def test_row_phase_unroll_shift(lib, case, layouts):
+    N, C, H, W, K, R, S, stride, pad, dil, shift = case
+    in_layout, out_layout = layouts
+    x = int8_uniform((N, C, H, W), 681)
+    w = int8_uniform((K, C, R, S), 682)
+    ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, in_layout, out_layout, 3)
+    es = [e for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_ROWPHASE_SHIFT]
+    assert len(es) == 1 and es[0].map_k == b2c.AXIS_SC and es[0].split_k == 1 and es[0].workspace_bytes > 0
+    check_against_oracle(x, w, stride, pad, dil, shift, 3, es[0].id, ref=ref, in_layout=in_layout, out_layout=out_layout)
+    # vertical dilation is outside this rewrite
+    d2 = lib.make_desc(N, C, H + 8, W, K, R, S, stride, pad, (2, 1), shift)
+    assert all(e.variant != b2c.VARIANT_ROWPHASE_SHIFT for e in lib.enumerate_embeddings(d2))
+
+
 def test_shift_execution_long_tile_walk(lib):
     # about twelve tiles per block of the persistent grid: the window ring and both accumulator
     # buffers wrap several times (cfg 1's layer at batch 1800)
@@ -362,7 +388,7 @@ def test_extreme_values_and_shift_clip(lib):
     x = np.full((1, 64, 6, 6), -128, dtype=np.int8)
     w = np.full((16, 64, 3, 3), -128, dtype=np.int8)
     ref = oracle.conv2d_int8(x, w, 1, 1, 1, 16)
-    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8):
+    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8, 9):
         d = lib.make_desc(1, 64, 6, 6, 16, 3, 3, 1, 1, 1, 16, out_mode=3)
         ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant]
         if ids:
