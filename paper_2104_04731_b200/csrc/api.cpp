@@ -558,11 +558,11 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
   // fastest is kept).  All schedules of the five lowest-overhead (axis map, layout variant)
   // groups are run on scratch tensors.
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  // (A shift variant belongs to the group of the view it executes: same rewrite, same weights.)
+  // (Variants of one family count as one candidate: a view and its shift execution, the row unrolls.)
   std::vector<int> groups;
   for (const b2c_embedding& e : all)
-    if (std::find(groups.begin(), groups.end(), shift_base_variant(e.variant)) == groups.end() && groups.size() < 5)
-      groups.push_back(shift_base_variant(e.variant));
+    if (std::find(groups.begin(), groups.end(), variant_family(e.variant)) == groups.end() && groups.size() < 5)
+      groups.push_back(variant_family(e.variant));
   size_t ws_max = 0;
   for (const b2c_embedding& e : all) ws_max = std::max(ws_max, (size_t)e.workspace_bytes);
   int8_t *x = nullptr, *w = nullptr;
@@ -592,7 +592,7 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
   int best = -1;
   float best_us = 0;
   for (size_t i = 0; i < all.size(); ++i) {
-    if (std::find(groups.begin(), groups.end(), shift_base_variant(all[i].variant)) == groups.end()) continue;
+    if (std::find(groups.begin(), groups.end(), variant_family(all[i].variant)) == groups.end()) continue;
     b2c_plan* p = nullptr;
     rc = create_plan_for(g, all[i], &p);
     if (rc != B2C_OK) break;

@@ -200,6 +200,13 @@ inline int shift_base_variant(int v) {
   return v == B2C_VARIANT_CP_SHIFT ? B2C_VARIANT_CP_TMA : (v == B2C_VARIANT_S2D_SHIFT ? B2C_VARIANT_SPACE_TO_DEPTH : v);
 }
 constexpr int kNumVariants = 10;
+// Family of a variant for the timed selection's "five best candidates": variants that share the
+// kind of rewrite (a view and its shift execution; row unroll with and without the stride phases)
+// count as one candidate with several schedules.
+inline int variant_family(int v) {
+  if (v == B2C_VARIANT_ROWPHASE_SHIFT) return B2C_VARIANT_ROW_UNROLL;
+  return shift_base_variant(v);
+}
 // Shared-memory geometry of the shift execution of a view; false if it does not apply (stride,
 // more than 256 output channels, rows wider than one copy, or window + weights beyond shared memory).
 struct ShiftGeom {
