@@ -117,7 +117,7 @@ struct ConvArgs {
   // image rows per channel block; the packed weights stay resident in shared memory.
   int sh_wps, sh_hp, sh_rows, sh_row_bytes, sh_ncb, sh_R, sh_cblk_bytes, sh_win_bytes, sh_w_bytes, sh_mtot;
   // two-dimensional tiles (remap == 3): tile t = (image, tile row, tile column); accumulator row m of
-  // a tile is pixel (m / kShiftTileW, m % kShiftTileW) of it; the window is one box per channel block
+  // a tile is pixel (m / tile_w, m % tile_w) of it (tile_w = sh_wps); the window is one box per channel block
   int sh_tiles_h, sh_tiles_w;
   FastDiv div_tiles_hw, div_tiles_w;
   int persistent_blocks_per_sm;  // blocks per SM the persistent grid is sized for (0: the mode's default)
@@ -187,9 +187,10 @@ inline bool is_shift_variant(int v) {
   return v == B2C_VARIANT_CP_SHIFT || v == B2C_VARIANT_S2D_SHIFT || v == B2C_VARIANT_ROWPHASE_SHIFT;
 }
 // The row-phase view has a single tap per filter row, so its tiles can be two-dimensional
-// (kShiftTileH x kShiftTileW output pixels): the window is then one box of
-// (kShiftTileH + R' - 1) x kShiftTileW pixels, tap r' the same tile read r' * kShiftTileW pixels on.
-constexpr int kShiftTileH = 8, kShiftTileW = 16;
+// (tile_h x tile_w output pixels, tile_w a power of two from kShiftTileW to 128, tile_h = 128 / tile_w):
+// the window is then one box of (tile_h + R' - 1) x tile_w pixels, tap r' the same tile read r' * tile_w
+// pixels on.
+constexpr int kShiftTileW = 16;
 // Row-phase unroll kernel: pixels per block and bytes of one input row segment a block stages
 // (counted from a 16-byte boundary); the C*stride_h segments of a block must fit in shared memory.
 constexpr int kRowPhaseTile = 128;

@@ -626,7 +626,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
           const int rem = t - img * (args.sh_tiles_h * args.sh_tiles_w);
           const int th = (int)args.div_tiles_w.div((uint32_t)rem), tw = rem - th * args.sh_tiles_w;
           for (int cblk = 0; cblk < args.sh_ncb; ++cblk)
-            tma_load_tiled_4d(dst + cblk * args.sh_cblk_bytes, &tmap_a, cblk * bk, tw * kShiftTileW, th * kShiftTileH, img,
+            tma_load_tiled_4d(dst + cblk * args.sh_cblk_bytes, &tmap_a, cblk * bk, tw * args.sh_wps, th * (kTileM / args.sh_wps), img,
                               full, leader);
         } else
         for (int j = 0; j < args.sh_rows; ++j) {
@@ -864,7 +864,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       out_img = (int)args.div_tiles_hw.div(tile);
       const int rem = (int)tile - out_img * (args.sh_tiles_h * args.sh_tiles_w);
       const int th = (int)args.div_tiles_w.div((uint32_t)rem), tw = rem - th * args.sh_tiles_w;
-      const int po = th * kShiftTileH + row / kShiftTileW, qo = tw * kShiftTileW + row % kShiftTileW;
+      const int tile_w = args.sh_wps, tile_h = kTileM / tile_w;  // tile width: a power of two
+      const int po = th * tile_h + row / tile_w, qo = tw * tile_w + (row & (tile_w - 1));
       row_valid = po < args.out_P && qo < args.out_Q;
       out_pq = po * args.out_Q + qo;
     } else if (args.remap == 2 && row_valid) {

@@ -110,12 +110,21 @@ bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg, bool tiles_2d) {
     // 8 x 16-pixel tiles over an unpadded view with one tap per filter row: the window is one box of
     // (8 + R - 1) rows of 16 pixels, and a tap moves the tile by one row of 16 pixels
     if (v.S != 1 || v.pad_h != 0 || v.pad_w != 0 || v.dil_h != 1) return false;
-    sg->wps = kShiftTileW;
+    // tile width: the widest power of two up to 128 that wastes at most 15 % of its columns on the
+    // ragged right edge (wide tiles give long contiguous output runs), else 16
+    int tile_w = kShiftTileW;
+    for (int tw = kTileM; tw > kShiftTileW; tw >>= 1)
+      if ((long long)((g.Q + tw - 1) / tw) * tw * 100 <= (long long)g.Q * 115) {
+        tile_w = tw;
+        break;
+      }
+    const int tile_h = kTileM / tile_w;
+    sg->wps = tile_w;
     sg->hp = v.H;
-    rows = kShiftTileH + v.R - 1;
+    rows = tile_h + v.R - 1;
     if (rows > 256) return false;
-    sg->tiles_h = (g.P + kShiftTileH - 1) / kShiftTileH;
-    sg->tiles_w = (g.Q + kShiftTileW - 1) / kShiftTileW;
+    sg->tiles_h = (g.P + tile_h - 1) / tile_h;
+    sg->tiles_w = (g.Q + tile_w - 1) / tile_w;
   } else {
     const int wp = v.W + 2 * v.pad_w;
     sg->wps = round_up(wp, 8);
