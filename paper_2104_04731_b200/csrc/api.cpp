@@ -299,7 +299,6 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
       // (n, h', w') <- input element, in the form the stencil-unroll kernel takes.  Weights: packed
       // column (tap, j) <- index into one KCRS filter.
       const long long sc = d.in_layout == B2C_LAYOUT_NCHW ? (long long)d.H * d.W : 1;
-      const long long sh = d.in_layout == B2C_LAYOUT_NCHW ? d.W : (long long)d.W * d.C;
       const long long sw = d.in_layout == B2C_LAYOUT_NCHW ? 1 : d.C;
       std::vector<GatherEntry> t(v.C, GatherEntry{-1, 0, 0});
       std::vector<int32_t> wt((size_t)v.R * v.S * v.C, -1);
@@ -323,17 +322,21 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
             for (int r = 0; r < d.R; ++r) wt[(size_t)r * v.C + j] = (c * d.R + r) * d.S + s;
           }
       } else {
-        for (int c = 0; c < d.C; ++c)
-          for (int dh = 0; dh < d.stride_h; ++dh)
-            for (int dw = 0; dw < d.stride_w; ++dw) {
-              const int j = (c * d.stride_h + dh) * d.stride_w + dw;
-              t[j] = GatherEntry{(int32_t)(c * sc + dh * sh + dw * sw), (int16_t)dh, (int16_t)dw};
-              for (int rp = 0; rp < v.R; ++rp)
-                for (int sp = 0; sp < v.S; ++sp) {
-                  const int r = rp * d.stride_h + dh, s = sp * d.stride_w + dw;
-                  if (r < d.R && s < d.S) wt[((size_t)rp * v.S + sp) * v.C + j] = (c * d.R + r) * d.S + s;
-                }
-            }
+        // space to depth with horizontal tap packing: scratch channel (ui, c, dh, dw) of pixel w' is phase
+        // (dh, dw) of channel c at scratch column w' + ui; tap s'' of the view stands for columns
+        // pack*s'' + ui (the activation rewrite has a kernel of its own and needs no table)
+        const int pack = s2d_pack_factor(g), cphase = d.C * d.stride_h * d.stride_w;
+        for (int ui = 0; ui < pack; ++ui)
+          for (int c = 0; c < d.C; ++c)
+            for (int dh = 0; dh < d.stride_h; ++dh)
+              for (int dw = 0; dw < d.stride_w; ++dw) {
+                const int j = ui * cphase + (c * d.stride_h + dh) * d.stride_w + dw;
+                for (int rp = 0; rp < v.R; ++rp)
+                  for (int sp = 0; sp < v.S; ++sp) {
+                    const int r = rp * d.stride_h + dh, s = (sp * pack + ui) * d.stride_w + dw;
+                    if (r < d.R && s < d.S) wt[((size_t)rp * v.S + sp) * v.C + j] = (c * d.R + r) * d.S + s;
+                  }
+              }
       }
       p->table_len = (int)t.size();
       if (cudaMalloc(&p->table, t.size() * sizeof(GatherEntry)) != cudaSuccess) return fail(B2C_E_CUDA);
@@ -675,8 +678,8 @@ static int run_rewrite(b2c_plan* p, const int8_t* x, void* ws, cudaStream_t st) 
       // space to depth: scratch pixel (n, h', w') holds the stride phases (c, dh, dw) of its window
       const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
       CUDA_TRY(launch_space_to_depth(x, scratch, v.N, v.H, v.W, d.C, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
-                                     v.C, a.x_stride_n, nchw ? (long long)d.H * d.W : 1, a.x_stride_h, a.x_stride_w,
-                                     st));
+                                     v.C, s2d_pack_factor(g), a.x_stride_n, nchw ? (long long)d.H * d.W : 1,
+                                     a.x_stride_h, a.x_stride_w, st));
     }
   } else if (p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
     CUDA_TRY(launch_im2col(x, scratch, p->table, g.Mg, g.PQ, g.Q, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,

@@ -247,6 +247,11 @@ struct WindowGeom {
   int rows, pitch, left, parts, bytes;
 };
 bool staged_window(const Geom& g, WindowGeom* w);
+// Space to depth, horizontal tap packing: when the stride phases of all channels fill at most a
+// quarter of the 32-byte channel block, each scratch pixel also carries the phases of its next pack - 1
+// horizontal neighbours, and the remaining convolution has ceil(S' / pack) taps per row at a
+// horizontal dilation of `pack` instead of S' (the bytes would otherwise be zero padding).
+int s2d_pack_factor(const Geom& g);
 // Staged stencil unroll with unit horizontal dilation: each (c, r) run of S taps is padded to a
 // multiple of 4 so that the A rows are built from aligned 32-bit words of the window.
 bool staged_word_mode(const Geom& g);
@@ -278,8 +283,8 @@ cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, 
                           int W, int stride_h, int stride_w, int pad_h, int pad_w, long long x_stride_n,
                           int x_stride_h, int x_stride_w, int K_pad, cudaStream_t st);
 cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, int Ws, int C, int H, int W, int sh,
-                                  int sw, int pad_h, int pad_w, int C_pad, long long stride_n, long long stride_c,
-                                  int stride_h, int stride_w, cudaStream_t st);
+                                  int sw, int pad_h, int pad_w, int C_pad, int pack, long long stride_n,
+                                  long long stride_c, int stride_h, int stride_w, cudaStream_t st);
 cudaError_t launch_row_phase_unroll(const int8_t* x, int8_t* out, int N, int Hs, int Q, int C, int H, int W, int S, int sh,
                                     int sw, int pad_h, int pad_w, int dil_w, int C_pad, long long stride_n,
                                     long long stride_c, int stride_h, int stride_w, cudaStream_t st);

@@ -340,12 +340,14 @@ __global__ void __launch_bounds__(256) phase_split_kernel(const int8_t* __restri
 __global__ void __launch_bounds__(256) space_to_depth_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ out,
                                                              unsigned total, FastDiv div_chunks, FastDiv div_ws,
                                                              FastDiv div_hs, int C, int H, int W, int sh, int sw,
-                                                             int pad_h, int pad_w, int C_pad, long long stride_n,
-                                                             int stride_c, int stride_h, int stride_w) {
+                                                             int pad_h, int pad_w, int C_pad, int pack,
+                                                             long long stride_n, int stride_c, int stride_h,
+                                                             int stride_w) {
   // (32-bit indices and multiply-shift divisions: a 64-bit division costs more than the 16 bytes moved)
   const int chunks = (int)div_chunks.d, Ws = (int)div_ws.d, Hs = (int)div_hs.d;
-  const int creal = C * sh * sw;
   const int phases = sh * sw;
+  const int cphase = C * phases;      // bytes of one scratch column's own phases
+  const int creal = pack * cphase;    // plus those of its pack - 1 right neighbours
   pdl_wait();
   for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
     const unsigned pix = div_chunks.div(i);
@@ -358,20 +360,25 @@ __global__ void __launch_bounds__(256) space_to_depth_kernel(const int8_t* __res
       const unsigned n = div_hs.div(t);
       const int hs = (int)(t - n * (unsigned)Hs);
       const int h0 = hs * sh - pad_h, w0 = ws * sw - pad_w;
-      int c = j0 / phases;
-      int rem = j0 - c * phases;
+      int ui = j0 / cphase;
+      int rem = j0 - ui * cphase;
+      int c = rem / phases;
+      rem -= c * phases;
       int dh = rem / sw, dw = rem - dh * sw;
       const int8_t* base = x + (long long)n * stride_n;
 #pragma unroll
       for (int e = 0; e < 16; ++e) {
-        const int h = h0 + dh, w = w0 + dw;
-        if (c < C && (unsigned)h < (unsigned)H && (unsigned)w < (unsigned)W)
+        const int h = h0 + dh, w = w0 + ui * sw + dw;
+        if (ui < pack && (unsigned)h < (unsigned)H && (unsigned)w < (unsigned)W)
           wv[e >> 2] |= (uint32_t)(uint8_t)base[c * stride_c + h * stride_h + w * stride_w] << (8 * (e & 3));
         if (++dw == sw) {
           dw = 0;
           if (++dh == sh) {
             dh = 0;
-            ++c;
+            if (++c == C) {
+              c = 0;
+              ++ui;
+            }
           }
         }
       }
@@ -389,7 +396,8 @@ constexpr int kS2dTile = 128;
 __global__ void __launch_bounds__(kS2dTile) space_to_depth_rows_kernel(const int8_t* __restrict__ x,
                                                                        int8_t* __restrict__ out, int Hs, int Ws, int C,
                                                                        int H, int W, int sh, int sw, int pad_h,
-                                                                       int pad_w, int C_pad, int seg, int ws_tiles) {
+                                                                       int pad_w, int C_pad, int pack, int seg,
+                                                                       int ws_tiles) {
   extern __shared__ __align__(16) uint8_t s2d_rows[];
   const int tile = blockIdx.x % ws_tiles;
   const int rowi = blockIdx.x / ws_tiles;  // (n, hs)
@@ -422,20 +430,23 @@ __global__ void __launch_bounds__(kS2dTile) space_to_depth_rows_kernel(const int
   const int ws = ws0 + threadIdx.x;
   if (ws >= Ws) return;
   const int off0 = threadIdx.x * sw + (wbeg - walign);
-  const int creal = C * sh * sw;
+  const int creal = pack * C * sh * sw;
   int8_t* dst = out + (((size_t)n * Hs + hs) * Ws + ws) * C_pad;
-  int c = 0, dh = 0, dw = 0;
+  int ui = 0, c = 0, dh = 0, dw = 0;
   for (int j0 = 0; j0 < C_pad; j0 += 16) {
     uint32_t wv[4] = {0, 0, 0, 0};
     if (j0 < creal) {
 #pragma unroll
       for (int e = 0; e < 16; ++e) {
-        if (c < C) wv[e >> 2] |= (uint32_t)s2d_rows[(c * sh + dh) * seg + off0 + dw] << (8 * (e & 3));
+        if (ui < pack) wv[e >> 2] |= (uint32_t)s2d_rows[(c * sh + dh) * seg + off0 + ui * sw + dw] << (8 * (e & 3));
         if (++dw == sw) {
           dw = 0;
           if (++dh == sh) {
             dh = 0;
-            ++c;
+            if (++c == C) {
+              c = 0;
+              ++ui;
+            }
           }
         }
       }
@@ -613,16 +624,16 @@ cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, 
 }
 
 cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, int Ws, int C, int H, int W, int sh,
-                                  int sw, int pad_h, int pad_w, int C_pad, long long stride_n, long long stride_c,
-                                  int stride_h, int stride_w, cudaStream_t st) {
+                                  int sw, int pad_h, int pad_w, int C_pad, int pack, long long stride_n,
+                                  long long stride_c, int stride_h, int stride_w, cudaStream_t st) {
   // Fast path: NCHW rows that are multiples of 16 bytes, row segments of a tile within 48 KB.
-  const int seg = ((kS2dTile * sw + sw + 15 + 15) / 16) * 16;  // bytes of one input row a tile reads, from a 16-byte boundary
+  const int seg = ((kS2dTile * sw + pack * sw + 15 + 15) / 16) * 16;  // bytes of one input row a tile reads, from a 16-byte boundary
   const long long smem = (long long)C * sh * seg;
   const long long blocks = (long long)N * Hs * ((Ws + kS2dTile - 1) / kS2dTile);
   if (stride_w == 1 && stride_h == W && stride_c == (long long)H * W && (W % 16) == 0 &&
       (reinterpret_cast<uintptr_t>(x) & 15) == 0 && smem <= 48 * 1024 && blocks < 0x7FFFFFFFLL && Ws >= 32)
     return launch_pdl(space_to_depth_rows_kernel, dim3((unsigned)blocks), dim3(kS2dTile), (size_t)smem, st, x, out, Hs, Ws, C,
-                      H, W, sh, sw, pad_h, pad_w, C_pad, seg, (Ws + kS2dTile - 1) / kS2dTile);
+                      H, W, sh, sw, pad_h, pad_w, C_pad, pack, seg, (Ws + kS2dTile - 1) / kS2dTile);
   // total 16-byte chunks of the scratch tensor; the planner keeps N*Hs*Ws*C_pad below 2^40 and one
   // image below 2^31 bytes, and the launch below is split so that each part's chunk count fits 32 bits
   const long long per_image = (long long)Hs * Ws * (C_pad / 16);
@@ -633,7 +644,7 @@ cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, i
     cudaError_t e = launch_pdl(space_to_depth_kernel, dim3(grid_for(total, 256)), dim3(256), 0, st,
                                x + (long long)n0 * stride_n, out + (long long)n0 * per_image * 16, (unsigned)total,
                                make_fastdiv((uint32_t)(C_pad / 16)), make_fastdiv((uint32_t)Ws), make_fastdiv((uint32_t)Hs),
-                               C, H, W, sh, sw, pad_h, pad_w, C_pad, stride_n, (int)stride_c, stride_h, stride_w);
+                               C, H, W, sh, sw, pad_h, pad_w, C_pad, pack, stride_n, (int)stride_c, stride_h, stride_w);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;

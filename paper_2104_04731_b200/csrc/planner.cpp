@@ -100,6 +100,13 @@ static bool view_fits_tensor_map(const TmaView& v) {
   return true;
 }
 
+int s2d_pack_factor(const Geom& g) {
+  const int cphase = g.d.C * g.d.stride_h * g.d.stride_w;
+  const int Sp = (g.d.S + g.d.stride_w - 1) / g.d.stride_w;
+  if (cphase > kMmaK / 4) return 1;  // worth the larger rewrite only when at least four columns share a pixel
+  return std::max(1, std::min(kMmaK / cphase, Sp));
+}
+
 bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg, bool tiles_2d) {
   if (v.stride_h != 1 || v.stride_w != 1 || g.d.K > 256) return false;
   sg->cb = cp_block_bytes(v.C);
@@ -198,7 +205,11 @@ bool tma_view_for(const Geom& g, int variant, TmaView* v) {
     // stride-1, unpadded R' x S' convolution over X' remains (R' = ceil(R / stride_h)).
     if (d.dil_h != 1 || d.dil_w != 1 || (d.stride_h == 1 && d.stride_w == 1)) return false;
     const int Rp = (d.R + d.stride_h - 1) / d.stride_h, Sp = (d.S + d.stride_w - 1) / d.stride_w;
-    *v = TmaView{d.N, round_up(d.C * d.stride_h * d.stride_w, kMmaK), g.P + Rp - 1, g.Q + Sp - 1, Rp, Sp, 1, 1, 0, 0, 1, 1};
+    // horizontal tap packing: X''[..][w'][(ui, c, dh, dw)] = X'[..][w' + ui][(c, dh, dw)], taps at w' + pack*s''
+    const int pack = s2d_pack_factor(g);
+    const int Sv = (Sp + pack - 1) / pack;
+    *v = TmaView{d.N, round_up(pack * d.C * d.stride_h * d.stride_w, kMmaK), g.P + Rp - 1, g.Q + pack * (Sv - 1), Rp, Sv,
+                 1, 1, 0, 0, 1, pack};
   } else if (variant == B2C_VARIANT_DILATION_PACK) {
     // Image Pack of a dilated convolution (Section 6.1): with h - pad_h = i*dil_h + a every tap of an
     // output pixel reads phase a of the image, X_a[j] = x[j*dil_h + a], at j = i + r.  The dil_h*dil_w

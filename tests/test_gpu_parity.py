@@ -317,6 +317,8 @@ def test_dense_layer_is_a_1x1_convolution(lib, batch, cin, cout):
     (4, 3, 40, 40, 64, 7, 7, 2, 3, 1, 6),            # stride 2: only through space to depth
     (2, 1, 33, 61, 32, 9, 21, 2, 0, 1, 5),           # single channel, wide kernel, stride 2
     (2, 5, 21, 23, 20, 4, 5, (3, 2), (1, 2), 1, 5),  # stride 3 x 2
+    (3, 2, 25, 27, 40, 5, 5, 2, 2, 1, 6),            # two channels, stride 2: three columns share a pixel (tap packing 3)
+    (2, 1, 19, 40, 16, 3, 7, (1, 2), (1, 3), 1, 4),  # horizontal stride only: 2 phase bytes, tap packing 4 of S' = 4
 ])
 @pytest.mark.parametrize("layouts", [(0, 0), (1, 1)])
 def test_shift_execution(lib, case, layouts):

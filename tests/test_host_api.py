@@ -136,6 +136,12 @@ def test_padding_inflates_weights_and_workspace(lib):
     assert ro.workspace_bytes == cfg.N * cfg.H * cfg.Q * 32          # (s, c) = 21 -> 32 channels per (n, h, q)
     # 3*2*2 = 12 -> 32 channels, R' = S' = 4; scratch sizes are rounded up to 256 bytes
     assert sd.workspace_bytes == -(-cfg.N * (cfg.P + 3) * (cfg.Q + 3) * 32 // 256) * 256
+    # single channel, 9 x 21 stride 2: 4 phase bytes per column, so eight columns share a 32-byte pixel and the
+    # S' = 11 taps of a row become 2 taps at dilation 8 over Q + 8 scratch columns (R' = 5)
+    c4 = CONFIGS[3]
+    d4 = b2c.make_desc(c4.N, c4.C, c4.H, c4.W, c4.K, c4.R, c4.S, c4.stride, c4.pad)
+    sd4 = next(e for e in b2c.enumerate_embeddings(d4) if e.variant == 5 and e.split_k == 1)
+    assert sd4.workspace_bytes == -(-c4.N * (c4.P + 4) * (c4.Q + 8) * 32 // 256) * 256
     assert ga.o_mac < ro.o_mac < cp.o_mac
     assert embs[0].variant in (2, 3)  # lowest overhead: stencil unroll formed inside the kernel
 
