@@ -182,10 +182,11 @@ void fill_common_args(b2c_plan* p) {
       a.div_wps = make_fastdiv((uint32_t)sg.wps);
       a.div_hp = make_fastdiv((uint32_t)sg.hp);
       a.remap = 2;
-      if (shift_tiles_2d(p->emb.variant)) {
+      if (sg.two_d) {
         a.remap = 3;
         a.sh_tiles_h = sg.tiles_h;
         a.sh_tiles_w = sg.tiles_w;
+        a.sh_valid_w = sg.valid_w;
         a.div_tiles_hw = make_fastdiv((uint32_t)(sg.tiles_h * sg.tiles_w));
         a.div_tiles_w = make_fastdiv((uint32_t)sg.tiles_w);
       }

@@ -118,7 +118,7 @@ struct ConvArgs {
   int sh_wps, sh_hp, sh_rows, sh_row_bytes, sh_ncb, sh_R, sh_cblk_bytes, sh_win_bytes, sh_w_bytes, sh_mtot;
   // two-dimensional tiles (remap == 3): tile t = (image, tile row, tile column); accumulator row m of
   // a tile is pixel (m / tile_w, m % tile_w) of it (tile_w = sh_wps); the window is one box per channel block
-  int sh_tiles_h, sh_tiles_w;
+  int sh_tiles_h, sh_tiles_w, sh_valid_w;  // sh_valid_w: columns of a tile that are outputs (tiles advance by it)
   FastDiv div_tiles_hw, div_tiles_w;
   int persistent_blocks_per_sm;  // blocks per SM the persistent grid is sized for (0: the mode's default)
   FastDiv div_wps, div_hp;
@@ -212,7 +212,7 @@ inline int variant_family(int v) {
 // more than 256 output channels, rows wider than one copy, or window + weights beyond shared memory).
 struct ShiftGeom {
   int wps, hp, rows, row_bytes, ncb, cb, cblk_bytes, win_bytes, w_bytes, tile_n, stages, blocks_per_sm;
-  int tiles_h, tiles_w;  // two-dimensional tiles only
+  int two_d, tiles_h, tiles_w, valid_w;  // two-dimensional tiles: pixel columns of a tile that are outputs
   long long mtot;
 };
 bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg, bool tiles_2d = false);

@@ -621,12 +621,13 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         uint32_t dst = a_base + s * a_stage_bytes;
         if (args.remap == 3) {
           // two-dimensional tile (image, tile row, tile column): the window is one box of sh_rows rows
-          // of 16 pixels per channel block
+          // of sh_wps pixels per channel block, from the tile's first window origin on
           const int img = (int)args.div_tiles_hw.div((uint32_t)t);
           const int rem = t - img * (args.sh_tiles_h * args.sh_tiles_w);
           const int th = (int)args.div_tiles_w.div((uint32_t)rem), tw = rem - th * args.sh_tiles_w;
           for (int cblk = 0; cblk < args.sh_ncb; ++cblk)
-            tma_load_tiled_4d(dst + cblk * args.sh_cblk_bytes, &tmap_a, cblk * bk, tw * args.sh_wps, th * (kTileM / args.sh_wps), img,
+            tma_load_tiled_4d(dst + cblk * args.sh_cblk_bytes, &tmap_a, cblk * bk, tw * args.sh_valid_w - args.pad_w,
+                              th * (kTileM / args.sh_wps) - args.pad_h, img,
                               full, leader);
         } else
         for (int j = 0; j < args.sh_rows; ++j) {
@@ -865,8 +866,9 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       const int rem = (int)tile - out_img * (args.sh_tiles_h * args.sh_tiles_w);
       const int th = (int)args.div_tiles_w.div((uint32_t)rem), tw = rem - th * args.sh_tiles_w;
       const int tile_w = args.sh_wps, tile_h = kTileM / tile_w;  // tile width: a power of two
-      const int po = th * tile_h + row / tile_w, qo = tw * tile_w + (row & (tile_w - 1));
-      row_valid = po < args.out_P && qo < args.out_Q;
+      const int col = row & (tile_w - 1);
+      const int po = th * tile_h + row / tile_w, qo = tw * args.sh_valid_w + col;
+      row_valid = col < args.sh_valid_w && po < args.out_P && qo < args.out_Q;
       out_pq = po * args.out_Q + qo;
     } else if (args.remap == 2 && row_valid) {
       // shift execution: row m is window origin (n, hp, wp) on the padded grid of sh_hp x sh_wps positions

@@ -113,10 +113,28 @@ bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg, bool tiles_2d) {
   sg->ncb = v.C / sg->cb;
   sg->tiles_h = sg->tiles_w = 0;
   long long rows;
-  if (tiles_2d) {
-    // 8 x 16-pixel tiles over an unpadded view with one tap per filter row: the window is one box of
-    // (8 + R - 1) rows of 16 pixels, and a tap moves the tile by one row of 16 pixels
+  sg->two_d = 0;
+  sg->valid_w = 0;
+  // Wide rows with several taps per filter row: a tile of 128 positions is one row of 128 window
+  // origins, of which the last (S - 1)*dil_w only serve as the taps' overhang (tiles advance by the
+  // valid width), and the window is one box of R rows (+1 for that overhang) of 128 pixels instead
+  // of whole padded rows.
+  const long long wp_full = round_up(v.W + 2 * v.pad_w, 8);
+  const int overhang = (v.S - 1) * v.dil_w;
+  if (!tiles_2d && v.S > 1 && v.dil_h == 1 && wp_full >= 192 && overhang <= kTileM / 4) {
+    sg->two_d = 1;
+    sg->wps = kTileM;
+    sg->valid_w = kTileM - overhang;
+    sg->hp = v.H + 2 * v.pad_h;
+    rows = v.R + 1;
+    if (rows > 256) return false;
+    sg->tiles_h = g.P;
+    sg->tiles_w = (g.Q + sg->valid_w - 1) / sg->valid_w;
+  } else if (tiles_2d) {
+    // tiles of 128/tw x tw pixels over an unpadded view with one tap per filter row: the window is one
+    // box of (128/tw + R - 1) rows of tw pixels, and a tap moves the tile by one row of tw pixels
     if (v.S != 1 || v.pad_h != 0 || v.pad_w != 0 || v.dil_h != 1) return false;
+    sg->two_d = 1;
     // tile width: the widest power of two up to 128 that wastes at most 15 % of its columns on the
     // ragged right edge (wide tiles give long contiguous output runs), else 16
     int tile_w = kShiftTileW;
@@ -127,6 +145,7 @@ bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg, bool tiles_2d) {
       }
     const int tile_h = kTileM / tile_w;
     sg->wps = tile_w;
+    sg->valid_w = tile_w;
     sg->hp = v.H;
     rows = tile_h + v.R - 1;
     if (rows > 256) return false;
@@ -166,7 +185,7 @@ bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg, bool tiles_2d) {
       sg->blocks_per_sm = bps;
     }
   }
-  sg->mtot = tiles_2d ? (long long)v.N * sg->tiles_h * sg->tiles_w * kTileM : (long long)v.N * sg->hp * sg->wps;
+  sg->mtot = sg->two_d ? (long long)v.N * sg->tiles_h * sg->tiles_w * kTileM : (long long)v.N * sg->hp * sg->wps;
   return sg->mtot <= 0x7FFFFF00LL;
 }
 
