@@ -323,15 +323,15 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
             for (int r = 0; r < d.R; ++r) wt[(size_t)r * v.C + j] = (c * d.R + r) * d.S + s;
           }
       } else {
-        // space to depth with horizontal tap packing: scratch channel (ui, c, dh, dw) of pixel w' is phase
+        // space to depth with horizontal tap packing: scratch channel (c, dh, ui, dw) of pixel w' is phase
         // (dh, dw) of channel c at scratch column w' + ui; tap s'' of the view stands for columns
         // pack*s'' + ui (the activation rewrite has a kernel of its own and needs no table)
-        const int pack = s2d_pack_factor(g), cphase = d.C * d.stride_h * d.stride_w;
+        const int pack = s2d_pack_factor(g);
         for (int ui = 0; ui < pack; ++ui)
           for (int c = 0; c < d.C; ++c)
             for (int dh = 0; dh < d.stride_h; ++dh)
               for (int dw = 0; dw < d.stride_w; ++dw) {
-                const int j = ui * cphase + (c * d.stride_h + dh) * d.stride_w + dw;
+                const int j = (((c * d.stride_h + dh) * pack) + ui) * d.stride_w + dw;
                 for (int rp = 0; rp < v.R; ++rp)
                   for (int sp = 0; sp < v.S; ++sp) {
                     const int r = rp * d.stride_h + dh, s = (sp * pack + ui) * d.stride_w + dw;

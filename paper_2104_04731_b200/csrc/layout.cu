@@ -345,9 +345,7 @@ __global__ void __launch_bounds__(256) space_to_depth_kernel(const int8_t* __res
                                                              int stride_w) {
   // (32-bit indices and multiply-shift divisions: a 64-bit division costs more than the 16 bytes moved)
   const int chunks = (int)div_chunks.d, Ws = (int)div_ws.d, Hs = (int)div_hs.d;
-  const int phases = sh * sw;
-  const int cphase = C * phases;      // bytes of one scratch column's own phases
-  const int creal = pack * cphase;    // plus those of its pack - 1 right neighbours
+  const int creal = pack * C * sh * sw;  // a column's own phases plus those of its pack - 1 right neighbours
   pdl_wait();
   for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
     const unsigned pix = div_chunks.div(i);
@@ -360,25 +358,23 @@ __global__ void __launch_bounds__(256) space_to_depth_kernel(const int8_t* __res
       const unsigned n = div_hs.div(t);
       const int hs = (int)(t - n * (unsigned)Hs);
       const int h0 = hs * sh - pad_h, w0 = ws * sw - pad_w;
-      int ui = j0 / cphase;
-      int rem = j0 - ui * cphase;
-      int c = rem / phases;
-      rem -= c * phases;
-      int dh = rem / sw, dw = rem - dh * sw;
+      // scratch channel j = ((c*sh + dh)*pack + ui)*sw + dw: the pack*sw bytes of one (c, dh) are
+      // consecutive input bytes of one row
+      const int run_len = pack * sw;
+      const int run = j0 / run_len;
+      int within = j0 - run * run_len;
+      int c = run / sh, dh = run - c * sh;
       const int8_t* base = x + (long long)n * stride_n;
 #pragma unroll
       for (int e = 0; e < 16; ++e) {
-        const int h = h0 + dh, w = w0 + ui * sw + dw;
-        if (ui < pack && (unsigned)h < (unsigned)H && (unsigned)w < (unsigned)W)
+        const int h = h0 + dh, w = w0 + within;
+        if (c < C && (unsigned)h < (unsigned)H && (unsigned)w < (unsigned)W)
           wv[e >> 2] |= (uint32_t)(uint8_t)base[c * stride_c + h * stride_h + w * stride_w] << (8 * (e & 3));
-        if (++dw == sw) {
-          dw = 0;
+        if (++within == run_len) {
+          within = 0;
           if (++dh == sh) {
             dh = 0;
-            if (++c == C) {
-              c = 0;
-              ++ui;
-            }
+            ++c;
           }
         }
       }
@@ -430,23 +426,38 @@ __global__ void __launch_bounds__(kS2dTile) space_to_depth_rows_kernel(const int
   const int ws = ws0 + threadIdx.x;
   if (ws >= Ws) return;
   const int off0 = threadIdx.x * sw + (wbeg - walign);
-  const int creal = pack * C * sh * sw;
+  // scratch channel j = ((c*sh + dh)*pack + ui)*sw + dw: the run of pack*sw bytes of one (c, dh) is
+  // pack*sw consecutive bytes of one staged row.  Runs that are whole words are copied word by word
+  // (an unaligned word = two aligned loads and a byte permute), others byte by byte.
+  const int run_len = pack * sw;
+  const int creal = C * sh * run_len;
   int8_t* dst = out + (((size_t)n * Hs + hs) * Ws + ws) * C_pad;
-  int ui = 0, c = 0, dh = 0, dw = 0;
+  int run = 0, within = 0;
   for (int j0 = 0; j0 < C_pad; j0 += 16) {
     uint32_t wv[4] = {0, 0, 0, 0};
     if (j0 < creal) {
+      if ((run_len & 3) == 0) {
 #pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        if (ui < pack) wv[e >> 2] |= (uint32_t)s2d_rows[(c * sh + dh) * seg + off0 + ui * sw + dw] << (8 * (e & 3));
-        if (++dw == sw) {
-          dw = 0;
-          if (++dh == sh) {
-            dh = 0;
-            if (++c == C) {
-              c = 0;
-              ++ui;
-            }
+        for (int k = 0; k < 4; ++k) {
+          if (j0 + 4 * k < creal) {
+            const int src = run * seg + off0 + within;
+            const uint32_t lo = *reinterpret_cast<const uint32_t*>(s2d_rows + (src & ~3));
+            const uint32_t hi = *reinterpret_cast<const uint32_t*>(s2d_rows + (src & ~3) + 4);
+            wv[k] = __byte_perm(lo, hi, 0x3210u + 0x1111u * (uint32_t)(src & 3));
+          }
+          within += 4;
+          if (within == run_len) {
+            within = 0;
+            ++run;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          if (j0 + e < creal) wv[e >> 2] |= (uint32_t)s2d_rows[run * seg + off0 + within] << (8 * (e & 3));
+          if (++within == run_len) {
+            within = 0;
+            ++run;
           }
         }
       }
