@@ -247,8 +247,8 @@ struct WindowGeom {
   int rows, pitch, left, parts, bytes;
 };
 bool staged_window(const Geom& g, WindowGeom* w);
-// Space to depth, horizontal tap packing: when the stride phases of all channels fill at most a
-// quarter of the 32-byte channel block, each scratch pixel also carries the phases of its next pack - 1
+// Space to depth, horizontal tap packing: when the stride phases of all channels fill at most half
+// of the 32-byte channel block, each scratch pixel also carries the phases of its next pack - 1
 // horizontal neighbours, and the remaining convolution has ceil(S' / pack) taps per row at a
 // horizontal dilation of `pack` instead of S' (the bytes would otherwise be zero padding).
 int s2d_pack_factor(const Geom& g);

@@ -103,7 +103,7 @@ static bool view_fits_tensor_map(const TmaView& v) {
 int s2d_pack_factor(const Geom& g) {
   const int cphase = g.d.C * g.d.stride_h * g.d.stride_w;
   const int Sp = (g.d.S + g.d.stride_w - 1) / g.d.stride_w;
-  if (cphase > kMmaK / 4) return 1;  // worth the larger rewrite only when at least four columns share a pixel
+  if (cphase > kMmaK / 2) return 1;
   return std::max(1, std::min(kMmaK / cphase, Sp));
 }
 

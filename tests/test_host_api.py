@@ -134,8 +134,9 @@ def test_padding_inflates_weights_and_workspace(lib):
     ro = next(e for e in embs if e.variant == 4 and e.split_k == 1)
     sd = next(e for e in embs if e.variant == 5 and e.split_k == 1)
     assert ro.workspace_bytes == cfg.N * cfg.H * cfg.Q * 32          # (s, c) = 21 -> 32 channels per (n, h, q)
-    # 3*2*2 = 12 -> 32 channels, R' = S' = 4; scratch sizes are rounded up to 256 bytes
-    assert sd.workspace_bytes == -(-cfg.N * (cfg.P + 3) * (cfg.Q + 3) * 32 // 256) * 256
+    # 3*2*2 = 12 phase bytes per column: two columns share a 32-byte pixel, so R' = 4 and S' = 4 -> 2 taps at
+    # dilation 2 over Q + 2 scratch columns; scratch sizes are rounded up to 256 bytes
+    assert sd.workspace_bytes == -(-cfg.N * (cfg.P + 3) * (cfg.Q + 2) * 32 // 256) * 256
     # single channel, 9 x 21 stride 2: 4 phase bytes per column, so eight columns share a 32-byte pixel and the
     # S' = 11 taps of a row become 2 taps at dilation 8 over Q + 8 scratch columns (R' = 5)
     c4 = CONFIGS[3]
