@@ -43,6 +43,8 @@ def _load():
         lib.oracle_conv2d_int8.restype = i32
         lib.oracle_conv2d_int8_act.argtypes = [vp, vp, vp, i32] + [i32] * 14 + [vp, vp, i32]
         lib.oracle_conv2d_int8_act.restype = i32
+        lib.oracle_conv2d_int8_grouped.argtypes = [vp, vp, vp, i32, i32] + [i32] * 14 + [vp, vp, i32]
+        lib.oracle_conv2d_int8_grouped.restype = i32
         lib.oracle_im2col.argtypes = [vp] + [i32] * 12 + [vp]
         lib.oracle_im2col.restype = None
         lib.oracle_gemm_abt.argtypes = [vp, vp, i64, i64, i64, vp]
@@ -79,9 +81,10 @@ def requant(acc: int, shift: int) -> int:
 
 
 def conv2d_int8(x, w, stride=1, pad=0, dilation=1, shift=0, want_i32=True, want_i8=True, threads=0, bias=None,
-                relu=False):
+                relu=False, groups=1):
     """x: int8 [N,C,H,W]; w: int8 [K,C,R,S] -> (y32 int32 [N,K,P,Q] or None, y8 int8 or None).
 
+    `groups` > 1: grouped convolution, w is [K, C/groups, R, S] (groups = C = K: depth-wise).
     Optional activation step before the outputs are written: per-output-channel int32 `bias` [K]
     added to the exact sum, then ReLU.  Raises OverflowError when a value leaves the int32 range.
     """
@@ -89,7 +92,8 @@ def conv2d_int8(x, w, stride=1, pad=0, dilation=1, shift=0, want_i32=True, want_
     w = np.ascontiguousarray(w, dtype=np.int8)
     N, C, H, W = x.shape
     K, C2, R, S = w.shape
-    assert C == C2
+    groups = int(groups)
+    assert groups >= 1 and C % groups == 0 and K % groups == 0 and C2 * groups == C  # w is [K][C/groups][R][S]
     sh, sw = _pair(stride)
     ph, pw = _pair(pad)
     dh, dw = _pair(dilation)
@@ -99,8 +103,8 @@ def conv2d_int8(x, w, stride=1, pad=0, dilation=1, shift=0, want_i32=True, want_
     if bias is not None:
         bias = np.ascontiguousarray(bias, dtype=np.int32)
         assert bias.shape == (K,)
-    rc = _load().oracle_conv2d_int8_act(
-        _ptr(x), _ptr(w), _ptr(bias), int(bool(relu)), N, C, H, W, K, R, S, sh, sw, ph, pw, dh, dw, int(shift),
+    rc = _load().oracle_conv2d_int8_grouped(
+        _ptr(x), _ptr(w), _ptr(bias), int(bool(relu)), groups, N, C, H, W, K, R, S, sh, sw, ph, pw, dh, dw, int(shift),
         _ptr(y32), _ptr(y8), int(threads)
     )
     if rc != 0:

@@ -62,6 +62,11 @@ int8_t oracle_requant(int64_t acc, int shift) {
  *   y32 = t;   y8 = clip(floor(t / 2^shift)).
  * t outside the int32 range is reported like an accumulator overflow.
  *
+ * Grouped convolution (Section 6.1 names depth-wise convolutions as the same low-channel problem):
+ * with `groups` > 1 the input channels and the filters are cut into that many equal groups, filter
+ * k (of group k / (K/groups)) has C/groups channels, w is [K][C/groups][R][S], and output channel k
+ * sums over the input channels of its own group only; groups = C = K is the depth-wise case.
+ *
  * The convolution itself:
  *   y[n][k][p][q] = sum_{c,r,s} x[n][c][p*stride_h - pad_h + r*dil_h][q*stride_w - pad_w + s*dil_w]
  *                               * w[k][c][r][s]        (terms outside the image are zero)
@@ -69,12 +74,13 @@ int8_t oracle_requant(int64_t acc, int shift) {
  * Returns 0, or 1 if some accumulator left the int32 range (outputs then undefined there).
  * `threads` > 0 sets the OpenMP team size used over the (n, k) loops; <= 0 keeps the default.
  */
-int oracle_conv2d_int8_act(const int8_t* x, const int8_t* w, const int32_t* bias, int relu,
-                           int N, int C, int H, int W, int K, int R, int S,
-                           int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
-                           int shift, int32_t* y32, int8_t* y8, int threads) {
+int oracle_conv2d_int8_grouped(const int8_t* x, const int8_t* w, const int32_t* bias, int relu, int groups,
+                               int N, int C, int H, int W, int K, int R, int S,
+                               int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                               int shift, int32_t* y32, int8_t* y8, int threads) {
   const int P = oracle_out_extent(H, R, stride_h, pad_h, dil_h);
   const int Q = oracle_out_extent(W, S, stride_w, pad_w, dil_w);
+  const int Cg = C / groups, Kg = K / groups; /* channels per group; the caller checks divisibility */
   int overflow = 0;
 #ifdef _OPENMP
   if (threads > 0) omp_set_num_threads(threads);
@@ -87,14 +93,15 @@ int oracle_conv2d_int8_act(const int8_t* x, const int8_t* w, const int32_t* bias
       for (int p = 0; p < P; ++p) {
         for (int q = 0; q < Q; ++q) {
           int64_t acc = 0;
-          for (int c = 0; c < C; ++c) {
+          const int c0 = (k / Kg) * Cg; /* first input channel of output channel k's group */
+          for (int c = 0; c < Cg; ++c) {
             for (int r = 0; r < R; ++r) {
               for (int s = 0; s < S; ++s) {
                 int h = p * stride_h - pad_h + r * dil_h;
                 int ww = q * stride_w - pad_w + s * dil_w;
                 if (h >= 0 && h < H && ww >= 0 && ww < W) {
-                  int xv = x[(((size_t)n * C + c) * H + h) * W + ww];
-                  int wv = w[(((size_t)k * C + c) * R + r) * S + s];
+                  int xv = x[(((size_t)n * C + c0 + c) * H + h) * W + ww];
+                  int wv = w[(((size_t)k * Cg + c) * R + r) * S + s];
                   acc += (int64_t)(xv * wv);
                 }
               }
@@ -112,6 +119,15 @@ int oracle_conv2d_int8_act(const int8_t* x, const int8_t* w, const int32_t* bias
     }
   }
   return overflow;
+}
+
+/* Dense convolution (one group) with the activation step. */
+int oracle_conv2d_int8_act(const int8_t* x, const int8_t* w, const int32_t* bias, int relu,
+                           int N, int C, int H, int W, int K, int R, int S,
+                           int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                           int shift, int32_t* y32, int8_t* y8, int threads) {
+  return oracle_conv2d_int8_grouped(x, w, bias, relu, 1, N, C, H, W, K, R, S, stride_h, stride_w, pad_h, pad_w, dil_h,
+                                    dil_w, shift, y32, y8, threads);
 }
 
 /* The convolution with the plain quantisation step only (no bias, no ReLU). */

@@ -288,3 +288,26 @@ def test_bias_and_relu_step():
     xp, wp = np.full((1, 5, 3, 3), 127, dtype=np.int8), np.full((6, 5, 3, 3), 127, dtype=np.int8)
     with pytest.raises(OverflowError):
         oracle.conv2d_int8(xp, wp, 1, 0, 1, 0, bias=big)
+
+
+@pytest.mark.parametrize("groups", [2, 3, 6])
+def test_grouped_conv_is_block_diagonal_dense_conv(groups):
+    """A grouped convolution is the dense convolution whose [K][C] filter matrix is block diagonal
+    (zeros where output channel and input channel belong to different groups); groups = C = K is the
+    depth-wise case.  Pins the group indexing against the dense path, which the other pins fix."""
+    C, K = 6, 12 if groups != 6 else 6
+    x = int8_uniform((2, C, 9, 7), 91)
+    w = int8_uniform((K, C // groups, 3, 2), 92)
+    Cg, Kg = C // groups, K // groups
+    dense = np.zeros((K, C, 3, 2), dtype=np.int8)
+    for k in range(K):
+        g = k // Kg
+        dense[k, g * Cg:(g + 1) * Cg] = w[k]
+    bias = (int8_uniform((K,), 93).astype(np.int32) * 77)
+    got = oracle.conv2d_int8(x, w, (2, 1), (1, 0), 1, 5, groups=groups, bias=bias, relu=True)
+    want = oracle.conv2d_int8(x, dense, (2, 1), (1, 0), 1, 5, bias=bias, relu=True)
+    assert np.array_equal(got[0], want[0]) and np.array_equal(got[1], want[1])
+    # one group is the dense convolution; depth-wise with all-ones data counts the taps inside the image
+    if groups == 6:
+        ones = oracle.conv2d_int8(np.ones((1, 6, 4, 4), np.int8), np.ones((6, 1, 3, 3), np.int8), 1, 1, 1, 0, groups=6)[0]
+        assert ones[0, :, 0, 0].tolist() == [4] * 6 and ones[0, :, 1, 1].tolist() == [9] * 6 and ones[0, :, 0, 2].tolist() == [6] * 6
