@@ -128,6 +128,19 @@ int b2c_enumerate(const b2c_conv_desc* desc, b2c_embedding* out, int32_t cap, in
  * owns its packed weights, lookup tables and a device status word; free it with b2c_plan_destroy. */
 int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_stream, b2c_plan** out);
 
+/* Grouped convolution (Section 6.1 names depth-wise convolutions as the same low-channel problem as
+ * the low-channel layers, without evaluating them).  `desc` describes the whole convolution: C input
+ * and K output channels, both multiples of `groups`; filter k belongs to group k / (K / groups), has
+ * C / groups channels and sums over the input channels of its own group only; the weight tensor
+ * given to b2c_plan_set_weights is int8 [K][C / groups][R][S]; groups == C == K is depth-wise.
+ * desc.in_layout and desc.out_layout must be B2C_LAYOUT_NCHW (UNSUPPORTED otherwise; INVALID_ARG when
+ * groups < 1 or does not divide C and K).  The plan runs one dense convolution per group on that
+ * group's channel slice of x and y in place (no scratch: b2c_plan_workspace_bytes is 0), each with
+ * the lowest-overhead stencil unroll formed inside the kernel; b2c_plan_info reports that embedding.
+ * All other plan calls (set_weights, set_activation with K bias values, run, device_status, destroy)
+ * apply as to any plan; the rewrite / run_rewritten halves are no-op and run respectively. */
+int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan** out);
+
 /* Copies the chosen embedding (with device_us if it was timed) to *chosen. */
 int b2c_plan_info(const b2c_plan* plan, b2c_embedding* chosen);
 

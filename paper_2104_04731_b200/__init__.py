@@ -30,6 +30,7 @@ EXPORTS = [
     "b2c_out_shape", "b2c_enumerate", "b2c_plan_create", "b2c_plan_info", "b2c_plan_workspace_bytes",
     "b2c_plan_set_weights", "b2c_conv2d_int8_run", "b2c_conv2d_int8", "b2c_conv2d_int8_host",
     "b2c_plan_rewrite_activations", "b2c_conv2d_int8_run_rewritten", "b2c_plan_footprint", "b2c_plan_set_activation",
+    "b2c_plan_create_grouped",
     "b2c_plan_device_status", "b2c_selftest_bounded_wait", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
     "b2c_status_string",
     "b2c_last_cuda_error",
@@ -89,6 +90,7 @@ def load():
     lib.b2c_plan_rewrite_activations.argtypes = [vp, vp, vp, vp]
     lib.b2c_conv2d_int8_run_rewritten.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.b2c_plan_set_activation.argtypes = [vp, vp, i32, vp]
+    lib.b2c_plan_create_grouped.argtypes = [pd, ctypes.c_int32, ctypes.POINTER(vp)]
     lib.b2c_plan_footprint.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
     lib.b2c_conv2d_int8.argtypes = [i32] * 11 + [vp] * 5
     lib.b2c_conv2d_int8_host.argtypes = [i32] * 11 + [vp] * 4
@@ -162,12 +164,16 @@ def _dptr(t):
 class Plan:
     """Owns a ``b2c_plan``.  ``run`` enqueues the whole path on the current torch stream."""
 
-    def __init__(self, desc: ConvDesc, policy_or_id: int = POLICY_MIN_OVERHEAD, stream=None):
+    def __init__(self, desc: ConvDesc, policy_or_id: int = POLICY_MIN_OVERHEAD, stream=None, groups: int = 1):
+        """groups > 1: grouped convolution (desc.C and desc.K are the totals, weights [K, C/groups, R, S])."""
         self._lib = load()
         self.desc = desc
         h = ctypes.c_void_p()
-        _check(self._lib.b2c_plan_create(ctypes.byref(desc), policy_or_id, _stream_ptr(stream), ctypes.byref(h)),
-               "b2c_plan_create")
+        if groups > 1:
+            _check(self._lib.b2c_plan_create_grouped(ctypes.byref(desc), groups, ctypes.byref(h)), "b2c_plan_create_grouped")
+        else:
+            _check(self._lib.b2c_plan_create(ctypes.byref(desc), policy_or_id, _stream_ptr(stream), ctypes.byref(h)),
+                   "b2c_plan_create")
         self._h = h
 
     def info(self) -> Embedding:

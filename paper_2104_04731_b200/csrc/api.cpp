@@ -38,6 +38,12 @@ struct b2c_plan {
   CUtensorMap tmap_b;
   // one-shot cache extras
   void* own_ws = nullptr;
+  // Grouped convolution: the plan owns one sub-plan per group (a dense convolution of C/groups
+  // input and K/groups output channels that reads its channel slice of x and writes its slice of
+  // y through the batch strides of the whole tensors); the group plan itself launches nothing.
+  int groups = 1;
+  std::vector<b2c_plan*> subs;
+  long long x_stride_n_whole = 0, y_stride_n_whole = 0;  // sub-plans: batch strides of the whole tensors
 };
 
 namespace {
@@ -129,6 +135,7 @@ void fill_common_args(b2c_plan* p) {
   a.table_len = p->table_len;
   a.table32 = p->table32;
   a.swap = is_swapped(p->emb) ? 1 : 0;
+  a.y_stride_n = (long long)d.K * p->g.PQ;
   a.out_PQ = p->g.PQ;
   a.out_P = p->g.P;
   a.out_Q = p->g.Q;
@@ -618,6 +625,56 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
   return create_plan_for(g, all[best], out);
 }
 
+int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan** out) {
+  if (!desc || !out || groups < 1) return B2C_E_INVALID_ARG;
+  *out = nullptr;
+  if (desc->C < 1 || desc->K < 1 || desc->C % groups != 0 || desc->K % groups != 0) return B2C_E_INVALID_ARG;
+  // whole tensors are NCHW / NKPQ: a group is then a contiguous channel slice of every image
+  if (desc->in_layout != B2C_LAYOUT_NCHW || desc->out_layout != B2C_LAYOUT_NCHW) return B2C_E_UNSUPPORTED;
+  b2c_conv_desc sd = *desc;
+  sd.C = desc->C / groups;
+  sd.K = desc->K / groups;
+  Geom sg;
+  int rc = resolve_geom(&sd, &sg);
+  if (rc != B2C_OK) return rc;
+  // Embedding of every group: the lowest-overhead unsplit stencil unroll formed inside the kernel
+  // (staged window where it fits, else the gather); both read their channel slice of x in place.
+  std::vector<b2c_embedding> all;
+  enumerate_embeddings(sg, &all);
+  int pick = -1;
+  for (size_t i = 0; i < all.size() && pick < 0; ++i)
+    if (all[i].split_k == 1 && !is_swapped(all[i]) && table_variant_legal(sg) &&
+        (all[i].variant == B2C_VARIANT_IM2COL_STAGED || all[i].variant == B2C_VARIANT_IM2COL_GATHER))
+      pick = (int)i;
+  if (pick < 0) return B2C_E_UNSUPPORTED;
+  b2c_plan* p = new (std::nothrow) b2c_plan();
+  if (!p) return B2C_E_INVALID_ARG;
+  p->g = sg;
+  p->g.d.C = desc->C;  // the group plan describes the whole convolution
+  p->g.d.K = desc->K;
+  p->emb = all[pick];
+  p->groups = groups;
+  cudaGetDevice(&p->device);
+  if (cudaMalloc(&p->status, sizeof(int)) != cudaSuccess || cudaMemset(p->status, 0, sizeof(int)) != cudaSuccess) {
+    set_last_cuda_error((int)cudaGetLastError());
+    b2c_plan_destroy(p);
+    return B2C_E_CUDA;
+  }
+  for (int gi = 0; gi < groups; ++gi) {
+    b2c_plan* sub = nullptr;
+    rc = create_plan_for(sg, all[pick], &sub);
+    if (rc != B2C_OK) {
+      b2c_plan_destroy(p);
+      return rc;
+    }
+    sub->x_stride_n_whole = (long long)desc->C * desc->H * desc->W;
+    sub->y_stride_n_whole = (long long)desc->K * sg.PQ;
+    p->subs.push_back(sub);
+  }
+  *out = p;
+  return B2C_OK;
+}
+
 int b2c_plan_info(const b2c_plan* plan, b2c_embedding* chosen) {
   if (!plan || !chosen) return B2C_E_INVALID_ARG;
   *chosen = plan->emb;
@@ -630,10 +687,27 @@ int b2c_plan_workspace_bytes(const b2c_plan* plan, size_t* bytes) {
   return B2C_OK;
 }
 
+static int set_weights_one(b2c_plan* p, const int8_t* w, cudaStream_t st);
+
 int b2c_plan_set_weights(b2c_plan* p, const int8_t* w, void* cuda_stream) {
   if (!p || !w) return B2C_E_INVALID_ARG;
   if (!aligned16(w)) return B2C_E_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (!p->subs.empty()) {
+    // w is [K][C/groups][R][S]: group g's filters are the g-th block of K/groups rows
+    const b2c_conv_desc& sd = p->subs[0]->g.d;
+    const size_t per_group = (size_t)sd.K * sd.C * sd.R * sd.S;
+    for (size_t gi = 0; gi < p->subs.size(); ++gi) {
+      int rc = set_weights_one(p->subs[gi], w + gi * per_group, st);
+      if (rc != B2C_OK) return rc;
+    }
+    p->weights_set = true;
+    return B2C_OK;
+  }
+  return set_weights_one(p, w, st);
+}
+
+static int set_weights_one(b2c_plan* p, const int8_t* w, cudaStream_t st) {
   const b2c_conv_desc& d = p->g.d;
   if (p->emb.variant == B2C_VARIANT_CP_TMA || p->emb.variant == B2C_VARIANT_DILATION_PACK ||
       p->emb.variant == B2C_VARIANT_CP_SHIFT)
@@ -698,6 +772,8 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   a.y8 = y8;
   a.bias = p->bias;
   a.relu = p->relu;
+  if (p->x_stride_n_whole) a.x_stride_n = p->x_stride_n_whole;
+  if (p->y_stride_n_whole) a.y_stride_n = p->y_stride_n_whole;
   const bool act = p->bias != nullptr || p->relu != 0;
   CUtensorMap tmap_a;
   std::memset(&tmap_a, 0, sizeof(tmap_a));
@@ -754,6 +830,17 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   int rc = check_run_args(p, x, true, y32, y8, true, ws);
   if (rc != B2C_OK) return rc;
   cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (!p->subs.empty()) {
+    // one dense convolution per group on its channel slice of x (NCHW) and of y (NKPQ)
+    const b2c_conv_desc& sd = p->subs[0]->g.d;
+    const size_t x_slice = (size_t)sd.C * sd.H * sd.W, y_slice = (size_t)sd.K * p->subs[0]->g.PQ;
+    for (size_t gi = 0; gi < p->subs.size(); ++gi) {
+      rc = run_convolve(p->subs[gi], x + gi * x_slice, y32 ? y32 + gi * y_slice : nullptr, y8 ? y8 + gi * y_slice : nullptr,
+                        nullptr, st);
+      if (rc != B2C_OK) return rc;
+    }
+    return B2C_OK;
+  }
   rc = run_rewrite(p, x, ws, st);
   if (rc != B2C_OK) return rc;
   return run_convolve(p, x, y32, y8, ws, st);
@@ -762,6 +849,7 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
 int b2c_plan_rewrite_activations(b2c_plan* p, const int8_t* x, void* ws, void* cuda_stream) {
   int rc = check_run_args(p, x, true, nullptr, nullptr, false, ws);
   if (rc != B2C_OK) return rc;
+  if (!p->subs.empty()) return B2C_OK;  // the group convolutions read x directly: nothing to rewrite
   return run_rewrite(p, x, ws, (cudaStream_t)cuda_stream);
 }
 
@@ -769,6 +857,7 @@ int b2c_conv2d_int8_run_rewritten(b2c_plan* p, const int8_t* x, int32_t* y32, in
   // x is still needed by the embeddings that have no rewrite (they read the input directly)
   int rc = check_run_args(p, x, p && p->ws_layout_bytes == 0, y32, y8, true, ws);
   if (rc != B2C_OK) return rc;
+  if (!p->subs.empty()) return b2c_conv2d_int8_run(p, x, y32, y8, ws, cuda_stream);
   return run_convolve(p, x, y32, y8, ws, (cudaStream_t)cuda_stream);
 }
 
@@ -784,6 +873,11 @@ int b2c_plan_set_activation(b2c_plan* p, const int32_t* bias_dev, int relu, void
     p->bias = nullptr;  // the buffer is kept for a later call
   }
   p->relu = relu;
+  // group plans: every group takes its own K/groups entries of the copy
+  for (size_t gi = 0; gi < p->subs.size(); ++gi) {
+    p->subs[gi]->bias = p->bias ? p->bias + gi * (size_t)p->subs[gi]->g.d.K : nullptr;
+    p->subs[gi]->relu = relu;
+  }
   return B2C_OK;
 }
 
@@ -791,6 +885,7 @@ int b2c_plan_footprint(const b2c_plan* p, size_t* rewritten_bytes, size_t* packe
   if (!p || !rewritten_bytes || !packed_weight_bytes) return B2C_E_INVALID_ARG;
   *rewritten_bytes = p->ws_layout_bytes;
   *packed_weight_bytes = p->w_packed_bytes;
+  for (const b2c_plan* sub : p->subs) *packed_weight_bytes += sub->w_packed_bytes;
   return B2C_OK;
 }
 
@@ -799,6 +894,12 @@ int b2c_plan_device_status(b2c_plan* p, int32_t* status) {
   int s = 0;
   CUDA_TRY(cudaMemcpy(&s, p->status, sizeof(int), cudaMemcpyDeviceToHost));
   if (s != 0) CUDA_TRY(cudaMemset(p->status, 0, sizeof(int)));
+  for (b2c_plan* sub : p->subs) {  // a group plan reports the first sub-plan status that is set
+    int32_t ss = 0;
+    int rc = b2c_plan_device_status(sub, &ss);
+    if (rc != B2C_OK) return rc;
+    if (s == 0) s = ss;
+  }
   *status = s;
   return B2C_OK;
 }
@@ -811,6 +912,7 @@ int b2c_selftest_bounded_wait(b2c_plan* p, void* cuda_stream) {
 
 void b2c_plan_destroy(b2c_plan* p) {
   if (!p) return;
+  for (b2c_plan* sub : p->subs) b2c_plan_destroy(sub);
   cudaFree(p->w_packed);
   cudaFree(p->table);
   cudaFree(p->table32);

@@ -122,6 +122,9 @@ struct ConvArgs {
   FastDiv div_tiles_hw, div_tiles_w;
   int persistent_blocks_per_sm;  // blocks per SM the persistent grid is sized for (0: the mode's default)
   FastDiv div_wps, div_hp;
+  // elements between consecutive images of the NKPQ output (K * P * Q, or more when this
+  // convolution writes one channel group of a wider tensor)
+  long long y_stride_n;
   // activation step applied to the complete sums before they are written: + bias[k] (nullptr: none),
   // then max(., 0) when relu != 0
   const int32_t* bias;

@@ -1069,7 +1069,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
       // Output index of (m, k): NKPQ -> (n*K + k)*PQ + pq ; NPQK -> m*K + k.
-      const long long base_nkpq = (long long)out_img * args.K * args.out_PQ + out_pq;
+      const long long base_nkpq = (long long)out_img * args.y_stride_n + out_pq;
       const long long base_npqk = args.remap ? ((long long)out_img * args.out_PQ + out_pq) * args.K : (long long)m * args.K;
       const int cols = args.tile_n >= 32 ? (args.tile_n >> 1) : 16;  // columns handled by this warp
       const int c_begin = half * cols;

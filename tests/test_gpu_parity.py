@@ -385,6 +385,47 @@ def test_shift_execution_many_tiles(lib):
     check_against_oracle(x, w, 1, 1, 1, 9, 3, e.id, ref=ref)
 
 
+# ---- grouped / depth-wise convolution: one dense convolution per group on channel slices in place --------
+@pytest.mark.parametrize("case", [
+    # N, C, H, W, K, groups, R, S, stride, pad, dil, shift, out_mode
+    (2, 8, 12, 16, 12, 2, 3, 3, 1, 1, 1, 6, 3),         # two groups of 4 -> 6 channels, rows of 16 bytes
+    (3, 12, 9, 7, 24, 4, 3, 2, (2, 1), (1, 0), 1, 5, 3),  # four groups, odd image: unaligned channel slices
+    (2, 6, 10, 10, 6, 6, 3, 3, 1, 1, 1, 4, 1),          # depth-wise, int32 only
+    (1, 16, 20, 20, 16, 16, 5, 5, 2, 2, 1, 5, 2),       # depth-wise 5x5 stride 2, int8 only
+    (2, 64, 7, 7, 128, 2, 1, 1, 1, 0, 1, 7, 3),         # pointwise, 64 output channels per group
+])
+def test_grouped_convolution(lib, case):
+    N, C, H, W, K, groups, R, S, stride, pad, dil, shift, out_mode = case
+    x = int8_uniform((N, C, H, W), 691)
+    w = int8_uniform((K, C // groups, R, S), 692)
+    bias = int8_uniform((K,), 693).astype(np.int32) * 211
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode=out_mode)
+    P, Q = lib.out_shape(d)
+    plan = lib.Plan(d, groups=groups)
+    assert plan.workspace_bytes() == 0 and plan.info().variant in (b2c.VARIANT_IM2COL_GATHER, b2c.VARIANT_IM2COL_STAGED)
+    xd, wd = to_dev(x), to_dev(w)
+    plan.set_weights(wd)
+    for use_bias, relu in [(False, False), (True, True)]:
+        ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift, groups=groups, bias=bias if use_bias else None, relu=relu)
+        plan.set_activation(to_dev(bias) if use_bias else None, relu)
+        y32 = torch.full((N, K, P, Q), -7777777, dtype=torch.int32, device="cuda") if out_mode & 1 else None
+        y8 = torch.full((N, K, P, Q), 77, dtype=torch.int8, device="cuda") if out_mode & 2 else None
+        plan.run(xd, y32, y8, None)
+        torch.cuda.synchronize()
+        assert plan.device_status() == b2c.OK
+        if y32 is not None:
+            assert np.array_equal(y32.cpu().numpy(), ref[0])
+        if y8 is not None:
+            assert np.array_equal(y8.cpu().numpy(), ref[1])
+    plan.destroy()
+    # argument checks: groups must divide both channel counts; whole tensors must be NCHW / NKPQ
+    raw = lib.load()
+    h = ctypes.c_void_p()
+    assert raw.b2c_plan_create_grouped(ctypes.byref(d), 5, ctypes.byref(h)) == b2c.E_INVALID_ARG
+    d_nhwc = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, 1, 0, out_mode)
+    assert raw.b2c_plan_create_grouped(ctypes.byref(d_nhwc), groups, ctypes.byref(h)) == b2c.E_UNSUPPORTED
+
+
 def test_extreme_values_and_shift_clip(lib):
     # -128 * -128 is the largest product; all-(-128) tensors with 9*64 taps reach 9437184.
     x = np.full((1, 64, 6, 6), -128, dtype=np.int8)
