@@ -115,20 +115,29 @@ bool shift_geom(const Geom& g, const TmaView& v, ShiftGeom* sg, bool tiles_2d) {
   long long rows;
   sg->two_d = 0;
   sg->valid_w = 0;
-  // Wide rows with several taps per filter row: a tile of 128 positions is one row of 128 window
-  // origins, of which the last (S - 1)*dil_w only serve as the taps' overhang (tiles advance by the
-  // valid width), and the window is one box of R rows (+1 for that overhang) of 128 pixels instead
-  // of whole padded rows.
-  const long long wp_full = round_up(v.W + 2 * v.pad_w, 8);
+  // Two-dimensional tiles for the multi-tap views: a tile is 128/pitch rows of `pitch` window origins
+  // (pitch a power of two), its window one TMA box of the rows those origins and their taps touch.
+  // Narrow rows (padded width up to 128, at most a quarter lost to rounding the pitch up): the pitch
+  // covers the whole padded row and a tile is several image rows.  Wide rows (padded width >= 192):
+  // one-row tiles of 128 origins of which the last (S - 1)*dil_w only serve as the taps' overhang
+  // (tiles advance by the valid width).  In between, and for anything else, the window is whole
+  // padded rows (below).
+  const int wp_real = v.W + 2 * v.pad_w;
+  const long long wp_full = round_up(wp_real, 8);
   const int overhang = (v.S - 1) * v.dil_w;
-  if (!tiles_2d && v.S > 1 && v.dil_h == 1 && wp_full >= 192 && overhang <= kTileM / 4) {
+  int pitch = 16;
+  while (pitch < wp_real) pitch <<= 1;
+  const bool narrow_2d = !tiles_2d && pitch <= kTileM && (long long)pitch * 100 <= wp_full * 125;
+  const bool wide_2d = !tiles_2d && v.S > 1 && wp_full >= 192 && overhang <= kTileM / 4;
+  if (narrow_2d || wide_2d) {
     sg->two_d = 1;
-    sg->wps = kTileM;
-    sg->valid_w = kTileM - overhang;
+    sg->wps = narrow_2d ? pitch : kTileM;
+    sg->valid_w = narrow_2d ? wp_real - overhang : kTileM - overhang;
     sg->hp = v.H + 2 * v.pad_h;
-    rows = v.R + 1;
+    const int tile_h = kTileM / sg->wps;
+    rows = tile_h + (long long)(v.R - 1) * v.dil_h + (overhang > 0 ? 1 : 0);
     if (rows > 256) return false;
-    sg->tiles_h = g.P;
+    sg->tiles_h = (g.P + tile_h - 1) / tile_h;
     sg->tiles_w = (g.Q + sg->valid_w - 1) / sg->valid_w;
   } else if (tiles_2d) {
     // tiles of 128/tw x tw pixels over an unpadded view with one tap per filter row: the window is one
