@@ -589,7 +589,15 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
   // The loops below keep stage index, phase bit, tap position and addresses as running
   // counters: each role is a single thread, so every integer division in a loop body would
   // cost hundreds of cycles of dependent issue.
-  if (warp == 0) {
+  // Which of the two single-thread roles sits in warp 0 and which in warp 1.  The warp that issues
+  // the MMAs holds up the other warps of its scheduler while it issues (a per-role clock timeline
+  // shows the epilogue warp with the same warp index modulo 4 finishing about one MMA-issue time
+  // after its siblings), so blocks that walk tiles side by side on one SM put it on different
+  // schedulers: persistent grids are sized in multiples of the SM count, and blocks b, b + 148, ..
+  // are taken to share an SM.
+  const int mma_warp = persistent ? 1 - (int)((blockIdx.x / kNumSMs) & 1u) : 1;
+  const int producer_warp = 1 - mma_warp;
+  if (warp == producer_warp) {
     // ---------------------------------------------------------------- TMA producer
     int s = 0;
     uint32_t ph = 0;
@@ -705,7 +713,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
+  } else if (warp == mma_warp) {
     // ---------------------------------------------------------------- MMA issuer
     {
       const uint32_t idesc = make_idesc_i8(args.tile_n);
