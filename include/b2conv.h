@@ -207,6 +207,27 @@ int b2c_conv2d_int8_host(int N, int C, int H, int W, int K, int R, int S, int st
                          int shift, const int8_t* x_host, const int8_t* w_host, int32_t* y_i32_host,
                          int8_t* y_i8_host);
 
+/* Streaming form for HOST tensors (the layer-by-layer inference loop of Section 4.3 fed from host
+ * memory): the plan keeps its weights, and each call enqueues, without waiting, the copy of one
+ * input batch to the device, the whole path of b2c_conv2d_int8_run on it and the copy of the
+ * outputs desc.out_mode selects back to the host.  The three steps run on three library-owned
+ * streams chained by events over a ring of three device buffer sets, so the copy of the next input
+ * and the read-back of the previous output overlap the kernels of the current call; a fourth call
+ * in flight blocks the host until the oldest one has finished.  x_host: int8 input in
+ * desc.in_layout; y_i32_host / y_i8_host: outputs in desc.out_layout (a selected output must be
+ * non-null, an unselected one is ignored).  The caller owns the host buffers, keeps them unchanged
+ * (x) and unread (y) until b2c_plan_host_sync returns, and should allocate them page-locked:
+ * pageable buffers give correct results but the copies then do not overlap.  Weights, bias and
+ * ReLU flag set on another stream must have completed before the first call.  The first call
+ * allocates the ring and a workspace (B2C_E_CUDA if that fails; nothing is then enqueued);
+ * b2c_plan_destroy frees them.  INVALID_ARG on null plan / x / selected output; NOT_READY without
+ * weights.  Not to be mixed with b2c_conv2d_int8_run on the same plan while calls are in flight. */
+int b2c_plan_run_host_async(b2c_plan* plan, const int8_t* x_host, int32_t* y_i32_host, int8_t* y_i8_host);
+
+/* Blocks until every b2c_plan_run_host_async of this plan has delivered its outputs to the host
+ * buffers.  B2C_OK when nothing is in flight; B2C_E_CUDA if a copy or kernel failed. */
+int b2c_plan_host_sync(b2c_plan* plan);
+
 /* Reads the plan's device status word (synchronises with the device).  *status is B2C_OK or
  * B2C_E_TIMEOUT if a kernel of this plan gave up on a bounded wait; the word is then cleared. */
 int b2c_plan_device_status(b2c_plan* plan, int32_t* status);

@@ -30,7 +30,7 @@ EXPORTS = [
     "b2c_out_shape", "b2c_enumerate", "b2c_plan_create", "b2c_plan_info", "b2c_plan_workspace_bytes",
     "b2c_plan_set_weights", "b2c_conv2d_int8_run", "b2c_conv2d_int8", "b2c_conv2d_int8_host",
     "b2c_plan_rewrite_activations", "b2c_conv2d_int8_run_rewritten", "b2c_plan_footprint", "b2c_plan_set_activation",
-    "b2c_plan_create_grouped",
+    "b2c_plan_create_grouped", "b2c_plan_run_host_async", "b2c_plan_host_sync",
     "b2c_plan_device_status", "b2c_selftest_bounded_wait", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
     "b2c_status_string",
     "b2c_last_cuda_error",
@@ -94,6 +94,8 @@ def load():
     lib.b2c_plan_footprint.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
     lib.b2c_conv2d_int8.argtypes = [i32] * 11 + [vp] * 5
     lib.b2c_conv2d_int8_host.argtypes = [i32] * 11 + [vp] * 4
+    lib.b2c_plan_run_host_async.argtypes = [vp, vp, vp, vp]
+    lib.b2c_plan_host_sync.argtypes = [vp]
     lib.b2c_plan_device_status.argtypes = [vp, pi32]
     lib.b2c_plan_destroy.argtypes = [vp]
     lib.b2c_selftest_bounded_wait.argtypes = [vp, vp]
@@ -207,6 +209,18 @@ class Plan:
         """Only the MMA kernel, epilogue and split finish on an already rewritten workspace (the "Op." half)."""
         _check(self._lib.b2c_conv2d_int8_run_rewritten(self._h, _dptr(x), _dptr(y32), _dptr(y8), _dptr(workspace),
                                                         _stream_ptr(stream)), "b2c_conv2d_int8_run_rewritten")
+
+    def run_host_async(self, x, y32=None, y8=None):
+        """Streaming call on numpy HOST arrays (page-locked for overlap): enqueues copy in, the whole path and
+        copy out, and returns; up to three calls are in flight.  The arrays stay untouched until host_sync()."""
+        def hp(a):
+            return a.ctypes.data_as(ctypes.c_void_p) if a is not None else None
+
+        _check(self._lib.b2c_plan_run_host_async(self._h, hp(x), hp(y32), hp(y8)), "b2c_plan_run_host_async")
+
+    def host_sync(self):
+        """Waits until every run_host_async of this plan has delivered its outputs."""
+        _check(self._lib.b2c_plan_host_sync(self._h), "b2c_plan_host_sync")
 
     def footprint(self) -> Tuple[int, int]:
         """(bytes of the rewritten activation operand, bytes of the packed weights)."""

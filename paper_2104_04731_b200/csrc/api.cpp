@@ -44,6 +44,25 @@ struct b2c_plan {
   int groups = 1;
   std::vector<b2c_plan*> subs;
   long long x_stride_n_whole = 0, y_stride_n_whole = 0;  // sub-plans: batch strides of the whole tensors
+  struct HostPipe* pipe = nullptr;  // streaming host-buffer calls: created by the first b2c_plan_run_host_async
+};
+
+// Device side of the streaming host-buffer calls: a ring of input / output buffers and three
+// streams (copy in, convolve, copy out) chained by events, so that the copy of call i + 1 and the
+// read-back of call i - 1 run beside the kernels of call i.
+struct HostPipe {
+  static constexpr int kSlots = 3;
+  struct Slot {
+    int8_t* x = nullptr;
+    int32_t* y32 = nullptr;
+    int8_t* y8 = nullptr;
+    cudaEvent_t in_done = nullptr, run_done = nullptr, out_done = nullptr;
+    bool used = false;
+  } slot[kSlots];
+  cudaStream_t s_in = nullptr, s_run = nullptr, s_out = nullptr;
+  void* ws = nullptr;
+  size_t x_bytes = 0, y_elems = 0;
+  int next = 0;
 };
 
 namespace {
@@ -910,8 +929,29 @@ int b2c_selftest_bounded_wait(b2c_plan* p, void* cuda_stream) {
   return B2C_OK;
 }
 
+static void destroy_pipe(HostPipe* hp) {
+  if (!hp) return;
+  if (hp->s_in) cudaStreamSynchronize(hp->s_in);
+  if (hp->s_run) cudaStreamSynchronize(hp->s_run);
+  if (hp->s_out) cudaStreamSynchronize(hp->s_out);
+  for (HostPipe::Slot& sl : hp->slot) {
+    cudaFree(sl.x);
+    cudaFree(sl.y32);
+    cudaFree(sl.y8);
+    if (sl.in_done) cudaEventDestroy(sl.in_done);
+    if (sl.run_done) cudaEventDestroy(sl.run_done);
+    if (sl.out_done) cudaEventDestroy(sl.out_done);
+  }
+  cudaFree(hp->ws);
+  if (hp->s_in) cudaStreamDestroy(hp->s_in);
+  if (hp->s_run) cudaStreamDestroy(hp->s_run);
+  if (hp->s_out) cudaStreamDestroy(hp->s_out);
+  delete hp;
+}
+
 void b2c_plan_destroy(b2c_plan* p) {
   if (!p) return;
+  destroy_pipe(p->pipe);
   for (b2c_plan* sub : p->subs) b2c_plan_destroy(sub);
   cudaFree(p->w_packed);
   cudaFree(p->table);
@@ -1007,6 +1047,67 @@ int b2c_conv2d_int8_host(int N, int C, int H, int W, int K, int R, int S, int st
   if (y32h) CUDA_TRY(cudaMemcpyAsync(y32h, dy32, g.y_elems * 4, cudaMemcpyDeviceToHost, st));
   if (y8h) CUDA_TRY(cudaMemcpyAsync(y8h, dy8, g.y_elems, cudaMemcpyDeviceToHost, st));
   CUDA_TRY(cudaStreamSynchronize(st));
+  return B2C_OK;
+}
+
+static int create_pipe(b2c_plan* p) {
+  HostPipe* hp = new (std::nothrow) HostPipe;
+  if (!hp) return B2C_E_CUDA;
+  p->pipe = hp;  // owned by the plan from here on: b2c_plan_destroy frees whatever was created
+  const b2c_conv_desc& d = p->g.d;
+  hp->x_bytes = (size_t)d.N * d.C * d.H * d.W;
+  hp->y_elems = (size_t)d.N * d.K * p->g.PQ;
+  CUDA_TRY(cudaStreamCreateWithFlags(&hp->s_in, cudaStreamNonBlocking));
+  CUDA_TRY(cudaStreamCreateWithFlags(&hp->s_run, cudaStreamNonBlocking));
+  CUDA_TRY(cudaStreamCreateWithFlags(&hp->s_out, cudaStreamNonBlocking));
+  if (p->ws_total) CUDA_TRY(cudaMalloc(&hp->ws, p->ws_total));
+  for (HostPipe::Slot& sl : hp->slot) {
+    CUDA_TRY(cudaMalloc((void**)&sl.x, hp->x_bytes + 256));
+    if (d.out_mode & B2C_OUT_I32) CUDA_TRY(cudaMalloc((void**)&sl.y32, hp->y_elems * 4));
+    if (d.out_mode & B2C_OUT_I8) CUDA_TRY(cudaMalloc((void**)&sl.y8, hp->y_elems));
+    CUDA_TRY(cudaEventCreateWithFlags(&sl.in_done, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventCreateWithFlags(&sl.run_done, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventCreateWithFlags(&sl.out_done, cudaEventDisableTiming));
+  }
+  return B2C_OK;
+}
+
+int b2c_plan_run_host_async(b2c_plan* p, const int8_t* xh, int32_t* y32h, int8_t* y8h) {
+  if (!p || !xh) return B2C_E_INVALID_ARG;
+  const int mode = p->g.d.out_mode;
+  if (((mode & B2C_OUT_I32) && !y32h) || ((mode & B2C_OUT_I8) && !y8h)) return B2C_E_INVALID_ARG;
+  if (!p->pipe) {
+    int rc = create_pipe(p);
+    if (rc != B2C_OK) {
+      destroy_pipe(p->pipe);
+      p->pipe = nullptr;
+      return rc;
+    }
+  }
+  HostPipe* hp = p->pipe;
+  HostPipe::Slot& sl = hp->slot[hp->next];
+  hp->next = (hp->next + 1) % HostPipe::kSlots;
+  // the slot's buffers are free once the read-back of the call that used them last has finished
+  if (sl.used) CUDA_TRY(cudaEventSynchronize(sl.out_done));
+  CUDA_TRY(cudaMemcpyAsync(sl.x, xh, hp->x_bytes, cudaMemcpyHostToDevice, hp->s_in));
+  CUDA_TRY(cudaEventRecord(sl.in_done, hp->s_in));
+  CUDA_TRY(cudaStreamWaitEvent(hp->s_run, sl.in_done, 0));
+  int rc = b2c_conv2d_int8_run(p, sl.x, sl.y32, sl.y8, hp->ws, hp->s_run);
+  if (rc != B2C_OK) return rc;
+  CUDA_TRY(cudaEventRecord(sl.run_done, hp->s_run));
+  CUDA_TRY(cudaStreamWaitEvent(hp->s_out, sl.run_done, 0));
+  if (mode & B2C_OUT_I32) CUDA_TRY(cudaMemcpyAsync(y32h, sl.y32, hp->y_elems * 4, cudaMemcpyDeviceToHost, hp->s_out));
+  if (mode & B2C_OUT_I8) CUDA_TRY(cudaMemcpyAsync(y8h, sl.y8, hp->y_elems, cudaMemcpyDeviceToHost, hp->s_out));
+  CUDA_TRY(cudaEventRecord(sl.out_done, hp->s_out));
+  sl.used = true;
+  return B2C_OK;
+}
+
+int b2c_plan_host_sync(b2c_plan* p) {
+  if (!p) return B2C_E_INVALID_ARG;
+  if (!p->pipe) return B2C_OK;  // nothing was enqueued
+  // every call ends with its read-back on the copy-out stream, which waits for the other two
+  CUDA_TRY(cudaStreamSynchronize(p->pipe->s_out));
   return B2C_OK;
 }
 

@@ -623,3 +623,60 @@ def test_large_grid_staged_window_walks_tiles(lib):
         ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == 3 and e.tile_n == tile_n and e.split_k == 1]
         assert ids
         check_against_oracle(x, w, 2, 3, 1, 7, 3, ids[0], ref=ref)
+
+
+# ---- streaming host-buffer calls: copy in, path and copy out of successive calls overlap ----------
+@pytest.mark.parametrize("policy", [b2c.POLICY_MIN_OVERHEAD, b2c.POLICY_AUTO_TIMED])
+def test_streaming_host_calls(lib, policy):
+    """Eleven calls with different inputs through a ring of three device buffer sets: every output must be
+    the oracle's for ITS input (a slot reused too early, or a read-back that overtakes its kernel, breaks one)."""
+    N, C, H, W, K, R, S, stride, pad, shift = 3, 24, 19, 17, 40, 3, 3, 2, 1, 6
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, shift=shift, out_mode=3)
+    w = int8_uniform((K, C, R, S), 911)
+    plan = lib.Plan(d, policy)
+    raw = lib.load()
+    plan.host_sync()  # nothing enqueued yet: returns at once
+    xs = [torch.from_numpy(int8_uniform((N, C, H, W), 920 + i)).pin_memory().numpy() for i in range(11)]
+    P, Q = lib.out_shape(d)
+    y32 = [torch.zeros((N, K, P, Q), dtype=torch.int32).pin_memory().numpy() for _ in xs]
+    y8 = [torch.zeros((N, K, P, Q), dtype=torch.int8).pin_memory().numpy() for _ in xs]
+    hp = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    assert raw.b2c_plan_run_host_async(plan._h, hp(xs[0]), hp(y32[0]), hp(y8[0])) == b2c.E_NOT_READY
+    plan.set_weights(to_dev(w))
+    torch.cuda.synchronize()
+    assert raw.b2c_plan_run_host_async(plan._h, hp(xs[0]), None, hp(y8[0])) == b2c.E_INVALID_ARG
+    assert raw.b2c_plan_run_host_async(plan._h, None, hp(y32[0]), hp(y8[0])) == b2c.E_INVALID_ARG
+    for i, x in enumerate(xs):
+        plan.run_host_async(x, y32[i], y8[i])
+    plan.host_sync()
+    for i, x in enumerate(xs):
+        want32, want8 = oracle.conv2d_int8(x, w, stride, pad, 1, shift)
+        assert np.array_equal(y32[i], want32), i
+        assert np.array_equal(y8[i], want8), i
+    assert plan.device_status() == b2c.OK
+    # pageable host memory: same results (the copies are then synchronous)
+    xp = int8_uniform((N, C, H, W), 990)
+    o32 = np.zeros((N, K, P, Q), dtype=np.int32)
+    o8 = np.zeros((N, K, P, Q), dtype=np.int8)
+    plan.run_host_async(xp, o32, o8)
+    plan.host_sync()
+    want32, want8 = oracle.conv2d_int8(xp, w, stride, pad, 1, shift)
+    assert np.array_equal(o32, want32) and np.array_equal(o8, want8)
+    plan.destroy()
+
+
+def test_streaming_host_calls_grouped(lib):
+    N, C, H, W, K, R, S, groups = 2, 32, 12, 12, 32, 3, 3, 4
+    d = lib.make_desc(N, C, H, W, K, R, S, 1, 1, out_mode=1)
+    w = int8_uniform((K, C // groups, R, S), 931)
+    plan = lib.Plan(d, groups=groups)
+    plan.set_weights(to_dev(w))
+    torch.cuda.synchronize()
+    xs = [torch.from_numpy(int8_uniform((N, C, H, W), 940 + i)).pin_memory().numpy() for i in range(5)]
+    ys = [torch.zeros((N, K, H, W), dtype=torch.int32).pin_memory().numpy() for _ in xs]
+    for x, y in zip(xs, ys):
+        plan.run_host_async(x, y)
+    plan.host_sync()
+    for x, y in zip(xs, ys):
+        assert np.array_equal(y, oracle.conv2d_int8(x, w, 1, 1, 1, 0, groups=groups)[0])
+    plan.destroy()
