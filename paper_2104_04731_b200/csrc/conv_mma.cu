@@ -544,6 +544,11 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
   int32_t* s_table32 = reinterpret_cast<int32_t*>(smem_extra);                    // A_STAGED
   uint8_t* s_window = smem_extra + ((args.table_len * 4 + 15) & ~15);             // A_STAGED
   constexpr bool kThreadsFormA = (AMODE == A_GATHER || AMODE == A_STAGED);
+  // A 16-column tile is drained by one warp per lane quadrant; the four warps of the second column
+  // half then have nothing to do (unless the threads also form the A operand) and stay out of the
+  // tile loop, so that they neither poll the barriers nor count in the accumulator hand-back.
+  const bool second_half_idle = !kThreadsFormA && args.tile_n < 32;
+  const int epilogue_warps = second_half_idle ? kGatherWarps / 2 : kGatherWarps;
 
   if (warp == 0) {
     if (lane < stages) {
@@ -554,8 +559,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       mbar_init(smem_u32(&ctl.tmem_full[0]), 1);
       if (persistent) {
         mbar_init(smem_u32(&ctl.tmem_full[1]), 1);
-        mbar_init(smem_u32(&ctl.tmem_empty[0]), kGatherWarps);
-        mbar_init(smem_u32(&ctl.tmem_empty[1]), kGatherWarps);
+        mbar_init(smem_u32(&ctl.tmem_empty[0]), epilogue_warps);
+        mbar_init(smem_u32(&ctl.tmem_empty[1]), epilogue_warps);
       }
       ctl.abort_flag = 0;
     }
@@ -851,16 +856,21 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     const int quad = warp & 3;          // TMEM lane quadrant this warp may read
     const int half = (warp - 2) >> 2;   // two warps share a quadrant and split the columns / chunks
     const int row = quad * 32 + lane;   // accumulator row = A-tile row
-    bool ok = true;
+    bool ok = !(second_half_idle && half == 1);
     int ti = 0;
     int s = 0;         // stage ring position of the A-forming threads (runs on across tiles)
     uint32_t ph = 0;
+    // two-dimensional tiles: the pixel of this row inside a tile does not change from tile to tile
+    // (the tile width is a power of two)
+    const int tile_w_log2 = args.remap == 3 ? 31 - __clz(args.sh_wps) : 0;
+    const int tile_h3 = kTileM >> tile_w_log2;
+    const int row_in_tile = row >> tile_w_log2, col_in_tile = row & ((1 << tile_w_log2) - 1);
     for (int t = tile_first; t < tile_end && ok; t += tile_step, ++ti) {
     B2C_TILE_ORIGIN(t)
     const unsigned m = (unsigned)m0 + (unsigned)row;
     bool row_valid = m < (unsigned)(args.swap ? args.K : args.Mg);
     int n_img = 0, pq = 0;
-    if (row_valid && !args.swap) {
+    if (row_valid && !args.swap && args.remap < 2) {
       n_img = (int)args.div_pq.div(m);
       pq = (int)(m - (unsigned)n_img * (unsigned)args.PQ);
     }
@@ -873,10 +883,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       out_img = (int)args.div_tiles_hw.div(tile);
       const int rem = (int)tile - out_img * (args.sh_tiles_h * args.sh_tiles_w);
       const int th = (int)args.div_tiles_w.div((uint32_t)rem), tw = rem - th * args.sh_tiles_w;
-      const int tile_w = args.sh_wps, tile_h = kTileM / tile_w;  // tile width: a power of two
-      const int col = row & (tile_w - 1);
-      const int po = th * tile_h + row / tile_w, qo = tw * args.sh_valid_w + col;
-      row_valid = col < args.sh_valid_w && po < args.out_P && qo < args.out_Q;
+      const int po = th * tile_h3 + row_in_tile, qo = tw * args.sh_valid_w + col_in_tile;
+      row_valid = col_in_tile < args.sh_valid_w && po < args.out_P && qo < args.out_Q;
       out_pq = po * args.out_Q + qo;
     } else if (args.remap == 2 && row_valid) {
       // shift execution: row m is window origin (n, hp, wp) on the padded grid of sh_hp x sh_wps positions
