@@ -27,8 +27,8 @@ constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s
 struct __align__(8) SharedCtl {
   unsigned long long full[8];
   unsigned long long empty[8];
-  unsigned long long tmem_full[2];   // accumulator buffer b complete (MMA warp -> epilogue warps)
-  unsigned long long tmem_empty[2];  // accumulator buffer b drained (epilogue warps -> MMA warp)
+  unsigned long long tmem_full[4];   // accumulator buffer b complete (MMA warp -> epilogue warps)
+  unsigned long long tmem_empty[4];  // accumulator buffer b drained (epilogue warps -> MMA warp)
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -513,7 +513,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
   const int tile_first = persistent ? (int)blockIdx.x : 0;
   const int tile_step = persistent ? (int)gridDim.x : 1;
   const int tile_end = persistent ? args.num_tiles : 1;
-  const int nbuf = persistent ? args.tmem_bufs : 1;
+  const int nbuf = persistent ? args.tmem_bufs : 1;  // a power of two, at most 4
+  const int nbuf_log2 = nbuf == 4 ? 2 : (nbuf == 2 ? 1 : 0);
 #define B2C_TILE_ORIGIN(t)                                                          \
   int m0, n0;                                                                       \
   if (persistent) {                                                                 \
@@ -548,7 +549,12 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
   // half then have nothing to do (unless the threads also form the A operand) and stay out of the
   // tile loop, so that they neither poll the barriers nor count in the accumulator hand-back.
   const bool second_half_idle = !kThreadsFormA && args.tile_n < 32;
-  const int epilogue_warps = second_half_idle ? kGatherWarps / 2 : kGatherWarps;
+  // Shift execution with two accumulator buffers: the two warps of a lane quadrant take turns, one
+  // draining the even tiles of the block's walk (buffer 0), the other the odd ones (buffer 1), each
+  // all columns of its tile.  The work per warp is the same as with split columns, but the per-tile
+  // fixed cost (barrier wait, tile coordinates, hand-back) is paid for every second tile only.
+  const bool alternate = persistent && AMODE == A_SHIFT && args.tmem_bufs >= 2;
+  const int epilogue_warps = (second_half_idle || alternate) ? kGatherWarps / 2 : kGatherWarps;
 
   if (warp == 0) {
     if (lane < stages) {
@@ -558,9 +564,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     if (lane == 8) {
       mbar_init(smem_u32(&ctl.tmem_full[0]), 1);
       if (persistent) {
-        mbar_init(smem_u32(&ctl.tmem_full[1]), 1);
-        mbar_init(smem_u32(&ctl.tmem_empty[0]), epilogue_warps);
-        mbar_init(smem_u32(&ctl.tmem_empty[1]), epilogue_warps);
+        for (int b = 1; b < 4; ++b) mbar_init(smem_u32(&ctl.tmem_full[b]), 1);
+        for (int b = 0; b < 4; ++b) mbar_init(smem_u32(&ctl.tmem_empty[b]), epilogue_warps);
       }
       ctl.abort_flag = 0;
     }
@@ -746,8 +751,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         const bool rows_as_taps = args.S == 1;
         const int sh_R = rows_as_taps ? 1 : args.sh_R, sh_S = rows_as_taps ? args.sh_R : args.S, sh_ncb = args.sh_ncb;
         for (int t = tile_first; t < tile_end && alive; t += tile_step, ++ti) {
-          const int buf = ti % nbuf;
-          const uint32_t use = (uint32_t)(ti / nbuf);
+          const int buf = ti & (nbuf - 1);
+          const uint32_t use = (uint32_t)(ti >> nbuf_log2);
           // (votes: the outcome of a wait is the same for all lanes, and saying so keeps the loop's
           // control flow, and with it the descriptor arithmetic, warp-uniform for the compiler)
           if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status))) break;
@@ -814,8 +819,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         alive = false;  // the generic stage loop below is not used
       }
       for (int t = tile_first; t < tile_end && alive; t += tile_step, ++ti) {
-      const int buf = persistent ? ti % nbuf : 0;
-      const uint32_t use = persistent ? (uint32_t)(ti / nbuf) : 0u;
+      const int buf = persistent ? (ti & (nbuf - 1)) : 0;
+      const uint32_t use = persistent ? (uint32_t)(ti >> nbuf_log2) : 0u;
       if (persistent) {
         // the epilogue must have drained this accumulator buffer (first use passes at once)
         if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status))) break;
@@ -856,7 +861,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     const int quad = warp & 3;          // TMEM lane quadrant this warp may read
     const int half = (warp - 2) >> 2;   // two warps share a quadrant and split the columns / chunks
     const int row = quad * 32 + lane;   // accumulator row = A-tile row
-    bool ok = !(second_half_idle && half == 1);
+    bool ok = alternate || !(second_half_idle && half == 1);
     int ti = 0;
     int s = 0;         // stage ring position of the A-forming threads (runs on across tiles)
     uint32_t ph = 0;
@@ -866,6 +871,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     const int tile_h3 = kTileM >> tile_w_log2;
     const int row_in_tile = row >> tile_w_log2, col_in_tile = row & ((1 << tile_w_log2) - 1);
     for (int t = tile_first; t < tile_end && ok; t += tile_step, ++ti) {
+    if (alternate && (ti & 1) != half) continue;
     B2C_TILE_ORIGIN(t)
     const unsigned m = (unsigned)m0 + (unsigned)row;
     bool row_valid = m < (unsigned)(args.swap ? args.K : args.Mg);
@@ -1079,16 +1085,16 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     }
 
     // ---- epilogue ----
-    const int buf = persistent ? ti % nbuf : 0;
-    const uint32_t use = persistent ? (uint32_t)(ti / nbuf) : 0u;
+    const int buf = persistent ? (ti & (nbuf - 1)) : 0;
+    const uint32_t use = persistent ? (uint32_t)(ti >> nbuf_log2) : 0u;
     if (ok) ok = mbar_wait(smem_u32(&ctl.tmem_full[buf]), use & 1u, &ctl, args.status);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
       // Output index of (m, k): NKPQ -> (n*K + k)*PQ + pq ; NPQK -> m*K + k.
       const long long base_nkpq = (long long)out_img * args.y_stride_n + out_pq;
       const long long base_npqk = args.remap ? ((long long)out_img * args.out_PQ + out_pq) * args.K : (long long)m * args.K;
-      const int cols = args.tile_n >= 32 ? (args.tile_n >> 1) : 16;  // columns handled by this warp
-      const int c_begin = half * cols;
+      const int cols = alternate ? args.tile_n : (args.tile_n >= 32 ? (args.tile_n >> 1) : 16);  // columns handled by this warp
+      const int c_begin = alternate ? 0 : half * cols;
       if (c_begin < args.tile_n) {
         const uint32_t taddr =
             tmem_acc + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * args.tmem_cols) + (uint32_t)c_begin;
