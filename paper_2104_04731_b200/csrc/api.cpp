@@ -246,7 +246,9 @@ void fill_common_args(b2c_plan* p) {
     a.ksteps_last = (p->K_pad - (a.num_kb - 1) * 128) / kMmaK;
     a.kb_per_tap = 1;
   }
-  // Pipeline depth: as many stages as the reduction slice has blocks, at most 6, within 160 KB.
+  // Pipeline depth: as many stages as the reduction slice has blocks, at most 6, within 196 KB (a
+  // block that is alone with its tile is paced by the copies it has in flight: a fourth 48 KB stage
+  // took 9 % off the 128 x 256 kernel of the 3x3 stride-2 256 -> 512 layer).
   // When the grid has more blocks than the machine has SMs, stay within 100 KB (but keep at least
   // two stages) so that two blocks are resident per SM: one block's epilogue and set-up then
   // overlap the other's main loop.
@@ -273,7 +275,7 @@ void fill_common_args(b2c_plan* p) {
       tiles_m * tiles_n < 0x7FFFFFFF)
     a.persistent = 2;
   a.tmem_bufs = (a.persistent && 2 * a.tmem_cols <= 512) ? 2 : 1;
-  const size_t budget = a.persistent == 1 ? 196 * 1024 : (a.persistent == 2 ? 68 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 160 * 1024));
+  const size_t budget = a.persistent == 1 ? 196 * 1024 : (a.persistent == 2 ? 68 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 196 * 1024));
   const size_t stage_bytes = (size_t)(kTileM + a.tile_n) * a.bk;
   // lookup table and staged window share the block's shared memory with the stages
   const size_t extra = p->amode == A_STAGED ? (size_t)p->win.bytes + 4 * (size_t)p->table_len + 64
