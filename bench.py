@@ -39,7 +39,7 @@ INT8_TO_BF16_RATIO = 2.0  # nominal dense int8 : bf16 tensor throughput on B200 
 
 # DRAM traffic of the dominant kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
 # per launch), valid only for the kernel source it was taken on; see profiles/.
-NCU_TRAFFIC = {"conv_mma_sha1": "f3ca284351610c736514d263cdb4837e9b89902d", "bytes_per_launch": 2859008}
+NCU_TRAFFIC = {"conv_mma_sha1": "8977bd1d72acdd803f1b71b95fed946eb0e61f2c", "bytes_per_launch": 2859008}
 
 
 def load_peaks():
