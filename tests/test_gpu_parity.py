@@ -376,13 +376,25 @@ def test_shift_execution_long_tile_walk(lib):
 
 
 def test_shift_execution_many_tiles(lib):
-    # enough tiles for every block of the persistent grid to walk several, both accumulator buffers in use
-    x = int8_uniform((40, 32, 28, 28), 673)
+    # enough tiles (2800) for every block of the persistent grid to walk several: both accumulator buffers
+    # wrap, and the two epilogue warps of each lane quadrant take alternate tiles (32 columns each)
+    x = int8_uniform((400, 32, 28, 28), 673)
     w = int8_uniform((32, 32, 3, 3), 674)
     ref = oracle.conv2d_int8(x, w, 1, 1, 1, 9)
-    d = lib.make_desc(40, 32, 28, 28, 32, 3, 3, 1, 1, 1, 9, out_mode=3)
+    d = lib.make_desc(400, 32, 28, 28, 32, 3, 3, 1, 1, 1, 9, out_mode=3)
     e = next(e for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_CP_SHIFT)
     check_against_oracle(x, w, 1, 1, 1, 9, 3, e.id, ref=ref)
+
+
+def test_shift_execution_four_accumulator_buffers(lib):
+    # 64-column tiles use a ring of four accumulator buffers; cfg 2's layer at batch 120 gives every block
+    # about eleven tiles, so the ring wraps more than twice (odd tile counts per block included)
+    x = int8_uniform((120, 64, 56, 56), 677)
+    w = int8_uniform((64, 64, 3, 3), 678)
+    ref = oracle.conv2d_int8(x, w, 1, 1, 1, 10)
+    d = lib.make_desc(120, 64, 56, 56, 64, 3, 3, 1, 1, 1, 10, out_mode=3)
+    e = next(e for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_CP_SHIFT)
+    check_against_oracle(x, w, 1, 1, 1, 10, 3, e.id, ref=ref)
 
 
 # ---- grouped / depth-wise convolution: one dense convolution per group on channel slices in place --------
