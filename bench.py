@@ -38,8 +38,10 @@ L2_BYTES = 126 * 1024 * 1024
 INT8_TO_BF16_RATIO = 2.0  # nominal dense int8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
 
 # DRAM traffic of the dominant kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
-# per launch), valid only for the kernel source it was taken on; see profiles/.
-NCU_TRAFFIC = {"conv_mma_sha1": "8977bd1d72acdd803f1b71b95fed946eb0e61f2c", "bytes_per_launch": 2859008}
+# per launch), valid only for the sources it was taken on (the kernel and the host code that picks its
+# tile, stage count and launch shape); see profiles/.
+KERNEL_SOURCES = ("conv_mma.cu", "api.cpp", "planner.cpp", "tma.cpp", "b2c_internal.h")
+NCU_TRAFFIC = {"conv_mma_sha1": "2f7f0c9ebef77a24137d8c3d4168093c86fde328", "bytes_per_launch": 2859008}
 
 
 def load_peaks():
@@ -647,7 +649,8 @@ def run_ours(args):
         achieved, peak, runit = ops / (op_us * 1e-6) / 1e12, peaks["bf16_tflops"] * INT8_TO_BF16_RATIO, "TFLOP/s"
     else:
         achieved, peak, runit = cfg.algorithmic_bytes / (op_us * 1e-6) / 1e9, peaks["hbm_gbs"], "GB/s"
-    sha = hashlib.sha1(open(os.path.join(ROOT, "paper_2104_04731_b200", "csrc", "conv_mma.cu"), "rb").read()).hexdigest()
+    sha = hashlib.sha1(b"".join(open(os.path.join(ROOT, "paper_2104_04731_b200", "csrc", f), "rb").read()
+                                for f in KERNEL_SOURCES)).hexdigest()
     traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["conv_mma_sha1"] == sha else None
     roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
                 "traffic": traffic, "kernel": "conv_mma_kernel", "kernel_us": op_us,
