@@ -207,8 +207,9 @@ int b2c_conv2d_int8_host(int N, int C, int H, int W, int K, int R, int S, int st
                          int shift, const int8_t* x_host, const int8_t* w_host, int32_t* y_i32_host,
                          int8_t* y_i8_host);
 
-/* Streaming form for HOST tensors (the layer-by-layer inference loop of Section 4.3 fed from host
- * memory): the plan keeps its weights, and each call enqueues, without waiting, the copy of one
+/* Streaming form for HOST tensors (the micro-benchmark of Section 5.1 runs packing, convolution,
+ * activation and unpacking on tensors that start and end in host memory; this is that loop with the
+ * copies across the host link pipelined around the path): the plan keeps its weights, and each call enqueues, without waiting, the copy of one
  * input batch to the device, the whole path of b2c_conv2d_int8_run on it and the copy of the
  * outputs desc.out_mode selects back to the host.  The three steps run on three library-owned
  * streams chained by events over a ring of three device buffer sets, so the copy of the next input
