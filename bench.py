@@ -192,6 +192,23 @@ class Instances:
         else:
             self.run_all()
 
+    def verify(self, which=(0, -1)):
+        """Compares the outputs the last step left in the given instances with the CPU oracle, element by
+        element (every instance has the same seeded input and weights)."""
+        import oracle
+        import torch
+
+        c = self.cfg
+        x, w = c.tensors()
+        ref32, ref8 = oracle.conv2d_int8(x, w, c.stride, c.pad, c.dilation, c.shift)
+        torch.cuda.synchronize()
+        for i in which:
+            if self.y32[i] is not None and not np.array_equal(self.y32[i].cpu().numpy(), ref32):
+                return False
+            if self.y8[i] is not None and not np.array_equal(self.y8[i].cpu().numpy(), ref8):
+                return False
+        return True
+
     def check_status(self, b2c):
         for p in self.plans:
             s = p.device_status()
@@ -252,6 +269,7 @@ def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, grap
         inst.capture(torch)
     ms = time_steps(torch, inst.step, steps, warmup, dist)
     inst.check_status(b2c)
+    verified = inst.verify()
     per_call_us = ms * 1e3 / (steps * G)
     emb = inst.emb.as_dict()
     launches = inst.launches_per_instance
@@ -270,13 +288,14 @@ def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, grap
         "op_us": op["us"] if op else None, "transf_us": max(0.0, per_call_us - op["us"]) if op else None, "cold": bool(G * cfg.algorithmic_bytes >= L2_BYTES), "combined_us": per_call_us, "tops": 2.0 * cfg.macs / (per_call_us * 1e-6) / 1e12,
         "roofline_us": t_roof, "bound": bound, "roofline_frac": t_roof / per_call_us,
         "embedding": {k: emb[k] for k in keys},
-        "launches_per_call": launches,
+        "launches_per_call": launches, "verified": verified,
     }
     if graph and streams > 1:
         conc = Instances(b2c, torch, cfg, G, b2c.POLICY_AUTO_TIMED_CONCURRENT)
         conc.capture(torch, streams=streams)
         ms_c = time_steps(torch, conc.step, steps, warmup, dist)
         conc.check_status(b2c)
+        res["concurrent_verified"] = conc.verify()
         us_c = ms_c * 1e3 / (steps * G)
         emb_c = conc.emb.as_dict()
         conc.destroy()
@@ -631,6 +650,10 @@ def run_ours(args):
     ms = time_steps(torch, inst.step, args.steps, args.warmup, dist, args.min_warm_s)
     inst.check_status(b2c)
     clocks = sampler.stop() if rank == 0 else None
+    # the timed graph did the work: first and last instance of the last step against the oracle
+    verified = inst.verify() if rank == 0 else None
+    if verified is False:
+        raise SystemExit("bench: the timed graph's output differs from the oracle")
     emb = inst.emb
     launches = inst.launches_per_instance * G * args.steps
     ops = 2.0 * cfg.macs
@@ -703,7 +726,7 @@ def run_ours(args):
                    "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k,
                                  "swapped": emb.map_m == b2c.AXIS_K, "planner_us": emb.device_us}},
         "roofline": roofline, "roofline_time_us": t_roof, "whole_path_roofline_frac": t_roof / per_call_us,
-        "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+        "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "verified": verified,
     }
     if cpu is not None:
         line["cpu_baseline"] = cpu
@@ -741,6 +764,16 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain script: start one rank per GPU (the same command a launcher would give)
+        import socket
+
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        return subprocess.call(cmd)
     return run_ours(args)
 
 

@@ -194,12 +194,26 @@ int b2c_plan_footprint(const b2c_plan* plan, size_t* rewritten_bytes, size_t* pa
 /* One-shot form of the paper's problem statement: NCHW int8 input, KCRS int8 weights, NKPQ
  * outputs (either may be NULL, not both), symmetric stride / pad / dilation.  All four tensor
  * pointers are DEVICE pointers.  Keeps plans and scratch in a library-owned cache keyed by
- * shape: the first call for a shape picks the embedding by timed selection (it allocates and
- * synchronises with the device, so make it outside any stream capture); later calls only
- * re-pack the weights and enqueue on `cuda_stream`. */
+ * (shape, output mode, device, cuda_stream): the first call for a key picks the embedding by
+ * timed selection (it allocates and synchronises with the device, so make it outside any stream
+ * capture); later calls only re-pack the weights and enqueue on `cuda_stream`.
+ * Ordering: every call re-packs w into its cached plan's weight buffer and runs in that plan's
+ * scratch.  Calls with the same key are ordered by their stream, so one call's buffers are never
+ * rewritten under another; calls on different streams use different cached plans and may overlap
+ * on the GPU.  Two host threads may call concurrently (the enqueue is serialised inside).
+ * A bounded device wait that expired inside a one-shot call is reported by b2c_oneshot_status. */
 int b2c_conv2d_int8(int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int dilation,
                     int shift, const int8_t* x_dev, const int8_t* w_dev, int32_t* y_i32_dev,
                     int8_t* y_i8_dev, void* cuda_stream);
+
+/* Device status of the one-shot cache on the current device: *status is B2C_OK, or B2C_E_TIMEOUT if a
+ * kernel enqueued by b2c_conv2d_int8 / b2c_conv2d_int8_host gave up on a bounded wait since the last
+ * query (the words are then cleared).  Waits for the device to be idle first. */
+int b2c_oneshot_status(int32_t* status);
+
+/* Frees every cached one-shot plan of the current device (packed weights, scratch, status words)
+ * after waiting for the device to be idle.  The next one-shot call of a shape selects again. */
+int b2c_oneshot_cache_clear(void);
 
 /* Same operation with HOST tensors: copies x and w to the device, runs, copies the requested
  * outputs back and synchronises.  Convenience for callers without device memory of their own. */
@@ -229,8 +243,10 @@ int b2c_plan_run_host_async(b2c_plan* plan, const int8_t* x_host, int32_t* y_i32
  * buffers.  B2C_OK when nothing is in flight; B2C_E_CUDA if a copy or kernel failed. */
 int b2c_plan_host_sync(b2c_plan* plan);
 
-/* Reads the plan's device status word (synchronises with the device).  *status is B2C_OK or
- * B2C_E_TIMEOUT if a kernel of this plan gave up on a bounded wait; the word is then cleared. */
+/* Reads the plan's device status word after waiting for ALL work on the current device to finish
+ * (cudaDeviceSynchronize: the plan does not know which streams its kernels were enqueued on).
+ * *status is B2C_OK or B2C_E_TIMEOUT if a kernel of this plan gave up on a bounded wait; the word is
+ * then cleared.  Not to be called while a stream is being captured. */
 int b2c_plan_device_status(b2c_plan* plan, int32_t* status);
 
 /* Failure-detection self-test (no counterpart in the paper): enqueues a one-block kernel that
@@ -239,11 +255,19 @@ int b2c_plan_device_status(b2c_plan* plan, int32_t* status);
  * word and returns normally; b2c_plan_device_status then reports it and the plan stays usable. */
 int b2c_selftest_bounded_wait(b2c_plan* plan, void* cuda_stream);
 
+/* The same self-test for the activation-pack kernel's wait on its bulk copies (no counterpart in the
+ * paper): one block waits for bytes that no copy delivers, gives up after about one second, records
+ * B2C_E_TIMEOUT in the plan's status word and returns normally. */
+int b2c_selftest_pack_wait(b2c_plan* plan, void* cuda_stream);
+
 void b2c_plan_destroy(b2c_plan* plan);
 
 /* Layout rewrites on their own (the Pad / Reorder / Stencil Unroll rules of Table 2), exposed so
  * they can be checked and timed separately.  b2c_pack_activations is asynchronous on
- * `cuda_stream`; b2c_im2col builds a temporary lookup table and synchronises the stream.
+ * `cuda_stream` (called on its own it has no status word: a block whose bounded wait for its
+ * bulk copies expires leaves its part of the output unwritten; inside a plan's run the same
+ * kernel records B2C_E_TIMEOUT in the plan's status word); b2c_im2col builds a temporary lookup
+ * table and synchronises the stream.
  * b2c_pack_activations: int8 NCHW [N][C][H][W] -> NHWC [N][H][W][C_pad], channels >= C zero;
  *   C_pad must be a multiple of 16 and >= C.
  * b2c_im2col: int8 input in desc.in_layout -> A[N*P*Q][K_pad], row m = (n, p, q), column
@@ -269,6 +293,11 @@ int b2c_im2col(const b2c_conv_desc* desc, const int8_t* x_dev, int8_t* a_dev, in
  *     calls whose kernels can overlap on the GPU (different streams, no ordering) race: order
  *     them on one stream or with events. */
 int b2c_im2col_noalloc(const b2c_conv_desc* desc, const int8_t* x_dev, int8_t* a_dev, int K_pad, void* cuda_stream);
+
+/* Host-side fault injection for tests (no counterpart in the paper): the n-th tensor-map encode
+ * from now on, counted over all threads, fails as if the driver had refused it (the call that
+ * needed it returns B2C_E_CUDA); n = 0 disarms.  Nothing on the device is touched. */
+int b2c_test_fail_nth_encode(int n);
 
 const char* b2c_status_string(int status);
 

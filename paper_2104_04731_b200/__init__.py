@@ -33,7 +33,7 @@ EXPORTS = [
     "b2c_plan_create_grouped", "b2c_plan_run_host_async", "b2c_plan_host_sync",
     "b2c_plan_device_status", "b2c_selftest_bounded_wait", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
     "b2c_status_string",
-    "b2c_last_cuda_error",
+    "b2c_last_cuda_error", "b2c_oneshot_status", "b2c_oneshot_cache_clear", "b2c_test_fail_nth_encode", "b2c_selftest_pack_wait",
 ]
 
 
@@ -99,6 +99,7 @@ def load():
     lib.b2c_plan_device_status.argtypes = [vp, pi32]
     lib.b2c_plan_destroy.argtypes = [vp]
     lib.b2c_selftest_bounded_wait.argtypes = [vp, vp]
+    lib.b2c_selftest_pack_wait.argtypes = [vp, vp]
     lib.b2c_plan_destroy.restype = None
     lib.b2c_pack_activations.argtypes = [vp, vp] + [i32] * 5 + [vp]
     lib.b2c_im2col.argtypes = [pd, vp, vp, i32, vp]
@@ -106,6 +107,9 @@ def load():
     lib.b2c_status_string.argtypes = [i32]
     lib.b2c_status_string.restype = ctypes.c_char_p
     lib.b2c_last_cuda_error.argtypes = []
+    lib.b2c_oneshot_status.argtypes = [pi32]
+    lib.b2c_oneshot_cache_clear.argtypes = []
+    lib.b2c_test_fail_nth_encode.argtypes = [i32]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("b2c_plan_destroy", "b2c_status_string"):
@@ -237,6 +241,10 @@ class Plan:
         """Enqueues the bounded-wait self-test; afterwards device_status() reports E_TIMEOUT once."""
         _check(self._lib.b2c_selftest_bounded_wait(self._h, _stream_ptr(stream)), "b2c_selftest_bounded_wait")
 
+    def selftest_pack_wait(self, stream=None):
+        """The same self-test for the activation-pack kernel's wait on its bulk copies."""
+        _check(self._lib.b2c_selftest_pack_wait(self._h, _stream_ptr(stream)), "b2c_selftest_pack_wait")
+
     def destroy(self):
         if getattr(self, "_h", None):
             self._lib.b2c_plan_destroy(self._h)
@@ -255,6 +263,23 @@ def conv2d_int8(x, w, stride=1, pad=0, dilation=1, shift=0, y32=None, y8=None, s
     K, _, R, S = w.shape
     _check(load().b2c_conv2d_int8(N, C, H, W, K, R, S, stride, pad, dilation, shift, _dptr(x), _dptr(w), _dptr(y32),
                                   _dptr(y8), _stream_ptr(stream)), "b2c_conv2d_int8")
+
+
+def oneshot_status() -> int:
+    """Status of the one-shot cache on the current device (E_TIMEOUT once after a bounded wait expired)."""
+    s = ctypes.c_int32()
+    _check(load().b2c_oneshot_status(ctypes.byref(s)), "b2c_oneshot_status")
+    return s.value
+
+
+def oneshot_cache_clear():
+    """Frees the plans and scratch the one-shot calls cached on the current device."""
+    _check(load().b2c_oneshot_cache_clear(), "b2c_oneshot_cache_clear")
+
+
+def test_fail_nth_encode(n: int):
+    """Host-side fault injection: the n-th tensor-map encode from now on fails (0 disarms)."""
+    _check(load().b2c_test_fail_nth_encode(n), "b2c_test_fail_nth_encode")
 
 
 def conv2d_int8_host(x, w, stride=1, pad=0, dilation=1, shift=0, y32=None, y8=None):

@@ -520,9 +520,16 @@ int time_plan(b2c_plan* p, const int8_t* x, const LaneBuffers* lane, int lanes, 
   return rc;
 }
 
+// Key of the one-shot cache: shape, output mode, device and the stream the call enqueues on.  Calls on
+// one stream are ordered by the stream; calls on different streams get plans (packed weights,
+// scratch, status word) of their own, so they may overlap on the GPU.
 struct ShapeKey {
   int v[12];
-  bool operator<(const ShapeKey& o) const { return std::memcmp(v, o.v, sizeof(v)) < 0; }
+  uintptr_t stream;
+  bool operator<(const ShapeKey& o) const {
+    const int c = std::memcmp(v, o.v, sizeof(v));
+    return c != 0 ? c < 0 : stream < o.stream;
+  }
 };
 std::mutex g_cache_mu;
 std::map<ShapeKey, b2c_plan*> g_cache;
@@ -626,17 +633,23 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
   cudaStreamSynchronize(st);
   int best = -1;
   float best_us = 0;
+  int first_error = B2C_OK;
   for (size_t i = 0; i < all.size(); ++i) {
     if (std::find(groups.begin(), groups.end(), variant_family(all[i].variant)) == groups.end()) continue;
+    // A candidate that cannot be built or run (a tensor map the driver refuses, an allocation that
+    // fails, a device wait that expires) is left out of the selection; the others are still timed.
     b2c_plan* p = nullptr;
     rc = create_plan_for(g, all[i], &p);
-    if (rc != B2C_OK) break;
-    rc = b2c_plan_set_weights(p, w, st);
+    if (rc == B2C_OK) rc = b2c_plan_set_weights(p, w, st);
     if (rc == B2C_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = B2C_E_CUDA;
     float us = -1;
     if (rc == B2C_OK) rc = time_plan(p, x, lane, lanes, &us);
     b2c_plan_destroy(p);
-    if (rc != B2C_OK) break;
+    if (rc != B2C_OK) {
+      if (first_error == B2C_OK) first_error = rc;
+      if (cudaGetLastError() != cudaSuccess && cudaDeviceSynchronize() != cudaSuccess) break;  // the context is lost
+      continue;
+    }
     all[i].device_us = us;
     if (best < 0 || us < best_us) {
       best = (int)i;
@@ -644,8 +657,7 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
     }
   }
   cleanup();
-  if (rc != B2C_OK) return rc;
-  if (best < 0) return B2C_E_UNSUPPORTED;
+  if (best < 0) return first_error != B2C_OK ? first_error : B2C_E_UNSUPPORTED;
   return create_plan_for(g, all[best], out);
 }
 
@@ -759,7 +771,7 @@ static int run_rewrite(b2c_plan* p, const int8_t* x, void* ws, cudaStream_t st) 
     const TmaView& v = p->view;
     const int base_variant = shift_base_variant(p->emb.variant);
     if (base_variant == B2C_VARIANT_CP_TMA) {
-      CUDA_TRY(launch_pack_activations(x, scratch, d.N, d.C, d.H, d.W, p->C_pad, st));
+      CUDA_TRY(launch_pack_activations(x, scratch, d.N, d.C, d.H, d.W, p->C_pad, st, p->status));
     } else if (base_variant == B2C_VARIANT_DILATION_PACK) {
       const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
       CUDA_TRY(launch_phase_split(x, scratch, d.N, d.C, d.H, d.W, d.dil_h, d.dil_w, v.H, v.W, v.C, a.x_stride_n,
@@ -916,6 +928,9 @@ int b2c_plan_footprint(const b2c_plan* p, size_t* rewritten_bytes, size_t* packe
 int b2c_plan_device_status(b2c_plan* p, int32_t* status) {
   if (!p || !status) return B2C_E_INVALID_ARG;
   int s = 0;
+  // (a plain cudaMemcpy only orders against blocking streams; kernels of this plan may run on
+  // non-blocking ones, so wait for the whole device first)
+  CUDA_TRY(cudaDeviceSynchronize());
   CUDA_TRY(cudaMemcpy(&s, p->status, sizeof(int), cudaMemcpyDeviceToHost));
   if (s != 0) CUDA_TRY(cudaMemset(p->status, 0, sizeof(int)));
   for (b2c_plan* sub : p->subs) {  // a group plan reports the first sub-plan status that is set
@@ -931,6 +946,12 @@ int b2c_plan_device_status(b2c_plan* p, int32_t* status) {
 int b2c_selftest_bounded_wait(b2c_plan* p, void* cuda_stream) {
   if (!p) return B2C_E_INVALID_ARG;
   CUDA_TRY(launch_bounded_wait_selftest(p->status, (cudaStream_t)cuda_stream));
+  return B2C_OK;
+}
+
+int b2c_selftest_pack_wait(b2c_plan* p, void* cuda_stream) {
+  if (!p) return B2C_E_INVALID_ARG;
+  CUDA_TRY(launch_pack_wait_selftest(p->status, (cudaStream_t)cuda_stream));
   return B2C_OK;
 }
 
@@ -983,7 +1004,8 @@ int b2c_conv2d_int8(int N, int C, int H, int W, int K, int R, int S, int stride,
   d.out_mode = (y32 ? B2C_OUT_I32 : 0) | (y8 ? B2C_OUT_I8 : 0);
   int dev = 0;
   cudaGetDevice(&dev);
-  ShapeKey key = {{N, C, H, W, K, R, S, stride, pad, dilation, shift, d.out_mode * 64 + dev}};
+  ShapeKey key = {{N, C, H, W, K, R, S, stride, pad, dilation, shift, d.out_mode * 64 + dev},
+                  reinterpret_cast<uintptr_t>(cuda_stream)};
   std::lock_guard<std::mutex> lock(g_cache_mu);
   b2c_plan* p = nullptr;
   auto it = g_cache.find(key);
@@ -1005,6 +1027,43 @@ int b2c_conv2d_int8(int N, int C, int H, int W, int K, int R, int S, int stride,
   int rc = b2c_plan_set_weights(p, w, cuda_stream);
   if (rc != B2C_OK) return rc;
   return b2c_conv2d_int8_run(p, x, y32, y8, p->own_ws, cuda_stream);
+}
+
+int b2c_oneshot_status(int32_t* status) {
+  if (!status) return B2C_E_INVALID_ARG;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  std::lock_guard<std::mutex> lock(g_cache_mu);
+  int32_t first = B2C_OK;
+  for (auto& kv : g_cache) {
+    if (kv.second->device != dev) continue;
+    int32_t s = B2C_OK;
+    int rc = b2c_plan_device_status(kv.second, &s);
+    if (rc != B2C_OK) return rc;
+    if (first == B2C_OK) first = s;
+  }
+  *status = first;
+  return B2C_OK;
+}
+
+int b2c_oneshot_cache_clear(void) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  std::lock_guard<std::mutex> lock(g_cache_mu);
+  bool synced = false;
+  for (auto it = g_cache.begin(); it != g_cache.end();) {
+    if (it->second->device != dev) {
+      ++it;
+      continue;
+    }
+    if (!synced) {
+      CUDA_TRY(cudaDeviceSynchronize());  // work enqueued by earlier one-shot calls may still use the buffers
+      synced = true;
+    }
+    b2c_plan_destroy(it->second);
+    it = g_cache.erase(it);
+  }
+  return B2C_OK;
 }
 
 int b2c_conv2d_int8_host(int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int dilation, int shift,
@@ -1119,7 +1178,7 @@ int b2c_plan_host_sync(b2c_plan* p) {
 int b2c_pack_activations(const int8_t* x, int8_t* out, int N, int C, int H, int W, int C_pad, void* cuda_stream) {
   if (!x || !out || N < 1 || C < 1 || H < 1 || W < 1 || C_pad < C || (C_pad % 16) != 0) return B2C_E_INVALID_ARG;
   if (!aligned16(x) || !aligned16(out)) return B2C_E_INVALID_ARG;
-  CUDA_TRY(launch_pack_activations(x, out, N, C, H, W, C_pad, (cudaStream_t)cuda_stream));
+  CUDA_TRY(launch_pack_activations(x, out, N, C, H, W, C_pad, (cudaStream_t)cuda_stream, nullptr));
   return B2C_OK;
 }
 

@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <vector>
 
 #include "b2conv.h"
@@ -168,6 +169,20 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 }
 #endif
 
+// Opt-in to more than 48 KB of dynamic shared memory for one kernel.  The attribute belongs to the
+// current device's context, so it is set once per (kernel, device): `done` holds one bit per device
+// ordinal (devices past 63 set it on every launch).  Safe from concurrent host threads.
+inline cudaError_t set_max_dynamic_smem_once(std::atomic<unsigned long long>& done, const void* kernel, int bytes) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && ((done.load(std::memory_order_acquire) >> dev) & 1ull)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && tracked) done.fetch_or(1ull << dev, std::memory_order_release);
+  return e;
+}
+
 // What the im2col-mode-TMA convolution kernel is given: an NHWC int8 tensor whose channel count is
 // a multiple of 32 and a filter geometry over it.  The channel-pack map uses the (padded) input
 // itself; the row-unroll and space-to-depth maps first rewrite the input into a scratch tensor for
@@ -274,8 +289,9 @@ void set_last_cuda_error(int e);
 int get_last_cuda_error();
 
 // --- kernel launchers (layout.cu, conv_mma.cu) -------------------------------------------------
+// status: device status word that a bounded wait of the kernel reports into, or nullptr
 cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, int H, int W, int C_pad,
-                                    cudaStream_t st);
+                                    cudaStream_t st, int* status);
 cudaError_t launch_pack_weights_cp(const int8_t* w, int8_t* out, int K, int C, int R, int S, int C_pad,
                                    cudaStream_t st);
 cudaError_t launch_pack_weights_table(const int8_t* w, int8_t* out, int K, int Kg, int cols, const int32_t* table,
@@ -300,5 +316,6 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
                             cudaStream_t st);
 size_t conv_mma_smem_bytes(int amode, const ConvArgs& args);
 cudaError_t launch_bounded_wait_selftest(int* status, cudaStream_t st);
+cudaError_t launch_pack_wait_selftest(int* status, cudaStream_t st);
 
 }  // namespace b2c

@@ -1299,13 +1299,9 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
   cudaError_t e;
 #define B2C_LAUNCH(MODE, PERS)                                                                             \
   {                                                                                                       \
-    static size_t configured = 0;                                                                         \
-    if (smem > configured) {                                                                              \
-      e = cudaFuncSetAttribute(conv_mma_kernel<MODE, PERS>, cudaFuncAttributeMaxDynamicSharedMemorySize,  \
-                               200 * 1024);                                                               \
-      if (e != cudaSuccess) return e;                                                                     \
-      configured = 200 * 1024;                                                                            \
-    }                                                                                                     \
+    static std::atomic<unsigned long long> configured{0};                                                 \
+    e = set_max_dynamic_smem_once(configured, (const void*)conv_mma_kernel<MODE, PERS>, 200 * 1024);      \
+    if (e != cudaSuccess) return e;                                                                       \
     e = launch_pdl_cluster(conv_mma_kernel<MODE, PERS>, grid, dim3(kThreads), smem, st,                   \
                            args.cluster_split ? args.split_k : 1, *tmap_a, *tmap_b, args);                \
     if (e != cudaSuccess) return e;                                                                       \

@@ -125,12 +125,59 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_kernel(const in
 // Groups of 16 rows are spaced 16 bytes further apart than their size, which makes the
 // transposing word reads of the store phase conflict free.  The store phase is the same register
 // transpose as in pack_activations_kernel.
-constexpr int kBulkWaitTries = 1 << 22;
+constexpr unsigned long long kPackWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s, as in the MMA kernel
+__device__ __forceinline__ unsigned long long pack_global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool pack_bar_try_wait(uint32_t bar) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar)
+      : "memory");
+  return ok != 0;
+}
+
+__device__ __forceinline__ bool pack_wait_bounded(uint32_t bar, int* status, bool reporter) {
+  bool done = false;
+  for (int tries = 0; tries < 64 && !done; ++tries) done = pack_bar_try_wait(bar);
+  if (!done) {
+    const unsigned long long t0 = pack_global_ns();
+    while (!(done = pack_bar_try_wait(bar)) && pack_global_ns() - t0 < kPackWaitLimitNs) {
+    }
+  }
+  if (!done) {
+    if (reporter && status != nullptr) atomicExch(status, B2C_E_TIMEOUT);
+    const unsigned long long t1 = pack_global_ns();
+    while (pack_global_ns() - t1 < 50000ull) __nanosleep(1000);
+  }
+  return done;
+}
+
+// One block waits, with the bounded wait of the bulk-copy pack kernel, on a barrier that expects
+// bytes no copy delivers; the wait gives up after its limit and reports through `status`.
+__global__ void pack_wait_selftest_kernel(int* status) {
+  __shared__ __align__(8) unsigned long long bar;
+  const uint32_t bar_a = (uint32_t)__cvta_generic_to_shared(&bar);
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"(16u) : "memory");
+  }
+  __syncthreads();
+  pack_wait_bounded(bar_a, status, threadIdx.x == 0);
+}
 
 template <bool kRowMode>
 __global__ void __launch_bounds__(kPackThreads) pack_activations_bulk_kernel(const int8_t* __restrict__ x,
                                                                              int8_t* __restrict__ out, int C, int HW,
-                                                                             int C_pad, int hw_tiles, int CT, int PT) {
+                                                                             int C_pad, int hw_tiles, int CT, int PT,
+                                                                             int* status) {
   extern __shared__ __align__(128) uint8_t btile[];
   __shared__ __align__(8) unsigned long long bar;
   const int n = blockIdx.x / hw_tiles;
@@ -169,20 +216,11 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_bulk_kernel(con
           : "memory");
     }
   }
-  // Bounded wait for the copies; on expiry the block gives up (its part of the output stays unwritten).
-  bool done = false;
-  for (int tries = 0; tries < kBulkWaitTries && !done; ++tries) {
-    uint32_t ok;
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n"
-        "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok)
-        : "r"(bar_a)
-        : "memory");
-    done = ok != 0;
-  }
-  if (!done) return;
+  // Bounded wait for the copies (every thread polls the barrier).  On expiry the block records
+  // B2C_E_TIMEOUT in the status word (when the caller gave one), leaves the copies that were issued
+  // some time to land before its shared memory is released, and returns; its part of the output
+  // stays unwritten.
+  if (!pack_wait_bounded(bar_a, status, t == 0)) return;
   // The next kernel may start its set-up once every block of this one has its tile in shared
   // memory (earlier, its resident blocks would only take shared memory away from this grid).
   pdl_launch_dependents();
@@ -573,7 +611,7 @@ int grid_for(long long total, int block) {
 }  // namespace
 
 cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, int H, int W, int C_pad,
-                                    cudaStream_t st) {
+                                    cudaStream_t st, int* status) {
   const int HW = H * W;
   int CT = C_pad >= 128 ? 128 : 64;
   const bool a16 = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
@@ -589,9 +627,9 @@ cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, 
     dim3 grid((unsigned)hw_tiles * (unsigned)N, (C_pad + CT - 1) / CT, 1);
     if (row_mode)
       return launch_pdl(pack_activations_bulk_kernel<true>, grid, dim3(kPackThreads), smem, st, x, out, C, HW, C_pad,
-                        hw_tiles, CT, PT);
+                        hw_tiles, CT, PT, status);
     return launch_pdl(pack_activations_bulk_kernel<false>, grid, dim3(kPackThreads), smem, st, x, out, C, HW, C_pad,
-                      hw_tiles, CT, PT);
+                      hw_tiles, CT, PT, status);
   }
   const int PT = HW > 128 ? 256 : (HW > 64 ? 128 : 64);
   const int hw_tiles = (HW + PT - 1) / PT;
@@ -603,6 +641,11 @@ cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, 
     return launch_pdl(pack_activations_kernel<4>, grid, dim3(kPackThreads), 0, st, x, out, C, HW, C_pad, hw_tiles, CT,
                       PT);
   return launch_pdl(pack_activations_kernel<1>, grid, dim3(kPackThreads), 0, st, x, out, C, HW, C_pad, hw_tiles, CT, PT);
+}
+
+cudaError_t launch_pack_wait_selftest(int* status, cudaStream_t st) {
+  pack_wait_selftest_kernel<<<1, 64, 0, st>>>(status);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_pack_weights_cp(const int8_t* w, int8_t* out, int K, int C, int R, int S, int C_pad,
@@ -675,12 +718,9 @@ cudaError_t launch_row_phase_unroll(const int8_t* x, int8_t* out, int N, int Hs,
                       (reinterpret_cast<uintptr_t>(x) & 15) == 0)
                          ? 1
                          : 0;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(row_phase_unroll_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowPhaseSmemMax);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static std::atomic<unsigned long long> configured{0};
+  cudaError_t ea = set_max_dynamic_smem_once(configured, (const void*)row_phase_unroll_kernel, kRowPhaseSmemMax);
+  if (ea != cudaSuccess) return ea;
   return launch_pdl(row_phase_unroll_kernel, dim3((unsigned)blocks), dim3(kS2dTile), (size_t)smem, st, x, out, Hs, Q, C, H,
                     W, S, sh, sw, pad_h, pad_w, dil_w, C_pad, seg, q_tiles, stride_n, stride_c, stride_h, stride_w, vec_ok);
 }

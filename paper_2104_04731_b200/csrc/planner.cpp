@@ -38,8 +38,13 @@ int resolve_geom(const b2c_conv_desc* d, Geom* g) {
   long long kg = (long long)d->C * d->R * d->S;
   if (g->P == 0 || g->Q == 0) return B2C_E_UNSUPPORTED;
   if (kg > kMaxKg) return B2C_E_UNSUPPORTED;
-  g->PQ = g->P * g->Q;
-  g->Mg = (long long)d->N * g->PQ;
+  // A padding of a million pixels per side serves no convolution and would let the products below
+  // leave 64 bits for extreme images; P*Q must fit 31 bits before anything is derived from it.
+  if (d->pad_h > (1 << 20) || d->pad_w > (1 << 20)) return B2C_E_UNSUPPORTED;
+  const long long pq = (long long)g->P * g->Q;
+  if (pq > 0x7FFFFF00LL) return B2C_E_UNSUPPORTED;
+  g->PQ = (int)pq;
+  g->Mg = (long long)d->N * pq;
   g->Kg = (int)kg;
   g->x_elems = (long long)d->N * d->C * d->H * d->W;
   g->w_elems = (long long)d->K * kg;

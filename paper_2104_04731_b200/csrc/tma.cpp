@@ -1,6 +1,7 @@
 // Tensor-map construction for the TMA loads of the MMA kernel.  The driver's encoders are
 // looked up at run time through cudaGetDriverEntryPoint, so the library has no link-time
 // dependency on libcuda and loads on machines without a driver.
+#include <atomic>
 #include <mutex>
 
 #include "b2c_internal.h"
@@ -19,9 +20,24 @@ static EncodeTiledFn g_tiled = nullptr;
 static EncodeIm2colFn g_im2col = nullptr;
 static std::once_flag g_once;
 static thread_local int g_last_cuda_error = 0;
-
 void set_last_cuda_error(int e) { g_last_cuda_error = e; }
 int get_last_cuda_error() { return g_last_cuda_error; }
+// Host-side fault injection for the tests: the n-th tensor-map encode from now on reports failure.
+static std::atomic<int> g_fail_countdown{0};
+static bool injected_failure() {
+  int n = g_fail_countdown.load();
+  while (n > 0) {
+    if (g_fail_countdown.compare_exchange_weak(n, n - 1)) {
+      if (n == 1) {
+        set_last_cuda_error((int)CUDA_ERROR_INVALID_VALUE);
+        return true;
+      }
+      return false;
+    }
+  }
+  return false;
+}
+
 
 static void resolve() {
   void* fn = nullptr;
@@ -47,6 +63,7 @@ static CUtensorMapSwizzle swizzle_of(int bytes) {
 int encode_tiled_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
                     uint32_t box_inner, uint32_t box_outer, int swizzle_bytes) {
   std::call_once(g_once, resolve);
+  if (injected_failure()) return B2C_E_CUDA;
   if (!g_tiled) {
     set_last_cuda_error((int)CUDA_ERROR_NOT_FOUND);
     return B2C_E_CUDA;
@@ -74,6 +91,7 @@ int encode_im2col_nhwc(CUtensorMap* map, const void* base, int C_pad, int W, int
                        int S, int R, int dil_w, int dil_h, int stride_w, int stride_h, int channels_per_pixel,
                        int pixels_per_column, int swizzle_bytes) {
   std::call_once(g_once, resolve);
+  if (injected_failure()) return B2C_E_CUDA;
   if (!g_im2col) {
     set_last_cuda_error((int)CUDA_ERROR_NOT_FOUND);
     return B2C_E_CUDA;
@@ -100,6 +118,7 @@ int encode_im2col_nhwc(CUtensorMap* map, const void* base, int C_pad, int W, int
 int encode_tiled_nhwc_rows(CUtensorMap* map, const void* base, int C_pad, int W, int H, int N, int box_c, int box_w,
                            int swizzle_bytes, int box_h) {
   std::call_once(g_once, resolve);
+  if (injected_failure()) return B2C_E_CUDA;
   if (!g_tiled) {
     set_last_cuda_error((int)CUDA_ERROR_NOT_FOUND);
     return B2C_E_CUDA;
@@ -121,3 +140,9 @@ int encode_tiled_nhwc_rows(CUtensorMap* map, const void* base, int C_pad, int W,
 }  // namespace b2c
 
 extern "C" int b2c_last_cuda_error(void) { return b2c::get_last_cuda_error(); }
+
+extern "C" int b2c_test_fail_nth_encode(int n) {
+  if (n < 0) return B2C_E_INVALID_ARG;
+  b2c::g_fail_countdown.store(n);
+  return B2C_OK;
+}

@@ -65,7 +65,7 @@ def test_config_every_embedding(lib, cfg):
         check_against_oracle(x, w, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, cfg.out_mode, e.id, ref=ref)
 
 
-@pytest.mark.parametrize("cfg", CONFIGS[:2] + CONFIGS[4:], ids=lambda c: c.name)
+@pytest.mark.parametrize("cfg", CONFIGS, ids=lambda c: c.name)
 @pytest.mark.parametrize("in_layout,out_layout", [(1, 1), (0, 1), (1, 0)])
 def test_config_layouts(lib, cfg, in_layout, out_layout):
     x, w, ref = cfg_reference(cfg)
@@ -568,7 +568,110 @@ def test_large_grid_persistent_tiles(lib, tile_n):
             check_against_oracle(x, w, 1, 1, 1, 9, 3, ids[0], ref=ref, in_layout=in_layout, out_layout=out_layout)
 
 
+# ---- the wide persistent schedule the large-batch benchmark runs: 128 x 256 tiles, two 256-column
+# accumulators (all of tensor memory), one block per SM walking 614 tiles -------------------------------
+_wide_ref = {}
+
+
+@pytest.mark.parametrize("in_layout", [0, 1])
+@pytest.mark.parametrize("out_mode", [1, 2, 3])
+def test_persistent_256_column_tiles(lib, in_layout, out_mode):
+    N, C, H, W, K, R, S = 800, 64, 14, 14, 512, 3, 3   # stride 2, pad 1: 39200 pixels = 307 row tiles x 2 column tiles
+    if "ref" not in _wide_ref:
+        x = int8_uniform((N, C, H, W), 711)
+        w = int8_uniform((K, C, R, S), 712)
+        _wide_ref["ref"] = (x, w, oracle.conv2d_int8(x, w, 2, 1, 1, 10))
+    x, w, ref = _wide_ref["ref"]
+    d = lib.make_desc(N, C, H, W, K, R, S, 2, 1, 1, 10, in_layout, 0, out_mode)
+    ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == 0 and e.tile_n == 256 and e.split_k == 1
+           and e.map_m == b2c.AXIS_NPQ]
+    assert ids
+    check_against_oracle(x, w, 2, 1, 1, 10, out_mode, ids[0], ref=ref, in_layout=in_layout)
+
+
+# ---- one-shot calls of one shape on two streams with different weights do not disturb each other ---------
+def test_one_shot_calls_on_two_streams(lib):
+    N, C, H, W, K, R, S = 2, 32, 20, 20, 48, 3, 3
+    x = int8_uniform((N, C, H, W), 721)
+    ws = [int8_uniform((K, C, R, S), 722 + i) for i in range(2)]
+    refs = [oracle.conv2d_int8(x, w, 1, 1, 1, 7) for w in ws]
+    xd = to_dev(x)
+    wd = [to_dev(w) for w in ws]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [[(torch.zeros(refs[0][0].shape, dtype=torch.int32, device="cuda"),
+              torch.zeros(refs[0][1].shape, dtype=torch.int8, device="cuda")) for _ in range(6)] for _ in range(2)]
+    torch.cuda.synchronize()
+    for rep in range(6):          # interleaved, nothing orders the two streams against each other
+        for i in range(2):
+            y32, y8 = outs[i][rep]
+            lib.conv2d_int8(xd, wd[i], 1, 1, 1, 7, y32, y8, stream=streams[i])
+    torch.cuda.synchronize()
+    assert lib.oneshot_status() == b2c.OK
+    for i in range(2):
+        for y32, y8 in outs[i]:
+            assert np.array_equal(y32.cpu().numpy(), refs[i][0])
+            assert np.array_equal(y8.cpu().numpy(), refs[i][1])
+    lib.oneshot_cache_clear()
+    y32, y8 = outs[0][0]
+    y32.zero_()
+    lib.conv2d_int8(xd, wd[1], 1, 1, 1, 7, y32, y8)   # selects again after the cache was cleared
+    torch.cuda.synchronize()
+    assert np.array_equal(y32.cpu().numpy(), refs[1][0])
+
+
+# ---- host-side fault injection: a tensor map the driver refuses ---------------------------------------
+def test_failed_descriptor_encode_is_reported_and_skipped(lib):
+    cfg = CONFIGS[0]
+    x, w, ref = cfg_reference(cfg)
+    d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
+                      out_mode=3)
+    try:
+        lib.test_fail_nth_encode(1)                  # the weight tensor map of the plan
+        with pytest.raises(b2c.B2CError) as err:
+            lib.Plan(d, b2c.POLICY_MIN_OVERHEAD)
+        assert err.value.code == b2c.E_CUDA
+        lib.test_fail_nth_encode(1)                  # first candidate of the timed selection cannot be built:
+        plan = lib.Plan(d, b2c.POLICY_AUTO_TIMED)    # it is left out, the others are still timed
+        lib.test_fail_nth_encode(0)
+        cp = [e.id for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_CP_TMA][0]
+        plan2 = lib.Plan(d, cp)
+        plan2.set_weights(to_dev(w))
+        ws2 = torch.zeros(max(16, plan2.workspace_bytes()), dtype=torch.uint8, device="cuda")
+        y32 = torch.zeros(ref[0].shape, dtype=torch.int32, device="cuda")
+        y8 = torch.zeros(ref[1].shape, dtype=torch.int8, device="cuda")
+        lib.test_fail_nth_encode(1)                  # the activation tensor map of a run
+        with pytest.raises(b2c.B2CError) as err:
+            plan2.run(to_dev(x), y32, y8, ws2)
+        assert err.value.code == b2c.E_CUDA
+        plan2.run(to_dev(x), y32, y8, ws2)           # the next run is not affected
+        torch.cuda.synchronize()
+        assert np.array_equal(y32.cpu().numpy(), ref[0])
+        plan2.destroy()
+    finally:
+        lib.test_fail_nth_encode(0)
+    assert plan.info().device_us > 0
+    plan.set_weights(to_dev(w))
+    y32 = torch.zeros(ref[0].shape, dtype=torch.int32, device="cuda")
+    y8 = torch.zeros(ref[1].shape, dtype=torch.int8, device="cuda")
+    ws = torch.zeros(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
+    plan.run(to_dev(x), y32, y8, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(y32.cpu().numpy(), ref[0]) and np.array_equal(y8.cpu().numpy(), ref[1])
+    plan.destroy()
+
+
 # ---- failure detection: a wait that cannot complete ends by itself and is reported --------------------
+def test_pack_kernel_wait_reports_timeout(lib):
+    d = lib.make_desc(1, 32, 8, 8, 16, 3, 3, 1, 1, 1, 0, out_mode=1)
+    plan = lib.Plan(d, b2c.POLICY_MIN_OVERHEAD)
+    plan.selftest_pack_wait()               # waits for bytes that no copy delivers: gives up after its limit
+    torch.cuda.synchronize()
+    assert plan.device_status() == b2c.E_TIMEOUT
+    assert plan.device_status() == b2c.OK
+    plan.destroy()
+
+
+
 def test_bounded_wait_reports_timeout_and_plan_stays_usable(lib):
     cfg = CONFIGS[0]
     x, w, ref = cfg_reference(cfg)

@@ -172,3 +172,22 @@ def test_swapped_map_is_listed_only_when_k_fills_half_a_tile(lib):
                 e8 = next(c for c in b2c.enumerate_embeddings(d8)
                           if (c.map_m, c.variant, c.tile_n, c.split_k) == (e.map_m, e.variant, e.tile_n, e.split_k))
                 assert e8.workspace_bytes >= 4 * M * K
+
+
+def test_output_extent_overflow_is_refused(lib):
+    # small image, huge padding: P = Q = 61000, P*Q beyond 31 bits
+    d = b2c.make_desc(1, 1, 1000, 1000, 1, 1, 1, 1, 30000, 1)
+    n = ctypes.c_int32()
+    assert b2c.load().b2c_enumerate(ctypes.byref(d), None, 0, ctypes.byref(n)) == b2c.E_UNSUPPORTED
+    # padding beyond any use
+    d = b2c.make_desc(1, 1, 8, 8, 1, 3, 3, 1, (1 << 20) + 1, 1)
+    assert b2c.load().b2c_enumerate(ctypes.byref(d), None, 0, ctypes.byref(n)) == b2c.E_UNSUPPORTED
+    # a large but representable extent is still listed
+    d = b2c.make_desc(1, 1, 1000, 1000, 1, 1, 1, 1, 5000, 1)
+    assert b2c.load().b2c_enumerate(ctypes.byref(d), None, 0, ctypes.byref(n)) == b2c.OK and n.value > 0
+
+
+def test_fault_injection_hook_arms_and_disarms(lib):
+    assert b2c.load().b2c_test_fail_nth_encode(-1) == b2c.E_INVALID_ARG
+    b2c.test_fail_nth_encode(3)
+    b2c.test_fail_nth_encode(0)

@@ -5,8 +5,8 @@ against cudaMalloc, a latency-critical loop, a process whose memory all belongs 
 They get the same matrix from a call that keeps its lookup table in a fixed array inside the
 library.  The table is shared by all calls and keeps what the last call wrote, so this test makes
 two calls in a row with different geometries (the second one shorter, so that stale entries of the
-first would show) and compares each, byte for byte, with b2c_im2col.  The file name makes pytest
-collect it last.
+first would show) and compares each, byte for byte, with b2c_im2col and with the CPU oracle's
+stencil-unroll matrix.  The file name makes pytest collect it last.
 """
 import ctypes
 
@@ -14,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2104_04731_b200 as b2c
 from paper_2104_04731_b200.synth import int8_uniform
 
@@ -33,16 +34,18 @@ def _both(lib, geom, in_layout, seed):
     lib.im2col(d, xd, ref, K_pad)          # existing entry point (allocates its table)
     lib.im2col_noalloc(d, xd, got, K_pad)  # the allocation-free one
     torch.cuda.synchronize()
-    return got.cpu().numpy(), ref.cpu().numpy()
+    want = oracle.im2col(x, R, S, stride, pad, dil)   # [N*P*Q][C*R*S], from the CPU oracle
+    return got.cpu().numpy(), ref.cpu().numpy(), want
 
 
 def test_two_calls_in_a_row_match_the_allocating_entry_point(lib):
     first = (2, 16, 13, 11, 3, 5, (2, 1), (1, 2), (1, 2))   # C*R*S = 240 -> K_pad 256
     second = (1, 3, 20, 21, 7, 7, 2, 3, 1)                   # C*R*S = 147 -> K_pad 160 (shorter table)
     for i, (geom, in_layout) in enumerate([(first, 0), (second, 1)]):
-        got, ref = _both(lib, geom, in_layout, 900 + i)
+        got, ref, want = _both(lib, geom, in_layout, 900 + i)
         assert np.array_equal(got, ref), "call %d differs from b2c_im2col" % (i + 1)
-        assert (got != 66).any()
+        assert np.array_equal(got[:, :want.shape[1]], want), "call %d differs from the oracle" % (i + 1)
+        assert not got[:, want.shape[1]:].any()
 
 
 def test_size_limit_is_reported_without_launching(lib):
