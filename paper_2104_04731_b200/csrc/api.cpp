@@ -275,6 +275,25 @@ void fill_common_args(b2c_plan* p) {
       tiles_m * tiles_n < 0x7FFFFFFF)
     a.persistent = 2;
   a.tmem_bufs = (a.persistent && 2 * a.tmem_cols <= 512) ? 2 : 1;
+  a.pair = p->emb.tile_m == 2 * kTileM ? 1 : 0;
+  if (a.pair) {
+    // Pair tiles of 256 rows; grids beyond one wave of pairs walk the tile list with one block per SM,
+    // two accumulator buffers and the deepest ring that fits; smaller grids keep two blocks per SM
+    // (one accumulator each, ring within half of the shared memory) so that one block's set-up and
+    // epilogue overlap the other's main loop.
+    const long long tiles_m2 = ((long long)a.Mg + 2 * kTileM - 1) / (2 * kTileM);
+    a.num_tiles = (int)std::min<long long>(tiles_m2 * tiles_n, 0x3FFFFFFF);
+    a.persistent = tiles_m2 * tiles_n > kNumSMs / 2 ? 1 : 0;
+    a.tmem_bufs = (a.persistent && 2 * a.tmem_cols <= 512) ? 2 : 1;
+    a.cluster_split = 0;
+    const size_t pair_stage = (size_t)(kTileM + a.tile_n / 2) * a.bk;
+    const size_t pair_budget = a.persistent ? 196 * 1024 : 100 * 1024;
+    int st = std::min(8, std::max(1, a.num_kb));
+    while (st > 2 && (size_t)st * pair_stage > pair_budget) --st;
+    a.stages = st;
+    a.stage_region = (int)((size_t)st * pair_stage);
+    return;
+  }
   const size_t budget = a.persistent == 1 ? 196 * 1024 : (a.persistent == 2 ? 68 * 1024 : (ctas > kNumSMs ? 100 * 1024 : 196 * 1024));
   const size_t stage_bytes = (size_t)(kTileM + a.tile_n) * a.bk;
   // lookup table and staged window share the block's shared memory with the stages
@@ -426,7 +445,7 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
   // Tensor map of the packed weights (plan-owned memory, so it is encoded once).
   // (Swapped map: the weights are the 128-row operand, so their box is 128 rows high.)
   int rc;
-  const int w_box_rows = is_swapped(emb) ? kTileM : emb.tile_n;
+  const int w_box_rows = is_swapped(emb) ? kTileM : (emb.tile_m == 2 * kTileM ? emb.tile_n / 2 : emb.tile_n);
   if (is_tma_view_variant(emb.variant)) {
     uint64_t cols = (uint64_t)p->view.R * p->view.S * p->view.C;
     rc = encode_tiled_2d(&p->tmap_b, p->w_packed, cols, d.K, cols, p->bk, w_box_rows, p->bk);
@@ -844,7 +863,10 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
     CUDA_TRY(cudaMemsetAsync(a.acc, 0, (size_t)g.y_elems * 4, st));
   }
 
-  CUDA_TRY(launch_conv_mma(p->amode, &tmap_a, &p->tmap_b, a, st));
+  if (a.pair)
+    CUDA_TRY(launch_conv_mma_pair(p->amode, &tmap_a, &p->tmap_b, a, st));
+  else
+    CUDA_TRY(launch_conv_mma(p->amode, &tmap_a, &p->tmap_b, a, st));
   if (need_finish)
     CUDA_TRY(launch_splitk_finish(a.acc, y32, y8, g.y_elems, d.shift, d.out_mode, p->bias, p->relu, d.K, g.PQ,
                                   d.out_layout == B2C_LAYOUT_NHWC ? 1 : 0, st));

@@ -122,6 +122,9 @@ struct ConvArgs {
   int sh_tiles_h, sh_tiles_w, sh_valid_w;  // sh_valid_w: columns of a tile that are outputs (tiles advance by it)
   FastDiv div_tiles_hw, div_tiles_w;
   int persistent_blocks_per_sm;  // blocks per SM the persistent grid is sized for (0: the mode's default)
+  // Two-SM schedule: a pair of blocks (cluster of two) owns a 256 x tile_n tile; num_tiles counts pair
+  // tiles, every block loads its own 128 A rows and tile_n / 2 B rows per stage.
+  int pair;
   FastDiv div_wps, div_hp;
   // elements between consecutive images of the NKPQ output (K * P * Q, or more when this
   // convolution writes one channel group of a wider tensor)
@@ -254,6 +257,16 @@ inline bool is_swapped(const b2c_embedding& e) { return e.map_m == B2C_AXIS_K; }
 // buffer, zero-fill or finish pass is needed.
 // (The variants that keep a lookup table or an input window in shared memory leave room for a
 // 128-column exchange tile at most.)
+// Two-SM schedule (tile_m = 256): a pair of blocks shares one accumulator tile of 256 fused pixels.  It
+// exists for the TMA-fed maps (operand A by im2col-mode or tiled TMA) without a split reduction, with
+// column tiles of 32 to 256 channels (each block loads tile_n / 2 weight rows, at least one 16-row
+// group), when the problem has more than one 128-row tile.
+inline bool pair_schedule_ok(int variant, int tile_n, int split_k, bool swap, long long rows) {
+  const bool tma_fed = variant == B2C_VARIANT_CP_TMA || variant == B2C_VARIANT_IM2COL_EXPLICIT ||
+                       variant == B2C_VARIANT_ROW_UNROLL || variant == B2C_VARIANT_SPACE_TO_DEPTH ||
+                       variant == B2C_VARIANT_DILATION_PACK;
+  return tma_fed && !swap && split_k == 1 && tile_n >= 32 && rows > kTileM;
+}
 inline bool cluster_split_ok(int variant, int tile_n, int split_k, bool swap = false) {
   // the swapped map and the phase pack (scattered output rows) meet their partial sums in global memory
   if (swap || variant == B2C_VARIANT_DILATION_PACK || is_shift_variant(variant)) return false;
@@ -315,6 +328,9 @@ cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, l
 cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,
                             cudaStream_t st);
 size_t conv_mma_smem_bytes(int amode, const ConvArgs& args);
+cudaError_t launch_conv_mma_pair(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,
+                                 cudaStream_t st);
+size_t conv_mma_pair_smem_bytes(const ConvArgs& args);
 cudaError_t launch_bounded_wait_selftest(int* status, cudaStream_t st);
 cudaError_t launch_pack_wait_selftest(int* status, cudaStream_t st);
 

@@ -1,0 +1,429 @@
+// Two-SM form of the convolution kernel: a pair of thread blocks on neighbouring SMs (a cluster
+// of two) owns one 256 x tile_n accumulator tile and issues tcgen05.mma.cta_group::2.kind::i8.
+// The GEMM intrinsic is still that of Section 5.1 (8-bit operands, 32-bit accumulation,
+// C_xy += A_xz * B_zy^T, B held transposed); what changes is how the operands are shared: each
+// block of the pair loads its own 128 rows of A (fused (n, p, q) pixels) and only HALF of the B
+// rows (tile_n / 2 output channels), and the tensor cores of both SMs read the two B halves from
+// both shared memories.  Per MMA cycle a block therefore takes a third fewer operand bytes from
+// L2 than the one-SM kernel with the same tile_n, which is what bounds the compute-bound shapes.
+//
+// Roles in each block: warp 0 TMA producer (own A rows, own B half; plain TMA loads that
+// complete on the block's own barrier, no cluster multicast), warp 1 MMA issue in the leader block
+// (cluster rank 0) and hand-over of "my half has landed" to the leader in the other block, warps
+// 2-9 epilogue of the block's own 128 accumulator rows (tcgen05.ld from the block's own tensor
+// memory, activation step, shift / clip, stores).  Barriers: full[s] of the leader counts its own
+// producer and the peer's hand-over; the leader's commits arrive on empty[s] and tmem_full[b] of
+// BOTH blocks (tcgen05.commit with a block mask); the epilogue warps of both blocks arrive on
+// the leader's tmem_empty[b].  Every wait is bounded as in the one-SM kernel.
+#include <algorithm>
+
+#include "conv_mma_common.cuh"
+
+namespace b2c {
+
+namespace {
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in block `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+  return remote;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Waits that pair with arrivals from the other block of the cluster.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+__device__ __noinline__ bool mbar_wait_cluster_slow(uint32_t bar, uint32_t parity, SharedCtl* ctl, int* status) {
+  const unsigned long long t0 = global_ns();
+  while (true) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if (ctl->abort_flag) return false;
+    if (global_ns() - t0 > kWaitLimitNs) {
+      ctl->abort_flag = 1;
+      atomicExch(status, B2C_E_TIMEOUT);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, SharedCtl* ctl, int* status) {
+#pragma unroll 1
+  for (int i = 0; i < 32; ++i)
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+  return mbar_wait_cluster_slow(bar, parity, ctl, status);
+}
+
+// Instruction descriptor of the two-SM MMA: as make_idesc_i8, with M = 256 (128 rows per block).
+__device__ __forceinline__ uint32_t make_idesc_i8_pair(int n) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
+// One reduction block of the pair: `ksteps` (1..4) two-SM MMAs over consecutive 32-byte slices.
+__device__ __forceinline__ void mma_i8_pair_block(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                  uint32_t accumulate, uint32_t on, int ksteps) {
+  asm volatile(
+      "{\n"
+      ".reg .pred pacc, ptrue, q0, q1, q2, q3;\n"
+      ".reg .b64 a1, a2, a3, b1, b2, b3;\n"
+      "setp.ne.b32 pacc, %4, 0;\n"
+      "setp.eq.b32 ptrue, 0, 0;\n"
+      "setp.ne.b32 q0, %5, 0;\n"
+      "setp.gt.and.s32 q1, %6, 1, q0;\n"
+      "setp.gt.and.s32 q2, %6, 2, q0;\n"
+      "setp.gt.and.s32 q3, %6, 3, q0;\n"
+      "add.u64 a1, %1, 2;\n"
+      "add.u64 b1, %2, 2;\n"
+      "add.u64 a2, %1, 4;\n"
+      "add.u64 b2, %2, 4;\n"
+      "add.u64 a3, %1, 6;\n"
+      "add.u64 b3, %2, 6;\n"
+      "@q0 tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, pacc;\n"
+      "@q1 tcgen05.mma.cta_group::2.kind::i8 [%0], a1, b1, %3, ptrue;\n"
+      "@q2 tcgen05.mma.cta_group::2.kind::i8 [%0], a2, b2, %3, ptrue;\n"
+      "@q3 tcgen05.mma.cta_group::2.kind::i8 [%0], a3, b3, %3, ptrue;\n"
+      "}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(on), "r"(ksteps)
+      : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in both blocks of the pair once every MMA
+// issued so far has completed.
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar, uint32_t on) {
+  asm volatile(
+      "{\n.reg .pred q;\n.reg .b16 m;\nsetp.ne.b32 q, %1, 0;\nmov.b16 m, 3;\n"
+      "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n}" ::"r"(bar),
+      "r"(on)
+      : "memory");
+}
+
+// PERSIST: 0 = one pair tile per cluster, two blocks resident per SM (one 256-column accumulator each,
+// stage ring within half of the shared memory); 1 = 74 clusters walk the tile list, one block per SM,
+// two accumulator buffers, the deepest stage ring that fits.
+template <int AMODE, int PERSIST>
+__global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
+    conv_mma_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                         const ConvArgs args) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ SharedCtl ctl;
+
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // 0: leader (issues the MMAs), 1: peer
+  const int pair_id = (int)(blockIdx.x >> 1);
+  const int num_pairs = (int)(gridDim.x >> 1);
+  constexpr bool persistent = PERSIST != 0;
+  const int tile_first = pair_id;
+  const int tile_step = num_pairs;
+  const int tile_end = args.num_tiles;
+  const int nbuf = persistent ? args.tmem_bufs : 1;  // 1 or 2
+  const int stages = args.stages;
+  const int bk = args.bk;
+  const int half_n = args.tile_n >> 1;  // B rows (output channels) this block loads
+  const uint32_t a_stage_bytes = (uint32_t)(kTileM * bk);
+  const uint32_t b_stage_bytes = (uint32_t)(half_n * bk);
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t a_base = smem_base;
+  const uint32_t b_base = smem_base + stages * a_stage_bytes;
+
+  if (warp == 0) {
+    if (lane < stages) {
+      // the leader's full barrier also counts the peer's "my half has landed"
+      mbar_init(smem_u32(&ctl.full[lane]), rank == 0 ? 2 : 1);
+      mbar_init(smem_u32(&ctl.empty[lane]), 1);
+    }
+    if (lane == 8) {
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(smem_u32(&ctl.tmem_full[b]), 1);
+        mbar_init(smem_u32(&ctl.tmem_empty[b]), 2 * kGatherWarps);  // the epilogue warps of both blocks
+      }
+      ctl.abort_flag = 0;
+    }
+    if (lane == 9) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+    if (lane == 10) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    // both blocks of the pair allocate the same columns together
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
+                 "r"(args.tmem_cols * nbuf)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  // the other block's barriers must be initialised before anything arrives on them
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_acc = __shfl_sync(0xffffffffu, ctl.tmem_base, 0);
+  pdl_wait();
+  pdl_launch_dependents();
+
+#define B2C_PAIR_TILE_ORIGIN(t)                                     \
+  const int mt_ = (int)args.div_tiles_n.div((uint32_t)(t));        \
+  const int m0 = mt_ * (2 * kTileM) + (int)rank * kTileM;          \
+  const int n0 = ((t) - mt_ * args.tiles_n) * args.tile_n;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer (both blocks)
+    int s = 0;
+    uint32_t ph = 0;
+    uint32_t a_dst = a_base, b_dst = b_base;
+    const uint32_t leader_lane = elect_one() ? 1u : 0u;
+    bool alive = true;
+    for (int t = tile_first; t < tile_end && alive; t += tile_step) {
+      B2C_PAIR_TILE_ORIGIN(t)
+      int n_img = 0, h_org = 0, w_org = 0, cb = 0, sx = 0, r = 0;
+      if (AMODE == A_IM2COL_TMA) {
+        n_img = (int)args.div_pq.div((uint32_t)m0);
+        const int rem = m0 - n_img * args.PQ;
+        const int p = (int)args.div_q.div((uint32_t)rem), q = rem - p * args.Q;
+        h_org = p * args.stride_h - args.pad_h;
+        w_org = q * args.stride_w - args.pad_w;
+      }
+      int kcol = 0;
+      const int wrow0 = n0 + (int)rank * half_n;  // first output channel of this block's B half
+      for (int kb = 0; kb < args.num_kb; ++kb) {
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.empty[s]), ph ^ 1u, &ctl, args.status))) {
+          alive = false;
+          break;
+        }
+        const uint32_t full = smem_u32(&ctl.full[s]);
+        mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes, leader_lane);
+        if (AMODE == A_TILED) {
+          tma_load_2d(a_dst, &tmap_a, kcol, m0, full, leader_lane);
+        } else {
+          tma_load_im2col_4d(a_dst, &tmap_a, cb * bk, w_org, h_org, n_img, full, (uint16_t)(sx * args.dil_w),
+                             (uint16_t)(r * args.dil_h), leader_lane);
+          if (++cb == args.kb_per_tap) {
+            cb = 0;
+            if (++sx == args.S) {
+              sx = 0;
+              ++r;
+            }
+          }
+        }
+        tma_load_2d(b_dst, &tmap_b, kcol, wrow0, full, leader_lane);
+        kcol += bk;
+        a_dst += a_stage_bytes;
+        b_dst += b_stage_bytes;
+        if (++s == stages) {
+          s = 0;
+          ph ^= 1u;
+          a_dst = a_base;
+          b_dst = b_base;
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1 && rank != 0) {
+    // ---------------------------------------------------------------- peer: hand-over of full stages
+    // Once this block's copies of a stage have landed, one lane arrives on the leader's full barrier.
+    int s = 0;
+    uint32_t ph = 0;
+    bool alive = true;
+    for (int t = tile_first; t < tile_end && alive; t += tile_step) {
+      for (int kb = 0; kb < args.num_kb; ++kb) {
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status))) {
+          alive = false;
+          break;
+        }
+        if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl.full[s]), 0u));
+        __syncwarp();
+        if (++s == stages) {
+          s = 0;
+          ph ^= 1u;
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- leader: MMA issue for the pair
+    const uint32_t idesc = make_idesc_i8_pair(args.tile_n);
+    const uint64_t adesc0 = make_smem_desc(a_base, bk);
+    const uint64_t bdesc0 = make_smem_desc(b_base, bk);
+    const uint64_t a_step = a_stage_bytes >> 4, b_step = b_stage_bytes >> 4;
+    uint64_t adesc = adesc0, bdesc = bdesc0;
+    int s = 0;
+    uint32_t ph = 0;
+    const uint32_t leader_lane = elect_one() ? 1u : 0u;
+    bool alive = true;
+    int ti = 0;
+    for (int t = tile_first; t < tile_end && alive; t += tile_step, ++ti) {
+      const int buf = persistent ? (ti & (nbuf - 1)) : 0;
+      const uint32_t use = persistent ? (uint32_t)(ti / nbuf) : 0u;
+      if (persistent) {
+        // the epilogue warps of both blocks must have drained this accumulator buffer
+        if (!__all_sync(0xffffffffu, mbar_wait_cluster(smem_u32(&ctl.tmem_empty[buf]), (use & 1u) ^ 1u, &ctl, args.status))) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      }
+      const uint32_t d_tmem = tmem_acc + (uint32_t)(buf * args.tmem_cols);
+      uint32_t accumulate = 0;
+      for (int kb = 0; kb < args.num_kb; ++kb) {
+        if (!__all_sync(0xffffffffu, mbar_wait_cluster(smem_u32(&ctl.full[s]), ph, &ctl, args.status))) {
+          alive = false;
+          break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int ksteps = (kb == args.num_kb - 1) ? args.ksteps_last : args.ksteps_full;
+        mma_i8_pair_block(d_tmem, adesc, bdesc, idesc, accumulate, leader_lane, ksteps);
+        mma_commit_pair(smem_u32(&ctl.empty[s]), leader_lane);
+        if (kb == args.num_kb - 1) mma_commit_pair(smem_u32(&ctl.tmem_full[buf]), leader_lane);
+        accumulate = 1;
+        adesc += a_step;
+        bdesc += b_step;
+        if (++s == stages) {
+          s = 0;
+          ph ^= 1u;
+          adesc = adesc0;
+          bdesc = bdesc0;
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------------------------------------------------------- epilogue warps (both blocks)
+    const int quad = warp & 3;         // TMEM lane quadrant this warp may read
+    const int half = (warp - 2) >> 2;  // the two warps of a quadrant split the columns
+    const int row = quad * 32 + lane;
+    const uint32_t leader_empty0 = map_to_rank(smem_u32(&ctl.tmem_empty[0]), 0u);
+    const uint32_t leader_empty1 = map_to_rank(smem_u32(&ctl.tmem_empty[1]), 0u);
+    bool ok = true;
+    int ti = 0;
+    for (int t = tile_first; t < tile_end && ok; t += tile_step, ++ti) {
+      B2C_PAIR_TILE_ORIGIN(t)
+      const unsigned m = (unsigned)m0 + (unsigned)row;
+      bool row_valid = m < (unsigned)args.Mg;
+      int n_img = 0, pq = 0;
+      if (row_valid) {
+        n_img = (int)args.div_pq.div(m);
+        pq = (int)(m - (unsigned)n_img * (unsigned)args.PQ);
+      }
+      int out_img = n_img, out_pq = pq;
+      if (args.remap == 1 && row_valid) {
+        // dilation phase pack: interleave the sub-image results back, drop rows outside the output
+        const int ps = (int)args.div_q.div((uint32_t)pq), qs = pq - ps * args.Q;
+        const int phases = args.ph_dh * args.ph_dw;
+        out_img = n_img / phases;
+        const int phs = n_img - out_img * phases;
+        const int a = phs / args.ph_dw, b = phs - a * args.ph_dw;
+        const int po = (ps - args.ph_pad_h) * args.ph_dh + a + args.out_pad_h;
+        const int qo = (qs - args.ph_pad_w) * args.ph_dw + b + args.out_pad_w;
+        row_valid = (unsigned)po < (unsigned)args.out_P && (unsigned)qo < (unsigned)args.out_Q;
+        out_pq = po * args.out_Q + qo;
+      }
+      const int buf = persistent ? (ti & (nbuf - 1)) : 0;
+      const uint32_t use = persistent ? (uint32_t)(ti / nbuf) : 0u;
+      ok = mbar_wait(smem_u32(&ctl.tmem_full[buf]), use & 1u, &ctl, args.status);
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (ok) {
+        const long long base_nkpq = (long long)out_img * args.y_stride_n + out_pq;
+        const long long base_npqk = args.remap ? ((long long)out_img * args.out_PQ + out_pq) * args.K : (long long)m * args.K;
+        const int cols = args.tile_n >> 1;  // tile_n >= 32
+        const int c_begin = half * cols;
+        const uint32_t taddr = tmem_acc + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * args.tmem_cols) + (uint32_t)c_begin;
+        if ((cols & 31) == 0) {
+          for (int c = 0; c < cols; c += 32)
+            epilogue_columns<32>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk, 0u);
+        } else {
+          for (int c = 0; c < cols; c += 16)
+            epilogue_columns<16>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk, 0u);
+        }
+        if (persistent) {
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(buf ? leader_empty1 : leader_empty0);
+        }
+      }
+    }
+  }
+#undef B2C_PAIR_TILE_ORIGIN
+
+  // ---------------------------------------------------------------- teardown
+  // No block of the pair leaves, or frees tensor memory, while the other may still read its shared
+  // memory, arrive on its barriers or write its accumulator.
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (ctl.abort_flag) {
+    if (threadIdx.x == 0) {
+      const unsigned long long t0 = global_ns();
+      while (global_ns() - t0 < 50000ull) __nanosleep(1000);
+    }
+    __syncthreads();
+  }
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(args.tmem_cols * nbuf)
+                 : "memory");
+  }
+}
+
+}  // namespace
+
+size_t conv_mma_pair_smem_bytes(const ConvArgs& a) { return 1024 + (size_t)a.stage_region; }
+
+cudaError_t launch_conv_mma_pair(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,
+                                 cudaStream_t st) {
+  const size_t smem = conv_mma_pair_smem_bytes(args);
+  int pairs = args.persistent ? std::min(args.num_tiles, kNumSMs / 2) : args.num_tiles;
+  dim3 grid((unsigned)(2 * pairs), 1, 1);
+  cudaError_t e;
+#define B2C_LAUNCH_PAIR(MODE, PERS)                                                                            \
+  {                                                                                                           \
+    static std::atomic<unsigned long long> configured{0};                                                     \
+    e = set_max_dynamic_smem_once(configured, (const void*)conv_mma_pair_kernel<MODE, PERS>, 200 * 1024);      \
+    if (e != cudaSuccess) return e;                                                                           \
+    cudaLaunchConfig_t cfg = {};                                                                              \
+    cfg.gridDim = grid;                                                                                       \
+    cfg.blockDim = dim3(kThreads);                                                                            \
+    cfg.dynamicSmemBytes = smem;                                                                              \
+    cfg.stream = st;                                                                                          \
+    cudaLaunchAttribute attr[2];                                                                              \
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                          \
+    attr[0].val.programmaticStreamSerializationAllowed = 1;                                                   \
+    attr[1].id = cudaLaunchAttributeClusterDimension;                                                         \
+    attr[1].val.clusterDim.x = 2;                                                                             \
+    attr[1].val.clusterDim.y = 1;                                                                             \
+    attr[1].val.clusterDim.z = 1;                                                                             \
+    cfg.attrs = attr;                                                                                         \
+    cfg.numAttrs = 2;                                                                                         \
+    if (PERS) {                                                                                               \
+      /* a persistent grid is one wave: as many pairs as the device keeps resident at once */                 \
+      int resident = 0;                                                                                       \
+      if (cudaOccupancyMaxActiveClusters(&resident, conv_mma_pair_kernel<MODE, PERS>, &cfg) == cudaSuccess && \
+          resident > 0 && resident < pairs) {                                                                 \
+        pairs = resident;                                                                                     \
+        cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);                                                      \
+      }                                                                                                       \
+      (void)cudaGetLastError();                                                                               \
+    }                                                                                                         \
+    e = cudaLaunchKernelEx(&cfg, conv_mma_pair_kernel<MODE, PERS>, *tmap_a, *tmap_b, args);                    \
+    if (e != cudaSuccess) return e;                                                                           \
+  }
+  if (amode == A_TILED && args.persistent) B2C_LAUNCH_PAIR(A_TILED, 1)
+  else if (amode == A_TILED) B2C_LAUNCH_PAIR(A_TILED, 0)
+  else if (amode == A_IM2COL_TMA && args.persistent) B2C_LAUNCH_PAIR(A_IM2COL_TMA, 1)
+  else if (amode == A_IM2COL_TMA) B2C_LAUNCH_PAIR(A_IM2COL_TMA, 0)
+  else return cudaErrorInvalidValue;
+#undef B2C_LAUNCH_PAIR
+  return cudaGetLastError();
+}
+
+}  // namespace b2c

@@ -296,18 +296,18 @@ bool staged_window(const Geom& g, WindowGeom* w) {
 }
 
 static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int tile_n, int split_k,
-                bool swap = false) {
+                bool swap = false, int tile_m = kTileM) {
   const b2c_conv_desc& d = g.d;
   b2c_embedding e;
   std::memset(&e, 0, sizeof(e));
   e.map_m = swap ? B2C_AXIS_K : B2C_AXIS_NPQ;
   e.map_n = swap ? B2C_AXIS_NPQ : B2C_AXIS_K;
   e.variant = variant;
-  e.tile_m = kTileM;
+  e.tile_m = tile_m;
   e.tile_n = tile_n;
   e.split_k = split_k;
   e.device_us = -1.0f;
-  long long M_pad = (g.Mg + kTileM - 1) / kTileM * kTileM;
+  long long M_pad = (g.Mg + tile_m - 1) / tile_m * tile_m;
   long long N_pad = (long long)round_up(d.K, tile_n);
   if (swap) {
     M_pad = (long long)round_up(d.K, kTileM);
@@ -322,7 +322,7 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
                   ? B2C_AXIS_C
                   : ((variant == B2C_VARIANT_ROW_UNROLL || variant == B2C_VARIANT_ROWPHASE_SHIFT) ? B2C_AXIS_SC
                                                                                                   : B2C_AXIS_C_PHASES);
-    if (!swap) M_pad = (view_rows(g, variant, v) + kTileM - 1) / kTileM * kTileM;
+    if (!swap) M_pad = (view_rows(g, variant, v) + tile_m - 1) / tile_m * tile_m;
     k_issued = (long long)v.R * v.S * v.C;
     long long packed = v.bytes();
     bool direct = shift_base_variant(variant) == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && v.C == d.C;
@@ -387,6 +387,8 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
         if (split > 1 && ctas * (split / 2) >= kNumSMs) break;
         add(out, g, variant, t, split);
       }
+      // two-SM schedule of the same map: 256-row tiles, each block of the pair loads half of the column tile
+      if (pair_schedule_ok(variant, t, 1, false, tiles_m * kTileM)) add(out, g, variant, t, 1, false, 2 * kTileM);
     }
     // Swapped axis map (M <- k, N <- fused pixels) for the TMA-fed variants: the 128 accumulator rows
     // are output channels, so it is only listed when K fills at least half of them; the pixel tile

@@ -589,6 +589,46 @@ def test_persistent_256_column_tiles(lib, in_layout, out_mode):
     check_against_oracle(x, w, 2, 1, 1, 10, out_mode, ids[0], ref=ref, in_layout=in_layout)
 
 
+# ---- two-SM schedule: a pair of blocks per 256-row tile, each loading half of the column tile -------------
+@pytest.mark.parametrize("case", [
+    # N, C, H, W, K, R, S, stride, pad, dil, shift
+    (32, 256, 14, 14, 512, 3, 3, 2, 1, 1, 10),     # the compute-bound benchmark shape: 7 x 2 pair tiles, the last one half empty
+    (3, 64, 20, 20, 129, 3, 3, 1, 1, 1, 9),        # ragged column tile (129 channels), 1200 pixels
+    (2, 32, 17, 13, 40, 2, 3, (1, 2), (0, 1), (2, 1), 7),   # 8-row-group ragged weights, dilation, odd pixel count
+    (5, 3, 30, 31, 96, 5, 5, 2, 2, 1, 6),          # low channel count: row-unroll / space-to-depth / explicit views
+    (1, 16, 33, 33, 64, 3, 3, 1, 2, 2, 8),         # dilated: the phase pack's scattered rows
+    (1, 128, 12, 11, 256, 1, 1, 1, 0, 1, 5),       # 1x1: 132 pixels, the second block of the pair nearly empty
+])
+@pytest.mark.parametrize("out_layout", [0, 1])
+def test_two_sm_schedule(lib, case, out_layout):
+    N, C, H, W, K, R, S, stride, pad, dil, shift = case
+    x = int8_uniform((N, C, H, W), 731)
+    w = int8_uniform((K, C, R, S), 732)
+    ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, 0, out_layout, 3)
+    pairs = [e for e in lib.enumerate_embeddings(d) if e.tile_m == 256]
+    assert pairs and all(e.split_k == 1 and e.map_m == b2c.AXIS_NPQ and e.tile_n >= 32 for e in pairs)
+    for e in pairs:
+        check_against_oracle(x, w, stride, pad, dil, shift, 3, e.id, ref=ref, out_layout=out_layout)
+
+
+@pytest.mark.parametrize("in_layout", [0, 1])
+@pytest.mark.parametrize("tile_n", [64, 256])
+def test_two_sm_schedule_walks_tiles(lib, in_layout, tile_n):
+    """More pair tiles than SM pairs: the clusters walk the tile list with two accumulator buffers."""
+    N, C, H, W, K, R, S = 800, 64, 14, 14, 512, 3, 3   # 39200 pixels = 154 pair row tiles x 2 (or 8) column tiles
+    if "ref" not in _wide_ref:
+        x = int8_uniform((N, C, H, W), 711)
+        w = int8_uniform((K, C, R, S), 712)
+        _wide_ref["ref"] = (x, w, oracle.conv2d_int8(x, w, 2, 1, 1, 10))
+    x, w, ref = _wide_ref["ref"]
+    d = lib.make_desc(N, C, H, W, K, R, S, 2, 1, 1, 10, in_layout, 0, 3)
+    for variant in (0, 1):
+        ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant and e.tile_n == tile_n and e.tile_m == 256]
+        assert ids
+        check_against_oracle(x, w, 2, 1, 1, 10, 3, ids[0], ref=ref, in_layout=in_layout)
+
+
 # ---- one-shot calls of one shape on two streams with different weights do not disturb each other ---------
 def test_one_shot_calls_on_two_streams(lib):
     N, C, H, W, K, R, S = 2, 32, 20, 20, 48, 3, 3

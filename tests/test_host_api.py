@@ -85,7 +85,9 @@ def test_enumeration_is_sorted_and_covers_variants(lib, cfg):
     assert costs == sorted(costs)
     assert {0, 1, 2} <= {e.variant for e in embs} <= {0, 1, 2, 3, 4, 5, 6, 7, 8, 9}
     for e in embs:
-        assert e.tile_m == 128 and e.tile_n in (16, 32, 64, 128, 256) and e.split_k >= 1
+        assert e.tile_m in (128, 256) and e.tile_n in (16, 32, 64, 128, 256) and e.split_k >= 1
+        if e.tile_m == 256:   # two-SM schedule: TMA-fed maps, no split, column tile of at least 32
+            assert e.variant in (0, 1, 4, 5, 6) and e.split_k == 1 and e.tile_n >= 32 and e.map_m == b2c.AXIS_NPQ
         assert (e.map_m, e.map_n) in ((b2c.AXIS_NPQ, b2c.AXIS_K), (b2c.AXIS_K, b2c.AXIS_NPQ))
         if e.map_m == b2c.AXIS_K:  # swapped map: TMA-fed variants only, and only when K fills half a tile
             assert e.variant in (0, 1, 4, 5) and cfg.K >= 64 and e.tile_n >= 32
@@ -104,8 +106,9 @@ def test_channel_pack_utilisation_law(lib):
         mac_min = N * K * 16 * 16 * C * R * S
         cp = [e for e in b2c.enumerate_embeddings(d)
               if e.variant == 0 and e.tile_n == 64 and e.split_k == 1 and e.map_m == b2c.AXIS_NPQ]
-        assert len(cp) == 1
-        assert (cp[0].o_mac + mac_min) * C == mac_min * C_pad
+        assert sorted(e.tile_m for e in cp) == [128, 256]   # one-SM and two-SM schedule of the same map
+        for e in cp:                                        # M = 512 is a multiple of both tile heights
+            assert (e.o_mac + mac_min) * C == mac_min * C_pad
         # the stencil-unroll maps pad the fused (c, r, s) axis to 32 instead
         kp = -(-C * R * S // 32) * 32
         un = [e for e in b2c.enumerate_embeddings(d) if e.variant == 2 and e.tile_n == 64 and e.split_k == 1]
