@@ -40,7 +40,7 @@ INT8_TO_BF16_RATIO = 2.0  # nominal dense int8 : bf16 tensor throughput on B200 
 # DRAM traffic of the dominant kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
 # per launch), valid only for the sources it was taken on (the kernel and the host code that picks its
 # tile, stage count and launch shape); see profiles/.
-KERNEL_SOURCES = ("conv_mma.cu", "api.cpp", "planner.cpp", "tma.cpp", "b2c_internal.h")
+KERNEL_SOURCES = ("conv_mma.cu", "conv_mma_pair.cu", "conv_mma_common.cuh", "api.cpp", "planner.cpp", "tma.cpp", "b2c_internal.h")
 NCU_TRAFFIC = {"conv_mma_sha1": "2f7f0c9ebef77a24137d8c3d4168093c86fde328", "bytes_per_launch": 2859008}
 
 
@@ -280,9 +280,10 @@ def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, grap
     warm.capture(torch, repeat=20)
     ms_w = time_steps(torch, warm.step, 10, 3, None, 0.0)
     warm.destroy()
-    op = op_only(b2c, torch, cfg, emb["variant"], emb["tile_n"], emb["split_k"], steps, warmup, graph, 1, emb["map_m"])
+    op = op_only(b2c, torch, cfg, emb["variant"], emb["tile_n"], emb["split_k"], steps, warmup, graph, 1, emb["map_m"],
+                 emb["tile_m"])
     t_roof, bound = roofline_time_us(cfg, peaks)
-    keys = ("id", "variant_name", "map_m", "tile_n", "split_k", "workspace_bytes", "o_mac", "o_data", "device_us")
+    keys = ("id", "variant_name", "map_m", "tile_m", "tile_n", "split_k", "workspace_bytes", "o_mac", "o_data", "device_us")
     res = {
         "shape": cfg.name, "instances": G, "warm_us": ms_w * 1e3 / (10 * 20),
         "op_us": op["us"] if op else None, "transf_us": max(0.0, per_call_us - op["us"]) if op else None, "cold": bool(G * cfg.algorithmic_bytes >= L2_BYTES), "combined_us": per_call_us, "tops": 2.0 * cfg.macs / (per_call_us * 1e-6) / 1e12,
@@ -339,8 +340,8 @@ def measure_scaled(b2c, torch, cfg, peaks, steps=10):
             raise RuntimeError("device status " + b2c.status_string(st))
         us = ms * 1e3 / steps
         return {"us": us, "tops": 2.0 * big.macs / (us * 1e-6) / 1e12, "roofline_frac": t_roof / us,
-                "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k,
-                              "swapped": emb.map_m == b2c.AXIS_K}}
+                "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_m": emb.tile_m, "tile_n": emb.tile_n,
+                              "split_k": emb.split_k, "swapped": emb.map_m == b2c.AXIS_K}}
 
     res = {"shape": big.name, "roofline_us": t_roof, "bound": bound, "bytes": big.algorithmic_bytes}
     res.update(one(0))
@@ -349,13 +350,14 @@ def measure_scaled(b2c, torch, cfg, peaks, steps=10):
     return res
 
 
-def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=True, streams=1, map_m=1):
+def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=True, streams=1, map_m=1, tile_m=128):
     """Device time of the MMA kernel alone: same embedding but with the layout rewrite already done
     (channel-pack map: NHWC input with padded channels; stencil-unroll in-kernel: unchanged)."""
     if emb_variant in (0, 7) and cfg.C % 32 == 0:
         d = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, 1, 0, cfg.out_mode)
         ids = [e.id for e in b2c.enumerate_embeddings(d)
-               if e.variant == emb_variant and e.tile_n == tile_n and e.split_k == split_k and e.map_m == map_m]
+               if e.variant == emb_variant and e.tile_n == tile_n and e.split_k == split_k and e.map_m == map_m
+               and e.tile_m == tile_m]
         if not ids:
             return None
         G = instances_for(cfg)
@@ -364,7 +366,8 @@ def op_only(b2c, torch, cfg, emb_variant, tile_n, split_k, steps, warmup, graph=
         # stencil unroll inside the kernel: there is no separate rewrite, the kernel is the whole path
         d = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift, 0, 0, cfg.out_mode)
         ids = [e.id for e in b2c.enumerate_embeddings(d)
-               if e.variant == emb_variant and e.tile_n == tile_n and e.split_k == split_k and e.map_m == map_m]
+               if e.variant == emb_variant and e.tile_n == tile_n and e.split_k == split_k and e.map_m == map_m
+               and e.tile_m == tile_m]
         G = instances_for(cfg)
         inst = Instances(b2c, torch, cfg, G, ids[0])
     else:
@@ -627,11 +630,11 @@ def run_ours(args):
     auto = b2c.POLICY_AUTO_TIMED_CONCURRENT if args.streams > 1 else b2c.POLICY_AUTO_TIMED
     policy = auto if args.embedding is None else args.embedding
     if args.pick:
-        v, tn, sk = (int(t) for t in args.pick.split(","))
+        v, tn, sk, tm = (tuple(int(t) for t in args.pick.split(",")) + (128,))[:4]
         d0 = b2c.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
                            0, 0, cfg.out_mode)
         policy = next(e.id for e in b2c.enumerate_embeddings(d0)
-                      if (e.variant, e.tile_n, e.split_k) == (v, tn, sk) and e.map_m == b2c.AXIS_NPQ)
+                      if (e.variant, e.tile_n, e.split_k, e.tile_m) == (v, tn, sk, tm) and e.map_m == b2c.AXIS_NPQ)
     graph = not args.no_graph
     if args.report == "candidates":
         rep = candidates_report(b2c, torch, CONFIGS + REPORT_EXTRA)
@@ -665,7 +668,7 @@ def run_ours(args):
     op = None
     if not args.no_op_pass:
         op = op_only(b2c, torch, cfg, emb.variant, emb.tile_n, emb.split_k, args.steps, args.warmup, graph, args.streams,
-                     emb.map_m)
+                     emb.map_m, emb.tile_m)
     t_roof, bound = roofline_time_us(cfg, peaks)
     op_us = op["us"] if op else per_call_us
     if bound == "tensor":
@@ -723,8 +726,8 @@ def run_ours(args):
                    "l2": "inputs larger than L2: %d distinct buffer sets per step (%.0f MB)" % (G, G * (cfg.algorithmic_bytes) / 1e6),
                    "cuda_graph": graph, "streams": args.streams if graph else 1,
                    "parallelism": "independent instances sharded over ranks, no collective",
-                   "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_n": emb.tile_n, "split_k": emb.split_k,
-                                 "swapped": emb.map_m == b2c.AXIS_K, "planner_us": emb.device_us}},
+                   "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_m": emb.tile_m, "tile_n": emb.tile_n,
+                                 "split_k": emb.split_k, "swapped": emb.map_m == b2c.AXIS_K, "planner_us": emb.device_us}},
         "roofline": roofline, "roofline_time_us": t_roof, "whole_path_roofline_frac": t_roof / per_call_us,
         "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "verified": verified,
     }
@@ -750,7 +753,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--headline-only", action="store_true", help="skip the per-shape and scaled-batch series")
-    ap.add_argument("--pick", default=None, help="embedding as variant,tile_n,split_k (instead of an id)")
+    ap.add_argument("--pick", default=None, help="embedding as variant,tile_n,split_k[,tile_m] (instead of an id)")
     ap.add_argument("--scaled", action="store_true", help="use the batch-scaled version of the shape as the workload")
     ap.add_argument("--instances", type=int, default=0, help="instances per step (default: enough to exceed L2)")
     ap.add_argument("--min-warm-s", type=float, default=0.2, help="extra time-based warm-up before the timed steps")

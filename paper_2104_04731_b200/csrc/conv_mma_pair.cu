@@ -7,14 +7,18 @@
 // both shared memories.  Per MMA cycle a block therefore takes a third fewer operand bytes from
 // L2 than the one-SM kernel with the same tile_n, which is what bounds the compute-bound shapes.
 //
-// Roles in each block: warp 0 TMA producer (own A rows, own B half; plain TMA loads that
-// complete on the block's own barrier, no cluster multicast), warp 1 MMA issue in the leader block
-// (cluster rank 0) and hand-over of "my half has landed" to the leader in the other block, warps
-// 2-9 epilogue of the block's own 128 accumulator rows (tcgen05.ld from the block's own tensor
-// memory, activation step, shift / clip, stores).  Barriers: full[s] of the leader counts its own
-// producer and the peer's hand-over; the leader's commits arrive on empty[s] and tmem_full[b] of
-// BOTH blocks (tcgen05.commit with a block mask); the epilogue warps of both blocks arrive on
-// the leader's tmem_empty[b].  Every wait is bounded as in the one-SM kernel.
+// Roles in each block: warp 0 TMA producer (own A rows, own B half, into the block's own shared
+// memory; no cluster multicast), warp 1 MMA issue in the leader block (cluster rank 0; idle in the
+// other block after the tensor-memory allocation), warps 2-9 epilogue of the block's own 128
+// accumulator rows (tcgen05.ld from the block's own tensor memory, activation step, shift / clip,
+// stores).  Barriers: the copies of BOTH blocks complete on the leader's full[s] (the loads carry
+// .cta_group::2, which lets a copy signal a barrier in the peer block; the leader's producer
+// announces the bytes of both), so the MMA thread waits on one barrier with no hand-over in
+// between (a hand-over by a thread of the peer, mbarrier.arrive.release.cluster on the leader's
+// barrier, measured about 0.8 us per stage and paced the whole kernel); the leader's commits
+// arrive on empty[s] and tmem_full[b] of BOTH blocks (tcgen05.commit with a block mask); the
+// epilogue warps of both blocks arrive on the leader's tmem_empty[b].  Every wait is bounded as
+// in the one-SM kernel.
 #include <algorithm>
 
 #include "conv_mma_common.cuh"
@@ -66,6 +70,27 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
   for (int i = 0; i < 32; ++i)
     if (mbar_try_wait_cluster(bar, parity)) return true;
   return mbar_wait_cluster_slow(bar, parity, ctl, status);
+}
+
+// TMA loads of a block of the pair: destination in the executing block's shared memory, completion
+// on `bar`, a shared::cluster address that may lie in either block of the pair (.cta_group::2).
+__device__ __forceinline__ void tma_pair_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar,
+                                                 uint32_t on) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %5, 0;\n"
+      "@q cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, %3}], "
+      "[%4];\n}" ::"r"(dst),
+      "l"(map), "r"(c0), "r"(c1), "r"(bar), "r"(on)
+      : "memory");
+}
+__device__ __forceinline__ void tma_pair_load_im2col_4d(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n,
+                                                        uint32_t bar, uint16_t off_w, uint16_t off_h, uint32_t on) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %9, 0;\n"
+      "@q cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, "
+      "%3, %4, %5}], [%6], {%7, %8};\n}" ::"r"(dst),
+      "l"(map), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"(off_w), "h"(off_h), "r"(on)
+      : "memory");
 }
 
 // Instruction descriptor of the two-SM MMA: as make_idesc_i8, with M = 256 (128 rows per block).
@@ -142,8 +167,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
 
   if (warp == 0) {
     if (lane < stages) {
-      // the leader's full barrier also counts the peer's "my half has landed"
-      mbar_init(smem_u32(&ctl.full[lane]), rank == 0 ? 2 : 1);
+      // full[] is used in the leader only: one arrival (its producer) plus the bytes of both blocks
+      mbar_init(smem_u32(&ctl.full[lane]), 1);
       mbar_init(smem_u32(&ctl.empty[lane]), 1);
     }
     if (lane == 8) {
@@ -203,13 +228,14 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
           alive = false;
           break;
         }
-        const uint32_t full = smem_u32(&ctl.full[s]);
-        mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes, leader_lane);
+        // both blocks' copies complete on the leader's barrier; the leader announces the bytes of both
+        const uint32_t full = map_to_rank(smem_u32(&ctl.full[s]), 0u);
+        if (rank == 0) mbar_arrive_expect_tx(smem_u32(&ctl.full[s]), 2u * (a_stage_bytes + b_stage_bytes), leader_lane);
         if (AMODE == A_TILED) {
-          tma_load_2d(a_dst, &tmap_a, kcol, m0, full, leader_lane);
+          tma_pair_load_2d(a_dst, &tmap_a, kcol, m0, full, leader_lane);
         } else {
-          tma_load_im2col_4d(a_dst, &tmap_a, cb * bk, w_org, h_org, n_img, full, (uint16_t)(sx * args.dil_w),
-                             (uint16_t)(r * args.dil_h), leader_lane);
+          tma_pair_load_im2col_4d(a_dst, &tmap_a, cb * bk, w_org, h_org, n_img, full, (uint16_t)(sx * args.dil_w),
+                                  (uint16_t)(r * args.dil_h), leader_lane);
           if (++cb == args.kb_per_tap) {
             cb = 0;
             if (++sx == args.S) {
@@ -218,7 +244,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
             }
           }
         }
-        tma_load_2d(b_dst, &tmap_b, kcol, wrow0, full, leader_lane);
+        tma_pair_load_2d(b_dst, &tmap_b, kcol, wrow0, full, leader_lane);
         kcol += bk;
         a_dst += a_stage_bytes;
         b_dst += b_stage_bytes;
@@ -232,26 +258,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
     }
     __syncwarp();
   } else if (warp == 1 && rank != 0) {
-    // ---------------------------------------------------------------- peer: hand-over of full stages
-    // Once this block's copies of a stage have landed, one lane arrives on the leader's full barrier.
-    int s = 0;
-    uint32_t ph = 0;
-    bool alive = true;
-    for (int t = tile_first; t < tile_end && alive; t += tile_step) {
-      for (int kb = 0; kb < args.num_kb; ++kb) {
-        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status))) {
-          alive = false;
-          break;
-        }
-        if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl.full[s]), 0u));
-        __syncwarp();
-        if (++s == stages) {
-          s = 0;
-          ph ^= 1u;
-        }
-      }
-    }
-    __syncwarp();
+    // (the peer's warp 1 only allocates and frees tensor memory)
   } else if (warp == 1) {
     // ---------------------------------------------------------------- leader: MMA issue for the pair
     const uint32_t idesc = make_idesc_i8_pair(args.tile_n);
@@ -275,7 +282,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
       const uint32_t d_tmem = tmem_acc + (uint32_t)(buf * args.tmem_cols);
       uint32_t accumulate = 0;
       for (int kb = 0; kb < args.num_kb; ++kb) {
-        if (!__all_sync(0xffffffffu, mbar_wait_cluster(smem_u32(&ctl.full[s]), ph, &ctl, args.status))) {
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl.full[s]), ph, &ctl, args.status))) {
           alive = false;
           break;
         }
