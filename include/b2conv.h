@@ -294,6 +294,17 @@ int b2c_im2col(const b2c_conv_desc* desc, const int8_t* x_dev, int8_t* a_dev, in
  *     them on one stream or with events. */
 int b2c_im2col_noalloc(const b2c_conv_desc* desc, const int8_t* x_dev, int8_t* a_dev, int K_pad, void* cuda_stream);
 
+/* Peak of the intrinsic itself on this device (Section 5.1: the GEMM core is the unit whose
+ * utilisation decides the operator time; this measures that unit alone).  Launches one block per SM
+ * that issues `mmas_per_block` (a multiple of 4, at most 2^22) tcgen05.mma.kind::i8 instructions of
+ * shape 128 x tile_n x 32 back to back on operands resident in shared memory, on `cuda_stream`, and
+ * waits for it.  *device_us: CUDA-event time of the launch (all SMs busy), so that
+ * 148 * mmas_per_block * 2*128*tile_n*32 / device_us is the device's int8 issue rate;
+ * *cycles_per_mma: median over the SMs of SM clock cycles per instruction.  tile_n in
+ * {16, 32, 64, 128, 256}.  Allocates a few KB and synchronises: not for use under stream capture.
+ * INVALID_ARG on bad arguments, B2C_E_CUDA / B2C_E_TIMEOUT on failure. */
+int b2c_measure_mma_rate(int tile_n, int mmas_per_block, float* device_us, float* cycles_per_mma, void* cuda_stream);
+
 /* Host-side fault injection for tests (no counterpart in the paper): the n-th tensor-map encode
  * from now on, counted over all threads, fails as if the driver had refused it (the call that
  * needed it returns B2C_E_CUDA); n = 0 disarms.  Nothing on the device is touched. */

@@ -33,7 +33,7 @@ EXPORTS = [
     "b2c_plan_create_grouped", "b2c_plan_run_host_async", "b2c_plan_host_sync",
     "b2c_plan_device_status", "b2c_selftest_bounded_wait", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
     "b2c_status_string",
-    "b2c_last_cuda_error", "b2c_oneshot_status", "b2c_oneshot_cache_clear", "b2c_test_fail_nth_encode", "b2c_selftest_pack_wait",
+    "b2c_last_cuda_error", "b2c_oneshot_status", "b2c_oneshot_cache_clear", "b2c_test_fail_nth_encode", "b2c_selftest_pack_wait", "b2c_measure_mma_rate",
 ]
 
 
@@ -108,6 +108,7 @@ def load():
     lib.b2c_status_string.restype = ctypes.c_char_p
     lib.b2c_last_cuda_error.argtypes = []
     lib.b2c_oneshot_status.argtypes = [pi32]
+    lib.b2c_measure_mma_rate.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float), vp]
     lib.b2c_oneshot_cache_clear.argtypes = []
     lib.b2c_test_fail_nth_encode.argtypes = [i32]
     for name in EXPORTS:
@@ -263,6 +264,14 @@ def conv2d_int8(x, w, stride=1, pad=0, dilation=1, shift=0, y32=None, y8=None, s
     K, _, R, S = w.shape
     _check(load().b2c_conv2d_int8(N, C, H, W, K, R, S, stride, pad, dilation, shift, _dptr(x), _dptr(w), _dptr(y32),
                                   _dptr(y8), _stream_ptr(stream)), "b2c_conv2d_int8")
+
+
+def measure_mma_rate(tile_n: int = 256, mmas_per_block: int = 20000, stream=None):
+    """(device_us, cycles_per_mma) of back-to-back 128 x tile_n x 32 int8 MMAs on all SMs, operands in shared memory."""
+    us, cyc = ctypes.c_float(), ctypes.c_float()
+    _check(load().b2c_measure_mma_rate(tile_n, mmas_per_block, ctypes.byref(us), ctypes.byref(cyc), _stream_ptr(stream)),
+           "b2c_measure_mma_rate")
+    return us.value, cyc.value
 
 
 def oneshot_status() -> int:

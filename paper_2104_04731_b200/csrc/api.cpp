@@ -45,6 +45,11 @@ struct b2c_plan {
   std::vector<b2c_plan*> subs;
   long long x_stride_n_whole = 0, y_stride_n_whole = 0;  // sub-plans: batch strides of the whole tensors
   struct HostPipe* pipe = nullptr;  // streaming host-buffer calls: created by the first b2c_plan_run_host_async
+  // The two-SM persistent channel-pack schedule can run the activation pack inside the MMA kernel
+  // (NCHW input whose rows have a bulk-copy form): run then launches one kernel, preceded by a memset
+  // of the work counters, which live in the workspace after the rewritten operand.
+  bool fused_pack = false;
+  size_t ws_ctl_offset = 0;  // bytes from the workspace start to the counters [1 + N] int
 };
 
 // Device side of the streaming host-buffer calls: a ring of input / output buffers and three
@@ -287,7 +292,20 @@ void fill_common_args(b2c_plan* p) {
     a.tmem_bufs = (a.persistent && 2 * a.tmem_cols <= 512) ? 2 : 1;
     a.cluster_split = 0;
     const size_t pair_stage = (size_t)(kTileM + a.tile_n / 2) * a.bk;
-    const size_t pair_budget = a.persistent ? 196 * 1024 : 100 * 1024;
+    size_t pair_budget = a.persistent ? 196 * 1024 : 100 * 1024;
+    // activation pack inside the kernel: NCHW input of the channel-pack map, persistent grid
+    a.pk_on = 0;
+    p->fused_pack = false;
+    if (a.persistent && p->emb.variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NCHW &&
+        fused_pack_geometry(d.C, d.H, d.W, p->C_pad, &a.pk_ct, &a.pk_pt, &a.pk_hw_tiles, &a.pk_ctiles, &a.pk_smem) &&
+        (long long)d.N * a.pk_hw_tiles * a.pk_ctiles < 0x7FFFFFFFLL) {
+      p->fused_pack = true;
+      a.pk_N = d.N;
+      a.pk_C = d.C;
+      a.pk_HW = d.H * d.W;
+      a.pk_Cpad = p->C_pad;
+      pair_budget = 224 * 1024 - (size_t)a.pk_smem;
+    }
     int st = std::min(8, std::max(1, a.num_kb));
     while (st > 2 && (size_t)st * pair_stage > pair_budget) --st;
     a.stages = st;
@@ -436,6 +454,10 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
   if (cudaMalloc(&p->w_packed, p->w_packed_bytes + 256) != cudaSuccess) return fail(B2C_E_CUDA);
   fill_common_args(p);
   p->ws_total = workspace_bytes_for(g, emb.variant, emb.tile_n, emb.split_k, is_swapped(emb));
+  if (p->fused_pack) {
+    p->ws_ctl_offset = (p->ws_total + 255) / 256 * 256;
+    p->ws_total = p->ws_ctl_offset + ((size_t)(d.N + 1) * sizeof(int) + 255) / 256 * 256;
+  }
   if (is_tma_view_variant(emb.variant)) {
     bool direct = shift_base_variant(emb.variant) == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC && p->C_pad == d.C;
     p->ws_layout_bytes = direct ? 0 : ((size_t)p->view.bytes() + 255) / 256 * 256;
@@ -641,7 +663,7 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
   for (int l = 0; l < lanes && alloc_ok; ++l)
     alloc_ok = cudaMalloc(&lane[l].y8, g.y_elems + 256) == cudaSuccess &&
                cudaMalloc(&lane[l].y32, g.y_elems * 4 + 256) == cudaSuccess &&
-               cudaMalloc(&lane[l].ws, ws_max + 256) == cudaSuccess;
+               cudaMalloc(&lane[l].ws, ws_max + 1024) == cudaSuccess;
   if (!alloc_ok) {
     set_last_cuda_error((int)cudaGetLastError());
     cleanup();
@@ -818,7 +840,8 @@ static int run_rewrite(b2c_plan* p, const int8_t* x, void* ws, cudaStream_t st) 
   return B2C_OK;
 }
 
-static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, cudaStream_t st) {
+static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, cudaStream_t st,
+                        bool fused_pack = false) {
   const b2c_conv_desc& d = p->g.d;
   const Geom& g = p->g;
   ConvArgs a = p->args;
@@ -863,9 +886,17 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
     CUDA_TRY(cudaMemsetAsync(a.acc, 0, (size_t)g.y_elems * 4, st));
   }
 
-  if (a.pair)
+  if (a.pair) {
+    a.pk_on = fused_pack ? 1 : 0;
+    if (fused_pack) {
+      // the kernel's pack warps rewrite x into the start of the workspace; its counters start at zero
+      a.pk_src = x;
+      a.pk_dst = reinterpret_cast<int8_t*>(wsb);
+      a.pk_ctl = reinterpret_cast<int*>(wsb + p->ws_ctl_offset);
+      CUDA_TRY(cudaMemsetAsync(a.pk_ctl, 0, (size_t)(d.N + 1) * sizeof(int), st));
+    }
     CUDA_TRY(launch_conv_mma_pair(p->amode, &tmap_a, &p->tmap_b, a, st));
-  else
+  } else
     CUDA_TRY(launch_conv_mma(p->amode, &tmap_a, &p->tmap_b, a, st));
   if (need_finish)
     CUDA_TRY(launch_splitk_finish(a.acc, y32, y8, g.y_elems, d.shift, d.out_mode, p->bias, p->relu, d.K, g.PQ,
@@ -899,6 +930,7 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
     }
     return B2C_OK;
   }
+  if (p->fused_pack && aligned16(x)) return run_convolve(p, x, y32, y8, ws, st, /*fused_pack=*/true);
   rc = run_rewrite(p, x, ws, st);
   if (rc != B2C_OK) return rc;
   return run_convolve(p, x, y32, y8, ws, st);

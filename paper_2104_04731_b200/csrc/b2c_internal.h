@@ -125,6 +125,15 @@ struct ConvArgs {
   // Two-SM schedule: a pair of blocks (cluster of two) owns a 256 x tile_n tile; num_tiles counts pair
   // tiles, every block loads its own 128 A rows and tile_n / 2 B rows per stage.
   int pair;
+  // Activation pack fused into the two-SM kernel (NCHW input, channel-pack map): four extra warps of
+  // every block rewrite the input into the NHWC scratch tensor that the kernel's own TMA loads read,
+  // in batches of pk_ct channels x pk_pt pixels of one image (units of 16 channels), taken from a
+  // global work counter in image order; pk_ctl[0] is that counter, pk_ctl[1 + n] counts the finished
+  // units of image n, and a tile's loads start once all units of its images are done.
+  const int8_t* pk_src;
+  int8_t* pk_dst;
+  int* pk_ctl;
+  int pk_on, pk_N, pk_C, pk_HW, pk_Cpad, pk_ct, pk_pt, pk_hw_tiles, pk_ctiles, pk_smem;
   FastDiv div_wps, div_hp;
   // elements between consecutive images of the NKPQ output (K * P * Q, or more when this
   // convolution writes one channel group of a wider tensor)
@@ -331,6 +340,8 @@ size_t conv_mma_smem_bytes(int amode, const ConvArgs& args);
 cudaError_t launch_conv_mma_pair(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,
                                  cudaStream_t st);
 size_t conv_mma_pair_smem_bytes(const ConvArgs& args);
+// Geometry of the fused activation pack; false when the tensor has no bulk-copy form.
+bool fused_pack_geometry(int C, int H, int W, int C_pad, int* ct, int* pt, int* hw_tiles, int* ctiles, int* smem);
 cudaError_t launch_bounded_wait_selftest(int* status, cudaStream_t st);
 cudaError_t launch_pack_wait_selftest(int* status, cudaStream_t st);
 

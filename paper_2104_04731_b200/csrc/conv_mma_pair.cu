@@ -135,15 +135,173 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar, uint32_t on) {
       : "memory");
 }
 
+constexpr int kPackWarps = 4;  // warps 10..13 of the fused form: activation pack
+constexpr int kPackGroup = 32 * kPackWarps;
+
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Pack role (Table 2: Pad, Split, Reorder of the activations, here inside the convolution kernel so
+// that the memory-bound rewrite runs beside the tensor-bound main loop).  Each of the four warps is
+// a pipeline of its own with one shared-memory buffer.  A warp takes a batch from the global
+// counter (one atomic per batch, issued one batch ahead): pk_ct channels x pk_pt pixels of one
+// image, i.e. up to four units of 16 channels.  The batch's channel rows arrive by bulk async copies
+// (one copy when the batch is contiguous in NCHW); every lane transposes 16 channels x 4 pixels in
+// registers and stores 16-byte pieces of the NHWC tensor.  When all lanes have read the buffer the
+// next batch's copies are started, and only then does the warp fence its stores and bump the
+// image's counter by the number of units: fence and copy latency overlap, and the other three
+// warps hide what is left.
+__device__ __forceinline__ void fused_pack_role(const ConvArgs& args, uint8_t* buf0, unsigned long long* bars,
+                                                SharedCtl* ctl, int pw, int lane) {
+  const int C = args.pk_C, HW = args.pk_HW, C_pad = args.pk_Cpad, PT = args.pk_pt, CT = args.pk_ct;
+  const int hw_tiles = args.pk_hw_tiles;
+  const int cgroups = args.pk_ctiles;                       // batches along the channel axis
+  const int bpi = hw_tiles * cgroups;                       // batches per image
+  const int total = args.pk_N * bpi;
+  const bool row_mode = hw_tiles > 1;
+  const int rp = row_mode ? PT : HW;                        // row pitch in shared memory
+  uint8_t* my_buf = buf0 + pw * (args.pk_smem / kPackWarps);
+  const uint32_t my_buf_a = smem_u32(my_buf);
+  const uint32_t bar = smem_u32(&bars[pw]);
+  uint32_t parity = 0u;
+
+  // starts the copies of a batch: channels [c0, min(c0 + CT, C)) x pixels [hw0, hw0 + npx) of image n
+  auto start_batch = [&](int n, int c0, int hw0, int npx) {
+    const int rows = max(0, min(CT, C - c0));
+    if (rows == 0) return;
+    if (lane == 0)
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)(rows * npx)) : "memory");
+    __syncwarp();
+    const int8_t* xin = args.pk_src + ((size_t)n * C + c0) * HW + hw0;
+    if (row_mode) {
+      for (int r = lane; r < rows; r += 32)
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                         my_buf_a + (uint32_t)(r * rp)),
+                     "l"(xin + (size_t)r * HW), "r"((uint32_t)npx), "r"(bar)
+                     : "memory");
+    } else if (lane == 0) {
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(my_buf_a),
+                   "l"(xin), "r"((uint32_t)(rows * HW)), "r"(bar)
+                   : "memory");
+    }
+  };
+  auto decode = [&](int batch, int* n, int* c0, int* hw0, int* npx) {
+    *n = batch / bpi;
+    const int rem = batch - *n * bpi;
+    const int hwt = rem / cgroups;
+    *c0 = (rem - hwt * cgroups) * CT;
+    *hw0 = hwt * PT;
+    *npx = min(PT, HW - *hw0);
+  };
+
+  int batch = 0, batch_next = 0;
+  if (lane == 0) batch = atomicAdd(args.pk_ctl, 1);
+  batch = __shfl_sync(0xffffffffu, batch, 0);
+  if (batch < total) {
+    int n, c0, hw0, npx;
+    decode(batch, &n, &c0, &hw0, &npx);
+    start_batch(n, c0, hw0, npx);
+  }
+  while (batch < total) {
+    if (lane == 0) batch_next = atomicAdd(args.pk_ctl, 1);  // used after this batch: its latency is hidden
+    int n, cg0, hw0, npx;
+    decode(batch, &n, &cg0, &hw0, &npx);
+    const int units = min(CT, C_pad - cg0) >> 4;
+    if (cg0 < C) {
+      if (!__all_sync(0xffffffffu, mbar_wait(bar, parity, ctl, args.status))) break;
+      parity ^= 1u;
+    }
+    // item = (group of 4 pixels, unit): the lanes of consecutive units of one pixel write consecutive
+    // 16-byte pieces, so a pixel's 64 bytes of this batch leave the SM as whole sectors
+    const int items = ((npx + 3) >> 2) * units;
+    for (int it = lane; it < items; it += 32) {
+      const int pg = it / units, k = it - pg * units;
+      const int c0 = cg0 + 16 * k;
+      uint32_t w[16];
+      if (c0 < C) {
+        const uint8_t* tile = my_buf + (16 * k) * rp + pg * 4;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) w[i] = *reinterpret_cast<const uint32_t*>(tile + i * rp);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) w[i] = 0;  // channels past C: the zero padding of the channel axis
+      }
+      int8_t* dst = args.pk_dst + ((size_t)n * HW + hw0 + pg * 4) * C_pad + c0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (pg * 4 + j < npx) {
+          uint32_t o[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t lo = __byte_perm(w[4 * q], w[4 * q + 1], j | ((4 + j) << 4));
+            const uint32_t hi = __byte_perm(w[4 * q + 2], w[4 * q + 3], j | ((4 + j) << 4));
+            o[q] = __byte_perm(lo, hi, 0x5410);
+          }
+          *reinterpret_cast<uint4*>(dst + (size_t)j * C_pad) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+      }
+    }
+    __syncwarp();  // every lane has read the buffer: the next batch's copies may land in it
+    batch_next = __shfl_sync(0xffffffffu, batch_next, 0);
+    if (batch_next < total) {
+      int n2, c2, h2, p2;
+      decode(batch_next, &n2, &c2, &h2, &p2);
+      start_batch(n2, c2, h2, p2);
+    }
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) atomicAdd(args.pk_ctl + 1 + n, units);
+    batch = batch_next;
+  }
+}
+
+// Producer side of the fused pack: the images a tile reads (rows m_first .. m_first + 127 of the fused
+// pixel axis) must be complete before its loads are issued.  Lanes poll different images; the
+// generic-proxy writes of the pack warps (any SM) are then ordered before this thread's TMA loads.
+__device__ __forceinline__ bool wait_images_packed(const ConvArgs& args, int m_first, int lane, SharedCtl* ctl) {
+  bool ok = true;
+  if (m_first < args.Mg) {
+    const int upi = args.pk_hw_tiles * (args.pk_Cpad >> 4);  // units of one image
+    const int n_a = (int)args.div_pq.div((uint32_t)m_first);
+    const int n_b = (int)args.div_pq.div((uint32_t)min(m_first + kTileM - 1, args.Mg - 1));
+    for (int n = n_a + lane; n <= n_b && ok; n += 32) {
+      const int* cnt = args.pk_ctl + 1 + n;
+      if (ld_acquire_gpu(cnt) >= upi) continue;
+      const unsigned long long t0 = global_ns();
+      while (ld_acquire_gpu(cnt) < upi) {
+        if (ctl->abort_flag) {
+          ok = false;
+          break;
+        }
+        if (global_ns() - t0 > kWaitLimitNs) {
+          ctl->abort_flag = 1;
+          atomicExch(args.status, B2C_E_TIMEOUT);
+          ok = false;
+          break;
+        }
+        __nanosleep(200);
+      }
+    }
+  }
+  ok = __all_sync(0xffffffffu, ok);
+  asm volatile("fence.proxy.async.global;" ::: "memory");
+  return ok;
+}
+
 // PERSIST: 0 = one pair tile per cluster, two blocks resident per SM (one 256-column accumulator each,
 // stage ring within half of the shared memory); 1 = 74 clusters walk the tile list, one block per SM,
 // two accumulator buffers, the deepest stage ring that fits.
-template <int AMODE, int PERSIST>
-__global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
+// PACK: the block has four more warps that run the activation pack (persistent channel-pack map only).
+template <int AMODE, int PERSIST, bool PACK>
+__global__ void __launch_bounds__(PACK ? kThreads + kPackGroup : kThreads, PERSIST == 1 ? 1 : 2)
     conv_mma_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                          const ConvArgs args) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ SharedCtl ctl;
+  __shared__ __align__(8) unsigned long long pack_bars[kPackWarps];
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
@@ -180,6 +338,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
     }
     if (lane == 9) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
     if (lane == 10) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+    if (PACK && lane >= 16 && lane < 16 + kPackWarps) mbar_init(smem_u32(&pack_bars[lane - 16]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -221,6 +380,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
         h_org = p * args.stride_h - args.pad_h;
         w_org = q * args.stride_w - args.pad_w;
       }
+      if (PACK && !wait_images_packed(args, m0, lane, &ctl)) break;
       int kcol = 0;
       const int wrow0 = n0 + (int)rank * half_n;  // first output channel of this block's B half
       for (int kb = 0; kb < args.num_kb; ++kb) {
@@ -303,6 +463,10 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
       }
     }
     __syncwarp();
+  } else if (PACK && warp >= 2 + kGatherWarps) {
+    // ---------------------------------------------------------------- activation pack (both blocks)
+    uint8_t* pack_buf = smem_raw + (smem_base - smem_u32(smem_raw)) + args.stage_region;
+    fused_pack_role(args, pack_buf, pack_bars, &ctl, warp - (2 + kGatherWarps), lane);
   } else {
     // ---------------------------------------------------------------- epilogue warps (both blocks)
     const int quad = warp & 3;         // TMEM lane quadrant this warp may read
@@ -384,7 +548,21 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 2)
 
 }  // namespace
 
-size_t conv_mma_pair_smem_bytes(const ConvArgs& a) { return 1024 + (size_t)a.stage_region; }
+size_t conv_mma_pair_smem_bytes(const ConvArgs& a) { return 1024 + (size_t)a.stage_region + (a.pk_on ? (size_t)a.pk_smem : 0); }
+
+bool fused_pack_geometry(int C, int H, int W, int C_pad, int* ct, int* pt, int* hw_tiles, int* ctiles, int* smem) {
+  const int HW = H * W;
+  // channels in whole groups of 16 and either the whole image per unit (a multiple of 4 pixels, at most
+  // 256) or pixel rows that are multiples of 16 bytes (units of 256 pixels)
+  if ((C % 16) != 0 || (HW % 4) != 0 || !(HW <= 256 || (HW % 16) == 0)) return false;
+  *pt = HW <= 256 ? HW : 128;
+  *hw_tiles = (HW + *pt - 1) / *pt;
+  *ct = 64;  // channels per batch (four units of 16)
+  *ctiles = (C_pad + *ct - 1) / *ct;
+  // one batch buffer per pack warp
+  *smem = 4 * ((*ct * *pt + 127) / 128 * 128);
+  return true;
+}
 
 cudaError_t launch_conv_mma_pair(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,
                                  cudaStream_t st) {
@@ -392,14 +570,14 @@ cudaError_t launch_conv_mma_pair(int amode, const CUtensorMap* tmap_a, const CUt
   int pairs = args.persistent ? std::min(args.num_tiles, kNumSMs / 2) : args.num_tiles;
   dim3 grid((unsigned)(2 * pairs), 1, 1);
   cudaError_t e;
-#define B2C_LAUNCH_PAIR(MODE, PERS)                                                                            \
+#define B2C_LAUNCH_PAIR(MODE, PERS, PACK)                                                                      \
   {                                                                                                           \
     static std::atomic<unsigned long long> configured{0};                                                     \
-    e = set_max_dynamic_smem_once(configured, (const void*)conv_mma_pair_kernel<MODE, PERS>, 200 * 1024);      \
+    e = set_max_dynamic_smem_once(configured, (const void*)conv_mma_pair_kernel<MODE, PERS, PACK>, 226 * 1024); \
     if (e != cudaSuccess) return e;                                                                           \
     cudaLaunchConfig_t cfg = {};                                                                              \
     cfg.gridDim = grid;                                                                                       \
-    cfg.blockDim = dim3(kThreads);                                                                            \
+    cfg.blockDim = dim3(PACK ? kThreads + kPackGroup : kThreads);                                             \
     cfg.dynamicSmemBytes = smem;                                                                              \
     cfg.stream = st;                                                                                          \
     cudaLaunchAttribute attr[2];                                                                              \
@@ -414,20 +592,21 @@ cudaError_t launch_conv_mma_pair(int amode, const CUtensorMap* tmap_a, const CUt
     if (PERS) {                                                                                               \
       /* a persistent grid is one wave: as many pairs as the device keeps resident at once */                 \
       int resident = 0;                                                                                       \
-      if (cudaOccupancyMaxActiveClusters(&resident, conv_mma_pair_kernel<MODE, PERS>, &cfg) == cudaSuccess && \
+      if (cudaOccupancyMaxActiveClusters(&resident, conv_mma_pair_kernel<MODE, PERS, PACK>, &cfg) == cudaSuccess && \
           resident > 0 && resident < pairs) {                                                                 \
         pairs = resident;                                                                                     \
         cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);                                                      \
       }                                                                                                       \
       (void)cudaGetLastError();                                                                               \
     }                                                                                                         \
-    e = cudaLaunchKernelEx(&cfg, conv_mma_pair_kernel<MODE, PERS>, *tmap_a, *tmap_b, args);                    \
+    e = cudaLaunchKernelEx(&cfg, conv_mma_pair_kernel<MODE, PERS, PACK>, *tmap_a, *tmap_b, args);                    \
     if (e != cudaSuccess) return e;                                                                           \
   }
-  if (amode == A_TILED && args.persistent) B2C_LAUNCH_PAIR(A_TILED, 1)
-  else if (amode == A_TILED) B2C_LAUNCH_PAIR(A_TILED, 0)
-  else if (amode == A_IM2COL_TMA && args.persistent) B2C_LAUNCH_PAIR(A_IM2COL_TMA, 1)
-  else if (amode == A_IM2COL_TMA) B2C_LAUNCH_PAIR(A_IM2COL_TMA, 0)
+  if (amode == A_TILED && args.persistent) B2C_LAUNCH_PAIR(A_TILED, 1, false)
+  else if (amode == A_TILED) B2C_LAUNCH_PAIR(A_TILED, 0, false)
+  else if (amode == A_IM2COL_TMA && args.persistent && args.pk_on) B2C_LAUNCH_PAIR(A_IM2COL_TMA, 1, true)
+  else if (amode == A_IM2COL_TMA && args.persistent) B2C_LAUNCH_PAIR(A_IM2COL_TMA, 1, false)
+  else if (amode == A_IM2COL_TMA) B2C_LAUNCH_PAIR(A_IM2COL_TMA, 0, false)
   else return cudaErrorInvalidValue;
 #undef B2C_LAUNCH_PAIR
   return cudaGetLastError();

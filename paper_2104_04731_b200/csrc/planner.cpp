@@ -342,6 +342,10 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
   e.o_mac = M_pad * N_pad * k_issued - mac_min;
   e.o_data = moved - data_min;
   e.workspace_bytes = (int64_t)workspace_bytes_for(g, variant, tile_n, split_k, swap);
+  // two-SM channel-pack schedule on NCHW input: room for the work counters of the pack that runs
+  // inside the MMA kernel (1 + N integers after the rewritten operand)
+  if (tile_m == 2 * kTileM && variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NCHW)
+    e.workspace_bytes = (e.workspace_bytes + 255) / 256 * 256 + ((int64_t)(d.N + 1) * 4 + 255) / 256 * 256;
   out->push_back(e);
 }
 

@@ -629,6 +629,53 @@ def test_two_sm_schedule_walks_tiles(lib, in_layout, tile_n):
         check_against_oracle(x, w, 2, 1, 1, 10, 3, ids[0], ref=ref, in_layout=in_layout)
 
 
+# ---- activation pack inside the two-SM kernel (NCHW input, persistent channel-pack schedule) -------------
+@pytest.mark.parametrize("case", [
+    # N, C, H, W, K, R, S, stride, pad, shift, tile_n
+    (100, 16, 14, 14, 64, 3, 3, 1, 1, 8, 64),     # whole image per unit, channels padded 16 -> 32
+    (8, 64, 56, 56, 64, 3, 3, 1, 1, 9, 64),       # units of 256 pixels (rows of 3136 pixels), ragged last unit
+    (60, 48, 20, 20, 96, 3, 3, 1, 1, 9, 32),      # 48 channels in 64-channel units: the last 16 are zero padding
+    (450, 32, 7, 9, 40, 2, 2, 1, 0, 7, 64),       # HW = 63 is no multiple of 4: falls back to the separate pack kernel
+])
+def test_fused_activation_pack(lib, case):
+    N, C, H, W, K, R, S, stride, pad, shift, tile_n = case
+    x = int8_uniform((N, C, H, W), 751)
+    w = int8_uniform((K, C, R, S), 752)
+    bias = (int8_uniform((K,), 753).astype(np.int32) * 1000)
+    ref = oracle.conv2d_int8(x, w, stride, pad, 1, shift, bias=bias, relu=True)
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, 1, shift, 0, 0, 3)
+    ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == 0 and e.tile_m == 256 and e.tile_n == tile_n]
+    assert ids
+    plan = lib.Plan(d, ids[0])
+    plan.set_weights(to_dev(w))
+    plan.set_activation(to_dev(bias), True)
+    y32 = torch.full(ref[0].shape, -7777777, dtype=torch.int32, device="cuda")
+    y8 = torch.full(ref[1].shape, 77, dtype=torch.int8, device="cuda")
+    ws = torch.empty(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xAB)
+    xd = to_dev(x)
+    for _ in range(2):   # twice: the counters in the workspace are cleared by every run
+        plan.run(xd, y32, y8, ws)
+    torch.cuda.synchronize()
+    assert plan.device_status() == b2c.OK
+    assert np.array_equal(y32.cpu().numpy(), ref[0]) and np.array_equal(y8.cpu().numpy(), ref[1])
+    # the rewritten operand the kernel left in the workspace is the oracle's NHWC, channel-padded tensor
+    C_pad = -(-C // 32) * 32
+    want = oracle.pack_nhwc_cpad(x, C_pad)
+    got = ws[:want.size].cpu().numpy().view(np.int8).reshape(want.shape)
+    assert np.array_equal(got, want)
+    g = torch.cuda.CUDAGraph()   # and once more from a captured graph, replayed twice
+    y32.fill_(-1)
+    with torch.cuda.graph(g):
+        plan.run(xd, y32, y8, ws)
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    assert plan.device_status() == b2c.OK
+    assert np.array_equal(y32.cpu().numpy(), ref[0]) and np.array_equal(y8.cpu().numpy(), ref[1])
+    plan.destroy()
+
+
 # ---- one-shot calls of one shape on two streams with different weights do not disturb each other ---------
 def test_one_shot_calls_on_two_streams(lib):
     N, C, H, W, K, R, S = 2, 32, 20, 20, 48, 3, 3
@@ -698,6 +745,17 @@ def test_failed_descriptor_encode_is_reported_and_skipped(lib):
     torch.cuda.synchronize()
     assert np.array_equal(y32.cpu().numpy(), ref[0]) and np.array_equal(y8.cpu().numpy(), ref[1])
     plan.destroy()
+
+
+# ---- issue-rate measurement of the intrinsic ------------------------------------------------------------
+def test_mma_rate_measurement_is_plausible(lib):
+    us, cyc = lib.measure_mma_rate(256, 4000)
+    # a 128 x 256 x 32 int8 MMA cannot take fewer cycles than 8192 MACs per clock per SM would allow
+    assert 100.0 < cyc < 400.0 and us > 0
+    us16, cyc16 = lib.measure_mma_rate(16, 4000)
+    assert cyc16 < cyc
+    with pytest.raises(b2c.B2CError):
+        lib.measure_mma_rate(48, 4000)
 
 
 # ---- failure detection: a wait that cannot complete ends by itself and is reported --------------------
