@@ -230,6 +230,9 @@ def max_over_ranks(torch, dist, value: float, device) -> float:
     return float(t.item())
 
 
+LAST_STEP_MS = []  # per-step device times of the most recent time_steps call (this rank)
+
+
 def time_steps(torch, fn, steps, warmup, dist=None, min_warm_s=0.2):
     for _ in range(warmup):
         fn()
@@ -242,13 +245,14 @@ def time_steps(torch, fn, steps, warmup, dist=None, min_warm_s=0.2):
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record()
+    for i in range(steps):
         fn()
-    e1.record()
+        ev[i + 1].record()
     torch.cuda.synchronize()
-    ms = max_over_ranks(torch, dist, e0.elapsed_time(e1), "cuda")
+    LAST_STEP_MS[:] = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+    ms = max_over_ranks(torch, dist, ev[0].elapsed_time(ev[steps]), "cuda")
     if dist is not None:
         dist.barrier()
     return ms
@@ -271,6 +275,7 @@ def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, grap
     inst.check_status(b2c)
     verified = inst.verify()
     per_call_us = ms * 1e3 / (steps * G)
+    st_sorted = sorted(LAST_STEP_MS)
     emb = inst.emb.as_dict()
     launches = inst.launches_per_instance
     inst.destroy()
@@ -286,6 +291,7 @@ def measure_shape(b2c, torch, cfg, steps, warmup, peaks, policy, dist=None, grap
     keys = ("id", "variant_name", "map_m", "tile_m", "tile_n", "split_k", "workspace_bytes", "o_mac", "o_data", "device_us")
     res = {
         "shape": cfg.name, "instances": G, "warm_us": ms_w * 1e3 / (10 * 20),
+        "combined_us_median": st_sorted[len(st_sorted) // 2] * 1e3 / G, "combined_us_min": st_sorted[0] * 1e3 / G,
         "op_us": op["us"] if op else None, "transf_us": max(0.0, per_call_us - op["us"]) if op else None, "cold": bool(G * cfg.algorithmic_bytes >= L2_BYTES), "combined_us": per_call_us, "tops": 2.0 * cfg.macs / (per_call_us * 1e-6) / 1e12,
         "roofline_us": t_roof, "bound": bound, "roofline_frac": t_roof / per_call_us,
         "embedding": {k: emb[k] for k in keys},
@@ -334,12 +340,25 @@ def measure_scaled(b2c, torch, cfg, peaks, steps=10):
         ws = torch.empty(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
         plan.set_weights(w)
         ms = time_steps(torch, lambda: plan.run(x, y32, y8, ws), steps, 3, None, 0.05)
+        per = sorted(LAST_STEP_MS)
+        # the two halves on their own (the paper's Transf. and Op. columns), and the layout kernel's achieved
+        # bandwidth on the bytes it reads and writes
+        data_b, _ = plan.footprint()
+        halves = {}
+        if data_b:
+            ms_t = time_steps(torch, lambda: plan.rewrite_activations(x, ws), steps, 3, None, 0.0)
+            ms_o = time_steps(torch, lambda: plan.run_rewritten(x, y32, y8, ws), steps, 3, None, 0.0)
+            moved = x.numel() + data_b
+            halves = {"transf_us": ms_t * 1e3 / steps, "op_us": ms_o * 1e3 / steps, "transf_bytes": moved,
+                      "transf_gbs": moved / (ms_t * 1e-3 / steps) / 1e9,
+                      "transf_frac_of_copy_bandwidth": moved / (ms_t * 1e-3 / steps) / 1e9 / peaks["hbm_gbs"]}
         st = plan.device_status()
         plan.destroy()
         if st != 0:
             raise RuntimeError("device status " + b2c.status_string(st))
         us = ms * 1e3 / steps
-        return {"us": us, "tops": 2.0 * big.macs / (us * 1e-6) / 1e12, "roofline_frac": t_roof / us,
+        return {"us": us, "us_median": per[len(per) // 2] * 1e3, "us_min": per[0] * 1e3, **halves,
+                "tops": 2.0 * big.macs / (us * 1e-6) / 1e12, "roofline_frac": t_roof / us,
                 "embedding": {"variant": b2c.VARIANT_NAMES[emb.variant], "tile_m": emb.tile_m, "tile_n": emb.tile_n,
                               "split_k": emb.split_k, "swapped": emb.map_m == b2c.AXIS_K}}
 
@@ -652,12 +671,14 @@ def run_ours(args):
         inst.capture(torch, streams=args.streams)
     ms = time_steps(torch, inst.step, args.steps, args.warmup, dist, args.min_warm_s)
     inst.check_status(b2c)
+    step_ms = sorted(LAST_STEP_MS)
     clocks = sampler.stop() if rank == 0 else None
     # the timed graph did the work: first and last instance of the last step against the oracle
     verified = inst.verify() if rank == 0 else None
     if verified is False:
         raise SystemExit("bench: the timed graph's output differs from the oracle")
     emb = inst.emb
+    inst_launches = inst.launches_per_instance
     launches = inst.launches_per_instance * G * args.steps
     ops = 2.0 * cfg.macs
     value = shard_report(world, G, ops, args.steps, ms)
@@ -671,6 +692,19 @@ def run_ours(args):
                      emb.map_m, emb.tile_m)
     t_roof, bound = roofline_time_us(cfg, peaks)
     op_us = op["us"] if op else per_call_us
+    op_steps = sorted(LAST_STEP_MS) if op else step_ms
+    # the same kernel with one launch in flight (one call after the other on one stream)
+    alone = None
+    if op and graph and args.streams > 1 and rank == 0:
+        alone = op_only(b2c, torch, cfg, emb.variant, emb.tile_n, emb.split_k, max(2, args.steps // 2), 3, graph, 1, emb.map_m,
+                        emb.tile_m)
+    # second denominator: this library's own issue-rate measurement of the intrinsic (no loads, all SMs)
+    issue = None
+    if rank == 0:
+        r_us, r_cyc = b2c.measure_mma_rate(256, 20000)
+        mma_ops = 2.0 * 128 * 256 * 32
+        issue = {"tile": "128x256x32", "mmas_per_sm": 20000, "device_us": r_us, "cycles_per_mma": r_cyc,
+                 "tops": 148 * 20000 * mma_ops / (r_us * 1e-6) / 1e12, "ops_per_clock_all_sms": 148 * mma_ops / r_cyc}
     if bound == "tensor":
         achieved, peak, runit = ops / (op_us * 1e-6) / 1e12, peaks["bf16_tflops"] * INT8_TO_BF16_RATIO, "TFLOP/s"
     else:
@@ -678,11 +712,25 @@ def run_ours(args):
     sha = hashlib.sha1(b"".join(open(os.path.join(ROOT, "paper_2104_04731_b200", "csrc", f), "rb").read()
                                 for f in KERNEL_SOURCES)).hexdigest()
     traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["conv_mma_sha1"] == sha else None
+    kname = "conv_mma_pair_kernel" if emb.tile_m == 256 else "conv_mma_kernel"
+    launches_per_step = (op["launches_per_call"] if op else inst_launches) * G
     roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
-                "traffic": traffic, "kernel": "conv_mma_kernel", "kernel_us": op_us,
+                "traffic": traffic, "kernel": kname, "kernel_us": op_us,
+                "kernel_us_median": op_steps[len(op_steps) // 2] * 1e3 / G, "kernel_us_min": op_steps[0] * 1e3 / G,
                 "kernel_us_note": "timed region / launches, %d launches in flight" % (args.streams if graph else 1),
+                "kernel_us_alone": alone["us"] if alone else None,
+                "frac_alone": (ops / (alone["us"] * 1e-6) / 1e12 / peak) if (alone and bound == "tensor") else None,
                 "peak_source": "%s bf16 burst x %.0f (nominal int8:bf16)" % (peaks["source"], INT8_TO_BF16_RATIO)
                 if bound == "tensor" else peaks["source"] + " copy bandwidth"}
+    if issue is not None and bound == "tensor":
+        # both denominators, and the fraction that does not depend on the clock the peaks were taken at:
+        # ops per SM clock of the timed kernel (time x median SM clock sampled during the run) against the
+        # ops per clock the intrinsic issues at
+        roofline["peak_i8_issue_rate"] = issue
+        roofline["frac_vs_issue_rate"] = achieved / issue["tops"]
+        roofline["frac_vs_larger_peak"] = achieved / max(peak, issue["tops"])
+        if clocks and clocks.get("sm_mhz"):
+            roofline["frac_clock_normalised"] = (ops / (op_us * 1e-6) / (clocks["sm_mhz"] * 1e6)) / issue["ops_per_clock_all_sms"]
 
     # ---- end to end through the host-buffer call ----------------------------------------------------
     e2e = None
@@ -723,6 +771,7 @@ def run_ours(args):
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "s8 x s8 -> s32", "data": "synthetic",
         "config": {"workload": cfg.name, "instances_per_step": G, "per_call_us": per_call_us,
+                   "per_call_us_median": step_ms[len(step_ms) // 2] * 1e3 / G, "per_call_us_min": step_ms[0] * 1e3 / G,
                    "l2": "inputs larger than L2: %d distinct buffer sets per step (%.0f MB)" % (G, G * (cfg.algorithmic_bytes) / 1e6),
                    "cuda_graph": graph, "streams": args.streams if graph else 1,
                    "parallelism": "independent instances sharded over ranks, no collective",

@@ -87,6 +87,12 @@ typedef struct {
                                       * stride phases (scratch [N][P + R' - 1][Q][(dh, s, c)], R' = ceil(R / stride_h)); what remains
                                       * is an R' x 1 stride-1 convolution, executed as operand shifts over 8 x 16-pixel tiles */
 
+#define B2C_VARIANT_IM2COL_WINDOW 10  /* low-channel shapes: stencil unroll formed in shared memory from a two-dimensional input
+                                      * window that one tiled TMA copy of the NCHW tensor stages per tile of tile_h x tile_w output
+                                      * pixels (zeros outside the image); builder warps write the swizzled A rows word by word,
+                                      * separate epilogue warps drain the accumulators; weights resident; needs NCHW input with
+                                      * rows that are multiples of 16 bytes and unit horizontal dilation */
+
 typedef struct {
   int32_t id;       /* index in the enumeration for this descriptor; pass to b2c_plan_create      */
   int32_t map_m, map_n, map_k; /* B2C_AXIS_*                                                      */

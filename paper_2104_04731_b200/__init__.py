@@ -20,11 +20,11 @@ OUT_I32, OUT_I8 = 1, 2
 AXIS_NPQ, AXIS_K, AXIS_C, AXIS_CRS, AXIS_SC, AXIS_C_PHASES = 1, 2, 3, 4, 5, 6
 VARIANT_CP_TMA, VARIANT_IM2COL_EXPLICIT, VARIANT_IM2COL_GATHER, VARIANT_IM2COL_STAGED = 0, 1, 2, 3
 VARIANT_ROW_UNROLL, VARIANT_SPACE_TO_DEPTH, VARIANT_DILATION_PACK = 4, 5, 6
-VARIANT_CP_SHIFT, VARIANT_S2D_SHIFT, VARIANT_ROWPHASE_SHIFT = 7, 8, 9
+VARIANT_CP_SHIFT, VARIANT_S2D_SHIFT, VARIANT_ROWPHASE_SHIFT, VARIANT_IM2COL_WINDOW = 7, 8, 9, 10
 POLICY_AUTO_TIMED, POLICY_MIN_OVERHEAD, POLICY_MIN_WORKSPACE, POLICY_AUTO_TIMED_CONCURRENT = -1, -2, -3, -4
 VARIANT_NAMES = {0: "channel_pack_tma_im2col", 1: "im2col_explicit", 2: "im2col_gather", 3: "im2col_staged_window",
                  4: "row_unroll_tma", 5: "space_to_depth_tma", 6: "dilation_phase_pack_tma",
-                 7: "channel_pack_shift", 8: "space_to_depth_shift", 9: "row_phase_unroll_shift"}
+                 7: "channel_pack_shift", 8: "space_to_depth_shift", 9: "row_phase_unroll_shift", 10: "im2col_tma_window"}
 
 EXPORTS = [
     "b2c_out_shape", "b2c_enumerate", "b2c_plan_create", "b2c_plan_info", "b2c_plan_workspace_bytes",

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "libb2conv.so")
-SOURCES = ["api.cpp", "planner.cpp", "tma.cpp", "layout.cu", "conv_mma.cu", "conv_mma_pair.cu", "mma_rate.cu"]
+SOURCES = ["api.cpp", "planner.cpp", "tma.cpp", "layout.cu", "conv_mma.cu", "conv_mma_pair.cu", "mma_rate.cu", "conv_mma_window.cu"]
 
 
 def _nvcc() -> str:

@@ -239,6 +239,40 @@ void fill_common_args(b2c_plan* p) {
       a.out_pad_h = d.pad_h;
       a.out_pad_w = d.pad_w;
     }
+  } else if (p->emb.variant == B2C_VARIANT_IM2COL_WINDOW) {
+    WindowTile wt;
+    window_tile_geom(p->g, &wt);  // legal: checked when the plan was created
+    p->amode = A_WINDOW;
+    p->K_pad = wt.K_pad;
+    p->bk = 128;
+    a.bk = 128;
+    a.num_kb = wt.num_kb;
+    a.ksteps_full = 4;
+    a.ksteps_last = (wt.K_pad - (wt.num_kb - 1) * 128) / kMmaK;
+    a.Mg = (int)wt.mtot;
+    a.wn_tile_w = wt.tile_w;
+    a.wn_win_w = wt.win_w;
+    a.wn_win_bytes = wt.win_bytes;
+    a.wn_box_bytes = wt.box_bytes;
+    a.wn_left = wt.left;
+    a.wn_off0 = wt.off0;
+    a.wn_chunks = wt.K_pad / 16;
+    a.sh_tiles_h = wt.tiles_h;
+    a.sh_tiles_w = wt.tiles_w;
+    a.div_tiles_hw = make_fastdiv((uint32_t)(wt.tiles_h * wt.tiles_w));
+    a.div_tiles_w = make_fastdiv((uint32_t)wt.tiles_w);
+    a.num_tiles = (int)((long long)d.N * wt.tiles_h * wt.tiles_w);
+    a.tiles_n = 1;
+    a.persistent = 2;
+    a.split_k = 1;
+    a.cluster_split = 0;
+    // accumulator ring: four buffers while two resident blocks' rings fit the 512 columns of tensor memory
+    const int per_sm = wt.smem * 2 + 4096 <= 227 * 1024 ? 2 : 1;
+    a.tmem_bufs = 4 * a.tmem_cols * per_sm <= 512 ? 4 : (2 * a.tmem_cols * per_sm <= 512 ? 2 : 1);
+    if (a.tmem_bufs == 1) a.tmem_bufs = 2;  // (tile_n = 256 leaves one block per SM by shared memory: two buffers fit)
+    a.stages = 3;
+    a.stage_region = 0;
+    return;
   } else {
     p->amode = p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT
                    ? A_TILED
@@ -424,6 +458,21 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
     if (cudaMalloc(&p->table, t.size() * sizeof(GatherEntry)) != cudaSuccess) return fail(B2C_E_CUDA);
     if (cudaMemcpy(p->table, t.data(), t.size() * sizeof(GatherEntry), cudaMemcpyHostToDevice) != cudaSuccess)
       return fail(B2C_E_CUDA);
+    if (emb.variant == B2C_VARIANT_IM2COL_WINDOW) {
+      WindowTile wt;
+      if (!window_tile_geom(g, &wt)) return fail(B2C_E_UNSUPPORTED);
+      // one entry per 32-bit word of an A row: byte offset of the word's first tap inside the window
+      // [c][row][byte]; words of the reduction padding point at the window's start (their weights are zero)
+      std::vector<int32_t> t32(K_pad / 4, 0);
+      for (int wi = 0; wi < K_pad / 4; ++wi) {
+        const int run = (wi * 4) / wt.S_run, s0 = (wi * 4) % wt.S_run;
+        if (run < d.C * d.R) t32[wi] = ((run / d.R) * wt.win_h + (run % d.R) * d.dil_h) * wt.win_w + s0;
+      }
+      p->table_len = (int)t32.size();
+      if (cudaMalloc(&p->table32, t32.size() * sizeof(int32_t)) != cudaSuccess) return fail(B2C_E_CUDA);
+      if (cudaMemcpy(p->table32, t32.data(), t32.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess)
+        return fail(B2C_E_CUDA);
+    }
     if (emb.variant == B2C_VARIANT_IM2COL_STAGED) {
       if (!staged_window(g, &p->win)) return fail(B2C_E_UNSUPPORTED);
       // reduction index (c, r, s) -> byte offset from the window position of the pixel's first tap
@@ -793,7 +842,10 @@ static int set_weights_one(b2c_plan* p, const int8_t* w, cudaStream_t st) {
     CUDA_TRY(launch_pack_weights_table(w, p->w_packed, d.K, p->g.Kg, p->view.R * p->view.S * p->view.C, p->wtable, st));
   else
     CUDA_TRY(launch_pack_weights_rows(w, p->w_packed, d.K, p->g.Kg, p->K_pad, d.S,
-                                      p->emb.variant == B2C_VARIANT_IM2COL_STAGED ? staged_run_len(p->g) : d.S, st));
+                                      p->emb.variant == B2C_VARIANT_IM2COL_STAGED
+                                          ? staged_run_len(p->g)
+                                          : (p->emb.variant == B2C_VARIANT_IM2COL_WINDOW ? round_up(d.S, 4) : d.S),
+                                      st));
   p->weights_set = true;
   return B2C_OK;
 }
@@ -869,6 +921,9 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   } else if (p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
     rc = encode_tiled_2d(&tmap_a, wsb, p->K_pad, (uint64_t)g.Mg, p->K_pad, 128, a.swap ? a.tile_n : kTileM, 128);
     if (rc != B2C_OK) return rc;
+  } else if (p->amode == A_WINDOW) {
+    rc = encode_tiled_nchw_window(&tmap_a, x, d.W, d.H, d.C, d.N, a.wn_win_w, a.wn_box_bytes / (d.C * a.wn_win_w));
+    if (rc != B2C_OK) return rc;
   } else {
     tmap_a = p->tmap_b;  // unused by the gather kernel; any valid map
   }
@@ -896,6 +951,8 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
       CUDA_TRY(cudaMemsetAsync(a.pk_ctl, 0, (size_t)(d.N + 1) * sizeof(int), st));
     }
     CUDA_TRY(launch_conv_mma_pair(p->amode, &tmap_a, &p->tmap_b, a, st));
+  } else if (p->amode == A_WINDOW) {
+    CUDA_TRY(launch_conv_mma_window(&tmap_a, &p->tmap_b, a, st));
   } else
     CUDA_TRY(launch_conv_mma(p->amode, &tmap_a, &p->tmap_b, a, st));
   if (need_finish)

@@ -63,7 +63,7 @@ inline FastDiv make_fastdiv(uint32_t d) {
   return f;
 }
 
-enum AMode { A_TILED = 0, A_IM2COL_TMA = 1, A_GATHER = 2, A_STAGED = 3, A_SHIFT = 4 };
+enum AMode { A_TILED = 0, A_IM2COL_TMA = 1, A_GATHER = 2, A_STAGED = 3, A_SHIFT = 4, A_WINDOW = 5 };
 
 // Everything the MMA kernel needs besides its two tensor maps.
 struct ConvArgs {
@@ -134,6 +134,11 @@ struct ConvArgs {
   int8_t* pk_dst;
   int* pk_ctl;
   int pk_on, pk_N, pk_C, pk_HW, pk_Cpad, pk_ct, pk_pt, pk_hw_tiles, pk_ctiles, pk_smem;
+  // Stencil unroll from a TMA-staged two-dimensional window (A_WINDOW): tiles of (128 / wn_tile_w) x
+  // wn_tile_w output pixels (sh_tiles_h x sh_tiles_w tiles per image); the window of a tile is C x win_h
+  // rows of wn_win_w bytes, its first byte wn_left columns left of the tile's first input column
+  // (wn_off0 = wn_left - pad_w bytes before the first tap); wn_chunks 16-byte chunks per A row.
+  int wn_tile_w, wn_win_w, wn_win_bytes, wn_box_bytes, wn_left, wn_off0, wn_chunks;
   FastDiv div_wps, div_hp;
   // elements between consecutive images of the NKPQ output (K * P * Q, or more when this
   // convolution writes one channel group of a wider tensor)
@@ -230,12 +235,13 @@ inline bool shift_tiles_2d(int v) { return v == B2C_VARIANT_ROWPHASE_SHIFT; }
 inline int shift_base_variant(int v) {
   return v == B2C_VARIANT_CP_SHIFT ? B2C_VARIANT_CP_TMA : (v == B2C_VARIANT_S2D_SHIFT ? B2C_VARIANT_SPACE_TO_DEPTH : v);
 }
-constexpr int kNumVariants = 10;
+constexpr int kNumVariants = 11;
 // Family of a variant for the timed selection's "five best candidates": variants that share the
 // kind of rewrite (a view and its shift execution; row unroll with and without the stride phases)
 // count as one candidate with several schedules.
 inline int variant_family(int v) {
   if (v == B2C_VARIANT_ROWPHASE_SHIFT) return B2C_VARIANT_ROW_UNROLL;
+  if (v == B2C_VARIANT_IM2COL_WINDOW) return B2C_VARIANT_IM2COL_STAGED;  // both form the unroll from a staged window
   return shift_base_variant(v);
 }
 // Shared-memory geometry of the shift execution of a view; false if it does not apply (stride,
@@ -298,6 +304,14 @@ bool staged_word_mode(const Geom& g);
 int staged_run_len(const Geom& g);  // taps per (c, r) run after padding
 int variant_k_pad(const Geom& g, int variant);  // padded reduction length of the stencil-unroll variants
 
+// Geometry of the TMA-staged window unroll (B2C_VARIANT_IM2COL_WINDOW); false if it does not apply.
+struct WindowTile {
+  int tile_w, tile_h, win_w, win_h, left, off0, S_run, K_pad, tiles_h, tiles_w, box_bytes, win_bytes, tile_n, num_kb;
+  long long mtot;  // accumulator rows issued: N * tiles_h * tiles_w * 128
+  size_t smem;
+};
+bool window_tile_geom(const Geom& g, WindowTile* wt);
+
 // --- tma.cpp -----------------------------------------------------------------------------------
 // Tensor-map encoders obtained through cudaGetDriverEntryPoint (no link-time libcuda dependency).
 int encode_tiled_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
@@ -307,6 +321,7 @@ int encode_tiled_nhwc_rows(CUtensorMap* map, const void* base, int C_pad, int W,
 int encode_im2col_nhwc(CUtensorMap* map, const void* base, int C_pad, int W, int H, int N, int pad_w, int pad_h,
                        int S, int R, int dil_w, int dil_h, int stride_w, int stride_h, int channels_per_pixel,
                        int pixels_per_column, int swizzle_bytes);
+int encode_tiled_nchw_window(CUtensorMap* map, const void* base, int W, int H, int C, int N, int box_w, int box_h);
 void set_last_cuda_error(int e);
 int get_last_cuda_error();
 
@@ -340,6 +355,8 @@ size_t conv_mma_smem_bytes(int amode, const ConvArgs& args);
 cudaError_t launch_conv_mma_pair(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,
                                  cudaStream_t st);
 size_t conv_mma_pair_smem_bytes(const ConvArgs& args);
+cudaError_t launch_conv_mma_window(const CUtensorMap* tmap_x, const CUtensorMap* tmap_b, const ConvArgs& args, cudaStream_t st);
+size_t conv_mma_window_smem_bytes(const ConvArgs& args);
 // Geometry of the fused activation pack; false when the tensor has no bulk-copy form.
 bool fused_pack_geometry(int C, int H, int W, int C_pad, int* ct, int* pt, int* hw_tiles, int* ctiles, int* smem);
 cudaError_t launch_bounded_wait_selftest(int* status, cudaStream_t st);

@@ -72,6 +72,7 @@ int im2col_k_pad(int Kg) { return round_up(Kg, kMmaK); }
 bool staged_word_mode(const Geom& g) { return g.d.dil_w == 1; }
 int staged_run_len(const Geom& g) { return staged_word_mode(g) ? round_up(g.d.S, 4) : g.d.S; }
 int variant_k_pad(const Geom& g, int variant) {
+  if (variant == B2C_VARIANT_IM2COL_WINDOW) return round_up(g.d.C * g.d.R * round_up(g.d.S, 4), kMmaK);
   if (variant == B2C_VARIANT_IM2COL_STAGED) return round_up(g.d.C * g.d.R * staged_run_len(g), kMmaK);
   return im2col_k_pad(g.Kg);
 }
@@ -295,6 +296,46 @@ bool staged_window(const Geom& g, WindowGeom* w) {
   return true;
 }
 
+bool window_tile_geom(const Geom& g, WindowTile* wt) {
+  const b2c_conv_desc& d = g.d;
+  // the window is one tiled TMA box of the NCHW tensor: rows must be multiples of 16 bytes, every box
+  // extent at most 256; words of an A row are unaligned words of a window row: unit horizontal dilation
+  if (d.in_layout != B2C_LAYOUT_NCHW || (d.W % 16) != 0 || d.dil_w != 1 || d.C > 64 || d.K > 256) return false;
+  wt->S_run = round_up(d.S, 4);
+  wt->K_pad = round_up(d.C * d.R * wt->S_run, kMmaK);
+  if (wt->K_pad > 1024) return false;
+  wt->num_kb = (wt->K_pad + 127) / 128;
+  wt->tile_n = 16;
+  while (wt->tile_n < d.K) wt->tile_n <<= 1;
+  wt->left = round_up(d.pad_w, 16);
+  wt->off0 = wt->left - d.pad_w;
+  long long best_tiles = -1;
+  for (int tw = kTileM; tw >= 16; tw >>= 1) {
+    const int th = kTileM / tw;
+    // last byte a row can touch: the last pixel's last (padded) tap, plus the second word of an unaligned read
+    const long long ww = round_up((int)std::min<long long>((long long)(tw - 1) * d.stride_w + wt->off0 + wt->S_run + 8, 1 << 20), 16);
+    const long long wh = (long long)(th - 1) * d.stride_h + (long long)(d.R - 1) * d.dil_h + 1;
+    if (ww > 256 || wh > 256 || (long long)d.C * wh * ww > 24 * 1024) continue;
+    const long long tiles = (long long)((g.P + th - 1) / th) * ((g.Q + tw - 1) / tw);
+    if (best_tiles < 0 || tiles < best_tiles) {
+      best_tiles = tiles;
+      wt->tile_w = tw;
+      wt->tile_h = th;
+      wt->win_w = (int)ww;
+      wt->win_h = (int)wh;
+    }
+  }
+  if (best_tiles < 0) return false;
+  wt->tiles_h = (g.P + wt->tile_h - 1) / wt->tile_h;
+  wt->tiles_w = (g.Q + wt->tile_w - 1) / wt->tile_w;
+  wt->box_bytes = d.C * wt->win_h * wt->win_w;
+  wt->win_bytes = round_up(wt->box_bytes + 32, 128);
+  wt->mtot = (long long)d.N * wt->tiles_h * wt->tiles_w * kTileM;
+  wt->smem = 1024 + 2 * (size_t)wt->num_kb * kTileM * 128 + (size_t)wt->num_kb * wt->tile_n * 128 + 3 * (size_t)wt->win_bytes +
+             (size_t)round_up(wt->K_pad, 128) + 256;
+  return wt->mtot <= 0x7FFFFF00LL && wt->smem <= 200 * 1024 && (long long)d.N * wt->tiles_h * wt->tiles_w < 0x7FFFFFFFLL;
+}
+
 static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int tile_n, int split_k,
                 bool swap = false, int tile_m = kTileM) {
   const b2c_conv_desc& d = g.d;
@@ -331,6 +372,8 @@ static void add(std::vector<b2c_embedding>* out, const Geom& g, int variant, int
     e.map_k = B2C_AXIS_CRS;
     int K_pad = variant_k_pad(g, variant);
     k_issued = K_pad;
+    WindowTile wt;
+    if (variant == B2C_VARIANT_IM2COL_WINDOW && window_tile_geom(g, &wt)) M_pad = wt.mtot;  // whole two-dimensional tiles
     if (variant == B2C_VARIANT_IM2COL_EXPLICIT)
       moved = g.x_elems + 2 * g.Mg * K_pad + (long long)d.K * K_pad + g.y_elems;
     else if (variant == B2C_VARIANT_IM2COL_STAGED)
@@ -365,6 +408,12 @@ void enumerate_embeddings(const Geom& g, std::vector<b2c_embedding>* out) {
         ((is_tma_view_variant(variant) ? view_rows(g, variant, view) : g.Mg) + kTileM - 1) / kTileM;
     WindowGeom wg;
     if (variant == B2C_VARIANT_IM2COL_STAGED && !staged_window(g, &wg)) continue;
+    if (variant == B2C_VARIANT_IM2COL_WINDOW) {
+      // one schedule: all output channels in one column tile (the weights are resident), no split
+      WindowTile wt;
+      if (window_tile_geom(g, &wt)) add(out, g, variant, wt.tile_n, 1);
+      continue;
+    }
     int num_kb;
     if (is_tma_view_variant(variant)) {
       num_kb = view.R * view.S * (view.C / cp_block_bytes(view.C));

@@ -137,6 +137,30 @@ int encode_tiled_nhwc_rows(CUtensorMap* map, const void* base, int C_pad, int W,
   return B2C_OK;
 }
 
+// NCHW int8 activation tensor seen as a 4-D tensor {W, H, C, N} in tiled mode without swizzle: one copy
+// fetches box_w bytes of box_h rows of all C channels of one image; columns left or right of the
+// image, rows above or below it and images past the batch read as zeros.  W must be a multiple of 16.
+int encode_tiled_nchw_window(CUtensorMap* map, const void* base, int W, int H, int C, int N, int box_w, int box_h) {
+  std::call_once(g_once, resolve);
+  if (injected_failure()) return B2C_E_CUDA;
+  if (!g_tiled) {
+    set_last_cuda_error((int)CUDA_ERROR_NOT_FOUND);
+    return B2C_E_CUDA;
+  }
+  cuuint64_t dims[4] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)C, (cuuint64_t)N};
+  cuuint64_t strides[3] = {(cuuint64_t)W, (cuuint64_t)W * H, (cuuint64_t)W * H * C};
+  cuuint32_t box[4] = {(cuuint32_t)box_w, (cuuint32_t)box_h, (cuuint32_t)C, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = g_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error((int)r);
+    return B2C_E_CUDA;
+  }
+  return B2C_OK;
+}
+
 }  // namespace b2c
 
 extern "C" int b2c_last_cuda_error(void) { return b2c::get_last_cuda_error(); }

@@ -69,7 +69,7 @@ def test_config_every_embedding(lib, cfg):
 @pytest.mark.parametrize("in_layout,out_layout", [(1, 1), (0, 1), (1, 0)])
 def test_config_layouts(lib, cfg, in_layout, out_layout):
     x, w, ref = cfg_reference(cfg)
-    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8, 9):
+    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10):
         d = lib.make_desc(cfg.N, cfg.C, cfg.H, cfg.W, cfg.K, cfg.R, cfg.S, cfg.stride, cfg.pad, cfg.dilation, cfg.shift,
                           in_layout, out_layout, 3)
         ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant]
@@ -105,7 +105,7 @@ def test_random_shapes(lib, case):
     ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
     d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode=3)
     embs = lib.enumerate_embeddings(d)
-    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8, 9):
+    for variant in (0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10):
         ids = [e.id for e in embs if e.variant == variant]
         for i in ids[:1] + ids[-1:]:
             check_against_oracle(x, w, stride, pad, dil, shift, 3, i, ref=ref)
@@ -627,6 +627,52 @@ def test_two_sm_schedule_walks_tiles(lib, in_layout, tile_n):
         ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == variant and e.tile_n == tile_n and e.tile_m == 256]
         assert ids
         check_against_oracle(x, w, 2, 1, 1, 10, 3, ids[0], ref=ref, in_layout=in_layout)
+
+
+# ---- stencil unroll from a TMA-staged two-dimensional window (low-channel shapes, NCHW rows of 16-byte multiples) ---
+@pytest.mark.parametrize("case", [
+    # N, C, H, W, K, R, S, stride, pad, dil, shift
+    (2, 3, 40, 48, 64, 7, 7, 2, 3, 1, 6),              # the 7x7 stride-2 stem class
+    (3, 1, 30, 96, 32, 9, 21, 2, 0, 1, 5),             # single channel, wide kernel: runs of 24 straddle 16-byte chunks
+    (2, 2, 17, 32, 17, 3, 3, 1, 1, 1, 4),              # 17 output channels in a 32-column tile, odd height
+    (1, 5, 33, 64, 130, 5, 4, (3, 1), (2, 3), (2, 1), 7),  # vertical dilation, stride 3 x 1, 130 channels (256-column tile)
+    (4, 1, 9, 16, 8, 3, 5, (1, 2), (1, 2), 1, 3),      # narrow image: 16-pixel-wide tiles
+    (2, 4, 20, 240, 40, 1, 1, 1, 0, 1, 2),             # 1x1 kernel: runs of one tap padded to four
+    (1, 16, 12, 16, 16, 3, 3, 1, 1, 1, 8),             # 16 channels: 576-byte rows, five reduction blocks
+])
+@pytest.mark.parametrize("out_layout,out_mode", [(0, 3), (1, 3), (0, 2)])
+def test_tma_window_unroll(lib, case, out_layout, out_mode):
+    N, C, H, W, K, R, S, stride, pad, dil, shift = case
+    x = int8_uniform((N, C, H, W), 761)
+    w = int8_uniform((K, C, R, S), 762)
+    ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, 0, out_layout, out_mode)
+    ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_IM2COL_WINDOW]
+    assert len(ids) == 1
+    check_against_oracle(x, w, stride, pad, dil, shift, out_mode, ids[0], ref=ref, out_layout=out_layout)
+
+
+def test_tma_window_unroll_walks_tiles(lib):
+    """More tiles than resident blocks (2 x 148): the rings of windows, operand buffers and accumulators wrap."""
+    N, C, H, W, K, R, S = 12, 3, 112, 112, 64, 7, 7   # stride 2: 56 x 56 outputs, 28 x 1 tiles per image... 336 tiles
+    x = int8_uniform((N, C, H, W), 763)
+    w = int8_uniform((K, C, R, S), 764)
+    bias = (int8_uniform((K,), 765).astype(np.int32) * 500)
+    ref = oracle.conv2d_int8(x, w, 2, 3, 1, 7, bias=bias, relu=True)
+    d = lib.make_desc(N, C, H, W, K, R, S, 2, 3, 1, 7, 0, 0, 3)
+    e = [e for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_IM2COL_WINDOW][0]
+    plan = lib.Plan(d, e.id)
+    plan.set_weights(to_dev(w))
+    plan.set_activation(to_dev(bias), True)
+    y32 = torch.full(ref[0].shape, -7777777, dtype=torch.int32, device="cuda")
+    y8 = torch.full(ref[1].shape, 77, dtype=torch.int8, device="cuda")
+    xd = to_dev(x)
+    for _ in range(2):
+        plan.run(xd, y32, y8, None)
+    torch.cuda.synchronize()
+    assert plan.device_status() == b2c.OK and plan.workspace_bytes() == 0
+    assert np.array_equal(y32.cpu().numpy(), ref[0]) and np.array_equal(y8.cpu().numpy(), ref[1])
+    plan.destroy()
 
 
 # ---- activation pack inside the two-SM kernel (NCHW input, persistent channel-pack schedule) -------------

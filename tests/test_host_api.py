@@ -83,7 +83,7 @@ def test_enumeration_is_sorted_and_covers_variants(lib, cfg):
     assert [e.id for e in embs] == list(range(len(embs)))
     costs = [e.o_mac + e.o_data for e in embs]
     assert costs == sorted(costs)
-    assert {0, 1, 2} <= {e.variant for e in embs} <= {0, 1, 2, 3, 4, 5, 6, 7, 8, 9}
+    assert {0, 1, 2} <= {e.variant for e in embs} <= {0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10}
     for e in embs:
         assert e.tile_m in (128, 256) and e.tile_n in (16, 32, 64, 128, 256) and e.split_k >= 1
         if e.tile_m == 256:   # two-SM schedule: TMA-fed maps, no split, column tile of at least 32
@@ -93,7 +93,7 @@ def test_enumeration_is_sorted_and_covers_variants(lib, cfg):
             assert e.variant in (0, 1, 4, 5) and cfg.K >= 64 and e.tile_n >= 32
         assert e.map_k == {0: b2c.AXIS_C, 6: b2c.AXIS_C, 7: b2c.AXIS_C, 4: b2c.AXIS_SC, 9: b2c.AXIS_SC, 5: b2c.AXIS_C_PHASES, 8: b2c.AXIS_C_PHASES}.get(e.variant, b2c.AXIS_CRS)
         assert e.o_mac >= 0 and e.o_data >= 0 and e.device_us == -1.0
-        if e.variant in (b2c.VARIANT_IM2COL_GATHER, b2c.VARIANT_IM2COL_STAGED) and e.split_k == 1:
+        if e.variant in (b2c.VARIANT_IM2COL_GATHER, b2c.VARIANT_IM2COL_STAGED, b2c.VARIANT_IM2COL_WINDOW) and e.split_k == 1:
             assert e.workspace_bytes == 0
 
 
