@@ -257,11 +257,13 @@ void fill_common_args(b2c_plan* p) {
     a.wn_left = wt.left;
     a.wn_off0 = wt.off0;
     a.wn_chunks = wt.K_pad / 16;
+    a.wn_linear = wt.linear;
+    a.sh_R = d.R;
     a.sh_tiles_h = wt.tiles_h;
     a.sh_tiles_w = wt.tiles_w;
     a.div_tiles_hw = make_fastdiv((uint32_t)(wt.tiles_h * wt.tiles_w));
     a.div_tiles_w = make_fastdiv((uint32_t)wt.tiles_w);
-    a.num_tiles = (int)((long long)d.N * wt.tiles_h * wt.tiles_w);
+    a.num_tiles = wt.linear ? (int)((wt.mtot + kTileM - 1) / kTileM) : (int)((long long)d.N * wt.tiles_h * wt.tiles_w);
     a.tiles_n = 1;
     a.persistent = 2;
     a.split_k = 1;
@@ -466,7 +468,10 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
       std::vector<int32_t> t32(K_pad / 4, 0);
       for (int wi = 0; wi < K_pad / 4; ++wi) {
         const int run = (wi * 4) / wt.S_run, s0 = (wi * 4) % wt.S_run;
-        if (run < d.C * d.R) t32[wi] = ((run / d.R) * wt.win_h + (run % d.R) * d.dil_h) * wt.win_w + s0;
+        if (run >= d.C * d.R) continue;
+        t32[wi] = ((run / d.R) * wt.win_h + (run % d.R) * d.dil_h) * wt.win_w + s0;
+        // linear tiles: + the filter row (bits 16-23) and the word of the run (bits 24-31) for the masks
+        if (wt.linear) t32[wi] |= ((run % d.R) << 16) | ((s0 >> 2) << 24);
       }
       p->table_len = (int)t32.size();
       if (cudaMalloc(&p->table32, t32.size() * sizeof(int32_t)) != cudaSuccess) return fail(B2C_E_CUDA);
@@ -922,8 +927,12 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
     rc = encode_tiled_2d(&tmap_a, wsb, p->K_pad, (uint64_t)g.Mg, p->K_pad, 128, a.swap ? a.tile_n : kTileM, 128);
     if (rc != B2C_OK) return rc;
   } else if (p->amode == A_WINDOW) {
-    rc = encode_tiled_nchw_window(&tmap_a, x, d.W, d.H, d.C, d.N, a.wn_win_w, a.wn_box_bytes / (d.C * a.wn_win_w));
-    if (rc != B2C_OK) return rc;
+    if (a.wn_linear) {
+      tmap_a = p->tmap_b;  // the images arrive by plain bulk copies; any valid map
+    } else {
+      rc = encode_tiled_nchw_window(&tmap_a, x, d.W, d.H, d.C, d.N, a.wn_win_w, a.wn_box_bytes / (d.C * a.wn_win_w));
+      if (rc != B2C_OK) return rc;
+    }
   } else {
     tmap_a = p->tmap_b;  // unused by the gather kernel; any valid map
   }

@@ -138,7 +138,9 @@ struct ConvArgs {
   // wn_tile_w output pixels (sh_tiles_h x sh_tiles_w tiles per image); the window of a tile is C x win_h
   // rows of wn_win_w bytes, its first byte wn_left columns left of the tile's first input column
   // (wn_off0 = wn_left - pad_w bytes before the first tap); wn_chunks 16-byte chunks per A row.
-  int wn_tile_w, wn_win_w, wn_win_bytes, wn_box_bytes, wn_left, wn_off0, wn_chunks;
+  // wn_linear: tiles are 128 consecutive fused pixels, the window holds whole images (wn_box_bytes each,
+  // behind a margin of wn_left bytes), taps outside the image are masked by the builders.
+  int wn_tile_w, wn_win_w, wn_win_bytes, wn_box_bytes, wn_left, wn_off0, wn_chunks, wn_linear;
   FastDiv div_wps, div_hp;
   // elements between consecutive images of the NKPQ output (K * P * Q, or more when this
   // convolution writes one channel group of a wider tensor)
@@ -307,6 +309,7 @@ int variant_k_pad(const Geom& g, int variant);  // padded reduction length of th
 // Geometry of the TMA-staged window unroll (B2C_VARIANT_IM2COL_WINDOW); false if it does not apply.
 struct WindowTile {
   int tile_w, tile_h, win_w, win_h, left, off0, S_run, K_pad, tiles_h, tiles_w, box_bytes, win_bytes, tile_n, num_kb;
+  int linear;      // small images: linear tiles over whole images staged by bulk copies (box_bytes = C*H*W, left = margin)
   long long mtot;  // accumulator rows issued: N * tiles_h * tiles_w * 128
   size_t smem;
 };

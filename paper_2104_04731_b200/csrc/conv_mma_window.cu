@@ -15,6 +15,11 @@
 // zero.  The packed weights stay resident in shared memory; one warp issues the MMAs; four epilogue
 // warps drain the accumulators (activation step, shift / clip, NKPQ or NPQK stores), so that the
 // operand build of tile t + 1, the MMAs of tile t and the stores of tile t - 1 overlap.
+// Small images (LINEAR form): when a whole image of C x H x W bytes is a multiple of 16 bytes and a few
+// KB, tiles are 128 consecutive fused (n, p, q) pixels instead, the window is the whole images those
+// pixels belong to, each fetched by one bulk copy of the NCHW tensor as it is (no zero padding in
+// shared memory), and the builders clear the taps that fall outside the image with per-row masks
+// (a bit per filter row, a byte mask per word of a run) computed once per tile and row.
 // Every wait is bounded as in the other kernels.
 #include <algorithm>
 
@@ -41,6 +46,7 @@ struct __align__(8) WindowCtl {
   SharedCtl base;  // abort flag and tensor-memory base (the bounded waits take this)
 };
 
+template <bool LINEAR>
 __global__ void __launch_bounds__(kWinThreads, 2)
     conv_mma_window_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_b,
                            const ConvArgs args) {
@@ -121,15 +127,32 @@ __global__ void __launch_bounds__(kWinThreads, 2)
     int s = 0;
     uint32_t ph = 0;
     for (int t = tile_first; t < tile_end; t += tile_step) {
-      const int img = (int)args.div_tiles_hw.div((uint32_t)t);
-      const int rem = t - img * tiles_per_image;
-      const int ty = (int)args.div_tiles_w.div((uint32_t)rem), tx = rem - ty * args.sh_tiles_w;
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&wc.win_empty[s]), ph ^ 1u, ctl, args.status))) break;
       const uint32_t full = smem_u32(&wc.win_full[s]);
-      mbar_arrive_expect_tx(full, (uint32_t)args.wn_box_bytes, leader);
-      // (the first column is a multiple of 16 bytes below the tile's first input column)
-      tma_load_tiled_4d(win_base + (uint32_t)s * win_bytes, &tmap_x, tx * args.wn_tile_w * args.stride_w - args.wn_left,
-                        ty * tile_h * args.stride_h - args.pad_h, 0, img, full, leader);
+      if (LINEAR) {
+        // the whole images of the tile's 128 pixels, one bulk copy each, behind the window's margin
+        const int m0 = t * kTileM;
+        const int n_a = (int)args.div_pq.div((uint32_t)m0);
+        const int n_b = (int)args.div_pq.div((uint32_t)min(m0 + kTileM - 1, args.Mg - 1));
+        const uint32_t img_bytes = (uint32_t)args.wn_box_bytes;
+        mbar_arrive_expect_tx(full, (uint32_t)(n_b - n_a + 1) * img_bytes, leader);
+        for (int n = n_a; n <= n_b; ++n) {
+          const uint32_t dst = win_base + (uint32_t)s * win_bytes + (uint32_t)args.wn_left + (uint32_t)(n - n_a) * img_bytes;
+          asm volatile(
+              "{\n.reg .pred q;\nsetp.ne.b32 q, %4, 0;\n"
+              "@q cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n}" ::"r"(dst),
+              "l"(args.x + (size_t)n * img_bytes), "r"(img_bytes), "r"(full), "r"(leader)
+              : "memory");
+        }
+      } else {
+        const int img = (int)args.div_tiles_hw.div((uint32_t)t);
+        const int rem = t - img * tiles_per_image;
+        const int ty = (int)args.div_tiles_w.div((uint32_t)rem), tx = rem - ty * args.sh_tiles_w;
+        mbar_arrive_expect_tx(full, (uint32_t)args.wn_box_bytes, leader);
+        // (the first column is a multiple of 16 bytes below the tile's first input column)
+        tma_load_tiled_4d(win_base + (uint32_t)s * win_bytes, &tmap_x, tx * args.wn_tile_w * args.stride_w - args.wn_left,
+                          ty * tile_h * args.stride_h - args.pad_h, 0, img, full, leader);
+      }
       if (++s == kWinStages) {
         s = 0;
         ph ^= 1u;
@@ -170,9 +193,11 @@ __global__ void __launch_bounds__(kWinThreads, 2)
     const int half = tid >> 7;  // warps 2-5 take the even 16-byte chunks of a row, warps 6-9 the odd ones
     const int ti_row = row >> tw_log2, tj = row & (args.wn_tile_w - 1);
     // byte offset of this row's first tap inside a window, and the permute selector of its alignment
-    const int tbase = ti_row * args.stride_h * args.wn_win_w + tj * args.stride_w + args.wn_off0;
-    const uint32_t sel = 0x3210u + 0x1111u * ((uint32_t)tbase & 3u);
-    const int tbase4 = tbase & ~3;
+    // (two-dimensional tiles: the same for every tile; linear tiles: set per tile below)
+    int tbase = ti_row * args.stride_h * args.wn_win_w + tj * args.stride_w + args.wn_off0;
+    uint32_t sel = 0x3210u + 0x1111u * ((uint32_t)tbase & 3u);
+    int tbase4 = tbase & ~3;
+    uint32_t rbits = 0, hm0 = 0, hm1 = 0;  // linear tiles: valid filter rows, byte masks of the two words of a run
     const uint32_t xr = (uint32_t)(row & 7);
     const uint32_t row_off = (uint32_t)row * 128u;
     const int nchunks = args.wn_chunks;  // 16-byte chunks of a row (K_pad / 16)
@@ -185,8 +210,56 @@ __global__ void __launch_bounds__(kWinThreads, 2)
       ok = mbar_wait(smem_u32(&wc.a_empty[ab]), (a_use & 1u) ^ 1u, ctl, args.status);
       if (ok) ok = mbar_wait(smem_u32(&wc.win_full[s]), ph, ctl, args.status);
       if (!ok) break;
-      const uint8_t* win = win_ptr + (size_t)s * win_bytes + tbase4;
+      if (LINEAR) {
+        // this row's pixel (n, p, q); rows past the last pixel build from the window's first image (never stored)
+        const unsigned m = (unsigned)t * kTileM + (unsigned)row;
+        const int n_a = (int)args.div_pq.div((uint32_t)t * kTileM);
+        int part = 0, p = 0, q = 0;
+        if (m < (unsigned)args.Mg) {
+          const int n = (int)args.div_pq.div(m);
+          const int pq = (int)(m - (unsigned)n * (unsigned)args.PQ);
+          p = (int)args.div_q.div((uint32_t)pq);
+          q = pq - p * args.Q;
+          part = n - n_a;
+        }
+        const int h0 = p * args.stride_h - args.pad_h, w0 = q * args.stride_w - args.pad_w;
+        tbase = args.wn_left + part * args.wn_box_bytes + h0 * args.W + w0;
+        sel = 0x3210u + 0x1111u * ((uint32_t)tbase & 3u);
+        tbase4 = tbase & ~3;
+        rbits = 0;
+        for (int r = 0; r < args.sh_R; ++r)
+          if ((unsigned)(h0 + r * args.dil_h) < (unsigned)args.H) rbits |= 1u << r;
+        hm0 = hm1 = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          if ((unsigned)(w0 + b) < (unsigned)args.W) hm0 |= 0xFFu << (8 * b);
+          if ((unsigned)(w0 + 4 + b) < (unsigned)args.W) hm1 |= 0xFFu << (8 * b);
+        }
+      }
+      const uint8_t* wslot = win_ptr + (size_t)s * win_bytes;
+      const uint8_t* win = wslot + tbase4;
       const uint32_t a_row = a_base + (uint32_t)ab * a_buf_bytes + row_off;
+      if (LINEAR) {
+        for (int ch = half; ch < nchunks; ch += 2) {
+          // table entry of a word: window offset (16 bits), filter row (8 bits), word of the run (8 bits)
+          const int4 e = *reinterpret_cast<const int4*>(s_table + ch * 4);
+          const int ev[4] = {e.x, e.y, e.z, e.w};
+          uint32_t wv[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int off = ev[i] & 0xFFFF, r = (ev[i] >> 16) & 0xFF, wi = ev[i] >> 24;
+            // (image rows are not multiples of 4 bytes here: the word's alignment depends on its offset too)
+            const int addr = tbase + off;
+            const uint8_t* src = wslot + (addr & ~3);
+            const uint32_t lo = *reinterpret_cast<const uint32_t*>(src);
+            const uint32_t hi = *reinterpret_cast<const uint32_t*>(src + 4);
+            const uint32_t mask = ((rbits >> r) & 1u) ? (wi ? hm1 : hm0) : 0u;
+            wv[i] = __byte_perm(lo, hi, 0x3210u + 0x1111u * ((uint32_t)addr & 3u)) & mask;
+          }
+          const uint32_t dst = a_row + (uint32_t)(ch >> 3) * a_block_bytes + ((((uint32_t)ch & 7u) ^ xr) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]), "r"(wv[3]));
+        }
+      } else
       for (int ch = half; ch < nchunks; ch += 2) {
         // the four words of this chunk: window offsets from the table (the same for the whole warp)
         const int4 off = *reinterpret_cast<const int4*>(s_table + ch * 4);
@@ -223,12 +296,21 @@ __global__ void __launch_bounds__(kWinThreads, 2)
     bool ok = true;
     int ti = 0;
     for (int t = tile_first; t < tile_end && ok; t += tile_step, ++ti) {
-      const int img = (int)args.div_tiles_hw.div((uint32_t)t);
-      const int rem = t - img * tiles_per_image;
-      const int ty = (int)args.div_tiles_w.div((uint32_t)rem), tx = rem - ty * args.sh_tiles_w;
-      const int po = ty * tile_h + ti_row, qo = tx * args.wn_tile_w + tj;
-      const bool row_valid = po < args.out_P && qo < args.out_Q;
-      const int out_pq = po * args.out_Q + qo;
+      int img, out_pq;
+      bool row_valid;
+      if (LINEAR) {
+        const unsigned m = (unsigned)t * kTileM + (unsigned)row;
+        row_valid = m < (unsigned)args.Mg;
+        img = row_valid ? (int)args.div_pq.div(m) : 0;
+        out_pq = row_valid ? (int)(m - (unsigned)img * (unsigned)args.PQ) : 0;
+      } else {
+        img = (int)args.div_tiles_hw.div((uint32_t)t);
+        const int rem = t - img * tiles_per_image;
+        const int ty = (int)args.div_tiles_w.div((uint32_t)rem), tx = rem - ty * args.sh_tiles_w;
+        const int po = ty * tile_h + ti_row, qo = tx * args.wn_tile_w + tj;
+        row_valid = po < args.out_P && qo < args.out_Q;
+        out_pq = po * args.out_Q + qo;
+      }
       const int tb = ti & (nbuf - 1);
       const uint32_t t_use = (uint32_t)(ti >> nbuf_log2);
       ok = mbar_wait(smem_u32(&wc.tmem_full[tb]), t_use & 1u, ctl, args.status);
@@ -276,13 +358,18 @@ size_t conv_mma_window_smem_bytes(const ConvArgs& a) {
 cudaError_t launch_conv_mma_window(const CUtensorMap* tmap_x, const CUtensorMap* tmap_b, const ConvArgs& args,
                                    cudaStream_t st) {
   const size_t smem = conv_mma_window_smem_bytes(args);
-  static std::atomic<unsigned long long> configured{0};
-  cudaError_t e = set_max_dynamic_smem_once(configured, (const void*)conv_mma_window_kernel, 226 * 1024);
+  static std::atomic<unsigned long long> configured{0}, configured_linear{0};
+  cudaError_t e = args.wn_linear
+                      ? set_max_dynamic_smem_once(configured_linear, (const void*)conv_mma_window_kernel<true>, 226 * 1024)
+                      : set_max_dynamic_smem_once(configured, (const void*)conv_mma_window_kernel<false>, 226 * 1024);
   if (e != cudaSuccess) return e;
   // blocks per SM by shared memory (at most two); the grid is one wave of resident blocks walking the tiles
   const int per_sm = smem * 2 + 4096 <= 227 * 1024 ? 2 : 1;
   const dim3 grid((unsigned)std::min(args.num_tiles, kNumSMs * per_sm), 1, 1);
-  e = launch_pdl(conv_mma_window_kernel, grid, dim3(kWinThreads), smem, st, *tmap_x, *tmap_b, args);
+  if (args.wn_linear)
+    e = launch_pdl(conv_mma_window_kernel<true>, grid, dim3(kWinThreads), smem, st, *tmap_x, *tmap_b, args);
+  else
+    e = launch_pdl(conv_mma_window_kernel<false>, grid, dim3(kWinThreads), smem, st, *tmap_x, *tmap_b, args);
   if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }

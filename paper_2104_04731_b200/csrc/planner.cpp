@@ -296,17 +296,55 @@ bool staged_window(const Geom& g, WindowGeom* w) {
   return true;
 }
 
+// Small images: whole images as the window, linear tiles.
+static bool window_linear_geom(const Geom& g, WindowTile* wt) {
+  const b2c_conv_desc& d = g.d;
+  const long long chw = (long long)d.C * d.H * d.W;
+  // an image is one bulk copy (16-byte multiple, a few KB); a tile of 128 consecutive pixels touches
+  // at most four images; runs of at most two words; the margin in front of the window covers the
+  // negative offsets of the padding (those taps are masked, but their addresses must be valid)
+  if ((chw % 16) != 0 || chw > 16 * 1024 || d.S > 8 || d.R > 32 || g.PQ < 43) return false;
+  if ((long long)d.pad_h * d.W + d.pad_w + 8 > 128) return false;
+  const int parts = (kTileM - 2) / g.PQ + 2;
+  wt->linear = 1;
+  wt->tile_w = kTileM;
+  wt->tile_h = 1;
+  wt->win_w = d.W;
+  wt->win_h = d.H;
+  wt->left = 128;
+  wt->off0 = 0;
+  wt->tiles_h = wt->tiles_w = 1;
+  wt->box_bytes = (int)chw;
+  // rows below the image that masked taps may address: up to (R-1)*dil_h rows past the last output row's first tap
+  const long long slack = round_up((int)((long long)(d.R - 1) * d.dil_h * d.W + d.S + 16), 128) + 128;
+  const long long win = 128 + (long long)parts * chw + slack;
+  if (win > 60 * 1024 || chw >= (1 << 16) || win >= (1 << 16)) return false;
+  wt->win_bytes = round_up((int)win, 128);
+  wt->mtot = g.Mg;
+  return true;
+}
+
 bool window_tile_geom(const Geom& g, WindowTile* wt) {
   const b2c_conv_desc& d = g.d;
-  // the window is one tiled TMA box of the NCHW tensor: rows must be multiples of 16 bytes, every box
-  // extent at most 256; words of an A row are unaligned words of a window row: unit horizontal dilation
-  if (d.in_layout != B2C_LAYOUT_NCHW || (d.W % 16) != 0 || d.dil_w != 1 || d.C > 64 || d.K > 256) return false;
+  // words of an A row are unaligned words of a window row: unit horizontal dilation
+  if (d.in_layout != B2C_LAYOUT_NCHW || d.dil_w != 1 || d.C > 64 || d.K > 256) return false;
+  wt->linear = 0;
   wt->S_run = round_up(d.S, 4);
   wt->K_pad = round_up(d.C * d.R * wt->S_run, kMmaK);
   if (wt->K_pad > 1024) return false;
   wt->num_kb = (wt->K_pad + 127) / 128;
   wt->tile_n = 16;
   while (wt->tile_n < d.K) wt->tile_n <<= 1;
+  // small images: linear tiles over whole images (no padded positions at all)
+  if (((d.W % 16) != 0 || g.PQ <= 1024) && window_linear_geom(g, wt)) {
+    wt->smem = 1024 + 2 * (size_t)wt->num_kb * kTileM * 128 + (size_t)wt->num_kb * wt->tile_n * 128 + 3 * (size_t)wt->win_bytes +
+               (size_t)round_up(wt->K_pad, 128) + 256;
+    return wt->mtot <= 0x7FFFFF00LL && wt->smem <= 200 * 1024;
+  }
+  wt->linear = 0;
+  // the window is one tiled TMA box of the NCHW tensor: rows must be multiples of 16 bytes, every box
+  // extent at most 256
+  if ((d.W % 16) != 0) return false;
   wt->left = round_up(d.pad_w, 16);
   wt->off0 = wt->left - d.pad_w;
   long long best_tiles = -1;

@@ -639,6 +639,12 @@ def test_two_sm_schedule_walks_tiles(lib, in_layout, tile_n):
     (4, 1, 9, 16, 8, 3, 5, (1, 2), (1, 2), 1, 3),      # narrow image: 16-pixel-wide tiles
     (2, 4, 20, 240, 40, 1, 1, 1, 0, 1, 2),             # 1x1 kernel: runs of one tap padded to four
     (1, 16, 12, 16, 16, 3, 3, 1, 1, 1, 8),             # 16 channels: 576-byte rows, five reduction blocks
+    # small images: linear tiles over whole images, border taps masked
+    (5, 16, 14, 14, 16, 3, 3, 1, 1, 1, 8),             # the 14 x 14, 16-channel shape: tiles span two images
+    (7, 2, 10, 8, 40, 3, 5, 2, 2, (2, 1), 5),          # stride 2, pad 2, vertical dilation; 20 pixels... too few: not listed
+    (9, 2, 20, 24, 33, 3, 5, (2, 1), (2, 1), (2, 1), 5),   # runs of two words, vertical dilation, 240 pixels per image
+    (3, 4, 9, 12, 8, 1, 1, 1, (1, 3), 1, 2),           # 1x1 kernel with padding: outputs that see only zeros
+    (6, 1, 16, 16, 64, 5, 8, (1, 2), (2, 4), 1, 6),    # 16-byte rows but small: the linear form is preferred; 8-tap runs
 ])
 @pytest.mark.parametrize("out_layout,out_mode", [(0, 3), (1, 3), (0, 2)])
 def test_tma_window_unroll(lib, case, out_layout, out_mode):
@@ -648,8 +654,23 @@ def test_tma_window_unroll(lib, case, out_layout, out_mode):
     ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift)
     d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, 0, out_layout, out_mode)
     ids = [e.id for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_IM2COL_WINDOW]
+    P, Q = lib.out_shape(d)
+    if W % 16 != 0 and P * Q < 43:
+        assert not ids   # neither form applies: rows are no 16-byte multiples and a tile would span too many images
+        return
     assert len(ids) == 1
     check_against_oracle(x, w, stride, pad, dil, shift, out_mode, ids[0], ref=ref, out_layout=out_layout)
+
+
+def test_window_unroll_small_images_walks_tiles(lib):
+    """Linear tiles over many small images: the rings wrap, tiles start inside one image and end in the next."""
+    N, C, H, W, K, R, S = 700, 16, 14, 14, 16, 3, 3   # 137200 pixels = 1072 tiles
+    x = int8_uniform((N, C, H, W), 766)
+    w = int8_uniform((K, C, R, S), 767)
+    ref = oracle.conv2d_int8(x, w, 1, 1, 1, 8)
+    d = lib.make_desc(N, C, H, W, K, R, S, 1, 1, 1, 8, 0, 0, 3)
+    e = [e for e in lib.enumerate_embeddings(d) if e.variant == b2c.VARIANT_IM2COL_WINDOW][0]
+    check_against_oracle(x, w, 1, 1, 1, 8, 3, e.id, ref=ref)
 
 
 def test_tma_window_unroll_walks_tiles(lib):
