@@ -36,6 +36,7 @@ extern "C" {
 #define B2C_E_CUDA (-4)                /* a CUDA runtime/driver call failed; see b2c_last_cuda_error */
 #define B2C_E_TIMEOUT (-5)             /* a bounded device-side wait expired (device status word) */
 #define B2C_E_NOT_READY (-6)           /* plan has no weights yet                                */
+#define B2C_E_BOUNDS (-7)              /* debug build only: a kernel computed an address outside its tensor (device status word) */
 
 /* ---- problem description -------------------------------------------------------------------- */
 /* Convolution y[n][k][p][q] = sum_{c,r,s} x[n][c][p*stride_h - pad_h + r*dil_h][q*stride_w - pad_w + s*dil_w] * w[k][c][r][s]
@@ -310,6 +311,26 @@ int b2c_im2col_noalloc(const b2c_conv_desc* desc, const int8_t* x_dev, int8_t* a
  * {16, 32, 64, 128, 256}.  Allocates a few KB and synchronises: not for use under stream capture.
  * INVALID_ARG on bad arguments, B2C_E_CUDA / B2C_E_TIMEOUT on failure. */
 int b2c_measure_mma_rate(int tile_n, int mmas_per_block, float* device_us, float* cycles_per_mma, void* cuda_stream);
+
+/* ---- debug build (no counterpart in the paper) ---------------------------------------------------
+ * libb2conv_debug.so is the same library compiled with -DB2C_DEBUG_BOUNDS.  In it every address a
+ * kernel computes by hand (loads of x, stores and atomics to the outputs and to the scratch; TMA
+ * copies are clipped by their tensor maps and need no check) is tested against the range of its
+ * tensor; the first access outside records B2C_E_BOUNDS, a site number and the byte offset from the
+ * range start in the plan's device status words and is skipped, later ones are only skipped.  The
+ * workspace gains a 64-byte guard band on either side (b2c_plan_workspace_bytes includes them; run
+ * repaints them and uses the middle).  It stands in for a memory checker where none can be run.
+ * b2c_debug_build: 1 in that library, 0 in the release one.
+ * b2c_plan_debug_info: site and byte offset of the report b2c_plan_device_status last returned.
+ * b2c_plan_check_canaries: waits for the device, reads the guard bands of `workspace_dev` (the
+ *   pointer given to run) and sets *intact to 0 if a byte changed; UNSUPPORTED in the release build.
+ * b2c_test_shrink_checked_ranges: test hook; every checked range is declared `bytes` shorter than it
+ *   is, so that in-range accesses near a tensor's end are reported and skipped (nothing out of range
+ *   is ever touched); 0 restores.  No effect in the release build. */
+int b2c_debug_build(void);
+int b2c_plan_debug_info(const b2c_plan* plan, int32_t* site, int64_t* byte_offset);
+int b2c_plan_check_canaries(b2c_plan* plan, const void* workspace_dev, int32_t* intact);
+int b2c_test_shrink_checked_ranges(long long bytes);
 
 /* Host-side fault injection for tests (no counterpart in the paper): the n-th tensor-map encode
  * from now on, counted over all threads, fails as if the driver had refused it (the call that

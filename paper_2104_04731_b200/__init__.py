@@ -11,10 +11,11 @@ import os
 from typing import List, Optional, Tuple
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libb2conv.so")
+# B2C_DEBUG_LIB=1 selects the debug build (bounds-checked kernels, guard bands round the workspace)
+LIB_PATH = os.path.join(_HERE, "libb2conv_debug.so" if os.environ.get("B2C_DEBUG_LIB") == "1" else "libb2conv.so")
 
 OK = 0
-E_INVALID_ARG, E_UNSUPPORTED, E_WORKSPACE_TOO_SMALL, E_CUDA, E_TIMEOUT, E_NOT_READY = -1, -2, -3, -4, -5, -6
+E_INVALID_ARG, E_UNSUPPORTED, E_WORKSPACE_TOO_SMALL, E_CUDA, E_TIMEOUT, E_NOT_READY, E_BOUNDS = -1, -2, -3, -4, -5, -6, -7
 LAYOUT_NCHW, LAYOUT_NHWC = 0, 1
 OUT_I32, OUT_I8 = 1, 2
 AXIS_NPQ, AXIS_K, AXIS_C, AXIS_CRS, AXIS_SC, AXIS_C_PHASES = 1, 2, 3, 4, 5, 6
@@ -33,7 +34,8 @@ EXPORTS = [
     "b2c_plan_create_grouped", "b2c_plan_run_host_async", "b2c_plan_host_sync",
     "b2c_plan_device_status", "b2c_selftest_bounded_wait", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
     "b2c_status_string",
-    "b2c_last_cuda_error", "b2c_oneshot_status", "b2c_oneshot_cache_clear", "b2c_test_fail_nth_encode", "b2c_selftest_pack_wait", "b2c_measure_mma_rate",
+    "b2c_last_cuda_error", "b2c_oneshot_status", "b2c_oneshot_cache_clear", "b2c_test_fail_nth_encode", "b2c_selftest_pack_wait", "b2c_measure_mma_rate", "b2c_debug_build", "b2c_plan_debug_info",
+    "b2c_plan_check_canaries", "b2c_test_shrink_checked_ranges",
 ]
 
 
@@ -108,6 +110,10 @@ def load():
     lib.b2c_status_string.restype = ctypes.c_char_p
     lib.b2c_last_cuda_error.argtypes = []
     lib.b2c_oneshot_status.argtypes = [pi32]
+    lib.b2c_debug_build.argtypes = []
+    lib.b2c_plan_debug_info.argtypes = [vp, pi32, ctypes.POINTER(ctypes.c_int64)]
+    lib.b2c_plan_check_canaries.argtypes = [vp, vp, pi32]
+    lib.b2c_test_shrink_checked_ranges.argtypes = [ctypes.c_longlong]
     lib.b2c_measure_mma_rate.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float), vp]
     lib.b2c_oneshot_cache_clear.argtypes = []
     lib.b2c_test_fail_nth_encode.argtypes = [i32]
@@ -242,6 +248,18 @@ class Plan:
         """Enqueues the bounded-wait self-test; afterwards device_status() reports E_TIMEOUT once."""
         _check(self._lib.b2c_selftest_bounded_wait(self._h, _stream_ptr(stream)), "b2c_selftest_bounded_wait")
 
+    def debug_info(self) -> Tuple[int, int]:
+        """(site, byte offset) of the out-of-range access the last device_status() reported (debug build)."""
+        site, off = ctypes.c_int32(), ctypes.c_int64()
+        _check(self._lib.b2c_plan_debug_info(self._h, ctypes.byref(site), ctypes.byref(off)), "b2c_plan_debug_info")
+        return site.value, off.value
+
+    def canaries_intact(self, workspace) -> bool:
+        """Debug build: True if the guard bands round `workspace` are untouched."""
+        ok = ctypes.c_int32()
+        _check(self._lib.b2c_plan_check_canaries(self._h, _dptr(workspace), ctypes.byref(ok)), "b2c_plan_check_canaries")
+        return bool(ok.value)
+
     def selftest_pack_wait(self, stream=None):
         """The same self-test for the activation-pack kernel's wait on its bulk copies."""
         _check(self._lib.b2c_selftest_pack_wait(self._h, _stream_ptr(stream)), "b2c_selftest_pack_wait")
@@ -272,6 +290,15 @@ def measure_mma_rate(tile_n: int = 256, mmas_per_block: int = 20000, stream=None
     _check(load().b2c_measure_mma_rate(tile_n, mmas_per_block, ctypes.byref(us), ctypes.byref(cyc), _stream_ptr(stream)),
            "b2c_measure_mma_rate")
     return us.value, cyc.value
+
+
+def debug_build() -> bool:
+    return bool(load().b2c_debug_build())
+
+
+def test_shrink_checked_ranges(nbytes: int):
+    """Debug-build test hook: declare every checked range `nbytes` shorter than it is (0 restores)."""
+    _check(load().b2c_test_shrink_checked_ranges(nbytes), "b2c_test_shrink_checked_ranges")
 
 
 def oneshot_status() -> int:

@@ -9,6 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "libb2conv.so")
+SO_DEBUG = os.path.join(HERE, "libb2conv_debug.so")  # -DB2C_DEBUG_BOUNDS: bounds-checked kernels, workspace guard bands
 SOURCES = ["api.cpp", "planner.cpp", "tma.cpp", "layout.cu", "conv_mma.cu", "conv_mma_pair.cu", "mma_rate.cu", "conv_mma_window.cu"]
 
 
@@ -19,17 +20,18 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def needs_build() -> bool:
-    if not os.path.exists(SO):
+def needs_build(so: str = SO) -> bool:
+    if not os.path.exists(so):
         return True
-    t = os.path.getmtime(SO)
+    t = os.path.getmtime(so)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "b2conv.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
-        return SO
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    so = SO_DEBUG if debug else SO
+    if not force and not needs_build(so):
+        return so
     cmd = [
         _nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
         "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-x", "cu",
@@ -37,12 +39,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
     ]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    tmp = SO + ".tmp.%d" % os.getpid()
+    if debug:
+        cmd += ["-DB2C_DEBUG_BOUNDS"]
+    tmp = so + ".tmp.%d" % os.getpid()
     cmd += ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
-    os.replace(tmp, SO)
-    return SO
+    os.replace(tmp, so)
+    return so
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

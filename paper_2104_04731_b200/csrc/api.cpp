@@ -2,6 +2,7 @@
 // MMA kernel with fused epilogue -> optional split-reduction finish), the one-shot calls and
 // the timed candidate selection.  See include/b2conv.h for the contract of each entry point.
 #include <algorithm>
+#include <atomic>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -50,6 +51,8 @@ struct b2c_plan {
   // of the work counters, which live in the workspace after the rewritten operand.
   bool fused_pack = false;
   size_t ws_ctl_offset = 0;  // bytes from the workspace start to the counters [1 + N] int
+  int dbg_site = 0;          // debug build: site and byte offset of the last reported out-of-range access
+  long long dbg_offset = 0;
 };
 
 // Device side of the streaming host-buffer calls: a ring of input / output buffers and three
@@ -71,6 +74,15 @@ struct HostPipe {
 };
 
 namespace {
+
+constexpr int kStatusWords = 4;     // [0] status, [1] site, [2..3] byte offset (debug build's bounds report)
+#ifdef B2C_DEBUG_BOUNDS
+constexpr size_t kCanaryBytes = 64;  // guard band on either side of the caller's workspace
+#else
+constexpr size_t kCanaryBytes = 0;
+#endif
+constexpr unsigned char kCanaryByte = 0xC5;
+std::atomic<long long> g_dbg_shrink{0};  // test hook: bytes taken off the end of every checked range
 
 #define CUDA_TRY(expr)                  \
   do {                                  \
@@ -392,8 +404,8 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
     b2c_plan_destroy(p);
     return code;
   };
-  if (cudaMalloc(&p->status, sizeof(int)) != cudaSuccess) return fail(B2C_E_CUDA);
-  if (cudaMemset(p->status, 0, sizeof(int)) != cudaSuccess) return fail(B2C_E_CUDA);
+  if (cudaMalloc(&p->status, kStatusWords * sizeof(int)) != cudaSuccess) return fail(B2C_E_CUDA);
+  if (cudaMemset(p->status, 0, kStatusWords * sizeof(int)) != cudaSuccess) return fail(B2C_E_CUDA);
   if (is_tma_view_variant(emb.variant)) {
     if (!tma_view_for(g, emb.variant, &p->view)) return fail(B2C_E_UNSUPPORTED);
     const TmaView& v = p->view;
@@ -642,6 +654,7 @@ const char* b2c_status_string(int s) {
     case B2C_E_CUDA: return "CUDA call failed";
     case B2C_E_TIMEOUT: return "bounded device wait expired";
     case B2C_E_NOT_READY: return "plan has no weights";
+    case B2C_E_BOUNDS: return "address outside its tensor (debug build)";
     default: return "unknown status";
   }
 }
@@ -786,7 +799,8 @@ int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan*
   p->emb = all[pick];
   p->groups = groups;
   cudaGetDevice(&p->device);
-  if (cudaMalloc(&p->status, sizeof(int)) != cudaSuccess || cudaMemset(p->status, 0, sizeof(int)) != cudaSuccess) {
+  if (cudaMalloc(&p->status, kStatusWords * sizeof(int)) != cudaSuccess ||
+      cudaMemset(p->status, 0, kStatusWords * sizeof(int)) != cudaSuccess) {
     set_last_cuda_error((int)cudaGetLastError());
     b2c_plan_destroy(p);
     return B2C_E_CUDA;
@@ -814,7 +828,7 @@ int b2c_plan_info(const b2c_plan* plan, b2c_embedding* chosen) {
 
 int b2c_plan_workspace_bytes(const b2c_plan* plan, size_t* bytes) {
   if (!plan || !bytes) return B2C_E_INVALID_ARG;
-  *bytes = plan->ws_total;
+  *bytes = plan->ws_total ? plan->ws_total + 2 * kCanaryBytes : 0;  // debug build: + the guard bands
   return B2C_OK;
 }
 
@@ -865,34 +879,41 @@ static int run_rewrite(b2c_plan* p, const int8_t* x, void* ws, cudaStream_t st) 
   const ConvArgs& a = p->args;
   if (!p->ws_layout_bytes) return B2C_OK;
   int8_t* scratch = static_cast<int8_t*>(ws);
+  Dbg dbg;
+  const long long shrink = g_dbg_shrink.load();
+  dbg.x_lo = x;
+  dbg.x_bytes = (long long)(d.N - 1) * a.x_stride_n + (long long)d.C * d.H * d.W - shrink;
+  dbg.ws_lo = ws;
+  dbg.ws_bytes = (long long)p->ws_layout_bytes - shrink;
+  dbg.status = p->status;
   if (is_tma_view_variant(p->emb.variant)) {
     const TmaView& v = p->view;
     const int base_variant = shift_base_variant(p->emb.variant);
     if (base_variant == B2C_VARIANT_CP_TMA) {
-      CUDA_TRY(launch_pack_activations(x, scratch, d.N, d.C, d.H, d.W, p->C_pad, st, p->status));
+      CUDA_TRY(launch_pack_activations(x, scratch, d.N, d.C, d.H, d.W, p->C_pad, st, p->status, dbg));
     } else if (base_variant == B2C_VARIANT_DILATION_PACK) {
       const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
       CUDA_TRY(launch_phase_split(x, scratch, d.N, d.C, d.H, d.W, d.dil_h, d.dil_w, v.H, v.W, v.C, a.x_stride_n,
-                                  nchw ? (long long)d.H * d.W : 1, a.x_stride_h, a.x_stride_w, st));
+                                  nchw ? (long long)d.H * d.W : 1, a.x_stride_h, a.x_stride_w, st, dbg));
     } else if (base_variant == B2C_VARIANT_ROWPHASE_SHIFT) {
       const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
       CUDA_TRY(launch_row_phase_unroll(x, scratch, v.N, v.H, v.W, d.C, d.H, d.W, d.S, d.stride_h, d.stride_w, d.pad_h,
                                        d.pad_w, d.dil_w, v.C, a.x_stride_n, nchw ? (long long)d.H * d.W : 1,
-                                       a.x_stride_h, a.x_stride_w, st));
+                                       a.x_stride_h, a.x_stride_w, st, dbg));
     } else if (base_variant == B2C_VARIANT_ROW_UNROLL) {
       // scratch pixel (n, h, q): window origin (h, q*stride_w - pad_w), channels (s, c)
       CUDA_TRY(launch_im2col(x, scratch, p->table, (long long)v.N * v.H * v.W, v.H * v.W, v.W, d.H, d.W, 1,
-                             d.stride_w, 0, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w, v.C, st));
+                             d.stride_w, 0, d.pad_w, a.x_stride_n, a.x_stride_h, a.x_stride_w, v.C, st, dbg));
     } else {
       // space to depth: scratch pixel (n, h', w') holds the stride phases (c, dh, dw) of its window
       const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;
       CUDA_TRY(launch_space_to_depth(x, scratch, v.N, v.H, v.W, d.C, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
                                      v.C, s2d_pack_factor(g), a.x_stride_n, nchw ? (long long)d.H * d.W : 1,
-                                     a.x_stride_h, a.x_stride_w, st));
+                                     a.x_stride_h, a.x_stride_w, st, dbg));
     }
   } else if (p->emb.variant == B2C_VARIANT_IM2COL_EXPLICIT) {
     CUDA_TRY(launch_im2col(x, scratch, p->table, g.Mg, g.PQ, g.Q, d.H, d.W, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
-                           a.x_stride_n, a.x_stride_h, a.x_stride_w, p->K_pad, st));
+                           a.x_stride_n, a.x_stride_h, a.x_stride_w, p->K_pad, st, dbg));
   }
   return B2C_OK;
 }
@@ -910,6 +931,19 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   if (p->x_stride_n_whole) a.x_stride_n = p->x_stride_n_whole;
   if (p->y_stride_n_whole) a.y_stride_n = p->y_stride_n_whole;
   const bool act = p->bias != nullptr || p->relu != 0;
+  {
+    const long long shrink = g_dbg_shrink.load();
+    const long long y_span = (long long)(d.N - 1) * a.y_stride_n + (long long)d.K * g.PQ;
+    a.dbg.x_lo = x;
+    a.dbg.x_bytes = x ? (long long)(d.N - 1) * a.x_stride_n + (long long)d.C * d.H * d.W - shrink : 0;
+    a.dbg.o32_lo = y32;
+    a.dbg.o32_bytes = (y_span - shrink) * 4;
+    a.dbg.o8_lo = y8;
+    a.dbg.o8_bytes = y_span - shrink;
+    a.dbg.ws_lo = ws;
+    a.dbg.ws_bytes = (long long)p->ws_total - shrink;
+    a.dbg.status = p->status;
+  }
   CUtensorMap tmap_a;
   std::memset(&tmap_a, 0, sizeof(tmap_a));
   uint8_t* wsb = static_cast<uint8_t*>(ws);
@@ -966,7 +1000,7 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
     CUDA_TRY(launch_conv_mma(p->amode, &tmap_a, &p->tmap_b, a, st));
   if (need_finish)
     CUDA_TRY(launch_splitk_finish(a.acc, y32, y8, g.y_elems, d.shift, d.out_mode, p->bias, p->relu, d.K, g.PQ,
-                                  d.out_layout == B2C_LAYOUT_NHWC ? 1 : 0, st));
+                                  d.out_layout == B2C_LAYOUT_NHWC ? 1 : 0, st, a.dbg));
   return B2C_OK;
 }
 
@@ -981,10 +1015,26 @@ static int check_run_args(b2c_plan* p, const int8_t* x, bool need_x, int32_t* y3
   return B2C_OK;
 }
 
+// Debug build: the caller's workspace is [guard band][scratch][guard band]; every run repaints the
+// bands and uses the middle.
+static void* guard_workspace(b2c_plan* p, void* ws, cudaStream_t st, int* rc) {
+  *rc = B2C_OK;
+  if (kCanaryBytes == 0 || !ws || !p->ws_total) return ws;
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  if (cudaMemsetAsync(w, kCanaryByte, kCanaryBytes, st) != cudaSuccess ||
+      cudaMemsetAsync(w + kCanaryBytes + p->ws_total, kCanaryByte, kCanaryBytes, st) != cudaSuccess) {
+    set_last_cuda_error((int)cudaGetLastError());
+    *rc = B2C_E_CUDA;
+  }
+  return w + kCanaryBytes;
+}
+
 int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, void* ws, void* cuda_stream) {
   int rc = check_run_args(p, x, true, y32, y8, true, ws);
   if (rc != B2C_OK) return rc;
   cudaStream_t st = (cudaStream_t)cuda_stream;
+  ws = guard_workspace(p, ws, st, &rc);
+  if (rc != B2C_OK) return rc;
   if (!p->subs.empty()) {
     // one dense convolution per group on its channel slice of x (NCHW) and of y (NKPQ)
     const b2c_conv_desc& sd = p->subs[0]->g.d;
@@ -1006,6 +1056,8 @@ int b2c_plan_rewrite_activations(b2c_plan* p, const int8_t* x, void* ws, void* c
   int rc = check_run_args(p, x, true, nullptr, nullptr, false, ws);
   if (rc != B2C_OK) return rc;
   if (!p->subs.empty()) return B2C_OK;  // the group convolutions read x directly: nothing to rewrite
+  ws = guard_workspace(p, ws, (cudaStream_t)cuda_stream, &rc);
+  if (rc != B2C_OK) return rc;
   return run_rewrite(p, x, ws, (cudaStream_t)cuda_stream);
 }
 
@@ -1014,6 +1066,7 @@ int b2c_conv2d_int8_run_rewritten(b2c_plan* p, const int8_t* x, int32_t* y32, in
   int rc = check_run_args(p, x, p && p->ws_layout_bytes == 0, y32, y8, true, ws);
   if (rc != B2C_OK) return rc;
   if (!p->subs.empty()) return b2c_conv2d_int8_run(p, x, y32, y8, ws, cuda_stream);
+  if (kCanaryBytes && ws && p->ws_total) ws = static_cast<uint8_t*>(ws) + kCanaryBytes;  // bands painted by the rewrite half
   return run_convolve(p, x, y32, y8, ws, (cudaStream_t)cuda_stream);
 }
 
@@ -1051,8 +1104,14 @@ int b2c_plan_device_status(b2c_plan* p, int32_t* status) {
   // (a plain cudaMemcpy only orders against blocking streams; kernels of this plan may run on
   // non-blocking ones, so wait for the whole device first)
   CUDA_TRY(cudaDeviceSynchronize());
-  CUDA_TRY(cudaMemcpy(&s, p->status, sizeof(int), cudaMemcpyDeviceToHost));
-  if (s != 0) CUDA_TRY(cudaMemset(p->status, 0, sizeof(int)));
+  int words[kStatusWords] = {0, 0, 0, 0};
+  CUDA_TRY(cudaMemcpy(words, p->status, sizeof(words), cudaMemcpyDeviceToHost));
+  s = words[0];
+  if (s != 0) {
+    p->dbg_site = words[1];
+    p->dbg_offset = ((long long)words[3] << 32) | (unsigned int)words[2];
+    CUDA_TRY(cudaMemset(p->status, 0, sizeof(words)));
+  }
   for (b2c_plan* sub : p->subs) {  // a group plan reports the first sub-plan status that is set
     int32_t ss = 0;
     int rc = b2c_plan_device_status(sub, &ss);
@@ -1060,6 +1119,49 @@ int b2c_plan_device_status(b2c_plan* p, int32_t* status) {
     if (s == 0) s = ss;
   }
   *status = s;
+  return B2C_OK;
+}
+
+int b2c_debug_build(void) {
+#ifdef B2C_DEBUG_BOUNDS
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+int b2c_plan_debug_info(const b2c_plan* p, int32_t* site, int64_t* byte_offset) {
+  if (!p || !site || !byte_offset) return B2C_E_INVALID_ARG;
+  *site = p->dbg_site;
+  *byte_offset = p->dbg_offset;
+  for (const b2c_plan* sub : p->subs)
+    if (*site == 0 && sub->dbg_site != 0) {
+      *site = sub->dbg_site;
+      *byte_offset = sub->dbg_offset;
+    }
+  return B2C_OK;
+}
+
+int b2c_plan_check_canaries(b2c_plan* p, const void* workspace_dev, int32_t* intact) {
+  if (!p || !intact) return B2C_E_INVALID_ARG;
+  if (kCanaryBytes == 0) return B2C_E_UNSUPPORTED;
+  *intact = 1;
+  if (!p->ws_total) return B2C_OK;
+  if (!workspace_dev) return B2C_E_INVALID_ARG;
+  CUDA_TRY(cudaDeviceSynchronize());
+  unsigned char band[2][64];
+  const unsigned char* w = static_cast<const unsigned char*>(workspace_dev);
+  CUDA_TRY(cudaMemcpy(band[0], w, kCanaryBytes, cudaMemcpyDeviceToHost));
+  CUDA_TRY(cudaMemcpy(band[1], w + kCanaryBytes + p->ws_total, kCanaryBytes, cudaMemcpyDeviceToHost));
+  for (int b = 0; b < 2; ++b)
+    for (size_t i = 0; i < kCanaryBytes; ++i)
+      if (band[b][i] != kCanaryByte) *intact = 0;
+  return B2C_OK;
+}
+
+int b2c_test_shrink_checked_ranges(long long bytes) {
+  if (bytes < 0) return B2C_E_INVALID_ARG;
+  g_dbg_shrink.store(bytes);
   return B2C_OK;
 }
 
@@ -1134,7 +1236,7 @@ int b2c_conv2d_int8(int N, int C, int H, int W, int K, int R, int S, int stride,
     int rc = b2c_plan_create(&d, B2C_POLICY_AUTO_TIMED, cuda_stream, &p);
     if (rc != B2C_OK) return rc;
     if (p->ws_total) {
-      if (cudaMalloc(&p->own_ws, p->ws_total) != cudaSuccess) {
+      if (cudaMalloc(&p->own_ws, p->ws_total + 2 * kCanaryBytes) != cudaSuccess) {
         set_last_cuda_error((int)cudaGetLastError());
         b2c_plan_destroy(p);
         return B2C_E_CUDA;
@@ -1244,7 +1346,7 @@ static int create_pipe(b2c_plan* p) {
   CUDA_TRY(cudaStreamCreateWithFlags(&hp->s_in, cudaStreamNonBlocking));
   CUDA_TRY(cudaStreamCreateWithFlags(&hp->s_run, cudaStreamNonBlocking));
   CUDA_TRY(cudaStreamCreateWithFlags(&hp->s_out, cudaStreamNonBlocking));
-  if (p->ws_total) CUDA_TRY(cudaMalloc(&hp->ws, p->ws_total));
+  if (p->ws_total) CUDA_TRY(cudaMalloc(&hp->ws, p->ws_total + 2 * kCanaryBytes));
   for (HostPipe::Slot& sl : hp->slot) {
     CUDA_TRY(cudaMalloc((void**)&sl.x, hp->x_bytes + 256));
     if (d.out_mode & B2C_OUT_I32) CUDA_TRY(cudaMalloc((void**)&sl.y32, hp->y_elems * 4));

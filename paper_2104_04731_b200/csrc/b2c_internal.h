@@ -63,6 +63,21 @@ inline FastDiv make_fastdiv(uint32_t d) {
   return f;
 }
 
+// Debug build (-DB2C_DEBUG_BOUNDS, libb2conv_debug.so): the address ranges every hand-computed global
+// access of a kernel must stay inside.  A null `lo` leaves that range unchecked.  In the release build
+// the struct travels along unused and every check below compiles to `true`.
+struct Dbg {
+  const void* x_lo = nullptr;    // the tensor the kernel reads with its own loads or bulk copies
+  long long x_bytes = 0;
+  const void* o32_lo = nullptr;  // int32 output
+  long long o32_bytes = 0;
+  const void* o8_lo = nullptr;   // int8 output
+  long long o8_bytes = 0;
+  const void* ws_lo = nullptr;   // scratch the kernel writes (rewritten operand, split-reduction sums, counters)
+  long long ws_bytes = 0;
+  int* status = nullptr;         // [0] status word, [1] site, [2..3] byte offset of the first bad access from its range start
+};
+
 enum AMode { A_TILED = 0, A_IM2COL_TMA = 1, A_GATHER = 2, A_STAGED = 3, A_SHIFT = 4, A_WINDOW = 5 };
 
 // Everything the MMA kernel needs besides its two tensor maps.
@@ -141,6 +156,7 @@ struct ConvArgs {
   // wn_linear: tiles are 128 consecutive fused pixels, the window holds whole images (wn_box_bytes each,
   // behind a margin of wn_left bytes), taps outside the image are masked by the builders.
   int wn_tile_w, wn_win_w, wn_win_bytes, wn_box_bytes, wn_left, wn_off0, wn_chunks, wn_linear;
+  Dbg dbg;  // debug build: ranges of x, the outputs and the scratch
   FastDiv div_wps, div_hp;
   // elements between consecutive images of the NKPQ output (K * P * Q, or more when this
   // convolution writes one channel group of a wider tensor)
@@ -157,6 +173,32 @@ struct ConvArgs {
 // next kernel may begin its own set-up.  Every kernel of this library follows that rule, so the
 // stream order of memory effects is unchanged; what overlaps is launch latency and block set-up.
 #ifdef __CUDACC__
+#ifdef B2C_DEBUG_BOUNDS
+// True when [p, p + n) lies inside [lo, lo + bytes) (or the range is unchecked).  Otherwise the first
+// offender records B2C_E_BOUNDS, its site and its byte offset from the range start in the status
+// words, and the caller skips the access.
+__device__ __forceinline__ bool b2c_dbg_in_range(int* status, int site, const void* lo, long long bytes, const void* p,
+                                                 long long n) {
+  if (lo == nullptr) return true;
+  const long long off = (const char*)p - (const char*)lo;
+  if (off >= 0 && off + n <= bytes) return true;
+  if (status != nullptr && atomicCAS(status, 0, B2C_E_BOUNDS) == 0) {
+    status[1] = site;
+    status[2] = (int)(off & 0xFFFFFFFFLL);
+    status[3] = (int)(off >> 32);
+  }
+  return false;
+}
+#define B2C_X_OK(d, site, p, n) b2c_dbg_in_range((d).status, site, (d).x_lo, (d).x_bytes, p, n)
+#define B2C_O32_OK(d, site, p, n) b2c_dbg_in_range((d).status, site, (d).o32_lo, (d).o32_bytes, p, n)
+#define B2C_O8_OK(d, site, p, n) b2c_dbg_in_range((d).status, site, (d).o8_lo, (d).o8_bytes, p, n)
+#define B2C_WS_OK(d, site, p, n) b2c_dbg_in_range((d).status, site, (d).ws_lo, (d).ws_bytes, p, n)
+#else
+#define B2C_X_OK(d, site, p, n) true
+#define B2C_O32_OK(d, site, p, n) true
+#define B2C_O8_OK(d, site, p, n) true
+#define B2C_WS_OK(d, site, p, n) true
+#endif
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -331,7 +373,7 @@ int get_last_cuda_error();
 // --- kernel launchers (layout.cu, conv_mma.cu) -------------------------------------------------
 // status: device status word that a bounded wait of the kernel reports into, or nullptr
 cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, int H, int W, int C_pad,
-                                    cudaStream_t st, int* status);
+                                    cudaStream_t st, int* status, const Dbg& dbg = Dbg());
 cudaError_t launch_pack_weights_cp(const int8_t* w, int8_t* out, int K, int C, int R, int S, int C_pad,
                                    cudaStream_t st);
 cudaError_t launch_pack_weights_table(const int8_t* w, int8_t* out, int K, int Kg, int cols, const int32_t* table,
@@ -340,18 +382,19 @@ cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg
                                      cudaStream_t st);
 cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, long long Mg, int PQ, int Q, int H,
                           int W, int stride_h, int stride_w, int pad_h, int pad_w, long long x_stride_n,
-                          int x_stride_h, int x_stride_w, int K_pad, cudaStream_t st);
+                          int x_stride_h, int x_stride_w, int K_pad, cudaStream_t st, const Dbg& dbg = Dbg());
 cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, int Ws, int C, int H, int W, int sh,
                                   int sw, int pad_h, int pad_w, int C_pad, int pack, long long stride_n,
-                                  long long stride_c, int stride_h, int stride_w, cudaStream_t st);
+                                  long long stride_c, int stride_h, int stride_w, cudaStream_t st, const Dbg& dbg = Dbg());
 cudaError_t launch_row_phase_unroll(const int8_t* x, int8_t* out, int N, int Hs, int Q, int C, int H, int W, int S, int sh,
                                     int sw, int pad_h, int pad_w, int dil_w, int C_pad, long long stride_n,
-                                    long long stride_c, int stride_h, int stride_w, cudaStream_t st);
+                                    long long stride_c, int stride_h, int stride_w, cudaStream_t st, const Dbg& dbg = Dbg());
 cudaError_t launch_phase_split(const int8_t* x, int8_t* out, int N, int C, int H, int W, int dh, int dw, int Hs, int Ws,
                                int C_pad, long long stride_n, long long stride_c, int stride_h, int stride_w,
-                               cudaStream_t st);
+                               cudaStream_t st, const Dbg& dbg = Dbg());
 cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, long long elems, int shift,
-                                 int out_mode, const int32_t* bias, int relu, int K, int PQ, int nhwc, cudaStream_t st);
+                                 int out_mode, const int32_t* bias, int relu, int K, int PQ, int nhwc, cudaStream_t st,
+                                 const Dbg& dbg = Dbg());
 cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensorMap* tmap_b, const ConvArgs& args,
                             cudaStream_t st);
 size_t conv_mma_smem_bytes(int amode, const ConvArgs& args);

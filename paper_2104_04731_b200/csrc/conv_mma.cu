@@ -473,7 +473,8 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
               const GatherEntry g = te[jj * 16 + e];
               const int h = h0 + g.dh, ww = w0 + g.dw;
               uint32_t v = 0;
-              if (g.off >= 0 && (unsigned)h < (unsigned)args.H && (unsigned)ww < (unsigned)args.W)
+              if (g.off >= 0 && (unsigned)h < (unsigned)args.H && (unsigned)ww < (unsigned)args.W &&
+                  B2C_X_OK(args.dbg, 30, base + g.off, 1))
                 v = (uint8_t)__ldg(base + g.off);
               wv[e >> 2] |= v << (8 * (e & 3));
             }
@@ -528,11 +529,12 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         if (row_live && col0 < args.W && col0 + 16 > 0) {
           const int8_t* src = args.x + (size_t)(img0 + part) * args.x_stride_n + ((size_t)c * args.H + h) * args.W + col0;
           if (vec_ok && col0 >= 0 && col0 + 16 <= args.W) {
-            val = __ldg(reinterpret_cast<const uint4*>(src));
+            if (B2C_X_OK(args.dbg, 31, src, 16)) val = __ldg(reinterpret_cast<const uint4*>(src));
           } else {
             uint32_t wv[4] = {0, 0, 0, 0};
             for (int b = 0; b < 16; ++b)
-              if ((unsigned)(col0 + b) < (unsigned)args.W) wv[b >> 2] |= (uint32_t)(uint8_t)__ldg(src + b) << (8 * (b & 3));
+              if ((unsigned)(col0 + b) < (unsigned)args.W && B2C_X_OK(args.dbg, 31, src + b, 1))
+                wv[b >> 2] |= (uint32_t)(uint8_t)__ldg(src + b) << (8 * (b & 3));
             val = make_uint4(wv[0], wv[1], wv[2], wv[3]);
           }
         }
@@ -722,6 +724,20 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
           const int c = cb + b * kGatherWarps;
           const int k = n0 + col_base + c;
           if (c >= cols_slice || k >= args.K || rows_valid == 0) continue;
+#ifdef B2C_DEBUG_BOUNDS
+          {
+            // the rows_valid output elements of channel k this lane writes, first and last
+            const unsigned m_l = mrow + (unsigned)rows_valid - 1u;
+            const int n_l = (int)args.div_pq.div(m_l);
+            const long long first = nhwc ? (long long)mrow * args.K + k : ((long long)n_img * args.K + k) * args.PQ + pq;
+            const long long last = nhwc ? (long long)m_l * args.K + k
+                                        : ((long long)n_l * args.K + k) * args.PQ + (int)(m_l - (unsigned)n_l * (unsigned)args.PQ);
+            bool okb = true;
+            if (args.out_mode & B2C_OUT_I32) okb = B2C_O32_OK(args.dbg, 32, args.y32 + first, 4) && B2C_O32_OK(args.dbg, 32, args.y32 + last, 4);
+            if (okb && (args.out_mode & B2C_OUT_I8)) okb = B2C_O8_OK(args.dbg, 33, args.y8 + first, 1) && B2C_O8_OK(args.dbg, 33, args.y8 + last, 1);
+            if (!okb) continue;
+          }
+#endif
 #pragma unroll
           for (int i = 0; i < 4; ++i) acc[b][i] = activate(args, acc[b][i], k);
           if (!nhwc && one_image) {

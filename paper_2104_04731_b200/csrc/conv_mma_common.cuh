@@ -89,7 +89,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, Share
     if (ctl->abort_flag) return false;
     if (global_ns() - t0 > kWaitLimitNs) {
       ctl->abort_flag = 1;
-      atomicExch(status, B2C_E_TIMEOUT);
+      atomicCAS(status, 0, B2C_E_TIMEOUT);
       return false;
     }
   }
@@ -303,6 +303,23 @@ __device__ __forceinline__ void store_columns(const ConvArgs& args, int32_t* v, 
   const int K = args.K;
   if (!row_valid || kbase >= K) return;
   const bool nhwc = args.out_layout == B2C_LAYOUT_NHWC;
+#ifdef B2C_DEBUG_BOUNDS
+  {
+    // first and last element this call can touch, in each tensor it writes
+    const int cnt = min(NC, K - kbase);
+    const long long first = nhwc ? base_npqk + kbase : base_nkpq + (long long)kbase * args.out_PQ;
+    const long long last = nhwc ? first + cnt - 1 : first + (long long)(cnt - 1) * args.out_PQ;
+    bool ok = true;
+    if (args.split_k > 1 && !args.cluster_split) {
+      ok = (args.acc == args.y32 ? B2C_O32_OK(args.dbg, 20, args.acc + first, 4) && B2C_O32_OK(args.dbg, 20, args.acc + last, 4)
+                                 : B2C_WS_OK(args.dbg, 20, args.acc + first, 4) && B2C_WS_OK(args.dbg, 20, args.acc + last, 4));
+    } else {
+      if (args.out_mode & B2C_OUT_I32) ok = B2C_O32_OK(args.dbg, 21, args.y32 + first, 4) && B2C_O32_OK(args.dbg, 21, args.y32 + last, 4);
+      if (ok && (args.out_mode & B2C_OUT_I8)) ok = B2C_O8_OK(args.dbg, 22, args.y8 + first, 1) && B2C_O8_OK(args.dbg, 22, args.y8 + last, 1);
+    }
+    if (!ok) return;
+  }
+#endif
   if (args.split_k > 1 && !args.cluster_split) {
     // Partial sums of the reduction slices meet in global memory; integer addition is
     // associative, so the order of arrival does not change the result.
@@ -386,6 +403,25 @@ __device__ __forceinline__ void store_columns_swapped(const ConvArgs& args, int3
                                                       int m_first) {
   if (!row_valid || m_first >= args.Mg) return;
   const int count = min(16, args.Mg - m_first);
+#ifdef B2C_DEBUG_BOUNDS
+  {
+    // output elements of pixels m_first .. m_first + count - 1 in channel k, first and last
+    const bool nh = args.out_layout == B2C_LAYOUT_NHWC;
+    const int m_last = m_first + count - 1;
+    const int n0_ = (int)args.div_pq.div((uint32_t)m_first), n1_ = (int)args.div_pq.div((uint32_t)m_last);
+    const long long first = nh ? (long long)m_first * args.K + k : ((long long)n0_ * args.K + k) * args.PQ + (m_first - n0_ * args.PQ);
+    const long long last = nh ? (long long)m_last * args.K + k : ((long long)n1_ * args.K + k) * args.PQ + (m_last - n1_ * args.PQ);
+    bool ok = true;
+    if (args.split_k > 1) {
+      ok = (args.acc == args.y32 ? B2C_O32_OK(args.dbg, 23, args.acc + first, 4) && B2C_O32_OK(args.dbg, 23, args.acc + last, 4)
+                                 : B2C_WS_OK(args.dbg, 23, args.acc + first, 4) && B2C_WS_OK(args.dbg, 23, args.acc + last, 4));
+    } else {
+      if (args.out_mode & B2C_OUT_I32) ok = B2C_O32_OK(args.dbg, 24, args.y32 + first, 4) && B2C_O32_OK(args.dbg, 24, args.y32 + last, 4);
+      if (ok && (args.out_mode & B2C_OUT_I8)) ok = B2C_O8_OK(args.dbg, 25, args.y8 + first, 1) && B2C_O8_OK(args.dbg, 25, args.y8 + last, 1);
+    }
+    if (!ok) return;
+  }
+#endif
   const int n_img = (int)args.div_pq.div((uint32_t)m_first);
   int pq = m_first - n_img * args.PQ;
   const bool nhwc = args.out_layout == B2C_LAYOUT_NHWC;

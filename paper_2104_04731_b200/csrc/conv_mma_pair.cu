@@ -60,7 +60,7 @@ __device__ __noinline__ bool mbar_wait_cluster_slow(uint32_t bar, uint32_t parit
     if (ctl->abort_flag) return false;
     if (global_ns() - t0 > kWaitLimitNs) {
       ctl->abort_flag = 1;
-      atomicExch(status, B2C_E_TIMEOUT);
+      atomicCAS(status, 0, B2C_E_TIMEOUT);
       return false;
     }
   }
@@ -172,6 +172,15 @@ __device__ __forceinline__ void fused_pack_role(const ConvArgs& args, uint8_t* b
   auto start_batch = [&](int n, int c0, int hw0, int npx) {
     const int rows = max(0, min(CT, C - c0));
     if (rows == 0) return;
+#ifdef B2C_DEBUG_BOUNDS
+    // the whole source block of the batch (first byte of the first row .. last byte of the last row);
+    // a refused batch completes its barrier phase without copying, so that its consumer's wait ends
+    if (!B2C_X_OK(args.dbg, 40, args.pk_src + ((size_t)n * C + c0) * HW + hw0, (long long)(rows - 1) * HW + npx)) {
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+      __syncwarp();
+      return;
+    }
+#endif
     if (lane == 0)
       asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)(rows * npx)) : "memory");
     __syncwarp();
@@ -240,7 +249,8 @@ __device__ __forceinline__ void fused_pack_role(const ConvArgs& args, uint8_t* b
             const uint32_t hi = __byte_perm(w[4 * q + 2], w[4 * q + 3], j | ((4 + j) << 4));
             o[q] = __byte_perm(lo, hi, 0x5410);
           }
-          *reinterpret_cast<uint4*>(dst + (size_t)j * C_pad) = make_uint4(o[0], o[1], o[2], o[3]);
+          if (B2C_WS_OK(args.dbg, 41, dst + (size_t)j * C_pad, 16))
+            *reinterpret_cast<uint4*>(dst + (size_t)j * C_pad) = make_uint4(o[0], o[1], o[2], o[3]);
         }
       }
     }
@@ -278,7 +288,7 @@ __device__ __forceinline__ bool wait_images_packed(const ConvArgs& args, int m_f
         }
         if (global_ns() - t0 > kWaitLimitNs) {
           ctl->abort_flag = 1;
-          atomicExch(args.status, B2C_E_TIMEOUT);
+          atomicCAS(args.status, 0, B2C_E_TIMEOUT);
           ok = false;
           break;
         }

@@ -135,8 +135,14 @@ __global__ void __launch_bounds__(kWinThreads, 2)
         const int n_a = (int)args.div_pq.div((uint32_t)m0);
         const int n_b = (int)args.div_pq.div((uint32_t)min(m0 + kTileM - 1, args.Mg - 1));
         const uint32_t img_bytes = (uint32_t)args.wn_box_bytes;
-        mbar_arrive_expect_tx(full, (uint32_t)(n_b - n_a + 1) * img_bytes, leader);
+        int copies = n_b - n_a + 1;
+#ifdef B2C_DEBUG_BOUNDS
+        for (int n = n_a; n <= n_b; ++n)
+          if (!B2C_X_OK(args.dbg, 50, args.x + (size_t)n * img_bytes, img_bytes)) --copies;  // refused below: not expected
+#endif
+        mbar_arrive_expect_tx(full, (uint32_t)copies * img_bytes, leader);
         for (int n = n_a; n <= n_b; ++n) {
+          if (!B2C_X_OK(args.dbg, 50, args.x + (size_t)n * img_bytes, img_bytes)) continue;
           const uint32_t dst = win_base + (uint32_t)s * win_bytes + (uint32_t)args.wn_left + (uint32_t)(n - n_a) * img_bytes;
           asm volatile(
               "{\n.reg .pred q;\nsetp.ne.b32 q, %4, 0;\n"

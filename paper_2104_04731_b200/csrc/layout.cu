@@ -27,7 +27,7 @@ constexpr int kPackSmem = kPackMaxC * (kPackMaxP + 4) + (kPackMaxC / 16) * 16;
 template <int VEC>
 __global__ void __launch_bounds__(kPackThreads) pack_activations_kernel(const int8_t* __restrict__ x,
                                                                         int8_t* __restrict__ out, int C, int HW,
-                                                                        int C_pad, int hw_tiles, int CT, int PT) {
+                                                                        int C_pad, int hw_tiles, int CT, int PT, Dbg dbg) {
   __shared__ __align__(16) uint8_t tile[kPackSmem];
   const int n = blockIdx.x / hw_tiles;
   const int c0 = blockIdx.y * CT;
@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_kernel(const in
       for (int k = 0; k < NW; ++k) v[k] = 0;
       if (row < rows) {
         const int8_t* src = xin + (size_t)row * HW + hw;
-        if (hw0 + hw + VEC <= HW) {
+        if (hw0 + hw + VEC <= HW && B2C_X_OK(dbg, 1, src, VEC)) {
           if constexpr (VEC == 16) {
             const uint4 q = *reinterpret_cast<const uint4*>(src);
             v[0] = q.x;
@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_kernel(const in
           }
         } else {
           for (int b = 0; b < VEC; ++b)
-            if (hw0 + hw + b < HW) v[b >> 2] |= (uint32_t)(uint8_t)src[b] << (8 * (b & 3));
+            if (hw0 + hw + b < HW && B2C_X_OK(dbg, 1, src + b, 1)) v[b >> 2] |= (uint32_t)(uint8_t)src[b] << (8 * (b & 3));
         }
       }
       uint32_t* dst = reinterpret_cast<uint32_t*>(&tile[row * pitch + (row >> 4) * 16 + hw]);
@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_kernel(const in
       const int row = i / PT;
       const int hw = i - row * PT;
       uint8_t v = 0;
-      if (row < rows && hw0 + hw < HW) v = (uint8_t)xin[(size_t)row * HW + hw];
+      if (row < rows && hw0 + hw < HW && B2C_X_OK(dbg, 1, xin + (size_t)row * HW + hw, 1)) v = (uint8_t)xin[(size_t)row * HW + hw];
       tile[row * pitch + (row >> 4) * 16 + hw] = v;
     }
   }
@@ -109,7 +109,8 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_kernel(const in
           const uint32_t hi = __byte_perm(w[4 * k + 2], w[4 * k + 3], j | ((4 + j) << 4));
           o[k] = __byte_perm(lo, hi, 0x5410);
         }
-        *reinterpret_cast<uint4*>(dst + (size_t)j * C_pad) = make_uint4(o[0], o[1], o[2], o[3]);
+        if (B2C_WS_OK(dbg, 2, dst + (size_t)j * C_pad, 16))
+          *reinterpret_cast<uint4*>(dst + (size_t)j * C_pad) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
   }
@@ -152,7 +153,7 @@ __device__ __forceinline__ bool pack_wait_bounded(uint32_t bar, int* status, boo
     }
   }
   if (!done) {
-    if (reporter && status != nullptr) atomicExch(status, B2C_E_TIMEOUT);
+    if (reporter && status != nullptr) atomicCAS(status, 0, B2C_E_TIMEOUT);
     const unsigned long long t1 = pack_global_ns();
     while (pack_global_ns() - t1 < 50000ull) __nanosleep(1000);
   }
@@ -177,7 +178,7 @@ template <bool kRowMode>
 __global__ void __launch_bounds__(kPackThreads) pack_activations_bulk_kernel(const int8_t* __restrict__ x,
                                                                              int8_t* __restrict__ out, int C, int HW,
                                                                              int C_pad, int hw_tiles, int CT, int PT,
-                                                                             int* status) {
+                                                                             int* status, Dbg dbg) {
   extern __shared__ __align__(128) uint8_t btile[];
   __shared__ __align__(8) unsigned long long bar;
   const int n = blockIdx.x / hw_tiles;
@@ -200,21 +201,29 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_bulk_kernel(con
   pdl_wait();
   const int8_t* xin = x + ((size_t)n * C + c0) * HW + hw0;
   if (kRowMode) {
-    if (t < rows) {
+    if (t < rows && B2C_X_OK(dbg, 3, xin + (size_t)t * HW, npx)) {
       const uint32_t dst = tile_a + (uint32_t)((t >> 4) * gs + (t & 15) * rp);
       asm volatile(
           "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
           "l"(xin + (size_t)t * HW), "r"((uint32_t)npx), "r"(bar_a)
           : "memory");
     }
+#ifdef B2C_DEBUG_BOUNDS
+    else if (t < rows)  // a refused copy: account for its bytes so that the barrier still completes
+      asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_a), "r"((uint32_t)npx) : "memory");
+#endif
   } else {
-    if (t < (rows >> 4)) {
+    if (t < (rows >> 4) && B2C_X_OK(dbg, 3, xin + (size_t)t * 16 * HW, 16 * HW)) {
       const uint32_t dst = tile_a + (uint32_t)(t * gs);
       asm volatile(
           "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
           "l"(xin + (size_t)t * 16 * HW), "r"((uint32_t)(16 * HW)), "r"(bar_a)
           : "memory");
     }
+#ifdef B2C_DEBUG_BOUNDS
+    else if (t < (rows >> 4))
+      asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_a), "r"((uint32_t)(16 * HW)) : "memory");
+#endif
   }
   // Bounded wait for the copies (every thread polls the barrier).  On expiry the block records
   // B2C_E_TIMEOUT in the status word (when the caller gave one), leaves the copies that were issued
@@ -252,7 +261,8 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_bulk_kernel(con
           const uint32_t hi = __byte_perm(w[4 * k + 2], w[4 * k + 3], j | ((4 + j) << 4));
           o[k] = __byte_perm(lo, hi, 0x5410);
         }
-        *reinterpret_cast<uint4*>(dst + (size_t)j * C_pad) = make_uint4(o[0], o[1], o[2], o[3]);
+        if (B2C_WS_OK(dbg, 2, dst + (size_t)j * C_pad, 16))
+          *reinterpret_cast<uint4*>(dst + (size_t)j * C_pad) = make_uint4(o[0], o[1], o[2], o[3]);
       }
     }
   }
@@ -306,7 +316,8 @@ __global__ void pack_weights_rows_kernel(const int8_t* __restrict__ w, int8_t* _
 __global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a,
                                                      const GatherEntry* __restrict__ table, long long Mg, int PQ, int Q,
                                                      int H, int W, int stride_h, int stride_w, int pad_h, int pad_w,
-                                                     long long x_stride_n, int x_stride_h, int x_stride_w, int K_pad) {
+                                                     long long x_stride_n, int x_stride_h, int x_stride_w, int K_pad,
+                                                     Dbg dbg) {
   const int chunks = K_pad >> 4;
   const long long total = Mg * chunks;
   pdl_wait();
@@ -325,10 +336,12 @@ __global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ 
       const GatherEntry g = table[ck * 16 + e];
       const int h = h0 + g.dh, ww = w0 + g.dw;
       uint32_t v = 0;
-      if (g.off >= 0 && (unsigned)h < (unsigned)H && (unsigned)ww < (unsigned)W) v = (uint8_t)base[g.off];
+      if (g.off >= 0 && (unsigned)h < (unsigned)H && (unsigned)ww < (unsigned)W && B2C_X_OK(dbg, 4, base + g.off, 1))
+        v = (uint8_t)base[g.off];
       wv[e >> 2] |= v << (8 * (e & 3));
     }
-    *reinterpret_cast<uint4*>(a + m * K_pad + ck * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+    if (B2C_WS_OK(dbg, 5, a + m * K_pad + ck * 16, 16))
+      *reinterpret_cast<uint4*>(a + m * K_pad + ck * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
   }
   pdl_launch_dependents();
 }
@@ -340,7 +353,7 @@ __global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ 
 __global__ void __launch_bounds__(256) phase_split_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ out, int N,
                                                           int C, int H, int W, int dh, int dw, int Hs, int Ws, int C_pad,
                                                           long long stride_n, long long stride_c, int stride_h,
-                                                          int stride_w) {
+                                                          int stride_w, Dbg dbg) {
   const int chunks = C_pad >> 4;
   const long long total = (long long)N * dh * dw * Hs * Ws * chunks;
   pdl_wait();
@@ -362,10 +375,11 @@ __global__ void __launch_bounds__(256) phase_split_kernel(const int8_t* __restri
 #pragma unroll
       for (int e = 0; e < 16; ++e) {
         const int c = ck * 16 + e;
-        if (c < C) wv[e >> 2] |= (uint32_t)(uint8_t)src[c * stride_c] << (8 * (e & 3));
+        if (c < C && B2C_X_OK(dbg, 6, src + c * stride_c, 1)) wv[e >> 2] |= (uint32_t)(uint8_t)src[c * stride_c] << (8 * (e & 3));
       }
     }
-    *reinterpret_cast<uint4*>(out + pix * C_pad + ck * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+    if (B2C_WS_OK(dbg, 7, out + pix * C_pad + ck * 16, 16))
+      *reinterpret_cast<uint4*>(out + pix * C_pad + ck * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
   }
   pdl_launch_dependents();
 }
@@ -380,7 +394,7 @@ __global__ void __launch_bounds__(256) space_to_depth_kernel(const int8_t* __res
                                                              FastDiv div_hs, int C, int H, int W, int sh, int sw,
                                                              int pad_h, int pad_w, int C_pad, int pack,
                                                              long long stride_n, int stride_c, int stride_h,
-                                                             int stride_w) {
+                                                             int stride_w, Dbg dbg) {
   // (32-bit indices and multiply-shift divisions: a 64-bit division costs more than the 16 bytes moved)
   const int chunks = (int)div_chunks.d, Ws = (int)div_ws.d, Hs = (int)div_hs.d;
   const int creal = pack * C * sh * sw;  // a column's own phases plus those of its pack - 1 right neighbours
@@ -406,7 +420,8 @@ __global__ void __launch_bounds__(256) space_to_depth_kernel(const int8_t* __res
 #pragma unroll
       for (int e = 0; e < 16; ++e) {
         const int h = h0 + dh, w = w0 + within;
-        if (c < C && (unsigned)h < (unsigned)H && (unsigned)w < (unsigned)W)
+        if (c < C && (unsigned)h < (unsigned)H && (unsigned)w < (unsigned)W &&
+            B2C_X_OK(dbg, 8, base + c * stride_c + h * stride_h + w * stride_w, 1))
           wv[e >> 2] |= (uint32_t)(uint8_t)base[c * stride_c + h * stride_h + w * stride_w] << (8 * (e & 3));
         if (++within == run_len) {
           within = 0;
@@ -417,7 +432,8 @@ __global__ void __launch_bounds__(256) space_to_depth_kernel(const int8_t* __res
         }
       }
     }
-    *reinterpret_cast<uint4*>(out + (size_t)i * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+    if (B2C_WS_OK(dbg, 9, out + (size_t)i * 16, 16))
+      *reinterpret_cast<uint4*>(out + (size_t)i * 16) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
   }
   pdl_launch_dependents();
 }
@@ -431,7 +447,7 @@ __global__ void __launch_bounds__(kS2dTile) space_to_depth_rows_kernel(const int
                                                                        int8_t* __restrict__ out, int Hs, int Ws, int C,
                                                                        int H, int W, int sh, int sw, int pad_h,
                                                                        int pad_w, int C_pad, int pack, int seg,
-                                                                       int ws_tiles) {
+                                                                       int ws_tiles, Dbg dbg) {
   extern __shared__ __align__(16) uint8_t s2d_rows[];
   const int tile = blockIdx.x % ws_tiles;
   const int rowi = blockIdx.x / ws_tiles;  // (n, hs)
@@ -448,13 +464,14 @@ __global__ void __launch_bounds__(kS2dTile) space_to_depth_rows_kernel(const int
     const int h = hs * sh + dh - pad_h;
     const int w = walign + v * 16;
     uint4 val = make_uint4(0, 0, 0, 0);
-    if ((unsigned)h < (unsigned)H && w >= 0 && w + 16 <= W)
-      val = __ldg(reinterpret_cast<const uint4*>(x + (((size_t)n * C + c) * H + h) * W + w));
-    else if ((unsigned)h < (unsigned)H && w + 16 > 0 && w < W) {
+    if ((unsigned)h < (unsigned)H && w >= 0 && w + 16 <= W) {
+      if (B2C_X_OK(dbg, 10, x + (((size_t)n * C + c) * H + h) * W + w, 16))
+        val = __ldg(reinterpret_cast<const uint4*>(x + (((size_t)n * C + c) * H + h) * W + w));
+    } else if ((unsigned)h < (unsigned)H && w + 16 > 0 && w < W) {
       uint32_t wv[4] = {0, 0, 0, 0};
       const int8_t* src = x + (((size_t)n * C + c) * H + h) * W;
       for (int b = 0; b < 16; ++b)
-        if ((unsigned)(w + b) < (unsigned)W) wv[b >> 2] |= (uint32_t)(uint8_t)src[w + b] << (8 * (b & 3));
+        if ((unsigned)(w + b) < (unsigned)W && B2C_X_OK(dbg, 10, src + w + b, 1)) wv[b >> 2] |= (uint32_t)(uint8_t)src[w + b] << (8 * (b & 3));
       val = make_uint4(wv[0], wv[1], wv[2], wv[3]);
     }
     *reinterpret_cast<uint4*>(s2d_rows + (size_t)r * seg + v * 16) = val;
@@ -500,7 +517,7 @@ __global__ void __launch_bounds__(kS2dTile) space_to_depth_rows_kernel(const int
         }
       }
     }
-    *reinterpret_cast<uint4*>(dst + j0) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+    if (B2C_WS_OK(dbg, 11, dst + j0, 16)) *reinterpret_cast<uint4*>(dst + j0) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
   }
 }
 
@@ -515,7 +532,7 @@ __global__ void __launch_bounds__(kS2dTile) row_phase_unroll_kernel(const int8_t
                                                                     int sw, int pad_h, int pad_w, int dil_w, int C_pad,
                                                                     int seg, int q_tiles, long long stride_n,
                                                                     long long stride_c, int stride_h, int stride_w,
-                                                                    int vec_ok) {
+                                                                    int vec_ok, Dbg dbg) {
   extern __shared__ __align__(16) uint8_t rp_rows[];
   const int tile = blockIdx.x % q_tiles;
   const int rowi = blockIdx.x / q_tiles;  // (n, hs)
@@ -535,12 +552,13 @@ __global__ void __launch_bounds__(kS2dTile) row_phase_unroll_kernel(const int8_t
       const int w = walign + v * 16;
       uint4 val = make_uint4(0, 0, 0, 0);
       if ((unsigned)h < (unsigned)H && w >= 0 && w + 16 <= W) {
-        val = __ldg(reinterpret_cast<const uint4*>(xn + c * stride_c + (long long)h * stride_h + w));
+        if (B2C_X_OK(dbg, 12, xn + c * stride_c + (long long)h * stride_h + w, 16))
+          val = __ldg(reinterpret_cast<const uint4*>(xn + c * stride_c + (long long)h * stride_h + w));
       } else if ((unsigned)h < (unsigned)H && w + 16 > 0 && w < W) {
         uint32_t wv[4] = {0, 0, 0, 0};
         const int8_t* src = xn + c * stride_c + (long long)h * stride_h;
         for (int b = 0; b < 16; ++b)
-          if ((unsigned)(w + b) < (unsigned)W) wv[b >> 2] |= (uint32_t)(uint8_t)src[w + b] << (8 * (b & 3));
+          if ((unsigned)(w + b) < (unsigned)W && B2C_X_OK(dbg, 12, src + w + b, 1)) wv[b >> 2] |= (uint32_t)(uint8_t)src[w + b] << (8 * (b & 3));
         val = make_uint4(wv[0], wv[1], wv[2], wv[3]);
       }
       *reinterpret_cast<uint4*>(rp_rows + (size_t)r * seg + v * 16) = val;
@@ -552,7 +570,8 @@ __global__ void __launch_bounds__(kS2dTile) row_phase_unroll_kernel(const int8_t
       const int h = hs * sh + dh - pad_h;
       const int w = walign + b;
       uint8_t val = 0;
-      if ((unsigned)h < (unsigned)H && (unsigned)w < (unsigned)W)
+      if ((unsigned)h < (unsigned)H && (unsigned)w < (unsigned)W &&
+          B2C_X_OK(dbg, 12, xn + c * stride_c + (long long)h * stride_h + (long long)w * stride_w, 1))
         val = (uint8_t)xn[c * stride_c + (long long)h * stride_h + (long long)w * stride_w];
       rp_rows[(size_t)r * seg + b] = val;
     }
@@ -580,7 +599,7 @@ __global__ void __launch_bounds__(kS2dTile) row_phase_unroll_kernel(const int8_t
         }
       }
     }
-    *reinterpret_cast<uint4*>(dst + j0) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+    if (B2C_WS_OK(dbg, 13, dst + j0, 16)) *reinterpret_cast<uint4*>(dst + j0) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
   }
 }
 
@@ -588,17 +607,18 @@ __global__ void __launch_bounds__(kS2dTile) row_phase_unroll_kernel(const int8_t
 // the shift-and-clip requantisation (arithmetic shift = floor division by 2^shift).
 __global__ void splitk_finish_kernel(const int32_t* __restrict__ acc, int32_t* __restrict__ y32,
                                      int8_t* __restrict__ y8, long long elems, int shift, int out_mode,
-                                     const int32_t* __restrict__ bias, int relu, int K, int PQ, int nhwc) {
+                                     const int32_t* __restrict__ bias, int relu, int K, int PQ, int nhwc, Dbg dbg) {
   pdl_wait();
   pdl_launch_dependents();
   const bool act = bias != nullptr || relu != 0;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < elems;
        i += (long long)gridDim.x * blockDim.x) {
+    if (!(acc == y32 ? B2C_O32_OK(dbg, 14, acc + i, 4) : B2C_WS_OK(dbg, 14, acc + i, 4))) continue;
     int v = acc[i];
     if (bias != nullptr) v += bias[nhwc ? (int)(i % K) : (int)((i / PQ) % K)];  // output channel of element i
     if (relu) v = max(v, 0);
-    if ((out_mode & B2C_OUT_I32) && (y32 != acc || act)) y32[i] = v;
-    if (out_mode & B2C_OUT_I8) y8[i] = (int8_t)max(-128, min(127, v >> shift));
+    if ((out_mode & B2C_OUT_I32) && (y32 != acc || act) && B2C_O32_OK(dbg, 15, y32 + i, 4)) y32[i] = v;
+    if ((out_mode & B2C_OUT_I8) && B2C_O8_OK(dbg, 16, y8 + i, 1)) y8[i] = (int8_t)max(-128, min(127, v >> shift));
   }
 }
 
@@ -611,7 +631,7 @@ int grid_for(long long total, int block) {
 }  // namespace
 
 cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, int H, int W, int C_pad,
-                                    cudaStream_t st, int* status) {
+                                    cudaStream_t st, int* status, const Dbg& dbg) {
   const int HW = H * W;
   int CT = C_pad >= 128 ? 128 : 64;
   const bool a16 = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
@@ -627,20 +647,20 @@ cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, 
     dim3 grid((unsigned)hw_tiles * (unsigned)N, (C_pad + CT - 1) / CT, 1);
     if (row_mode)
       return launch_pdl(pack_activations_bulk_kernel<true>, grid, dim3(kPackThreads), smem, st, x, out, C, HW, C_pad,
-                        hw_tiles, CT, PT, status);
+                        hw_tiles, CT, PT, status, dbg);
     return launch_pdl(pack_activations_bulk_kernel<false>, grid, dim3(kPackThreads), smem, st, x, out, C, HW, C_pad,
-                      hw_tiles, CT, PT, status);
+                      hw_tiles, CT, PT, status, dbg);
   }
   const int PT = HW > 128 ? 256 : (HW > 64 ? 128 : 64);
   const int hw_tiles = (HW + PT - 1) / PT;
   dim3 grid((unsigned)hw_tiles * (unsigned)N, (C_pad + CT - 1) / CT, 1);
   if ((HW % 16) == 0 && a16)
     return launch_pdl(pack_activations_kernel<16>, grid, dim3(kPackThreads), 0, st, x, out, C, HW, C_pad, hw_tiles, CT,
-                      PT);
+                      PT, dbg);
   if ((HW % 4) == 0 && a16)
     return launch_pdl(pack_activations_kernel<4>, grid, dim3(kPackThreads), 0, st, x, out, C, HW, C_pad, hw_tiles, CT,
-                      PT);
-  return launch_pdl(pack_activations_kernel<1>, grid, dim3(kPackThreads), 0, st, x, out, C, HW, C_pad, hw_tiles, CT, PT);
+                      PT, dbg);
+  return launch_pdl(pack_activations_kernel<1>, grid, dim3(kPackThreads), 0, st, x, out, C, HW, C_pad, hw_tiles, CT, PT, dbg);
 }
 
 cudaError_t launch_pack_wait_selftest(int* status, cudaStream_t st) {
@@ -671,15 +691,15 @@ cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg
 
 cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, long long Mg, int PQ, int Q, int H,
                           int W, int stride_h, int stride_w, int pad_h, int pad_w, long long x_stride_n,
-                          int x_stride_h, int x_stride_w, int K_pad, cudaStream_t st) {
+                          int x_stride_h, int x_stride_w, int K_pad, cudaStream_t st, const Dbg& dbg) {
   const long long total = Mg * (K_pad / 16);
   return launch_pdl(im2col_kernel, dim3(grid_for(total, 256)), dim3(256), 0, st, x, a, table, Mg, PQ, Q, H, W, stride_h,
-                    stride_w, pad_h, pad_w, x_stride_n, x_stride_h, x_stride_w, K_pad);
+                    stride_w, pad_h, pad_w, x_stride_n, x_stride_h, x_stride_w, K_pad, dbg);
 }
 
 cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, int Ws, int C, int H, int W, int sh,
                                   int sw, int pad_h, int pad_w, int C_pad, int pack, long long stride_n,
-                                  long long stride_c, int stride_h, int stride_w, cudaStream_t st) {
+                                  long long stride_c, int stride_h, int stride_w, cudaStream_t st, const Dbg& dbg) {
   // Fast path: NCHW rows that are multiples of 16 bytes, row segments of a tile within 48 KB.
   const int seg = ((kS2dTile * sw + pack * sw + 15 + 15) / 16) * 16;  // bytes of one input row a tile reads, from a 16-byte boundary
   const long long smem = (long long)C * sh * seg;
@@ -687,7 +707,7 @@ cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, i
   if (stride_w == 1 && stride_h == W && stride_c == (long long)H * W && (W % 16) == 0 &&
       (reinterpret_cast<uintptr_t>(x) & 15) == 0 && smem <= 48 * 1024 && blocks < 0x7FFFFFFFLL && Ws >= 32)
     return launch_pdl(space_to_depth_rows_kernel, dim3((unsigned)blocks), dim3(kS2dTile), (size_t)smem, st, x, out, Hs, Ws, C,
-                      H, W, sh, sw, pad_h, pad_w, C_pad, pack, seg, (Ws + kS2dTile - 1) / kS2dTile);
+                      H, W, sh, sw, pad_h, pad_w, C_pad, pack, seg, (Ws + kS2dTile - 1) / kS2dTile, dbg);
   // total 16-byte chunks of the scratch tensor; the planner keeps N*Hs*Ws*C_pad below 2^40 and one
   // image below 2^31 bytes, and the launch below is split so that each part's chunk count fits 32 bits
   const long long per_image = (long long)Hs * Ws * (C_pad / 16);
@@ -698,7 +718,7 @@ cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, i
     cudaError_t e = launch_pdl(space_to_depth_kernel, dim3(grid_for(total, 256)), dim3(256), 0, st,
                                x + (long long)n0 * stride_n, out + (long long)n0 * per_image * 16, (unsigned)total,
                                make_fastdiv((uint32_t)(C_pad / 16)), make_fastdiv((uint32_t)Ws), make_fastdiv((uint32_t)Hs),
-                               C, H, W, sh, sw, pad_h, pad_w, C_pad, pack, stride_n, (int)stride_c, stride_h, stride_w);
+                               C, H, W, sh, sw, pad_h, pad_w, C_pad, pack, stride_n, (int)stride_c, stride_h, stride_w, dbg);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
@@ -706,7 +726,7 @@ cudaError_t launch_space_to_depth(const int8_t* x, int8_t* out, int N, int Hs, i
 
 cudaError_t launch_row_phase_unroll(const int8_t* x, int8_t* out, int N, int Hs, int Q, int C, int H, int W, int S, int sh,
                                     int sw, int pad_h, int pad_w, int dil_w, int C_pad, long long stride_n,
-                                    long long stride_c, int stride_h, int stride_w, cudaStream_t st) {
+                                    long long stride_c, int stride_h, int stride_w, cudaStream_t st, const Dbg& dbg) {
   // bytes of one input row a tile of kS2dTile pixels reads, counted from a 16-byte boundary
   static_assert(kRowPhaseTile == kS2dTile, "one pixel per thread");
   const int seg = row_phase_seg(sw, S, dil_w);
@@ -722,21 +742,22 @@ cudaError_t launch_row_phase_unroll(const int8_t* x, int8_t* out, int N, int Hs,
   cudaError_t ea = set_max_dynamic_smem_once(configured, (const void*)row_phase_unroll_kernel, kRowPhaseSmemMax);
   if (ea != cudaSuccess) return ea;
   return launch_pdl(row_phase_unroll_kernel, dim3((unsigned)blocks), dim3(kS2dTile), (size_t)smem, st, x, out, Hs, Q, C, H,
-                    W, S, sh, sw, pad_h, pad_w, dil_w, C_pad, seg, q_tiles, stride_n, stride_c, stride_h, stride_w, vec_ok);
+                    W, S, sh, sw, pad_h, pad_w, dil_w, C_pad, seg, q_tiles, stride_n, stride_c, stride_h, stride_w, vec_ok, dbg);
 }
 
 cudaError_t launch_phase_split(const int8_t* x, int8_t* out, int N, int C, int H, int W, int dh, int dw, int Hs, int Ws,
                                int C_pad, long long stride_n, long long stride_c, int stride_h, int stride_w,
-                               cudaStream_t st) {
+                               cudaStream_t st, const Dbg& dbg) {
   const long long total = (long long)N * dh * dw * Hs * Ws * (C_pad / 16);
   return launch_pdl(phase_split_kernel, dim3(grid_for(total, 256)), dim3(256), 0, st, x, out, N, C, H, W, dh, dw, Hs, Ws,
-                    C_pad, stride_n, stride_c, stride_h, stride_w);
+                    C_pad, stride_n, stride_c, stride_h, stride_w, dbg);
 }
 
 cudaError_t launch_splitk_finish(const int32_t* acc, int32_t* y32, int8_t* y8, long long elems, int shift,
-                                 int out_mode, const int32_t* bias, int relu, int K, int PQ, int nhwc, cudaStream_t st) {
+                                 int out_mode, const int32_t* bias, int relu, int K, int PQ, int nhwc, cudaStream_t st,
+                                 const Dbg& dbg) {
   return launch_pdl(splitk_finish_kernel, dim3(grid_for(elems, 256)), dim3(256), 0, st, acc, y32, y8, elems, shift,
-                    out_mode, bias, relu, K, PQ, nhwc);
+                    out_mode, bias, relu, K, PQ, nhwc, dbg);
 }
 
 }  // namespace b2c
