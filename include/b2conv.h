@@ -141,9 +141,11 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
  * C / groups channels and sums over the input channels of its own group only; the weight tensor
  * given to b2c_plan_set_weights is int8 [K][C / groups][R][S]; groups == C == K is depth-wise.
  * desc.in_layout and desc.out_layout must be B2C_LAYOUT_NCHW (UNSUPPORTED otherwise; INVALID_ARG when
- * groups < 1 or does not divide C and K).  The plan runs one dense convolution per group on that
- * group's channel slice of x and y in place (no scratch: b2c_plan_workspace_bytes is 0), each with
- * the lowest-overhead stencil unroll formed inside the kernel; b2c_plan_info reports that embedding.
+ * groups < 1 or does not divide C and K).  The plan runs all groups in ONE launch of the MMA kernel
+ * (the group is a grid axis: every block convolves its group's channel slice of x into that
+ * group's slice of y in place, with the filters of all groups packed once into one matrix; no
+ * scratch: b2c_plan_workspace_bytes is 0), with the lowest-overhead stencil unroll formed inside
+ * the kernel; b2c_plan_info reports that embedding.
  * All other plan calls (set_weights, set_activation with K bias values, run, device_status, destroy)
  * apply as to any plan; the rewrite / run_rewritten halves are no-op and run respectively. */
 int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan** out);

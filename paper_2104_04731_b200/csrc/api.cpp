@@ -44,6 +44,7 @@ struct b2c_plan {
   // y through the batch strides of the whole tensors); the group plan itself launches nothing.
   int groups = 1;
   std::vector<b2c_plan*> subs;
+  int group_count = 1;  // on the sub-plan of a group plan: groups run by one launch (blockIdx.z = group)
   long long x_stride_n_whole = 0, y_stride_n_whole = 0;  // sub-plans: batch strides of the whole tensors
   struct HostPipe* pipe = nullptr;  // streaming host-buffer calls: created by the first b2c_plan_run_host_async
   // The two-SM persistent channel-pack schedule can run the activation pack inside the MMA kernel
@@ -172,6 +173,8 @@ void fill_common_args(b2c_plan* p) {
   a.table32 = p->table32;
   a.swap = is_swapped(p->emb) ? 1 : 0;
   a.y_stride_n = (long long)d.K * p->g.PQ;
+  a.groups = p->group_count;
+  a.group_x_stride = (long long)d.C * d.H * d.W;
   a.out_PQ = p->g.PQ;
   a.out_P = p->g.P;
   a.out_Q = p->g.Q;
@@ -308,7 +311,8 @@ void fill_common_args(b2c_plan* p) {
   int per_cta_kb = (a.num_kb + a.split_k - 1) / a.split_k;
   int stages = std::min(6, std::max(1, per_cta_kb));
   const long long ctas = a.swap ? ((p->g.Mg + a.tile_n - 1) / a.tile_n) * ((d.K + kTileM - 1) / kTileM) * a.split_k
-                                : (((long long)a.Mg + kTileM - 1) / kTileM) * ((d.K + a.tile_n - 1) / a.tile_n) * a.split_k;
+                                : (((long long)a.Mg + kTileM - 1) / kTileM) * ((d.K + a.tile_n - 1) / a.tile_n) * a.split_k *
+                                      p->group_count;
   // Large TMA-fed problems run persistently: one block per SM walks the tile list with two
   // accumulator buffers in tensor memory and the deepest stage ring that fits.
   const long long tiles_m = ((long long)a.Mg + kTileM - 1) / kTileM;
@@ -393,11 +397,12 @@ void fill_common_args(b2c_plan* p) {
   a.stages = stages;
 }
 
-int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
+int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out, int group_count = 1) {
   b2c_plan* p = new (std::nothrow) b2c_plan();
   if (!p) return B2C_E_INVALID_ARG;
   p->g = g;
   p->emb = emb;
+  p->group_count = group_count;
   cudaGetDevice(&p->device);
   const b2c_conv_desc& d = g.d;
   auto fail = [&](int code) {
@@ -465,7 +470,7 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
     }
   } else {
     int K_pad = variant_k_pad(g, emb.variant);
-    p->w_packed_bytes = (size_t)d.K * K_pad;
+    p->w_packed_bytes = (size_t)d.K * K_pad * group_count;  // grouped: the filters of all groups, one block of K rows each
     std::vector<GatherEntry> t;
     build_table(g, K_pad, &t);
     p->table_len = K_pad;
@@ -484,6 +489,17 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
         t32[wi] = ((run / d.R) * wt.win_h + (run % d.R) * d.dil_h) * wt.win_w + s0;
         // linear tiles: + the filter row (bits 16-23) and the word of the run (bits 24-31) for the masks
         if (wt.linear) t32[wi] |= ((run % d.R) << 16) | ((s0 >> 2) << 24);
+      }
+      if (!wt.linear) {
+        // two-dimensional tiles: the low two bits of a chunk's first entry say how its four words lie
+        // (offsets are multiples of 4): 0 = 16 consecutive bytes, 1 = two runs of 8 bytes, 2 = anything else
+        for (int ch = 0; ch + 3 < (int)t32.size(); ch += 4) {
+          const int o0 = t32[ch], o1 = t32[ch + 1], o2 = t32[ch + 2], o3 = t32[ch + 3];
+          int kind = 2;
+          if (o1 == o0 + 4 && o2 == o0 + 8 && o3 == o0 + 12) kind = 0;
+          else if (o1 == o0 + 4 && o3 == o2 + 4) kind = 1;
+          t32[ch] = o0 | kind;
+        }
       }
       p->table_len = (int)t32.size();
       if (cudaMalloc(&p->table32, t32.size() * sizeof(int32_t)) != cudaSuccess) return fail(B2C_E_CUDA);
@@ -538,7 +554,7 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out) {
     uint64_t cols = (uint64_t)p->view.R * p->view.S * p->view.C;
     rc = encode_tiled_2d(&p->tmap_b, p->w_packed, cols, d.K, cols, p->bk, w_box_rows, p->bk);
   } else {
-    rc = encode_tiled_2d(&p->tmap_b, p->w_packed, p->K_pad, d.K, p->K_pad, 128, w_box_rows, 128);
+    rc = encode_tiled_2d(&p->tmap_b, p->w_packed, p->K_pad, (uint64_t)d.K * group_count, p->K_pad, 128, w_box_rows, 128);
   }
   if (rc != B2C_OK) return fail(rc);
   *out = p;
@@ -805,17 +821,16 @@ int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan*
     b2c_plan_destroy(p);
     return B2C_E_CUDA;
   }
-  for (int gi = 0; gi < groups; ++gi) {
-    b2c_plan* sub = nullptr;
-    rc = create_plan_for(sg, all[pick], &sub);
-    if (rc != B2C_OK) {
-      b2c_plan_destroy(p);
-      return rc;
-    }
-    sub->x_stride_n_whole = (long long)desc->C * desc->H * desc->W;
-    sub->y_stride_n_whole = (long long)desc->K * sg.PQ;
-    p->subs.push_back(sub);
+  // one sub-plan runs all groups in one launch (the group is a grid axis of the kernel)
+  b2c_plan* sub = nullptr;
+  rc = create_plan_for(sg, all[pick], &sub, groups);
+  if (rc != B2C_OK) {
+    b2c_plan_destroy(p);
+    return rc;
   }
+  sub->x_stride_n_whole = (long long)desc->C * desc->H * desc->W;
+  sub->y_stride_n_whole = (long long)desc->K * sg.PQ;
+  p->subs.push_back(sub);
   *out = p;
   return B2C_OK;
 }
@@ -840,12 +855,9 @@ int b2c_plan_set_weights(b2c_plan* p, const int8_t* w, void* cuda_stream) {
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (!p->subs.empty()) {
     // w is [K][C/groups][R][S]: group g's filters are the g-th block of K/groups rows
-    const b2c_conv_desc& sd = p->subs[0]->g.d;
-    const size_t per_group = (size_t)sd.K * sd.C * sd.R * sd.S;
-    for (size_t gi = 0; gi < p->subs.size(); ++gi) {
-      int rc = set_weights_one(p->subs[gi], w + gi * per_group, st);
-      if (rc != B2C_OK) return rc;
-    }
+    // (one pack launch: the rows of all groups have the same format)
+    int rc = set_weights_one(p->subs[0], w, st);
+    if (rc != B2C_OK) return rc;
     p->weights_set = true;
     return B2C_OK;
   }
@@ -860,7 +872,7 @@ static int set_weights_one(b2c_plan* p, const int8_t* w, cudaStream_t st) {
   else if (is_tma_view_variant(p->emb.variant))
     CUDA_TRY(launch_pack_weights_table(w, p->w_packed, d.K, p->g.Kg, p->view.R * p->view.S * p->view.C, p->wtable, st));
   else
-    CUDA_TRY(launch_pack_weights_rows(w, p->w_packed, d.K, p->g.Kg, p->K_pad, d.S,
+    CUDA_TRY(launch_pack_weights_rows(w, p->w_packed, d.K * p->group_count, p->g.Kg, p->K_pad, d.S,
                                       p->emb.variant == B2C_VARIANT_IM2COL_STAGED
                                           ? staged_run_len(p->g)
                                           : (p->emb.variant == B2C_VARIANT_IM2COL_WINDOW ? round_up(d.S, 4) : d.S),
@@ -933,9 +945,9 @@ static int run_convolve(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   const bool act = p->bias != nullptr || p->relu != 0;
   {
     const long long shrink = g_dbg_shrink.load();
-    const long long y_span = (long long)(d.N - 1) * a.y_stride_n + (long long)d.K * g.PQ;
+    const long long y_span = (long long)(d.N - 1) * a.y_stride_n + (long long)d.K * g.PQ * a.groups;
     a.dbg.x_lo = x;
-    a.dbg.x_bytes = x ? (long long)(d.N - 1) * a.x_stride_n + (long long)d.C * d.H * d.W - shrink : 0;
+    a.dbg.x_bytes = x ? (long long)(d.N - 1) * a.x_stride_n + (long long)d.C * d.H * d.W * a.groups - shrink : 0;
     a.dbg.o32_lo = y32;
     a.dbg.o32_bytes = (y_span - shrink) * 4;
     a.dbg.o8_lo = y8;
@@ -1036,15 +1048,8 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   ws = guard_workspace(p, ws, st, &rc);
   if (rc != B2C_OK) return rc;
   if (!p->subs.empty()) {
-    // one dense convolution per group on its channel slice of x (NCHW) and of y (NKPQ)
-    const b2c_conv_desc& sd = p->subs[0]->g.d;
-    const size_t x_slice = (size_t)sd.C * sd.H * sd.W, y_slice = (size_t)sd.K * p->subs[0]->g.PQ;
-    for (size_t gi = 0; gi < p->subs.size(); ++gi) {
-      rc = run_convolve(p->subs[gi], x + gi * x_slice, y32 ? y32 + gi * y_slice : nullptr, y8 ? y8 + gi * y_slice : nullptr,
-                        nullptr, st);
-      if (rc != B2C_OK) return rc;
-    }
-    return B2C_OK;
+    // one launch: every group convolves its channel slice of x (NCHW) into its slice of y (NKPQ)
+    return run_convolve(p->subs[0], x, y32, y8, nullptr, st);
   }
   if (p->fused_pack && aligned16(x)) return run_convolve(p, x, y32, y8, ws, st, /*fused_pack=*/true);
   rc = run_rewrite(p, x, ws, st);
@@ -1083,9 +1088,9 @@ int b2c_plan_set_activation(b2c_plan* p, const int32_t* bias_dev, int relu, void
   }
   p->relu = relu;
   // group plans: every group takes its own K/groups entries of the copy
-  for (size_t gi = 0; gi < p->subs.size(); ++gi) {
-    p->subs[gi]->bias = p->bias ? p->bias + gi * (size_t)p->subs[gi]->g.d.K : nullptr;
-    p->subs[gi]->relu = relu;
+  for (b2c_plan* sub : p->subs) {  // (the kernel indexes the bias by group)
+    sub->bias = p->bias;
+    sub->relu = relu;
   }
   return B2C_OK;
 }

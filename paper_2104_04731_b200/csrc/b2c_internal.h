@@ -156,6 +156,11 @@ struct ConvArgs {
   // wn_linear: tiles are 128 consecutive fused pixels, the window holds whole images (wn_box_bytes each,
   // behind a margin of wn_left bytes), taps outside the image are masked by the builders.
   int wn_tile_w, wn_win_w, wn_win_bytes, wn_box_bytes, wn_left, wn_off0, wn_chunks, wn_linear;
+  // Grouped convolution in one launch (in-kernel stencil unroll, NCHW / NKPQ): blockIdx.z is the group;
+  // group g reads channels [g*C, (g+1)*C) of x (group_x_stride elements further on per group), uses rows
+  // [g*K, (g+1)*K) of the packed weights and of the bias, and writes output channels [g*K, (g+1)*K).
+  int groups;
+  long long group_x_stride;
   Dbg dbg;  // debug build: ranges of x, the outputs and the scratch
   FastDiv div_wps, div_hp;
   // elements between consecutive images of the NKPQ output (K * P * Q, or more when this
@@ -348,6 +353,7 @@ bool staged_word_mode(const Geom& g);
 int staged_run_len(const Geom& g);  // taps per (c, r) run after padding
 int variant_k_pad(const Geom& g, int variant);  // padded reduction length of the stencil-unroll variants
 
+constexpr int kWindowStages = 6;  // input windows in flight per block of the window unroll kernel
 // Geometry of the TMA-staged window unroll (B2C_VARIANT_IM2COL_WINDOW); false if it does not apply.
 struct WindowTile {
   int tile_w, tile_h, win_w, win_h, left, off0, S_run, K_pad, tiles_h, tiles_w, box_bytes, win_bytes, tile_n, num_kb;

@@ -60,8 +60,11 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     m0 = (int)blockIdx.x * kTileM;                                                  \
     n0 = (int)blockIdx.y * args.tile_n;                                             \
   }
-  const int kb_begin = (int)((unsigned)blockIdx.z * (unsigned)args.num_kb / (unsigned)args.split_k);
-  const int kb_end = (int)((unsigned)(blockIdx.z + 1) * (unsigned)args.num_kb / (unsigned)args.split_k);
+  // blockIdx.z: reduction slice of a split reduction, or the group of a grouped convolution (never both)
+  const int grp = args.groups > 1 ? (int)blockIdx.z : 0;
+  const unsigned zslice = args.groups > 1 ? 0u : blockIdx.z;
+  const int kb_begin = (int)(zslice * (unsigned)args.num_kb / (unsigned)args.split_k);
+  const int kb_end = (int)((zslice + 1u) * (unsigned)args.num_kb / (unsigned)args.split_k);
   const int stages = args.stages;
   const int bk = args.bk;
   const uint32_t a_stage_bytes = AMODE == A_SHIFT ? (uint32_t)args.sh_win_bytes : (uint32_t)(kTileM * bk);
@@ -225,7 +228,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         const uint32_t full = smem_u32(&ctl.full[s]);
         if (kThreadsFormA) {
           mbar_arrive_expect_tx(full, b_stage_bytes, leader);
-          tma_load_2d(b_dst, &tmap_b, kcol, n0, full, leader);
+          tma_load_2d(b_dst, &tmap_b, kcol, n0 + grp * args.K, full, leader);
         } else if (AMODE == A_TILED) {
           mbar_arrive_expect_tx(full, a_stage_bytes + b_stage_bytes, leader);
           tma_load_2d(swap ? b_dst : a_dst, &tmap_a, kcol, pix0, full, leader);
@@ -451,7 +454,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
       const int p = (int)args.div_q.div((uint32_t)pq), q = pq - p * args.Q;
       const int h0 = row_valid ? p * args.stride_h - args.pad_h : -(1 << 29);
       const int w0 = q * args.stride_w - args.pad_w;
-      const int8_t* base = args.x + n_img * args.x_stride_n + (long long)(row_valid ? h0 : 0) * args.x_stride_h +
+      const int8_t* base = args.x + grp * args.group_x_stride + n_img * args.x_stride_n + (long long)(row_valid ? h0 : 0) * args.x_stride_h +
                            (long long)w0 * args.x_stride_w;
       const uint32_t row_off = (uint32_t)row * 128u;
       const uint32_t xr = (uint32_t)(row & 7);
@@ -527,7 +530,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         const int col0 = v16 * 16 - args.win_left;  // image column of the first byte of this vector
         uint4 val = make_uint4(0, 0, 0, 0);
         if (row_live && col0 < args.W && col0 + 16 > 0) {
-          const int8_t* src = args.x + (size_t)(img0 + part) * args.x_stride_n + ((size_t)c * args.H + h) * args.W + col0;
+          const int8_t* src = args.x + grp * args.group_x_stride + (size_t)(img0 + part) * args.x_stride_n + ((size_t)c * args.H + h) * args.W + col0;
           if (vec_ok && col0 >= 0 && col0 + 16 <= args.W) {
             if (B2C_X_OK(args.dbg, 31, src, 16)) val = __ldg(reinterpret_cast<const uint4*>(src));
           } else {
@@ -625,7 +628,7 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
       // Output index of (m, k): NKPQ -> (n*K + k)*PQ + pq ; NPQK -> m*K + k.
-      const long long base_nkpq = (long long)out_img * args.y_stride_n + out_pq;
+      const long long base_nkpq = (long long)out_img * args.y_stride_n + out_pq + (long long)grp * args.K * args.out_PQ;
       const long long base_npqk = args.remap ? ((long long)out_img * args.out_PQ + out_pq) * args.K : (long long)m * args.K;
       const int cols = alternate ? args.tile_n : (args.tile_n >= 32 ? (args.tile_n >> 1) : 16);  // columns handled by this warp
       const int c_begin = alternate ? 0 : half * cols;
@@ -645,11 +648,11 @@ __global__ void __launch_bounds__(kThreads, PERSIST == 1 ? 1 : 3) conv_mma_kerne
         } else if ((cols & 31) == 0) {
           for (int c = 0; c < cols; c += 32)
             epilogue_columns<32>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk,
-                                 xch ? xch + (uint32_t)c * (kTileM * 4) : 0u);
+                                 xch ? xch + (uint32_t)c * (kTileM * 4) : 0u, grp * args.K);
         } else {
           for (int c = 0; c < cols; c += 16)
             epilogue_columns<16>(args, taddr + (uint32_t)c, n0 + c_begin + c, row_valid, base_nkpq, base_npqk,
-                                 xch ? xch + (uint32_t)c * (kTileM * 4) : 0u);
+                                 xch ? xch + (uint32_t)c * (kTileM * 4) : 0u, grp * args.K);
         }
       }
       if (persistent) {
@@ -844,6 +847,7 @@ cudaError_t launch_conv_mma(int amode, const CUtensorMap* tmap_a, const CUtensor
     const int per_sm = args.persistent_blocks_per_sm > 0 ? args.persistent_blocks_per_sm : (args.persistent == 2 ? 3 : 1);
     grid = dim3((unsigned)std::min(args.num_tiles, kNumSMs * per_sm), 1, 1);
   }
+  if (args.groups > 1) grid.z = (unsigned)args.groups;  // (grouped plans never split the reduction)
   cudaError_t e;
 #define B2C_LAUNCH(MODE, PERS)                                                                             \
   {                                                                                                       \

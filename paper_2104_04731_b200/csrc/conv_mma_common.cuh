@@ -299,7 +299,7 @@ __device__ __forceinline__ void tmem_ld<32>(uint32_t taddr, int32_t* v) {
 // are added into a zeroed int32 buffer instead.
 template <int NC>
 __device__ __forceinline__ void store_columns(const ConvArgs& args, int32_t* v, int kbase, bool row_valid,
-                                              long long base_nkpq, long long base_npqk) {
+                                              long long base_nkpq, long long base_npqk, int bias_off = 0) {
   const int K = args.K;
   if (!row_valid || kbase >= K) return;
   const bool nhwc = args.out_layout == B2C_LAYOUT_NHWC;
@@ -335,7 +335,7 @@ __device__ __forceinline__ void store_columns(const ConvArgs& args, int32_t* v, 
   if (args.bias != nullptr || args.relu) {
 #pragma unroll
     for (int j = 0; j < NC; ++j)
-      if (kbase + j < K) v[j] = activate(args, v[j], kbase + j);
+      if (kbase + j < K) v[j] = activate(args, v[j], bias_off + kbase + j);
   }
   if (!nhwc) {
     // NKPQ: for a fixed column the 32 lanes of a warp hold 32 consecutive pixels, so every
@@ -500,7 +500,8 @@ __device__ __forceinline__ void store_columns_swapped(const ConvArgs& args, int3
 
 template <int NC>
 __device__ __forceinline__ void epilogue_columns(const ConvArgs& args, uint32_t taddr, int kbase, bool row_valid,
-                                                 long long base_nkpq, long long base_npqk, uint32_t exchange_addr) {
+                                                 long long base_nkpq, long long base_npqk, uint32_t exchange_addr,
+                                                 int bias_off = 0) {
   int32_t v[NC];
   __syncwarp();
   tmem_ld<NC>(taddr, v);  // warp-collective: executed by all lanes
@@ -511,7 +512,7 @@ __device__ __forceinline__ void epilogue_columns(const ConvArgs& args, uint32_t 
       asm volatile("st.shared.b32 [%0], %1;" ::"r"(exchange_addr + (uint32_t)j * (kTileM * 4)), "r"(v[j]) : "memory");
     return;
   }
-  store_columns<NC>(args, v, kbase, row_valid, base_nkpq, base_npqk);
+  store_columns<NC>(args, v, kbase, row_valid, base_nkpq, base_npqk, bias_off);
 }
 
 }  // namespace

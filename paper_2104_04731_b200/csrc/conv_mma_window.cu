@@ -32,9 +32,28 @@ namespace {
 constexpr int kBuildWarps = 8;   // warps 2..9
 constexpr int kEpiWarps = 4;     // warps 10..13 (one per tensor-memory lane quadrant)
 constexpr int kWinThreads = 64 + 32 * (kBuildWarps + kEpiWarps);
-constexpr int kWinStages = 3;    // input windows in flight
+constexpr int kWinStages = kWindowStages;  // input windows in flight
 constexpr int kABufs = 2;        // A operand buffers
 
+// Bounded wait with back-off: the roles of this kernel wait for whole tiles (a microsecond or so), and
+// fourteen warps polling shared-memory barriers compete with the builders for the same memory pipe, so
+// a waiting warp sleeps between polls.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, SharedCtl* ctl, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  while (true) {
+    __nanosleep(100);
+    if (mbar_try_wait(bar, parity)) return true;
+    if (ctl->abort_flag) return false;
+    if (global_ns() - t0 > kWaitLimitNs) {
+      ctl->abort_flag = 1;
+      atomicCAS(status, 0, B2C_E_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+static_assert(kWinStages <= 8, "one lane per window barrier");
 struct __align__(8) WindowCtl {
   unsigned long long win_full[kWinStages];
   unsigned long long win_empty[kWinStages];
@@ -78,20 +97,20 @@ __global__ void __launch_bounds__(kWinThreads, 2)
       mbar_init(smem_u32(&wc.win_full[lane]), 1);
       mbar_init(smem_u32(&wc.win_empty[lane]), kBuildWarps);
     }
-    if (lane >= 4 && lane < 4 + kABufs) {
-      mbar_init(smem_u32(&wc.a_full[lane - 4]), kBuildWarps);
-      mbar_init(smem_u32(&wc.a_empty[lane - 4]), 1);
+    if (lane >= 8 && lane < 8 + kABufs) {
+      mbar_init(smem_u32(&wc.a_full[lane - 8]), kBuildWarps);
+      mbar_init(smem_u32(&wc.a_empty[lane - 8]), 1);
     }
-    if (lane >= 8 && lane < 12) {
-      mbar_init(smem_u32(&wc.tmem_full[lane - 8]), 1);
-      mbar_init(smem_u32(&wc.tmem_empty[lane - 8]), kEpiWarps);
+    if (lane >= 12 && lane < 16) {
+      mbar_init(smem_u32(&wc.tmem_full[lane - 12]), 1);
+      mbar_init(smem_u32(&wc.tmem_empty[lane - 12]), kEpiWarps);
     }
-    if (lane == 12) {
+    if (lane == 16) {
       mbar_init(smem_u32(&wc.w_full), 1);
       ctl->abort_flag = 0;
     }
-    if (lane == 13) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
-    if (lane == 14) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+    if (lane == 17) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+    if (lane == 18) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -127,7 +146,7 @@ __global__ void __launch_bounds__(kWinThreads, 2)
     int s = 0;
     uint32_t ph = 0;
     for (int t = tile_first; t < tile_end; t += tile_step) {
-      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&wc.win_empty[s]), ph ^ 1u, ctl, args.status))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait_relaxed(smem_u32(&wc.win_empty[s]), ph ^ 1u, ctl, args.status))) break;
       const uint32_t full = smem_u32(&wc.win_full[s]);
       if (LINEAR) {
         // the whole images of the tile's 128 pixels, one bulk copy each, behind the window's margin
@@ -213,8 +232,8 @@ __global__ void __launch_bounds__(kWinThreads, 2)
     for (int t = tile_first; t < tile_end && ok; t += tile_step, ++ti) {
       const int ab = ti & (kABufs - 1);
       const uint32_t a_use = (uint32_t)(ti / kABufs);
-      ok = mbar_wait(smem_u32(&wc.a_empty[ab]), (a_use & 1u) ^ 1u, ctl, args.status);
-      if (ok) ok = mbar_wait(smem_u32(&wc.win_full[s]), ph, ctl, args.status);
+      ok = mbar_wait_relaxed(smem_u32(&wc.a_empty[ab]), (a_use & 1u) ^ 1u, ctl, args.status);
+      if (ok) ok = mbar_wait_relaxed(smem_u32(&wc.win_full[s]), ph, ctl, args.status);
       if (!ok) break;
       if (LINEAR) {
         // this row's pixel (n, p, q); rows past the last pixel build from the window's first image (never stored)
@@ -265,22 +284,62 @@ __global__ void __launch_bounds__(kWinThreads, 2)
           const uint32_t dst = a_row + (uint32_t)(ch >> 3) * a_block_bytes + ((((uint32_t)ch & 7u) ^ xr) << 4);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(wv[0]), "r"(wv[1]), "r"(wv[2]), "r"(wv[3]));
         }
-      } else
-      for (int ch = half; ch < nchunks; ch += 2) {
-        // the four words of this chunk: window offsets from the table (the same for the whole warp)
-        const int4 off = *reinterpret_cast<const int4*>(s_table + ch * 4);
-        uint32_t lo0 = *reinterpret_cast<const uint32_t*>(win + off.x);
-        uint32_t hi0 = *reinterpret_cast<const uint32_t*>(win + off.x + 4);
-        uint32_t lo1 = off.y == off.x + 4 ? hi0 : *reinterpret_cast<const uint32_t*>(win + off.y);
-        uint32_t hi1 = *reinterpret_cast<const uint32_t*>(win + off.y + 4);
-        uint32_t lo2 = off.z == off.y + 4 ? hi1 : *reinterpret_cast<const uint32_t*>(win + off.z);
-        uint32_t hi2 = *reinterpret_cast<const uint32_t*>(win + off.z + 4);
-        uint32_t lo3 = off.w == off.z + 4 ? hi2 : *reinterpret_cast<const uint32_t*>(win + off.w);
-        uint32_t hi3 = *reinterpret_cast<const uint32_t*>(win + off.w + 4);
-        const uint32_t w0 = __byte_perm(lo0, hi0, sel), w1 = __byte_perm(lo1, hi1, sel);
-        const uint32_t w2 = __byte_perm(lo2, hi2, sel), w3 = __byte_perm(lo3, hi3, sel);
-        const uint32_t dst = a_row + (uint32_t)(ch >> 3) * a_block_bytes + ((((uint32_t)ch & 7u) ^ xr) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w0), "r"(w1), "r"(w2), "r"(w3));
+      } else {
+        // 32-bit shared-memory addresses and explicit ld.shared: no generic-pointer arithmetic in the loop.
+        // The table gives each chunk's four word offsets; the low two bits of the first say how they lie:
+        // 0 = one run of 16 consecutive bytes (five aligned loads), 1 = two runs of 8 (three loads each),
+        // 2 = four separate words.
+        const uint32_t win_s = win_base + (uint32_t)s * win_bytes + (uint32_t)tbase4;
+        const uint32_t tab_s = win_base + kWinStages * win_bytes;
+        for (int ch = half; ch < nchunks; ch += 2) {
+          uint32_t o0, o1, o2, o3;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(o0), "=r"(o1), "=r"(o2), "=r"(o3) : "r"(tab_s + (uint32_t)ch * 16u));
+          const uint32_t kind = o0 & 3u;
+          const uint32_t a0 = win_s + (o0 & ~3u);
+          uint32_t w0, w1, w2, w3;
+          if (kind == 0u) {
+            uint32_t v0, v1, v2, v3, v4;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v0) : "r"(a0));
+            asm volatile("ld.shared.b32 %0, [%1+4];" : "=r"(v1) : "r"(a0));
+            asm volatile("ld.shared.b32 %0, [%1+8];" : "=r"(v2) : "r"(a0));
+            asm volatile("ld.shared.b32 %0, [%1+12];" : "=r"(v3) : "r"(a0));
+            asm volatile("ld.shared.b32 %0, [%1+16];" : "=r"(v4) : "r"(a0));
+            w0 = __byte_perm(v0, v1, sel);
+            w1 = __byte_perm(v1, v2, sel);
+            w2 = __byte_perm(v2, v3, sel);
+            w3 = __byte_perm(v3, v4, sel);
+          } else if (kind == 1u) {
+            const uint32_t a2 = win_s + o2;
+            uint32_t v0, v1, v2, u0, u1, u2;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v0) : "r"(a0));
+            asm volatile("ld.shared.b32 %0, [%1+4];" : "=r"(v1) : "r"(a0));
+            asm volatile("ld.shared.b32 %0, [%1+8];" : "=r"(v2) : "r"(a0));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(u0) : "r"(a2));
+            asm volatile("ld.shared.b32 %0, [%1+4];" : "=r"(u1) : "r"(a2));
+            asm volatile("ld.shared.b32 %0, [%1+8];" : "=r"(u2) : "r"(a2));
+            w0 = __byte_perm(v0, v1, sel);
+            w1 = __byte_perm(v1, v2, sel);
+            w2 = __byte_perm(u0, u1, sel);
+            w3 = __byte_perm(u1, u2, sel);
+          } else {
+            const uint32_t a1 = win_s + o1, a2 = win_s + o2, a3 = win_s + o3;
+            uint32_t l0, h0, l1, h1, l2, h2, l3, h3;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(l0) : "r"(a0));
+            asm volatile("ld.shared.b32 %0, [%1+4];" : "=r"(h0) : "r"(a0));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(l1) : "r"(a1));
+            asm volatile("ld.shared.b32 %0, [%1+4];" : "=r"(h1) : "r"(a1));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(l2) : "r"(a2));
+            asm volatile("ld.shared.b32 %0, [%1+4];" : "=r"(h2) : "r"(a2));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(l3) : "r"(a3));
+            asm volatile("ld.shared.b32 %0, [%1+4];" : "=r"(h3) : "r"(a3));
+            w0 = __byte_perm(l0, h0, sel);
+            w1 = __byte_perm(l1, h1, sel);
+            w2 = __byte_perm(l2, h2, sel);
+            w3 = __byte_perm(l3, h3, sel);
+          }
+          const uint32_t dst = a_row + (uint32_t)(ch >> 3) * a_block_bytes + ((((uint32_t)ch & 7u) ^ xr) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w0), "r"(w1), "r"(w2), "r"(w3));
+        }
       }
       // the window has been read; the A rows are visible to the tensor core's async proxy
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -319,7 +378,7 @@ __global__ void __launch_bounds__(kWinThreads, 2)
       }
       const int tb = ti & (nbuf - 1);
       const uint32_t t_use = (uint32_t)(ti >> nbuf_log2);
-      ok = mbar_wait(smem_u32(&wc.tmem_full[tb]), t_use & 1u, ctl, args.status);
+      ok = mbar_wait_relaxed(smem_u32(&wc.tmem_full[tb]), t_use & 1u, ctl, args.status);
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       if (!ok) break;
       const long long base_nkpq = (long long)img * args.y_stride_n + out_pq;

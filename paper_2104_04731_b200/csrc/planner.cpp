@@ -337,7 +337,7 @@ bool window_tile_geom(const Geom& g, WindowTile* wt) {
   while (wt->tile_n < d.K) wt->tile_n <<= 1;
   // small images: linear tiles over whole images (no padded positions at all)
   if (((d.W % 16) != 0 || g.PQ <= 1024) && window_linear_geom(g, wt)) {
-    wt->smem = 1024 + 2 * (size_t)wt->num_kb * kTileM * 128 + (size_t)wt->num_kb * wt->tile_n * 128 + 3 * (size_t)wt->win_bytes +
+    wt->smem = 1024 + 2 * (size_t)wt->num_kb * kTileM * 128 + (size_t)wt->num_kb * wt->tile_n * 128 + kWindowStages * (size_t)wt->win_bytes +
                (size_t)round_up(wt->K_pad, 128) + 256;
     return wt->mtot <= 0x7FFFFF00LL && wt->smem <= 200 * 1024;
   }
@@ -369,7 +369,7 @@ bool window_tile_geom(const Geom& g, WindowTile* wt) {
   wt->box_bytes = d.C * wt->win_h * wt->win_w;
   wt->win_bytes = round_up(wt->box_bytes + 32, 128);
   wt->mtot = (long long)d.N * wt->tiles_h * wt->tiles_w * kTileM;
-  wt->smem = 1024 + 2 * (size_t)wt->num_kb * kTileM * 128 + (size_t)wt->num_kb * wt->tile_n * 128 + 3 * (size_t)wt->win_bytes +
+  wt->smem = 1024 + 2 * (size_t)wt->num_kb * kTileM * 128 + (size_t)wt->num_kb * wt->tile_n * 128 + kWindowStages * (size_t)wt->win_bytes +
              (size_t)round_up(wt->K_pad, 128) + 256;
   return wt->mtot <= 0x7FFFFF00LL && wt->smem <= 200 * 1024 && (long long)d.N * wt->tiles_h * wt->tiles_w < 0x7FFFFFFFLL;
 }

@@ -397,7 +397,7 @@ def test_shift_execution_four_accumulator_buffers(lib):
     check_against_oracle(x, w, 1, 1, 1, 10, 3, e.id, ref=ref)
 
 
-# ---- grouped / depth-wise convolution: one dense convolution per group on channel slices in place --------
+# ---- grouped / depth-wise convolution: one launch, the group is a grid axis of the kernel ------------------
 @pytest.mark.parametrize("case", [
     # N, C, H, W, K, groups, R, S, stride, pad, dil, shift, out_mode
     (2, 8, 12, 16, 12, 2, 3, 3, 1, 1, 1, 6, 3),         # two groups of 4 -> 6 channels, rows of 16 bytes
@@ -405,6 +405,8 @@ def test_shift_execution_four_accumulator_buffers(lib):
     (2, 6, 10, 10, 6, 6, 3, 3, 1, 1, 1, 4, 1),          # depth-wise, int32 only
     (1, 16, 20, 20, 16, 16, 5, 5, 2, 2, 1, 5, 2),       # depth-wise 5x5 stride 2, int8 only
     (2, 64, 7, 7, 128, 2, 1, 1, 1, 0, 1, 7, 3),         # pointwise, 64 output channels per group
+    (2, 256, 14, 14, 256, 256, 3, 3, 1, 1, 1, 4, 3),    # depth-wise, 256 channels: 256 groups in one launch
+    (40, 32, 28, 28, 64, 8, 3, 3, 2, 1, 1, 6, 3),       # many tiles per group: the persistent walk with a group axis
 ])
 def test_grouped_convolution(lib, case):
     N, C, H, W, K, groups, R, S, stride, pad, dil, shift, out_mode = case
