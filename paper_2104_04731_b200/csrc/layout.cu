@@ -268,6 +268,76 @@ __global__ void __launch_bounds__(kPackThreads) pack_activations_bulk_kernel(con
   }
 }
 
+// Activation pack for large batches of small images whose channels all fit one tile (C a multiple of 16,
+// at most 64; H*W a multiple of 4, at most 256): the images of a batch tensor are then contiguous, so one
+// block fetches `ipb` whole images with ONE bulk copy (several KB in flight per block instead of one
+// 16-channel group) and transposes them as the kernels above do.  Channels C .. C_pad-1 are written as zeros.
+__global__ void __launch_bounds__(kPackThreads) pack_small_images_kernel(const int8_t* __restrict__ x,
+                                                                        int8_t* __restrict__ out, int N, int C, int HW,
+                                                                        int C_pad, int ipb, int* status, Dbg dbg) {
+  extern __shared__ __align__(128) uint8_t btile[];
+  __shared__ __align__(8) unsigned long long bar;
+  const int t = threadIdx.x;
+  const int n0 = blockIdx.x * ipb;
+  const int nimg = min(ipb, N - n0);
+  const int img_bytes = C * HW;
+  const uint32_t bar_a = (uint32_t)__cvta_generic_to_shared(&bar);
+  const uint32_t tile_a = (uint32_t)__cvta_generic_to_shared(btile);
+  const int8_t* xin = x + (size_t)n0 * img_bytes;
+  if (t == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  pdl_wait();
+  if (t == 0) {
+    const uint32_t bytes = (uint32_t)(nimg * img_bytes);
+    if (B2C_X_OK(dbg, 17, xin, bytes)) {
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"(bytes) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(tile_a),
+                   "l"(xin), "r"(bytes), "r"(bar_a)
+                   : "memory");
+    } else {
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_a) : "memory");  // refused (debug build): nothing to wait for
+    }
+  }
+  if (!pack_wait_bounded(bar_a, status, t == 0)) return;
+  pdl_launch_dependents();
+  const int chunks = C_pad >> 4;            // 16-channel chunks of an output pixel
+  const int pgs = (HW + 3) >> 2;            // groups of 4 pixels of an image
+  const int items = nimg * pgs * chunks;
+  for (int it = t; it < items; it += kPackThreads) {
+    const int ch = it % chunks;
+    const int r = it / chunks;
+    const int pg = r % pgs;
+    const int i = r / pgs;
+    uint32_t w[16];
+    if (ch * 16 < C) {
+      const uint8_t* src = btile + (size_t)i * img_bytes + (ch * 16) * HW + pg * 4;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) w[k] = *reinterpret_cast<const uint32_t*>(src + k * HW);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) w[k] = 0;
+    }
+    int8_t* dst = out + ((size_t)(n0 + i) * HW + pg * 4) * C_pad + ch * 16;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (pg * 4 + j < HW) {
+        uint32_t o[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const uint32_t lo = __byte_perm(w[4 * k], w[4 * k + 1], j | ((4 + j) << 4));
+          const uint32_t hi = __byte_perm(w[4 * k + 2], w[4 * k + 3], j | ((4 + j) << 4));
+          o[k] = __byte_perm(lo, hi, 0x5410);
+        }
+        if (B2C_WS_OK(dbg, 18, dst + (size_t)j * C_pad, 16))
+          *reinterpret_cast<uint4*>(dst + (size_t)j * C_pad) = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+    }
+  }
+}
+
 // Channel-pack weights: out[k][(r*S + s)][c_pad] = w[k][c][r][s], zeros for c >= C.
 __global__ void pack_weights_cp_kernel(const int8_t* __restrict__ w, int8_t* __restrict__ out, int K, int C, int RS,
                                        int C_pad) {
@@ -635,6 +705,13 @@ cudaError_t launch_pack_activations(const int8_t* x, int8_t* out, int N, int C, 
   const int HW = H * W;
   int CT = C_pad >= 128 ? 128 : 64;
   const bool a16 = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+  // large batches of small images with few channels: several whole images per block
+  if (a16 && (C % 16) == 0 && C <= 64 && (HW % 4) == 0 && HW <= 256 && C * HW <= 12 * 1024 && N >= 8 * kNumSMs) {
+    const int ipb = std::max(1, std::min(16, (24 * 1024) / (C * HW)));
+    const size_t smem = (size_t)ipb * C * HW;
+    return launch_pdl(pack_small_images_kernel, dim3((unsigned)((N + ipb - 1) / ipb)), dim3(kPackThreads), smem, st, x, out, N, C,
+                      HW, C_pad, ipb, status, dbg);
+  }
   // Bulk-copy kernels: channels in whole groups of 16 and either the whole image per tile
   // (H*W <= 256, a multiple of 4) or rows that are multiples of 16 bytes.
   if (a16 && (C % 16) == 0 && (HW % 4) == 0 && (HW <= 256 || (HW % 16) == 0)) {

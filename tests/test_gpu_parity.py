@@ -25,7 +25,8 @@ def cfg_reference(cfg):
 
 # ---- layout kernels on their own ---------------------------------------------------------------------
 @pytest.mark.parametrize("shape,C_pad", [((1, 16, 14, 14), 32), ((2, 3, 30, 23), 16), ((3, 70, 9, 13), 96),
-                                         ((2, 256, 14, 14), 256), ((1, 1, 96, 480), 32), ((2, 64, 56, 56), 64)])
+                                         ((2, 256, 14, 14), 256), ((1, 1, 96, 480), 32), ((2, 64, 56, 56), 64),
+                                         ((1500, 16, 14, 14), 32), ((1203, 48, 6, 10), 64)])   # large batches of small images
 def test_pack_activations(lib, shape, C_pad):
     x = int8_uniform(shape, 301)
     want = oracle.pack_nhwc_cpad(x, C_pad)
