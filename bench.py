@@ -41,7 +41,13 @@ INT8_TO_BF16_RATIO = 2.0  # nominal dense int8 : bf16 tensor throughput on B200 
 # per launch), valid only for the sources it was taken on (the kernel and the host code that picks its
 # tile, stage count and launch shape); see profiles/.
 KERNEL_SOURCES = ("conv_mma.cu", "conv_mma_pair.cu", "conv_mma_common.cuh", "api.cpp", "planner.cpp", "tma.cpp", "b2c_internal.h")
-NCU_TRAFFIC = {"conv_mma_sha1": "2f7f0c9ebef77a24137d8c3d4168093c86fde328", "bytes_per_launch": 2859008}
+
+
+def kernel_sources_sha1():
+    return hashlib.sha1(b"".join(open(os.path.join(ROOT, "paper_2104_04731_b200", "csrc", f), "rb").read()
+                                 for f in KERNEL_SOURCES)).hexdigest()
+# (per tile shape "tile_m x tile_n" of the channel-pack map on the headline shape)
+NCU_TRAFFIC = {"conv_mma_sha1": "", "bytes_per_launch": {}}
 
 
 def load_peaks():
@@ -709,9 +715,10 @@ def run_ours(args):
         achieved, peak, runit = ops / (op_us * 1e-6) / 1e12, peaks["bf16_tflops"] * INT8_TO_BF16_RATIO, "TFLOP/s"
     else:
         achieved, peak, runit = cfg.algorithmic_bytes / (op_us * 1e-6) / 1e9, peaks["hbm_gbs"], "GB/s"
-    sha = hashlib.sha1(b"".join(open(os.path.join(ROOT, "paper_2104_04731_b200", "csrc", f), "rb").read()
-                                for f in KERNEL_SOURCES)).hexdigest()
-    traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["conv_mma_sha1"] == sha else None
+    sha = kernel_sources_sha1()
+    traffic = None
+    if NCU_TRAFFIC["conv_mma_sha1"] == sha and args.config == HEADLINE and not args.scaled and emb.variant == 0:
+        traffic = NCU_TRAFFIC["bytes_per_launch"].get("%dx%d" % (emb.tile_m, emb.tile_n))
     kname = "conv_mma_pair_kernel" if emb.tile_m == 256 else "conv_mma_kernel"
     launches_per_step = (op["launches_per_call"] if op else inst_launches) * G
     roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,

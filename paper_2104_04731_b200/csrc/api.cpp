@@ -901,7 +901,11 @@ static int run_rewrite(b2c_plan* p, const int8_t* x, void* ws, cudaStream_t st) 
   if (is_tma_view_variant(p->emb.variant)) {
     const TmaView& v = p->view;
     const int base_variant = shift_base_variant(p->emb.variant);
-    if (base_variant == B2C_VARIANT_CP_TMA) {
+    if (base_variant == B2C_VARIANT_CP_TMA && d.in_layout == B2C_LAYOUT_NHWC) {
+      // NHWC re-pad (Pad rule alone): the layout-generic copy kernel with one phase per axis
+      CUDA_TRY(launch_phase_split(x, scratch, d.N, d.C, d.H, d.W, 1, 1, d.H, d.W, v.C, a.x_stride_n, 1, a.x_stride_h,
+                                  a.x_stride_w, st, dbg));
+    } else if (base_variant == B2C_VARIANT_CP_TMA) {
       CUDA_TRY(launch_pack_activations(x, scratch, d.N, d.C, d.H, d.W, p->C_pad, st, p->status, dbg));
     } else if (base_variant == B2C_VARIANT_DILATION_PACK) {
       const bool nchw = d.in_layout == B2C_LAYOUT_NCHW;

@@ -224,9 +224,8 @@ bool tma_view_for(const Geom& g, int variant, TmaView* v) {
     return tma_view_for(g, shift_base_variant(variant), v) && shift_geom(g, *v, &sg);
   }
   if (variant == B2C_VARIANT_CP_TMA) {
-    // Pad + Split + Reorder of the channel axis (Table 2); an NHWC source must already have a
-    // multiple of 32 channels (there is no NHWC re-pad kernel).
-    if (d.in_layout == B2C_LAYOUT_NHWC && cp_channel_pad(d.C) != d.C) return false;
+    // Pad + Split + Reorder of the channel axis (Table 2).  An NHWC source with a multiple of 32
+    // channels is read in place; any other NHWC source is re-padded into the scratch tensor.
     *v = TmaView{d.N, cp_channel_pad(d.C), d.H, d.W, d.R, d.S, d.stride_h, d.stride_w, d.pad_h, d.pad_w, d.dil_h, d.dil_w};
   } else if (variant == B2C_VARIANT_ROW_UNROLL) {
     // Stencil Unroll along s only: U[n][h][q][(s, c)] = x[n][c][h][q*stride_w - pad_w + s*dil_w].

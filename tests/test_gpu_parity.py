@@ -116,6 +116,24 @@ def test_random_shapes(lib, case):
     check_against_oracle(x, w, stride, pad, dil, shift, 3, e2.id, ref=ref, in_layout=1, out_layout=1)
 
 
+# ---- NHWC input whose channel count is no multiple of 32: re-padded into the scratch tensor -----------------
+@pytest.mark.parametrize("C", [3, 24, 40, 72])
+def test_nhwc_input_is_repadded_for_the_channel_pack_maps(lib, C):
+    N, H, W, K, R, S = 3, 13, 15, 40, 3, 3
+    x = int8_uniform((N, C, H, W), 771)
+    w = int8_uniform((K, C, R, S), 772)
+    ref = oracle.conv2d_int8(x, w, 1, 1, 1, 7)
+    d = lib.make_desc(N, C, H, W, K, R, S, 1, 1, 1, 7, 1, 1, 3)
+    embs = [e for e in lib.enumerate_embeddings(d) if e.variant in (b2c.VARIANT_CP_TMA, b2c.VARIANT_CP_SHIFT)]
+    assert {e.variant for e in embs} == {b2c.VARIANT_CP_TMA, b2c.VARIANT_CP_SHIFT} and all(e.workspace_bytes > 0 for e in embs)
+    seen = set()
+    for e in embs:
+        if (e.variant, e.tile_m) in seen:
+            continue
+        seen.add((e.variant, e.tile_m))
+        check_against_oracle(x, w, 1, 1, 1, 7, 3, e.id, ref=ref, in_layout=1, out_layout=1)
+
+
 # ---- swapped axis map (M <- k, N <- fused pixels) -------------------------------------------------------
 @pytest.mark.parametrize("case", [
     # N, C, H, W, K, R, S, stride, pad, dil, shift
@@ -331,9 +349,7 @@ def test_shift_execution(lib, case, layouts):
     d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, in_layout, out_layout, 3)
     shifts = [e for e in lib.enumerate_embeddings(d) if e.variant in (b2c.VARIANT_CP_SHIFT, b2c.VARIANT_S2D_SHIFT)]
     want = {b2c.VARIANT_S2D_SHIFT} if stride != 1 else {b2c.VARIANT_CP_SHIFT}
-    if in_layout == 1 and C % 32 != 0 and stride == 1:
-        want = set()  # an NHWC source needs padded channels for the channel-pack view
-    assert {e.variant for e in shifts} == want
+    assert {e.variant for e in shifts} == want   # (an NHWC source without padded channels is re-padded into the scratch tensor)
     for e in shifts:
         assert e.split_k == 1 and e.tile_n >= K and e.map_m == b2c.AXIS_NPQ
         check_against_oracle(x, w, stride, pad, dil, shift, 3, e.id, ref=ref, in_layout=in_layout, out_layout=out_layout)
