@@ -54,7 +54,7 @@ int8_t oracle_requant(int64_t acc, int shift) {
 
 /*
  * The definition (Figure 5 step 1; Table 2 access [n, i + k]), followed by the vector unit's
- * "activation and quantization operations" (Section 5.1; the micro-benchmark of Section 5.2 runs
+ * "activation and quantization operations" (Section 5.1, which also describes the micro-benchmark that runs
  * pack -> conv -> activation -> unpack).  The paper does not say which activation; the reading
  * taken here is an optional per-output-channel int32 bias and an optional ReLU, both applied to
  * the exact sum before the outputs are written:
