@@ -264,7 +264,7 @@ def time_steps(torch, fn, steps, warmup, dist=None, min_warm_s=0.2):
     return ms
 
 
-def instances_for(cfg, min_bytes=2 * L2_BYTES, lo=8, hi=256):
+def instances_for(cfg, min_bytes=8 * L2_BYTES, lo=8, hi=256):
     per = cfg.algorithmic_bytes + cfg.N * cfg.C * cfg.H * cfg.W  # plus a packed copy of the input
     return int(max(lo, min(hi, -(-min_bytes // per))))
 

@@ -341,6 +341,24 @@ __device__ __forceinline__ void store_columns(const ConvArgs& args, int32_t* v, 
     // NKPQ: for a fixed column the 32 lanes of a warp hold 32 consecutive pixels, so every
     // store instruction writes one contiguous run.
     const long long o = base_nkpq + (long long)kbase * args.out_PQ;
+    if (kbase + NC <= K && (long long)NC * args.out_PQ < 0x7FFFFFFFLL) {
+      // all NC channels exist: no per-column test, and every address is the base plus a 32-bit
+      // offset, so the columns are independent instructions
+      const int pq = args.out_PQ, shift = args.shift;
+      if (args.out_mode & B2C_OUT_I32) {
+        int32_t* dst = args.y32 + o;
+#pragma unroll
+        for (int j = 0; j < NC; ++j) dst[j * pq] = v[j];
+      }
+      if (args.out_mode & B2C_OUT_I8) {
+        int8_t* dst = args.y8 + o;
+#pragma unroll
+        for (int j = 0; j < NC; ++j) {
+          dst[j * pq] = requant(v[j], shift);
+        }
+      }
+      return;
+    }
     if (args.out_mode & B2C_OUT_I32) {
       int32_t* dst = args.y32 + o;
 #pragma unroll

@@ -366,7 +366,10 @@ __global__ void __launch_bounds__(PACK ? kThreads + kPackGroup : kThreads, PERSI
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = __shfl_sync(0xffffffffu, ctl.tmem_base, 0);
   pdl_wait();
-  pdl_launch_dependents();
+  // The next kernel of the stream may start its set-up once the leader has issued its last MMA (its
+  // blocks then wait in griddepcontrol.wait while this grid's epilogue runs).  An earlier start would
+  // park waiting blocks on SMs that blocks of other streams could be using.
+  if (rank != 0) pdl_launch_dependents();
 
 #define B2C_PAIR_TILE_ORIGIN(t)                                     \
   const int mt_ = (int)args.div_tiles_n.div((uint32_t)(t));        \
@@ -472,6 +475,7 @@ __global__ void __launch_bounds__(PACK ? kThreads + kPackGroup : kThreads, PERSI
         }
       }
     }
+    pdl_launch_dependents();
     __syncwarp();
   } else if (PACK && warp >= 2 + kGatherWarps) {
     // ---------------------------------------------------------------- activation pack (both blocks)
