@@ -109,8 +109,8 @@ typedef struct {
 #define B2C_POLICY_AUTO_TIMED (-1)   /* time the 5 lowest-overhead candidates, keep the fastest (Section 6.1) */
 #define B2C_POLICY_MIN_OVERHEAD (-2) /* lowest |[o_mac, o_data] . [1, 1]| without timing (Section 4.4)        */
 #define B2C_POLICY_MIN_WORKSPACE (-3) /* smallest scratch footprint (Table 4)                                 */
-#define B2C_POLICY_AUTO_TIMED_CONCURRENT (-4) /* as AUTO_TIMED, but every candidate is timed as eight independent
-                                        * runs on eight streams at once and the highest throughput wins: for callers
+#define B2C_POLICY_AUTO_TIMED_CONCURRENT (-4) /* as AUTO_TIMED, but every candidate is timed as sixteen independent
+                                        * runs on sixteen streams at once and the highest throughput wins: for callers
                                         * that keep several independent convolutions in flight, where a schedule
                                         * with fewer, wider tiles beats the one with the shortest single-run time */
 
@@ -127,7 +127,7 @@ int b2c_out_shape(const b2c_conv_desc* desc, int32_t* P, int32_t* Q);
 int b2c_enumerate(const b2c_conv_desc* desc, b2c_embedding* out, int32_t cap, int32_t* count);
 
 /* Creates a plan for `desc` on the current device.  `policy_or_id` is a B2C_POLICY_* value or
- * an embedding id from b2c_enumerate.  AUTO_TIMED (and AUTO_TIMED_CONCURRENT, with eight sets of
+ * an embedding id from b2c_enumerate.  AUTO_TIMED (and AUTO_TIMED_CONCURRENT, with sixteen sets of
  * output and scratch buffers) allocates temporary device buffers, captures
  * each candidate's launches in a CUDA graph on a private stream, replays it and keeps the
  * fastest; it synchronises with the device and must not be called while a stream of the calling

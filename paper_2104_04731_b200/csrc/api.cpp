@@ -566,7 +566,7 @@ int create_plan_for(const Geom& g, const b2c_embedding& emb, b2c_plan** out, int
 // With lanes > 1 every iteration enqueues one run per lane, each lane on a stream of its own
 // (forked from and joined back into the first) with its own outputs and scratch, so that kernels
 // of different lanes may overlap on the GPU; *us is then the time per run at that concurrency.
-constexpr int kMaxLanes = 8;
+constexpr int kMaxLanes = 16;
 struct LaneBuffers {
   int32_t* y32;
   int8_t* y8;
