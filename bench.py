@@ -571,6 +571,36 @@ def candidates_report(b2c, torch, shapes):
     return out
 
 
+def grouped_report(b2c, torch, N=8, C=256, H=28, W=28, R=3, stride=1, pad=1, shift=6):
+    """Depth-wise layer (Section 6.1 names it as the same low-channel problem): all groups in one launch
+    against the same layer written as a dense convolution with block-diagonal weights (zeros elsewhere)."""
+    rng = np.random.default_rng(2104)
+    xh = rng.integers(-128, 128, (N, C, H, W), dtype=np.int8)
+    wg = rng.integers(-128, 128, (C, 1, R, R), dtype=np.int8)
+    wd = np.zeros((C, C, R, R), dtype=np.int8)
+    wd[np.arange(C), np.arange(C)] = wg[:, 0]
+    d = b2c.make_desc(N, C, H, W, C, R, R, stride, pad, 1, shift, 0, 0, 2)
+    P = (H + 2 * pad - R) // stride + 1
+    x = torch.from_numpy(xh).cuda()
+    y8 = torch.empty((N, C, P, P), dtype=torch.int8, device="cuda")
+    rows, outs = [], []
+    for name, groups, wh, policy in (("grouped, one launch", C, wg, 0),
+                                     ("dense, block-diagonal weights", 1, wd, b2c.POLICY_AUTO_TIMED)):
+        plan = b2c.Plan(d, policy, groups=groups) if groups > 1 else b2c.Plan(d, policy)
+        ws = torch.empty(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
+        plan.set_weights(torch.from_numpy(wh).cuda())
+        us = _graph_us(torch, lambda: plan.run(x, None, y8, ws))
+        if plan.device_status() != 0:
+            raise RuntimeError("device status")
+        e = plan.info()
+        rows.append({"form": name, "us": us, "embedding": b2c.VARIANT_NAMES[e.variant], "tile_n": e.tile_n,
+                     "weight_elements": int(wh.size)})
+        outs.append(y8.clone())
+        plan.destroy()
+    return {"shape": "depthwise_n%d_c%d_%dx%d_%dx%d" % (N, C, H, W, R, R), "rows": rows,
+            "same_result": bool(torch.equal(outs[0], outs[1]))}
+
+
 def print_candidates_markdown(report):
     for sh in report:
         ref = next((r for r in sh["rows"] if r["reference"]), None)
@@ -664,8 +694,16 @@ def run_ours(args):
     graph = not args.no_graph
     if args.report == "candidates":
         rep = candidates_report(b2c, torch, CONFIGS + REPORT_EXTRA)
-        print(json.dumps({"report": "candidates", "shapes": rep}))
+        grps = [grouped_report(b2c, torch, N=n) for n in (8, 128)]
+        print(json.dumps({"report": "candidates", "shapes": rep, "grouped": grps}))
         print_candidates_markdown(rep)
+        for grp in grps:
+            print("\n### %s (grouped / depth-wise, Section 6.1)" % grp["shape"])
+            print("| form | us | embedding | tile_n | weight elements |")
+            print("|---|---|---|---|---|")
+            for r in grp["rows"]:
+                print("| %s | %.2f | %s | %d | %d |" % (r["form"], r["us"], r["embedding"], r["tile_n"], r["weight_elements"]))
+            print("(same int8 output from both forms: %s)" % grp["same_result"])
         return 0
 
     sampler = ClockSampler(local)

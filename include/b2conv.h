@@ -144,8 +144,13 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
  * groups < 1 or does not divide C and K).  The plan runs all groups in ONE launch of the MMA kernel
  * (the group is a grid axis: every block convolves its group's channel slice of x into that
  * group's slice of y in place, with the filters of all groups packed once into one matrix; no
- * scratch: b2c_plan_workspace_bytes is 0), with the lowest-overhead stencil unroll formed inside
- * the kernel; b2c_plan_info reports that embedding.
+ * scratch: b2c_plan_workspace_bytes is 0), with a stencil unroll formed inside the kernel (the
+ * staged window where it fits, else the gather); b2c_plan_info reports that embedding.
+ * Narrow groups are merged: m consecutive groups (m the smallest divisor of `groups` that brings a
+ * merged group to 32 output channels, within 1024 reduction elements) run as one group of m times
+ * the channels with block-diagonal filters; b2c_plan_set_weights expands the filters into a buffer
+ * the plan owns (zeros between the groups) before it packs them.  Results are those of the grouped
+ * convolution; only the number of tiles and the idle share of each MMA change.
  * All other plan calls (set_weights, set_activation with K bias values, run, device_status, destroy)
  * apply as to any plan; the rewrite / run_rewritten halves are no-op and run respectively. */
 int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan** out);

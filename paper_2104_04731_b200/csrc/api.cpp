@@ -45,6 +45,11 @@ struct b2c_plan {
   int groups = 1;
   std::vector<b2c_plan*> subs;
   int group_count = 1;  // on the sub-plan of a group plan: groups run by one launch (blockIdx.z = group)
+  // Group merge (group plan): `merge` consecutive groups run as ONE group of merge x the channels with
+  // block-diagonal filters (zeros between the groups), so that narrow groups fill the MMA's columns and
+  // reduction depth; w_expanded holds the expanded filters [K][merge * C/groups][R][S].
+  int merge = 1;
+  int8_t* w_expanded = nullptr;  // device, plan-owned
   long long x_stride_n_whole = 0, y_stride_n_whole = 0;  // sub-plans: batch strides of the whole tensors
   struct HostPipe* pipe = nullptr;  // streaming host-buffer calls: created by the first b2c_plan_run_host_async
   // The two-SM persistent channel-pack schedule can run the activation pack inside the MMA kernel
@@ -794,20 +799,43 @@ int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan*
   if (desc->C < 1 || desc->K < 1 || desc->C % groups != 0 || desc->K % groups != 0) return B2C_E_INVALID_ARG;
   // whole tensors are NCHW / NKPQ: a group is then a contiguous channel slice of every image
   if (desc->in_layout != B2C_LAYOUT_NCHW || desc->out_layout != B2C_LAYOUT_NCHW) return B2C_E_UNSUPPORTED;
+  // Narrow groups are merged: a depth-wise layer run group by group gives every MMA one useful column and
+  // nine useful reduction elements.  m consecutive groups as one group with block-diagonal filters spend m
+  // times the MACs (which are idle anyway) for 1/m of the tiles: the smallest divisor m of `groups` that
+  // brings a merged group to 32 output channels, within 1024 reduction elements.
+  const int cg = desc->C / groups, kg = desc->K / groups;
+  int merge = 1;
+  for (int m = 1; m <= groups; ++m) {
+    if (groups % m != 0) continue;
+    if ((long long)m * cg * desc->R * desc->S > 1024 && m > 1) break;
+    merge = m;
+    if (m * kg >= 32) break;
+  }
   b2c_conv_desc sd = *desc;
-  sd.C = desc->C / groups;
-  sd.K = desc->K / groups;
+  sd.C = cg * merge;
+  sd.K = kg * merge;
   Geom sg;
   int rc = resolve_geom(&sd, &sg);
   if (rc != B2C_OK) return rc;
+  const int run_groups = groups / merge;
   // Embedding of every group: the lowest-overhead unsplit stencil unroll formed inside the kernel
   // (staged window where it fits, else the gather); both read their channel slice of x in place.
   std::vector<b2c_embedding> all;
   enumerate_embeddings(sg, &all);
+  // (the staged window before the gather: it builds the operand from shared memory with word loads; of
+  // one variant's schedules the one whose column tile holds a whole group, else the widest)
   int pick = -1;
-  for (size_t i = 0; i < all.size() && pick < 0; ++i)
-    if (all[i].split_k == 1 && !is_swapped(all[i]) && table_variant_legal(sg) &&
-        (all[i].variant == B2C_VARIANT_IM2COL_STAGED || all[i].variant == B2C_VARIANT_IM2COL_GATHER))
+  auto better = [&](const b2c_embedding& a, const b2c_embedding& b) {
+    const bool as = a.variant == B2C_VARIANT_IM2COL_STAGED, bs = b.variant == B2C_VARIANT_IM2COL_STAGED;
+    if (as != bs) return as;
+    const bool af = a.tile_n >= sd.K, bf = b.tile_n >= sd.K;
+    if (af != bf) return af;
+    return af ? a.tile_n < b.tile_n : a.tile_n > b.tile_n;
+  };
+  for (size_t i = 0; i < all.size(); ++i)
+    if (all[i].split_k == 1 && !is_swapped(all[i]) && all[i].tile_m == kTileM && table_variant_legal(sg) &&
+        (all[i].variant == B2C_VARIANT_IM2COL_STAGED || all[i].variant == B2C_VARIANT_IM2COL_GATHER) &&
+        (pick < 0 || better(all[i], all[pick])))
       pick = (int)i;
   if (pick < 0) return B2C_E_UNSUPPORTED;
   b2c_plan* p = new (std::nothrow) b2c_plan();
@@ -817,6 +845,7 @@ int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan*
   p->g.d.K = desc->K;
   p->emb = all[pick];
   p->groups = groups;
+  p->merge = merge;
   cudaGetDevice(&p->device);
   if (cudaMalloc(&p->status, kStatusWords * sizeof(int)) != cudaSuccess ||
       cudaMemset(p->status, 0, kStatusWords * sizeof(int)) != cudaSuccess) {
@@ -826,10 +855,17 @@ int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan*
   }
   // one sub-plan runs all groups in one launch (the group is a grid axis of the kernel)
   b2c_plan* sub = nullptr;
-  rc = create_plan_for(sg, all[pick], &sub, groups);
+  rc = create_plan_for(sg, all[pick], &sub, run_groups);
   if (rc != B2C_OK) {
     b2c_plan_destroy(p);
     return rc;
+  }
+  if (merge > 1 &&
+      cudaMalloc(&p->w_expanded, (size_t)desc->K * sd.C * desc->R * desc->S + 256) != cudaSuccess) {
+    set_last_cuda_error((int)cudaGetLastError());
+    b2c_plan_destroy(sub);
+    b2c_plan_destroy(p);
+    return B2C_E_CUDA;
   }
   sub->x_stride_n_whole = (long long)desc->C * desc->H * desc->W;
   sub->y_stride_n_whole = (long long)desc->K * sg.PQ;
@@ -859,7 +895,13 @@ int b2c_plan_set_weights(b2c_plan* p, const int8_t* w, void* cuda_stream) {
   if (!p->subs.empty()) {
     // w is [K][C/groups][R][S]: group g's filters are the g-th block of K/groups rows
     // (one pack launch: the rows of all groups have the same format)
-    int rc = set_weights_one(p->subs[0], w, st);
+    const int8_t* src = w;
+    if (p->merge > 1) {
+      const b2c_conv_desc& d = p->g.d;  // (the whole convolution)
+      CUDA_TRY(launch_expand_group_weights(w, p->w_expanded, d.K, d.C / p->groups, d.K / p->groups, p->merge, d.R * d.S, st));
+      src = p->w_expanded;
+    }
+    int rc = set_weights_one(p->subs[0], src, st);
     if (rc != B2C_OK) return rc;
     p->weights_set = true;
     return B2C_OK;
@@ -1214,6 +1256,7 @@ void b2c_plan_destroy(b2c_plan* p) {
   destroy_pipe(p->pipe);
   for (b2c_plan* sub : p->subs) b2c_plan_destroy(sub);
   cudaFree(p->w_packed);
+  cudaFree(p->w_expanded);
   cudaFree(p->table);
   cudaFree(p->table32);
   cudaFree(p->wtable);

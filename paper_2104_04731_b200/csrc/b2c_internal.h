@@ -384,6 +384,9 @@ cudaError_t launch_pack_weights_cp(const int8_t* w, int8_t* out, int K, int C, i
                                    cudaStream_t st);
 cudaError_t launch_pack_weights_table(const int8_t* w, int8_t* out, int K, int Kg, int cols, const int32_t* table,
                                       cudaStream_t st);
+// Filters of a grouped convolution [K][cg][RS] expanded for groups merged m at a time: [K][m * cg][RS],
+// row k holds its own cg channels at channel offset ((k / kg) % m) * cg and zeros elsewhere.
+cudaError_t launch_expand_group_weights(const int8_t* w, int8_t* out, int K, int cg, int kg, int m, int RS, cudaStream_t st);
 cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg, int K_pad, int S, int S_run,
                                      cudaStream_t st);
 cudaError_t launch_im2col(const int8_t* x, int8_t* a, const GatherEntry* table, long long Mg, int PQ, int Q, int H,

@@ -759,6 +759,29 @@ cudaError_t launch_pack_weights_table(const int8_t* w, int8_t* out, int K, int K
   return cudaGetLastError();
 }
 
+namespace {
+__global__ void expand_group_weights_kernel(const int8_t* __restrict__ w, int8_t* __restrict__ out, int K, int cg, int kg,
+                                            int m, int RS) {
+  pdl_wait();
+  const long long row = (long long)m * cg * RS;  // elements of one expanded filter
+  const long long total = (long long)K * row;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int k = (int)(i / row);
+    const int rem = (int)(i - (long long)k * row);
+    const int c = rem / RS, t = rem - c * RS;
+    const int slot = (k / kg) % m;  // which of the merged groups filter k belongs to
+    out[i] = (c / cg == slot) ? w[((long long)k * cg + (c - slot * cg)) * RS + t] : (int8_t)0;
+  }
+  pdl_launch_dependents();
+}
+}  // namespace
+
+cudaError_t launch_expand_group_weights(const int8_t* w, int8_t* out, int K, int cg, int kg, int m, int RS, cudaStream_t st) {
+  const long long total = (long long)K * m * cg * RS;
+  const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
+  return launch_pdl(expand_group_weights_kernel, dim3((unsigned)std::max(1, blocks)), dim3(256), 0, st, w, out, K, cg, kg, m, RS);
+}
+
 cudaError_t launch_pack_weights_rows(const int8_t* w, int8_t* out, int K, int Kg, int K_pad, int S, int S_run,
                                      cudaStream_t st) {
   const long long total = (long long)K * K_pad;
