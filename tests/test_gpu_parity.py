@@ -424,6 +424,7 @@ def test_shift_execution_four_accumulator_buffers(lib):
     (2, 64, 7, 7, 128, 2, 1, 1, 1, 0, 1, 7, 3),         # pointwise, 64 output channels per group
     (2, 256, 14, 14, 256, 256, 3, 3, 1, 1, 1, 4, 3),    # depth-wise, 256 channels: 256 groups in one launch
     (40, 32, 28, 28, 64, 8, 3, 3, 2, 1, 1, 6, 3),       # many tiles per group: the persistent walk with a group axis
+    (2, 48, 9, 9, 96, 48, 3, 3, 1, 1, 1, 5, 3),         # 48 groups of 1 -> 2 channels: merged 16 at a time, three merged groups
 ])
 def test_grouped_convolution(lib, case):
     N, C, H, W, K, groups, R, S, stride, pad, dil, shift, out_mode = case
