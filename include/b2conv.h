@@ -319,6 +319,14 @@ int b2c_im2col_noalloc(const b2c_conv_desc* desc, const int8_t* x_dev, int8_t* a
  * INVALID_ARG on bad arguments, B2C_E_CUDA / B2C_E_TIMEOUT on failure. */
 int b2c_measure_mma_rate(int tile_n, int mmas_per_block, float* device_us, float* cycles_per_mma, void* cuda_stream);
 
+/* The same for the two-SM form (tcgen05.mma.cta_group::2.kind::i8, 256 x tile_n x 32 per instruction,
+ * issued by the leader of each of the device's 74 block pairs; every block holds 128 rows of A and
+ * tile_n / 2 rows of B and its tensor core reads the other half of B from its peer's shared memory):
+ * 74 * mmas_per_pair * 2*256*tile_n*32 / device_us is the issue rate of the two-SM schedule, the
+ * ceiling of the kernel that uses it.  tile_n in {64, 128, 256}; *cycles_per_mma: median over the
+ * pairs.  Same allocation, synchronisation and error behaviour as b2c_measure_mma_rate. */
+int b2c_measure_mma_rate_pair(int tile_n, int mmas_per_pair, float* device_us, float* cycles_per_mma, void* cuda_stream);
+
 /* ---- debug build (no counterpart in the paper) ---------------------------------------------------
  * libb2conv_debug.so is the same library compiled with -DB2C_DEBUG_BOUNDS.  In it every address a
  * kernel computes by hand (loads of x, stores and atomics to the outputs and to the scratch; TMA

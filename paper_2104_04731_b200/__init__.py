@@ -34,7 +34,7 @@ EXPORTS = [
     "b2c_plan_create_grouped", "b2c_plan_run_host_async", "b2c_plan_host_sync",
     "b2c_plan_device_status", "b2c_selftest_bounded_wait", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
     "b2c_status_string",
-    "b2c_last_cuda_error", "b2c_oneshot_status", "b2c_oneshot_cache_clear", "b2c_test_fail_nth_encode", "b2c_selftest_pack_wait", "b2c_measure_mma_rate", "b2c_debug_build", "b2c_plan_debug_info",
+    "b2c_last_cuda_error", "b2c_oneshot_status", "b2c_oneshot_cache_clear", "b2c_test_fail_nth_encode", "b2c_selftest_pack_wait", "b2c_measure_mma_rate", "b2c_measure_mma_rate_pair", "b2c_debug_build", "b2c_plan_debug_info",
     "b2c_plan_check_canaries", "b2c_test_shrink_checked_ranges",
 ]
 
@@ -115,6 +115,7 @@ def load():
     lib.b2c_plan_check_canaries.argtypes = [vp, vp, pi32]
     lib.b2c_test_shrink_checked_ranges.argtypes = [ctypes.c_longlong]
     lib.b2c_measure_mma_rate.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float), vp]
+    lib.b2c_measure_mma_rate_pair.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float), vp]
     lib.b2c_oneshot_cache_clear.argtypes = []
     lib.b2c_test_fail_nth_encode.argtypes = [i32]
     for name in EXPORTS:
@@ -289,6 +290,14 @@ def measure_mma_rate(tile_n: int = 256, mmas_per_block: int = 20000, stream=None
     us, cyc = ctypes.c_float(), ctypes.c_float()
     _check(load().b2c_measure_mma_rate(tile_n, mmas_per_block, ctypes.byref(us), ctypes.byref(cyc), _stream_ptr(stream)),
            "b2c_measure_mma_rate")
+    return us.value, cyc.value
+
+
+def measure_mma_rate_pair(tile_n: int = 256, mmas_per_pair: int = 20000, stream=None):
+    """(device_us, cycles_per_mma) of back-to-back two-SM 256 x tile_n x 32 int8 MMAs on all 74 block pairs."""
+    us, cyc = ctypes.c_float(), ctypes.c_float()
+    _check(load().b2c_measure_mma_rate_pair(tile_n, mmas_per_pair, ctypes.byref(us), ctypes.byref(cyc), _stream_ptr(stream)),
+           "b2c_measure_mma_rate_pair")
     return us.value, cyc.value
 
 

@@ -843,6 +843,11 @@ def test_mma_rate_measurement_is_plausible(lib):
     assert cyc16 < cyc
     with pytest.raises(b2c.B2CError):
         lib.measure_mma_rate(48, 4000)
+    # two-SM form: 256 x 256 x 32 per instruction; a pair cannot beat two SMs' worth of MACs per clock
+    us2, cyc2 = lib.measure_mma_rate_pair(256, 4000)
+    assert 100.0 < cyc2 < 600.0 and us2 > 0
+    with pytest.raises(b2c.B2CError):
+        lib.measure_mma_rate_pair(32, 4000)
 
 
 # ---- failure detection: a wait that cannot complete ends by itself and is reported --------------------
