@@ -155,6 +155,19 @@ int b2c_plan_create(const b2c_conv_desc* desc, int32_t policy_or_id, void* cuda_
  * apply as to any plan; the rewrite / run_rewritten halves are no-op and run respectively. */
 int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan** out);
 
+/* Grouped convolution with the form chosen by timing (Section 6.1's timed choice among candidates, applied
+ * to the merge factor).  Two forms are built and run on scratch tensors: the in-place form of
+ * b2c_plan_create_grouped, and the full merge: the dense convolution of the whole tensors with
+ * block-diagonal filters (all other filter elements zero), itself chosen by B2C_POLICY_AUTO_TIMED.  The
+ * full merge spends `groups` times the MACs and may need scratch (b2c_plan_workspace_bytes is then that of
+ * its embedding, and run takes the workspace like any dense plan); it is considered when the expanded
+ * filters [K][C][R][S] are at most 16 MB.  The faster form is returned; b2c_plan_info reports its
+ * embedding with the measured device_us.  Weights, activation, run and results are as for
+ * b2c_plan_create_grouped.  Allocates temporary device buffers and synchronises with the device like
+ * B2C_POLICY_AUTO_TIMED; `cuda_stream` is used for buffer initialisation.  Errors as
+ * b2c_plan_create_grouped; when the full merge cannot be built or timed the in-place form is returned. */
+int b2c_plan_create_grouped_timed(const b2c_conv_desc* desc, int32_t groups, void* cuda_stream, b2c_plan** out);
+
 /* Copies the chosen embedding (with device_us if it was timed) to *chosen. */
 int b2c_plan_info(const b2c_plan* plan, b2c_embedding* chosen);
 

@@ -31,7 +31,7 @@ EXPORTS = [
     "b2c_out_shape", "b2c_enumerate", "b2c_plan_create", "b2c_plan_info", "b2c_plan_workspace_bytes",
     "b2c_plan_set_weights", "b2c_conv2d_int8_run", "b2c_conv2d_int8", "b2c_conv2d_int8_host",
     "b2c_plan_rewrite_activations", "b2c_conv2d_int8_run_rewritten", "b2c_plan_footprint", "b2c_plan_set_activation",
-    "b2c_plan_create_grouped", "b2c_plan_run_host_async", "b2c_plan_host_sync",
+    "b2c_plan_create_grouped", "b2c_plan_create_grouped_timed", "b2c_plan_run_host_async", "b2c_plan_host_sync",
     "b2c_plan_device_status", "b2c_selftest_bounded_wait", "b2c_plan_destroy", "b2c_pack_activations", "b2c_im2col", "b2c_im2col_noalloc",
     "b2c_status_string",
     "b2c_last_cuda_error", "b2c_oneshot_status", "b2c_oneshot_cache_clear", "b2c_test_fail_nth_encode", "b2c_selftest_pack_wait", "b2c_measure_mma_rate", "b2c_measure_mma_rate_pair", "b2c_debug_build", "b2c_plan_debug_info",
@@ -93,6 +93,7 @@ def load():
     lib.b2c_conv2d_int8_run_rewritten.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.b2c_plan_set_activation.argtypes = [vp, vp, i32, vp]
     lib.b2c_plan_create_grouped.argtypes = [pd, ctypes.c_int32, ctypes.POINTER(vp)]
+    lib.b2c_plan_create_grouped_timed.argtypes = [pd, ctypes.c_int32, vp, ctypes.POINTER(vp)]
     lib.b2c_plan_footprint.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
     lib.b2c_conv2d_int8.argtypes = [i32] * 11 + [vp] * 5
     lib.b2c_conv2d_int8_host.argtypes = [i32] * 11 + [vp] * 4
@@ -179,11 +180,15 @@ class Plan:
     """Owns a ``b2c_plan``.  ``run`` enqueues the whole path on the current torch stream."""
 
     def __init__(self, desc: ConvDesc, policy_or_id: int = POLICY_MIN_OVERHEAD, stream=None, groups: int = 1):
-        """groups > 1: grouped convolution (desc.C and desc.K are the totals, weights [K, C/groups, R, S])."""
+        """groups > 1: grouped convolution (desc.C and desc.K are the totals, weights [K, C/groups, R, S]); with a
+        timed policy the form (in place, or all groups merged into a dense convolution) is chosen by timing."""
         self._lib = load()
         self.desc = desc
         h = ctypes.c_void_p()
-        if groups > 1:
+        if groups > 1 and policy_or_id in (POLICY_AUTO_TIMED, POLICY_AUTO_TIMED_CONCURRENT):
+            _check(self._lib.b2c_plan_create_grouped_timed(ctypes.byref(desc), groups, _stream_ptr(stream), ctypes.byref(h)),
+                   "b2c_plan_create_grouped_timed")
+        elif groups > 1:
             _check(self._lib.b2c_plan_create_grouped(ctypes.byref(desc), groups, ctypes.byref(h)), "b2c_plan_create_grouped")
         else:
             _check(self._lib.b2c_plan_create(ctypes.byref(desc), policy_or_id, _stream_ptr(stream), ctypes.byref(h)),

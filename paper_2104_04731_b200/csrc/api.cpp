@@ -50,6 +50,9 @@ struct b2c_plan {
   // reduction depth; w_expanded holds the expanded filters [K][merge * C/groups][R][S].
   int merge = 1;
   int8_t* w_expanded = nullptr;  // device, plan-owned
+  // Group plan whose one sub-plan is the DENSE convolution of the whole tensors with block-diagonal filters
+  // (every group merged): it runs like any dense plan, rewrite and scratch included.
+  bool dense_sub = false;
   long long x_stride_n_whole = 0, y_stride_n_whole = 0;  // sub-plans: batch strides of the whole tensors
   struct HostPipe* pipe = nullptr;  // streaming host-buffer calls: created by the first b2c_plan_run_host_async
   // The two-SM persistent channel-pack schedule can run the activation pack inside the MMA kernel
@@ -874,6 +877,83 @@ int b2c_plan_create_grouped(const b2c_conv_desc* desc, int32_t groups, b2c_plan*
   return B2C_OK;
 }
 
+int b2c_plan_create_grouped_timed(const b2c_conv_desc* desc, int32_t groups, void* cuda_stream, b2c_plan** out) {
+  if (!desc || !out) return B2C_E_INVALID_ARG;
+  *out = nullptr;
+  b2c_plan* inplace = nullptr;
+  int rc = b2c_plan_create_grouped(desc, groups, &inplace);
+  if (rc != B2C_OK) return rc;
+  // The other form: every group merged, i.e. the dense convolution with block-diagonal filters through the
+  // timed selection of dense plans.  It pays `groups` times the MACs and has the rewrite and the scratch
+  // of its embedding; on this device it still wins for a few hundred groups.
+  const long long dense_w = (long long)desc->K * desc->C * desc->R * desc->S;
+  if (groups < 2 || dense_w > (16ll << 20)) {
+    *out = inplace;
+    return B2C_OK;
+  }
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  b2c_plan* dense = nullptr;
+  if (b2c_plan_create(desc, B2C_POLICY_AUTO_TIMED, cuda_stream, &dense) != B2C_OK || dense->emb.device_us <= 0) {
+    b2c_plan_destroy(dense);
+    *out = inplace;
+    return B2C_OK;
+  }
+  // time the in-place form on scratch tensors, as the dense candidates were
+  const Geom& g = dense->g;
+  int8_t *x = nullptr, *w = nullptr;
+  LaneBuffers lane = {};
+  float us = -1;
+  bool ok = cudaMalloc(&x, g.x_elems + 256) == cudaSuccess && cudaMalloc(&w, g.w_elems + 256) == cudaSuccess &&
+            cudaMalloc(&lane.y8, g.y_elems + 256) == cudaSuccess && cudaMalloc(&lane.y32, g.y_elems * 4 + 256) == cudaSuccess &&
+            cudaMalloc(&lane.ws, 1024) == cudaSuccess;
+  if (ok) {
+    cudaMemsetAsync(x, 1, g.x_elems, st);
+    cudaMemsetAsync(w, 1, g.w_elems, st);  // (the grouped filter tensor is smaller than the dense one)
+    ok = b2c_plan_set_weights(inplace, w, st) == B2C_OK && cudaStreamSynchronize(st) == cudaSuccess &&
+         time_plan(inplace, x, &lane, 1, &us) == B2C_OK;
+    inplace->weights_set = false;  // the caller's filters are still to come
+  }
+  cudaFree(x);
+  cudaFree(w);
+  cudaFree(lane.y8);
+  cudaFree(lane.y32);
+  cudaFree(lane.ws);
+  if (!ok) (void)cudaGetLastError();
+  if (!ok || us <= dense->emb.device_us) {  // (an in-place form that could not be timed is still the safe choice)
+    b2c_plan_destroy(dense);
+    inplace->emb.device_us = us;
+    *out = inplace;
+    return B2C_OK;
+  }
+  // wrap the dense plan: filters expanded at set_weights, everything else is the dense plan's own path
+  b2c_plan* p = new (std::nothrow) b2c_plan();
+  bool made = p != nullptr;
+  if (made) {
+    p->g = dense->g;
+    p->emb = dense->emb;
+    p->groups = groups;
+    p->merge = groups;
+    p->dense_sub = true;
+    p->ws_total = dense->ws_total;
+    p->ws_layout_bytes = dense->ws_layout_bytes;
+    cudaGetDevice(&p->device);
+    made = cudaMalloc(&p->status, kStatusWords * sizeof(int)) == cudaSuccess &&
+           cudaMemset(p->status, 0, kStatusWords * sizeof(int)) == cudaSuccess &&
+           cudaMalloc(&p->w_expanded, (size_t)dense_w + 256) == cudaSuccess;
+  }
+  if (!made) {
+    set_last_cuda_error((int)cudaGetLastError());
+    b2c_plan_destroy(p);
+    b2c_plan_destroy(dense);
+    *out = inplace;
+    return B2C_OK;
+  }
+  p->subs.push_back(dense);
+  b2c_plan_destroy(inplace);
+  *out = p;
+  return B2C_OK;
+}
+
 int b2c_plan_info(const b2c_plan* plan, b2c_embedding* chosen) {
   if (!plan || !chosen) return B2C_E_INVALID_ARG;
   *chosen = plan->emb;
@@ -1096,14 +1176,15 @@ int b2c_conv2d_int8_run(b2c_plan* p, const int8_t* x, int32_t* y32, int8_t* y8, 
   cudaStream_t st = (cudaStream_t)cuda_stream;
   ws = guard_workspace(p, ws, st, &rc);
   if (rc != B2C_OK) return rc;
-  if (!p->subs.empty()) {
+  if (!p->subs.empty() && !p->dense_sub) {
     // one launch: every group convolves its channel slice of x (NCHW) into its slice of y (NKPQ)
     return run_convolve(p->subs[0], x, y32, y8, nullptr, st);
   }
-  if (p->fused_pack && aligned16(x)) return run_convolve(p, x, y32, y8, ws, st, /*fused_pack=*/true);
-  rc = run_rewrite(p, x, ws, st);
+  b2c_plan* r = p->dense_sub ? p->subs[0] : p;  // (all groups merged: the dense plan's own path)
+  if (r->fused_pack && aligned16(x)) return run_convolve(r, x, y32, y8, ws, st, /*fused_pack=*/true);
+  rc = run_rewrite(r, x, ws, st);
   if (rc != B2C_OK) return rc;
-  return run_convolve(p, x, y32, y8, ws, st);
+  return run_convolve(r, x, y32, y8, ws, st);
 }
 
 int b2c_plan_rewrite_activations(b2c_plan* p, const int8_t* x, void* ws, void* cuda_stream) {

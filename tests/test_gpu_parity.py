@@ -458,6 +458,38 @@ def test_grouped_convolution(lib, case):
     assert raw.b2c_plan_create_grouped(ctypes.byref(d_nhwc), groups, ctypes.byref(h)) == b2c.E_UNSUPPORTED
 
 
+@pytest.mark.parametrize("case", [
+    (2, 256, 14, 14, 256, 256, 3, 3, 1, 1, 1, 4, 3),    # depth-wise, 256 channels: the full merge wins on this device
+    (3, 12, 9, 7, 24, 4, 3, 2, (2, 1), (1, 0), 1, 5, 3),  # four groups, odd image
+    (2, 64, 7, 7, 128, 2, 1, 1, 1, 0, 1, 7, 2),         # pointwise, two wide groups
+])
+def test_grouped_convolution_form_chosen_by_timing(lib, case):
+    N, C, H, W, K, groups, R, S, stride, pad, dil, shift, out_mode = case
+    x = int8_uniform((N, C, H, W), 695)
+    w = int8_uniform((K, C // groups, R, S), 696)
+    bias = int8_uniform((K,), 697).astype(np.int32) * 101
+    d = lib.make_desc(N, C, H, W, K, R, S, stride, pad, dil, shift, out_mode=out_mode)
+    P, Q = lib.out_shape(d)
+    plan = lib.Plan(d, b2c.POLICY_AUTO_TIMED, groups=groups)
+    assert plan.info().device_us > 0
+    ws = torch.empty(max(16, plan.workspace_bytes()), dtype=torch.uint8, device="cuda")
+    plan.set_weights(to_dev(w))
+    xd = to_dev(x)
+    for use_bias, relu in [(False, False), (True, True)]:
+        ref = oracle.conv2d_int8(x, w, stride, pad, dil, shift, groups=groups, bias=bias if use_bias else None, relu=relu)
+        plan.set_activation(to_dev(bias) if use_bias else None, relu)
+        y32 = torch.full((N, K, P, Q), -7777777, dtype=torch.int32, device="cuda") if out_mode & 1 else None
+        y8 = torch.full((N, K, P, Q), 77, dtype=torch.int8, device="cuda") if out_mode & 2 else None
+        plan.run(xd, y32, y8, ws)
+        torch.cuda.synchronize()
+        assert plan.device_status() == b2c.OK
+        if y32 is not None:
+            assert np.array_equal(y32.cpu().numpy(), ref[0])
+        if y8 is not None:
+            assert np.array_equal(y8.cpu().numpy(), ref[1])
+    plan.destroy()
+
+
 def test_extreme_values_and_shift_clip(lib):
     # -128 * -128 is the largest product; all-(-128) tensors with 9*64 taps reach 9437184.
     x = np.full((1, 64, 6, 6), -128, dtype=np.int8)
